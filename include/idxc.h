@@ -1,0 +1,186 @@
+/*
+ * idxc -- lightning-indexer scoring, causal top-k selection and the IndexCache
+ * Full/Shared layer schedule for one NVIDIA B200 (sm_100a).
+ *
+ * Plain C ABI. Every pointer is a DEVICE pointer unless its comment says HOST.
+ * The caller owns every buffer; the library allocates no device memory. All
+ * work is enqueued on the CUDA stream passed in (a cudaStream_t cast to
+ * void*, NULL = the legacy default stream) and the calls return without
+ * synchronising. Every call returns an idxc_status; nothing throws or aborts.
+ * Inputs are assumed finite (NaN / Inf scores give an unspecified selection).
+ *
+ * Notation follows the paper: L sequence length, H_I indexer heads, d_I indexer
+ * head dimension, k_top selected tokens per query (k = 2048 in the paper),
+ * N layers, pattern string c over {F, S}. Positions and layers are 0-based.
+ */
+#ifndef IDXC_H_
+#define IDXC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    IDXC_OK = 0,
+    IDXC_ERR_INVALID_ARG = 1,    /* null / misaligned pointer, size out of range, inconsistent sizes      */
+    IDXC_ERR_UNSUPPORTED = 2,    /* a valid request this build has no kernel for (H_I, d_I, dtype combo)  */
+    IDXC_ERR_WORKSPACE = 3,      /* workspace missing or smaller than the matching *_workspace_bytes()    */
+    IDXC_ERR_PATTERN = 4,        /* pattern string invalid, or layers visited out of order                */
+    IDXC_ERR_CUDA = 5,           /* a CUDA runtime/driver call failed (launch, tensor-map encode, ...)    */
+    IDXC_ERR_DEVICE_TIMEOUT = 6  /* a bounded device-side wait gave up; results of that launch are void   */
+} idxc_status;
+
+/* Storage type of q and k. w and the scales are always fp32.
+ * IDXC_FP8_E4M3 is the finite-only e4m3 ("FN": max 448, no infinities) with one
+ * fp32 scale per token: value = code * scale. */
+typedef enum { IDXC_BF16 = 0, IDXC_FP8_E4M3 = 1 } idxc_dtype;
+
+/* flags (bitwise or) */
+#define IDXC_FLAG_COPY_SHARED 0x1u  /* schedule: S layers copy the cached indices into topk_buf instead of aliasing */
+#define IDXC_FLAG_SIMT_SCORER 0x2u  /* debugging aid: score with the plain CUDA-core kernel instead of tcgen05     */
+
+/* Limits checked before any launch. */
+#define IDXC_MAX_K_TOP 2048
+#define IDXC_MAX_HEADS 64
+
+const char* idxc_status_string(idxc_status s);
+
+/* ---------------------------------------------------------------------------
+ * Prefill: indexer scores and causal top-k for a block of query positions.
+ *
+ * Operation (Sec. 2.1 "DeepSeek Sparse Attention": the lightning indexer scores
+ * all preceding tokens with a multi-head ReLU-gated dot product; Sec. 3
+ * "Notation": T_t = Top-k(I_t)):
+ *     I[t, s] = sum_h w[t, h] * max(q[t, h, :] . k[s, :], 0)      for s <= t
+ *     T[t]    = the min(k_top, t + 1) positions s <= t with the largest I[t, s]
+ * Ties go to the lowest position. T[t] is written in ascending position order
+ * and padded with -1 up to k_top entries. With IDXC_FP8_E4M3 the dot product
+ * uses the codes and the result is multiplied by q_scale[t] * k_scale[s].
+ *
+ *   q        [q_len, H_I, d_I] row-major; row r is position t = q_begin + r
+ *   k        [L_k, d_I] row-major, L_k >= q_begin + q_len
+ *   w        [q_len, H_I] fp32
+ *   q_scale  [q_len] fp32, k_scale [L_k] fp32: IDXC_FP8_E4M3 only, else NULL
+ *   scores_out  NULL, or [q_len, ld_scores] fp32 (ld_scores >= L_k, a multiple of 4;
+ *               base 16-byte aligned). Only entries s <= t are written.
+ *   topk_out    NULL, or [q_len, k_top] int32
+ *   workspace   at least idxc_prefill_workspace_bytes(...) bytes, 256-byte aligned;
+ *               contents are scratch. With scores_out == NULL the scores go through it
+ *               in query chunks, so its size does not grow with q_len beyond a cap.
+ * A full prefill is q_begin = 0, q_len = L_k = L; chunked prefill calls this once
+ * per chunk with the full K and gives the same rows.
+ * Supported: d_I in {64, 128}; H_I in {16, 32, 64}; 1 <= k_top <= 2048;
+ * q, k, w 16-byte aligned. Other sizes return IDXC_ERR_UNSUPPORTED / INVALID_ARG
+ * before anything is launched.
+ * ------------------------------------------------------------------------- */
+size_t idxc_prefill_workspace_bytes(int64_t q_len, int64_t L_k, int H_I, int d_I, int k_top,
+                                    idxc_dtype dt, uint32_t flags);
+
+idxc_status idxc_indexer_prefill(const void* q, const void* k, const float* w,
+                                 const float* q_scale, const float* k_scale,
+                                 int64_t q_begin, int64_t q_len, int64_t L_k,
+                                 int H_I, int d_I, int k_top, idxc_dtype dt,
+                                 float* scores_out, int64_t ld_scores, int32_t* topk_out,
+                                 void* workspace, size_t workspace_bytes, uint32_t flags,
+                                 void* cuda_stream);
+
+/* ---------------------------------------------------------------------------
+ * Decode: one new query per sequence against that sequence's cached indexer keys
+ * (Sec. 4.2 "Decode": a per-token indexer pass over the full context).
+ *     I[b, s] = sum_h w[b, h] * max(q_step[b, h, :] . K_b[s, :], 0)   for s < lens[b]
+ *     T[b]    = Top-k over s in [0, lens[b]), same order / tie / padding rules
+ *
+ *   q_step    [B, H_I, d_I]
+ *   k_cache   base of a [rows, d_I] row-major array; sequence b owns rows
+ *             k_offsets[b] .. k_offsets[b] + lens[b] - 1 (the new token's key included)
+ *   cache_rows  number of rows of k_cache that may be addressed (bounds the tensor map)
+ *   w         [B, H_I] fp32
+ *   q_scale   [B], k_scale [cache_rows] (same row indexing as k_cache): FP8 only
+ *   k_offsets [B] int64, lens [B] int32 (device memory, read by the kernels)
+ *   max_len   HOST upper bound on lens[b]; sizes the grid and the workspace
+ *   scores_out NULL or [B, ld_scores] fp32, ld_scores >= max_len, multiple of 4
+ *   topk_out  NULL or [B, k_top] int32
+ * ------------------------------------------------------------------------- */
+size_t idxc_decode_workspace_bytes(int B, int64_t max_len, int H_I, int d_I, int k_top,
+                                   idxc_dtype dt, uint32_t flags);
+
+idxc_status idxc_indexer_decode(const void* q_step, const void* k_cache, int64_t cache_rows,
+                                const float* w, const float* q_scale, const float* k_scale,
+                                const int64_t* k_offsets, const int32_t* lens,
+                                int B, int64_t max_len, int H_I, int d_I, int k_top, idxc_dtype dt,
+                                float* scores_out, int64_t ld_scores, int32_t* topk_out,
+                                void* workspace, size_t workspace_bytes, uint32_t flags,
+                                void* cuda_stream);
+
+/* ---------------------------------------------------------------------------
+ * Top-k alone (Sec. 3 "Notation"), for rows of fp32 scores already in memory.
+ * Row r has length lens[r] if lens != NULL (device int32), else
+ * first_len + r * len_step (len_step = 1: causal rows; 0: equal rows), clamped to
+ * [0, ld]. scores: [n_rows, ld] fp32, 16-byte aligned, ld a multiple of 4.
+ * Same order / tie / padding rules as above. Needs no workspace.
+ * ------------------------------------------------------------------------- */
+idxc_status idxc_topk_rows(const float* scores, int64_t ld, int64_t n_rows,
+                           int64_t first_len, int64_t len_step, const int32_t* lens,
+                           int k_top, int32_t* topk_out, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------
+ * IndexCache layer schedule (Sec. 3 "Overview", Figure 2(b)).
+ * pattern c_0 .. c_{N-1} over {'F','S'}: an F (Full) layer runs its indexer and its
+ * result becomes the cached index tensor; an S (Shared) layer returns the cached
+ * tensor of f(l) = max{ j < l : c_j = F } without running anything. c_0 must be 'F'.
+ * The schedule object is HOST state only (the pattern, f(l), the cached pointer and
+ * counters); it is not thread-safe. Layers of one forward pass are visited in
+ * increasing order; idxc_schedule_begin_pass() forgets the cached tensor.
+ * ------------------------------------------------------------------------- */
+typedef struct idxc_schedule idxc_schedule;
+
+idxc_status idxc_schedule_create(const char* pattern /* HOST, N chars */, int N, idxc_schedule** out /* HOST */);
+void        idxc_schedule_destroy(idxc_schedule* s);
+idxc_status idxc_schedule_begin_pass(idxc_schedule* s);
+/* f(layer); equals layer on F layers. src_layer is a HOST pointer. */
+idxc_status idxc_schedule_source(const idxc_schedule* s, int layer, int* src_layer);
+/* HOST outputs: number of F and S layers in the pattern, indexer launches made so far. */
+idxc_status idxc_schedule_stats(const idxc_schedule* s, int* n_full, int* n_shared, int64_t* indexer_calls);
+
+/* One layer of a prefill pass. On an F layer: runs idxc_indexer_prefill with the given
+ * arguments into topk_buf ([q_len, k_top] int32, required) and caches it. On an S layer:
+ * q, k, w, scales, scores_out and workspace are ignored (may be NULL) and nothing is
+ * launched; *topk_result (HOST out) is the cached pointer, i.e. it aliases the F layer's
+ * buffer, which the caller must therefore keep intact until the next F layer. With
+ * IDXC_FLAG_COPY_SHARED an S layer instead copies the cached tensor into topk_buf
+ * (one device-to-device copy) and returns topk_buf. Visiting an S layer whose source
+ * layer was not the last F layer run in this pass returns IDXC_ERR_PATTERN. */
+idxc_status idxc_schedule_prefill_layer(idxc_schedule* s, int layer,
+                                        const void* q, const void* k, const float* w,
+                                        const float* q_scale, const float* k_scale,
+                                        int64_t q_begin, int64_t q_len, int64_t L_k,
+                                        int H_I, int d_I, int k_top, idxc_dtype dt,
+                                        float* scores_out, int64_t ld_scores, int32_t* topk_buf,
+                                        void* workspace, size_t workspace_bytes, uint32_t flags,
+                                        void* cuda_stream, const int32_t** topk_result);
+
+/* One layer of a decode step; same rules, wrapping idxc_indexer_decode ([B, k_top]). */
+idxc_status idxc_schedule_decode_layer(idxc_schedule* s, int layer,
+                                       const void* q_step, const void* k_cache, int64_t cache_rows,
+                                       const float* w, const float* q_scale, const float* k_scale,
+                                       const int64_t* k_offsets, const int32_t* lens,
+                                       int B, int64_t max_len, int H_I, int d_I, int k_top, idxc_dtype dt,
+                                       float* scores_out, int64_t ld_scores, int32_t* topk_buf,
+                                       void* workspace, size_t workspace_bytes, uint32_t flags,
+                                       void* cuda_stream, const int32_t** topk_result);
+
+/* Synchronises the stream, then returns IDXC_OK, IDXC_ERR_CUDA, or
+ * IDXC_ERR_DEVICE_TIMEOUT if any kernel of this library recorded a bounded wait that
+ * ran out since the last poll (the record is cleared). */
+idxc_status idxc_poll_device_status(void* cuda_stream);
+
+/* Number of kernel launches this library has made in this process (all streams). */
+int64_t idxc_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* IDXC_H_ */

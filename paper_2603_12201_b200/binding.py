@@ -1,0 +1,288 @@
+"""Python binding of the idxc C-ABI library: argument marshalling only.
+
+Every step of the path (scoring, selection, schedule bookkeeping) runs inside
+``libidxc.so``; torch is used for device memory and streams. There is no CPU or
+eager fallback: if the library is missing or a call fails, an exception is raised.
+Function names mirror ``include/idxc.h``.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import torch
+
+_LIB_PATH = Path(__file__).resolve().parent / "libidxc.so"
+
+OK = 0
+ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_PATTERN, ERR_CUDA, ERR_DEVICE_TIMEOUT = 1, 2, 3, 4, 5, 6
+BF16, FP8_E4M3 = 0, 1
+FLAG_COPY_SHARED = 0x1
+FLAG_SIMT_SCORER = 0x2
+
+EXPORTED_SYMBOLS = [
+    "idxc_status_string", "idxc_prefill_workspace_bytes", "idxc_indexer_prefill", "idxc_decode_workspace_bytes",
+    "idxc_indexer_decode", "idxc_topk_rows", "idxc_schedule_create", "idxc_schedule_destroy",
+    "idxc_schedule_begin_pass", "idxc_schedule_source", "idxc_schedule_stats", "idxc_schedule_prefill_layer",
+    "idxc_schedule_decode_layer", "idxc_poll_device_status", "idxc_launch_count",
+]
+
+
+class IdxcError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded library; raises if it has not been built (run paper_2603_12201_b200/build.py)."""
+    global _lib
+    if _lib is None:
+        if not _LIB_PATH.exists():
+            raise RuntimeError(f"{_LIB_PATH} is missing: build it with `python -m paper_2603_12201_b200.build` "
+                               "(there is no fallback path)")
+        L = ctypes.CDLL(str(_LIB_PATH))
+        vp, i64, i32, u32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_uint32, ctypes.c_size_t
+        L.idxc_status_string.restype = ctypes.c_char_p
+        L.idxc_status_string.argtypes = [i32]
+        L.idxc_launch_count.restype = i64
+        L.idxc_prefill_workspace_bytes.restype = sz
+        L.idxc_prefill_workspace_bytes.argtypes = [i64, i64, i32, i32, i32, i32, u32]
+        L.idxc_decode_workspace_bytes.restype = sz
+        L.idxc_decode_workspace_bytes.argtypes = [i32, i64, i32, i32, i32, i32, u32]
+        prefill_args = [vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, i32, i32, vp, i64, vp, vp, sz, u32, vp]
+        decode_args = [vp, vp, i64, vp, vp, vp, vp, vp, i32, i64, i32, i32, i32, i32, vp, i64, vp, vp, sz, u32, vp]
+        L.idxc_indexer_prefill.restype = i32
+        L.idxc_indexer_prefill.argtypes = prefill_args
+        L.idxc_indexer_decode.restype = i32
+        L.idxc_indexer_decode.argtypes = decode_args
+        L.idxc_topk_rows.restype = i32
+        L.idxc_topk_rows.argtypes = [vp, i64, i64, i64, i64, vp, i32, vp, vp]
+        L.idxc_schedule_create.restype = i32
+        L.idxc_schedule_create.argtypes = [ctypes.c_char_p, i32, ctypes.POINTER(vp)]
+        L.idxc_schedule_destroy.restype = None
+        L.idxc_schedule_destroy.argtypes = [vp]
+        L.idxc_schedule_begin_pass.restype = i32
+        L.idxc_schedule_begin_pass.argtypes = [vp]
+        L.idxc_schedule_source.restype = i32
+        L.idxc_schedule_source.argtypes = [vp, i32, ctypes.POINTER(i32)]
+        L.idxc_schedule_stats.restype = i32
+        L.idxc_schedule_stats.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i64)]
+        L.idxc_schedule_prefill_layer.restype = i32
+        L.idxc_schedule_prefill_layer.argtypes = [vp, i32] + prefill_args + [ctypes.POINTER(vp)]
+        L.idxc_schedule_decode_layer.restype = i32
+        L.idxc_schedule_decode_layer.argtypes = [vp, i32] + decode_args + [ctypes.POINTER(vp)]
+        L.idxc_poll_device_status.restype = i32
+        L.idxc_poll_device_status.argtypes = [vp]
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().idxc_status_string(int(status)).decode()
+
+
+def launch_count() -> int:
+    return int(lib().idxc_launch_count())
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise IdxcError(status, where)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _dtype_of(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return BF16
+    if t.dtype == torch.float8_e4m3fn:
+        return FP8_E4M3
+    raise TypeError(f"q/k must be bfloat16 or float8_e4m3fn, got {t.dtype}")
+
+
+def _dev(t: torch.Tensor, name: str, dtype=None):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError(f"{name} must live on a CUDA device (this library has no CPU path)")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{name}: expected {dtype}, got {t.dtype}")
+    return t
+
+
+def prefill_workspace_bytes(q_len, L_k, H, d, k_top, dt=BF16, flags=0) -> int:
+    return int(lib().idxc_prefill_workspace_bytes(q_len, L_k, H, d, k_top, dt, flags))
+
+
+def decode_workspace_bytes(B, max_len, H, d, k_top, dt=BF16, flags=0) -> int:
+    return int(lib().idxc_decode_workspace_bytes(B, max_len, H, d, k_top, dt, flags))
+
+
+def alloc_workspace(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def _prefill_marshal(q, k, w, q_scale, k_scale, q_begin, k_top, scores_out, topk_out, workspace, flags, stream):
+    _dev(q, "q"); _dev(k, "k"); _dev(w, "w", torch.float32)
+    _dev(q_scale, "q_scale", torch.float32); _dev(k_scale, "k_scale", torch.float32)
+    _dev(scores_out, "scores_out", torch.float32); _dev(topk_out, "topk_out", torch.int32); _dev(workspace, "workspace")
+    dt = _dtype_of(q)
+    if k.dtype != q.dtype:
+        raise TypeError("q and k must have the same dtype")
+    q_len, H, d = q.shape
+    L_k = k.shape[0]
+    if k.shape[1] != d or tuple(w.shape) != (q_len, H):
+        raise ValueError("shape mismatch between q, k and w")
+    ld = 0
+    if scores_out is not None:
+        if scores_out.dim() != 2 or scores_out.shape[0] != q_len:
+            raise ValueError("scores_out must be [q_len, ld]")
+        ld = scores_out.shape[1]
+    if topk_out is not None and tuple(topk_out.shape) != (q_len, k_top):
+        raise ValueError("topk_out must be [q_len, k_top]")
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    return [_ptr(q), _ptr(k), _ptr(w), _ptr(q_scale), _ptr(k_scale), int(q_begin), q_len, L_k, H, d, int(k_top), dt,
+            _ptr(scores_out), ld, _ptr(topk_out), _ptr(workspace), ws_bytes, int(flags), _stream(stream)]
+
+
+def indexer_prefill(q, k, w, k_top, q_scale=None, k_scale=None, q_begin=0, scores_out=None, topk_out=None,
+                    workspace=None, flags=0, stream=None):
+    """idxc_indexer_prefill. Writes into scores_out / topk_out (either may be None, not both)."""
+    args = _prefill_marshal(q, k, w, q_scale, k_scale, q_begin, k_top, scores_out, topk_out, workspace, flags, stream)
+    _check(lib().idxc_indexer_prefill(*args), "idxc_indexer_prefill")
+
+
+def _decode_marshal(q_step, k_cache, w, q_scale, k_scale, k_offsets, lens, max_len, k_top, scores_out, topk_out,
+                    workspace, flags, stream):
+    _dev(q_step, "q_step"); _dev(k_cache, "k_cache"); _dev(w, "w", torch.float32)
+    _dev(q_scale, "q_scale", torch.float32); _dev(k_scale, "k_scale", torch.float32)
+    _dev(k_offsets, "k_offsets", torch.int64); _dev(lens, "lens", torch.int32)
+    _dev(scores_out, "scores_out", torch.float32); _dev(topk_out, "topk_out", torch.int32); _dev(workspace, "workspace")
+    dt = _dtype_of(q_step)
+    if k_cache.dtype != q_step.dtype:
+        raise TypeError("q_step and k_cache must have the same dtype")
+    B, H, d = q_step.shape
+    if k_cache.shape[1] != d or tuple(w.shape) != (B, H) or k_offsets.shape[0] != B or lens.shape[0] != B:
+        raise ValueError("shape mismatch between q_step, k_cache, w, k_offsets and lens")
+    ld = 0
+    if scores_out is not None:
+        if scores_out.dim() != 2 or scores_out.shape[0] != B:
+            raise ValueError("scores_out must be [B, ld]")
+        ld = scores_out.shape[1]
+    if topk_out is not None and tuple(topk_out.shape) != (B, k_top):
+        raise ValueError("topk_out must be [B, k_top]")
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    return [_ptr(q_step), _ptr(k_cache), k_cache.shape[0], _ptr(w), _ptr(q_scale), _ptr(k_scale), _ptr(k_offsets),
+            _ptr(lens), B, int(max_len), H, d, int(k_top), dt, _ptr(scores_out), ld, _ptr(topk_out), _ptr(workspace),
+            ws_bytes, int(flags), _stream(stream)]
+
+
+def indexer_decode(q_step, k_cache, w, k_offsets, lens, max_len, k_top, q_scale=None, k_scale=None, scores_out=None,
+                   topk_out=None, workspace=None, flags=0, stream=None):
+    """idxc_indexer_decode. ``max_len`` is a host upper bound on ``lens``."""
+    args = _decode_marshal(q_step, k_cache, w, q_scale, k_scale, k_offsets, lens, max_len, k_top, scores_out,
+                           topk_out, workspace, flags, stream)
+    _check(lib().idxc_indexer_decode(*args), "idxc_indexer_decode")
+
+
+def topk_rows(scores, k_top, topk_out, first_len=0, len_step=0, lens=None, stream=None):
+    """idxc_topk_rows on a [n_rows, ld] fp32 tensor."""
+    _dev(scores, "scores", torch.float32); _dev(topk_out, "topk_out", torch.int32); _dev(lens, "lens", torch.int32)
+    n_rows, ld = scores.shape
+    if tuple(topk_out.shape) != (n_rows, k_top):
+        raise ValueError("topk_out must be [n_rows, k_top]")
+    _check(lib().idxc_topk_rows(_ptr(scores), ld, n_rows, int(first_len), int(len_step), _ptr(lens), int(k_top),
+                                _ptr(topk_out), _stream(stream)), "idxc_topk_rows")
+
+
+def poll_device_status(stream=None):
+    """Synchronises the stream and raises if a kernel recorded a bounded-wait timeout."""
+    _check(lib().idxc_poll_device_status(_stream(stream)), "idxc_poll_device_status")
+
+
+class Schedule:
+    """idxc_schedule: the Full/Shared layer pattern and the cached index tensor (host state)."""
+
+    def __init__(self, pattern: str):
+        self._h = ctypes.c_void_p()
+        self.pattern = pattern
+        raw = pattern.encode("ascii", errors="replace")
+        _check(lib().idxc_schedule_create(raw, len(raw), ctypes.byref(self._h)), "idxc_schedule_create")
+        self._keep = {}          # topk buffers by data_ptr, so a returned alias can be mapped back to its tensor
+
+    def close(self):
+        if self._h:
+            lib().idxc_schedule_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def begin_pass(self):
+        self._keep.clear()
+        _check(lib().idxc_schedule_begin_pass(self._h), "idxc_schedule_begin_pass")
+
+    def source(self, layer: int) -> int:
+        out = ctypes.c_int()
+        _check(lib().idxc_schedule_source(self._h, layer, ctypes.byref(out)), "idxc_schedule_source")
+        return out.value
+
+    def stats(self):
+        nf, ns, calls = ctypes.c_int(), ctypes.c_int(), ctypes.c_int64()
+        _check(lib().idxc_schedule_stats(self._h, ctypes.byref(nf), ctypes.byref(ns), ctypes.byref(calls)),
+               "idxc_schedule_stats")
+        return nf.value, ns.value, calls.value
+
+    def _result(self, res_ptr, topk_buf):
+        if topk_buf is not None:
+            self._keep[topk_buf.data_ptr()] = topk_buf
+        t = self._keep.get(res_ptr.value)
+        if t is None:
+            raise RuntimeError("schedule returned a pointer to a buffer this object has not seen")
+        return t
+
+    def prefill_layer(self, layer, q=None, k=None, w=None, k_top=0, q_scale=None, k_scale=None, q_begin=0, q_len=None,
+                      scores_out=None, topk_buf=None, workspace=None, flags=0, stream=None):
+        """One layer of a prefill pass. S layers need only k_top and q_len (inputs may be None).
+        Returns the tensor holding this layer's indices (the F layer's buffer on S layers)."""
+        res = ctypes.c_void_p()
+        if q is None:
+            if q_len is None:
+                raise ValueError("q_len is required when q is None")
+            args = [None, None, None, None, None, int(q_begin), int(q_len), 0, 0, 0, int(k_top), BF16, None, 0,
+                    _ptr(_dev(topk_buf, "topk_buf", torch.int32)), None, 0, int(flags), _stream(stream)]
+        else:
+            args = _prefill_marshal(q, k, w, q_scale, k_scale, q_begin, k_top, scores_out, topk_buf, workspace, flags, stream)
+        _check(lib().idxc_schedule_prefill_layer(self._h, layer, *args, ctypes.byref(res)), "idxc_schedule_prefill_layer")
+        return self._result(res, topk_buf)
+
+    def decode_layer(self, layer, q_step=None, k_cache=None, w=None, k_offsets=None, lens=None, max_len=0, k_top=0,
+                     q_scale=None, k_scale=None, B=None, scores_out=None, topk_buf=None, workspace=None, flags=0,
+                     stream=None):
+        res = ctypes.c_void_p()
+        if q_step is None:
+            if B is None:
+                raise ValueError("B is required when q_step is None")
+            args = [None, None, 0, None, None, None, None, None, int(B), int(max_len), 0, 0, int(k_top), BF16, None, 0,
+                    _ptr(_dev(topk_buf, "topk_buf", torch.int32)), None, 0, int(flags), _stream(stream)]
+        else:
+            args = _decode_marshal(q_step, k_cache, w, q_scale, k_scale, k_offsets, lens, max_len, k_top, scores_out,
+                                   topk_buf, workspace, flags, stream)
+        _check(lib().idxc_schedule_decode_layer(self._h, layer, *args, ctypes.byref(res)), "idxc_schedule_decode_layer")
+        return self._result(res, topk_buf)

@@ -1,0 +1,390 @@
+// C-ABI layer: argument validation, TMA tensor-map encoding, launch sequencing and the
+// host-side IndexCache schedule object. No device memory is allocated here.
+#include <atomic>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/idxc.h"
+#include "kernels.h"
+
+namespace idxc {
+
+__device__ unsigned int g_device_status = 0;   // first bounded-wait failure since the last poll
+
+namespace {
+
+std::atomic<int64_t> g_launches{0};
+
+struct DeviceInfo {
+    bool ready = false;
+    bool ok = false;
+    int sm_count = 0;
+    unsigned int* status_ptr = nullptr;
+    decltype(&cuTensorMapEncodeTiled) encode = nullptr;
+};
+
+DeviceInfo& device_info() {
+    static DeviceInfo info;
+    if (!info.ready) {
+        info.ready = true;
+        int dev = 0;
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&info.sm_count, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
+            cudaGetSymbolAddress(reinterpret_cast<void**>(&info.status_ptr), g_device_status) == cudaSuccess &&
+            cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess && fn != nullptr) {
+            info.encode = reinterpret_cast<decltype(&cuTensorMapEncodeTiled)>(fn);
+            info.ok = true;
+        }
+    }
+    return info;
+}
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
+
+constexpr int64_t kMinChunkRows = 32;
+constexpr int64_t kPreferredScratchBytes = int64_t(8) << 30;
+
+// Row-major [rows, d] operand, 128-byte swizzle, box = 128 bytes x box_rows rows.
+bool encode_operand_map(CUtensorMap* map, const void* base, int64_t rows, int d, bool fp8, int box_rows) {
+    DeviceInfo& di = device_info();
+    const cuuint64_t gdim[2] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t gstride[1] = {static_cast<cuuint64_t>(d) * (fp8 ? 1u : 2u)};
+    const cuuint32_t box[2] = {fp8 ? 128u : 64u, static_cast<cuuint32_t>(box_rows)};
+    const cuuint32_t estr[2] = {1u, 1u};
+    CUresult r = di.encode(map, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                           const_cast<void*>(base), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+idxc_status check_common(int H, int d, int k_top, idxc_dtype dt, uint32_t flags) {
+    if (dt != IDXC_BF16 && dt != IDXC_FP8_E4M3) return IDXC_ERR_INVALID_ARG;
+    if (k_top < 1 || k_top > IDXC_MAX_K_TOP) return IDXC_ERR_INVALID_ARG;
+    if (H < 1 || H > IDXC_MAX_HEADS || d < 1) return IDXC_ERR_INVALID_ARG;
+    if (flags & ~(IDXC_FLAG_COPY_SHARED | IDXC_FLAG_SIMT_SCORER)) return IDXC_ERR_INVALID_ARG;
+    if (!(flags & IDXC_FLAG_SIMT_SCORER) && !score_tc_supported(H, d, dt == IDXC_FP8_E4M3)) return IDXC_ERR_UNSUPPORTED;
+    return IDXC_OK;
+}
+
+idxc_status launch_scorer(const ScoreArgs& a, bool decode, uint32_t flags, cudaStream_t stream) {
+    if (flags & IDXC_FLAG_SIMT_SCORER) {
+        g_launches += 1;
+        return launch_score_simt(a, stream) == cudaSuccess ? IDXC_OK : IDXC_ERR_CUDA;
+    }
+    DeviceInfo& di = device_info();
+    CUtensorMap q_map, k_map;
+    const int q_box_rows = decode ? a.H : 256;
+    if (!encode_operand_map(&q_map, a.q, a.n_rows * a.H, a.d, a.fp8 != 0, q_box_rows)) return IDXC_ERR_CUDA;
+    if (!encode_operand_map(&k_map, a.k, a.k_rows, a.d, a.fp8 != 0, 128)) return IDXC_ERR_CUDA;
+    cudaError_t e = decode ? launch_score_decode_tc(a, q_map, k_map, di.status_ptr, di.sm_count, stream)
+                           : launch_score_prefill_tc(a, q_map, k_map, di.status_ptr, di.sm_count, stream);
+    g_launches += 1;
+    return e == cudaSuccess ? IDXC_OK : IDXC_ERR_CUDA;
+}
+
+}  // namespace
+}  // namespace idxc
+
+using namespace idxc;
+
+struct idxc_schedule {
+    std::string pattern;
+    std::vector<int> src;
+    int n_full = 0;
+    int n_shared = 0;
+    int64_t indexer_calls = 0;
+    int cache_layer = -1;              // F layer whose indices are cached, -1: none yet in this pass
+    const int32_t* cache_ptr = nullptr;
+    int64_t cache_rows = 0;
+    int cache_k_top = 0;
+};
+
+extern "C" {
+
+const char* idxc_status_string(idxc_status s) {
+    switch (s) {
+        case IDXC_OK: return "ok";
+        case IDXC_ERR_INVALID_ARG: return "invalid argument";
+        case IDXC_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+        case IDXC_ERR_WORKSPACE: return "workspace missing or too small";
+        case IDXC_ERR_PATTERN: return "invalid pattern or layer order";
+        case IDXC_ERR_CUDA: return "CUDA call failed";
+        case IDXC_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+int64_t idxc_launch_count(void) { return g_launches.load(); }
+
+size_t idxc_prefill_workspace_bytes(int64_t q_len, int64_t L_k, int H_I, int d_I, int k_top, idxc_dtype dt,
+                                    uint32_t flags) {
+    (void)L_k; (void)H_I; (void)d_I; (void)k_top; (void)dt; (void)flags;
+    if (q_len <= 0) return 0;
+    // scratch rows of round_up(L_k, 32) floats; L_k bounds q_begin + q_len
+    const int64_t ld = round_up(L_k > q_len ? L_k : q_len, 32);
+    int64_t rows = round_up(q_len, kMinChunkRows);
+    const int64_t cap = (kPreferredScratchBytes / (ld * 4)) / kMinChunkRows * kMinChunkRows;
+    if (rows > cap) rows = cap < kMinChunkRows ? kMinChunkRows : cap;
+    return static_cast<size_t>(rows * ld * 4);
+}
+
+idxc_status idxc_indexer_prefill(const void* q, const void* k, const float* w, const float* q_scale,
+                                 const float* k_scale, int64_t q_begin, int64_t q_len, int64_t L_k, int H_I,
+                                 int d_I, int k_top, idxc_dtype dt, float* scores_out, int64_t ld_scores,
+                                 int32_t* topk_out, void* workspace, size_t workspace_bytes, uint32_t flags,
+                                 void* cuda_stream) {
+    idxc_status st = check_common(H_I, d_I, k_top, dt, flags);
+    if (st != IDXC_OK) return st;
+    if (q_begin < 0 || q_len < 0 || L_k < q_begin + q_len || L_k > (int64_t(1) << 30)) return IDXC_ERR_INVALID_ARG;
+    if (!scores_out && !topk_out) return IDXC_ERR_INVALID_ARG;
+    if (q_len == 0) return IDXC_OK;
+    if (!q || !k || !w || !aligned(q, 16) || !aligned(k, 16) || !aligned(w, 16)) return IDXC_ERR_INVALID_ARG;
+    const bool fp8 = dt == IDXC_FP8_E4M3;
+    if (fp8 && (!q_scale || !k_scale)) return IDXC_ERR_INVALID_ARG;
+    if (scores_out && (ld_scores < L_k || (ld_scores & 3) || !aligned(scores_out, 16))) return IDXC_ERR_INVALID_ARG;
+    if (topk_out && !aligned(topk_out, 4)) return IDXC_ERR_INVALID_ARG;
+    if (!device_info().ok) return IDXC_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int64_t elem = fp8 ? 1 : 2;
+
+    ScoreArgs a{};
+    a.k = k; a.k_scale = fp8 ? k_scale : nullptr; a.k_offsets = nullptr; a.lens = nullptr;
+    a.k_rows = L_k; a.max_len = 0; a.H = H_I; a.d = d_I; a.fp8 = fp8 ? 1 : 0;
+
+    auto run_rows = [&](int64_t r0, int64_t nr, float* sc, int64_t ld) -> idxc_status {
+        a.q = static_cast<const char*>(q) + r0 * H_I * d_I * elem;
+        a.w = w + r0 * H_I;
+        a.q_scale = fp8 ? q_scale + r0 : nullptr;
+        a.q_begin = q_begin + r0;
+        a.n_rows = nr;
+        a.scores = sc;
+        a.ld = ld;
+        idxc_status s2 = launch_scorer(a, false, flags, stream);
+        if (s2 != IDXC_OK) return s2;
+        if (topk_out) {
+            g_launches += 1;
+            if (launch_topk_rows(sc, ld, nr, q_begin + r0 + 1, 1, nullptr, k_top, topk_out + r0 * k_top, stream) != cudaSuccess)
+                return IDXC_ERR_CUDA;
+        }
+        return IDXC_OK;
+    };
+
+    if (scores_out) return run_rows(0, q_len, scores_out, ld_scores);
+
+    // scores go through the workspace in query chunks
+    const int64_t ld = round_up(q_begin + q_len, 32);
+    if (!workspace || !aligned(workspace, 256)) return IDXC_ERR_WORKSPACE;
+    int64_t chunk = static_cast<int64_t>(workspace_bytes / static_cast<size_t>(ld * 4)) / kMinChunkRows * kMinChunkRows;
+    if (chunk < kMinChunkRows) return IDXC_ERR_WORKSPACE;
+    for (int64_t r0 = 0; r0 < q_len; r0 += chunk) {
+        const int64_t nr = q_len - r0 < chunk ? q_len - r0 : chunk;
+        st = run_rows(r0, nr, static_cast<float*>(workspace), ld);
+        if (st != IDXC_OK) return st;
+    }
+    return IDXC_OK;
+}
+
+size_t idxc_decode_workspace_bytes(int B, int64_t max_len, int H_I, int d_I, int k_top, idxc_dtype dt, uint32_t flags) {
+    (void)H_I; (void)d_I; (void)k_top; (void)dt; (void)flags;
+    if (B <= 0 || max_len <= 0) return 0;
+    return static_cast<size_t>(B) * static_cast<size_t>(round_up(max_len, 32)) * 4;
+}
+
+idxc_status idxc_indexer_decode(const void* q_step, const void* k_cache, int64_t cache_rows, const float* w,
+                                const float* q_scale, const float* k_scale, const int64_t* k_offsets,
+                                const int32_t* lens, int B, int64_t max_len, int H_I, int d_I, int k_top,
+                                idxc_dtype dt, float* scores_out, int64_t ld_scores, int32_t* topk_out,
+                                void* workspace, size_t workspace_bytes, uint32_t flags, void* cuda_stream) {
+    idxc_status st = check_common(H_I, d_I, k_top, dt, flags);
+    if (st != IDXC_OK) return st;
+    if (B < 0 || max_len < 0 || max_len > (int64_t(1) << 30) || cache_rows < 0 || cache_rows > (int64_t(1) << 31) - 256)
+        return IDXC_ERR_INVALID_ARG;
+    if (!scores_out && !topk_out) return IDXC_ERR_INVALID_ARG;
+    if (B == 0) return IDXC_OK;
+    if (!q_step || !k_cache || !w || !k_offsets || !lens) return IDXC_ERR_INVALID_ARG;
+    if (!aligned(q_step, 16) || !aligned(k_cache, 16) || !aligned(k_offsets, 8) || !aligned(lens, 4)) return IDXC_ERR_INVALID_ARG;
+    const bool fp8 = dt == IDXC_FP8_E4M3;
+    if (fp8 && (!q_scale || !k_scale)) return IDXC_ERR_INVALID_ARG;
+    if (scores_out && (ld_scores < max_len || (ld_scores & 3) || !aligned(scores_out, 16))) return IDXC_ERR_INVALID_ARG;
+    if (!device_info().ok) return IDXC_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    float* sc = scores_out;
+    int64_t ld = ld_scores;
+    if (!sc) {
+        ld = round_up(max_len, 32);
+        if (max_len > 0 && (!workspace || !aligned(workspace, 256) ||
+                            workspace_bytes < static_cast<size_t>(B) * static_cast<size_t>(ld) * 4))
+            return IDXC_ERR_WORKSPACE;
+        sc = static_cast<float*>(workspace);
+    }
+    ScoreArgs a{};
+    a.q = q_step; a.k = k_cache; a.w = w;
+    a.q_scale = fp8 ? q_scale : nullptr; a.k_scale = fp8 ? k_scale : nullptr;
+    a.k_offsets = k_offsets; a.lens = lens; a.q_begin = 0; a.n_rows = B; a.k_rows = cache_rows;
+    a.max_len = max_len; a.H = H_I; a.d = d_I; a.fp8 = fp8 ? 1 : 0; a.scores = sc; a.ld = ld;
+    if (max_len > 0) {
+        st = launch_scorer(a, true, flags, stream);
+        if (st != IDXC_OK) return st;
+    }
+    if (topk_out) {
+        g_launches += 1;
+        if (launch_topk_rows(sc, ld, B, 0, 0, lens, k_top, topk_out, stream) != cudaSuccess) return IDXC_ERR_CUDA;
+    }
+    return IDXC_OK;
+}
+
+idxc_status idxc_topk_rows(const float* scores, int64_t ld, int64_t n_rows, int64_t first_len, int64_t len_step,
+                           const int32_t* lens, int k_top, int32_t* topk_out, void* cuda_stream) {
+    if (k_top < 1 || k_top > IDXC_MAX_K_TOP || n_rows < 0 || ld < 0 || (ld & 3) || ld > (int64_t(1) << 30))
+        return IDXC_ERR_INVALID_ARG;
+    if (n_rows == 0) return IDXC_OK;
+    if (!scores || !topk_out || !aligned(scores, 16) || !aligned(topk_out, 4)) return IDXC_ERR_INVALID_ARG;
+    if (!lens && (first_len < 0 || len_step < 0)) return IDXC_ERR_INVALID_ARG;
+    g_launches += 1;
+    return launch_topk_rows(scores, ld, n_rows, first_len, len_step, lens, k_top, topk_out,
+                            static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? IDXC_OK : IDXC_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------ schedule (Figure 2(b))
+
+idxc_status idxc_schedule_create(const char* pattern, int N, idxc_schedule** out) {
+    if (!out) return IDXC_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!pattern || N < 1) return IDXC_ERR_PATTERN;
+    for (int l = 0; l < N; ++l)
+        if (pattern[l] != 'F' && pattern[l] != 'S') return IDXC_ERR_PATTERN;
+    if (pattern[0] != 'F') return IDXC_ERR_PATTERN;   // the first layer seeds the indices
+    idxc_schedule* s = new (std::nothrow) idxc_schedule();
+    if (!s) return IDXC_ERR_INVALID_ARG;
+    s->pattern.assign(pattern, pattern + N);
+    s->src.resize(N);
+    int last_full = 0;
+    for (int l = 0; l < N; ++l) {
+        if (pattern[l] == 'F') { last_full = l; ++s->n_full; } else { ++s->n_shared; }
+        s->src[l] = last_full;                          // f(l) = nearest preceding F layer (l itself on F layers)
+    }
+    *out = s;
+    return IDXC_OK;
+}
+
+void idxc_schedule_destroy(idxc_schedule* s) { delete s; }
+
+idxc_status idxc_schedule_begin_pass(idxc_schedule* s) {
+    if (!s) return IDXC_ERR_INVALID_ARG;
+    s->cache_layer = -1;
+    s->cache_ptr = nullptr;
+    s->cache_rows = 0;
+    s->cache_k_top = 0;
+    return IDXC_OK;
+}
+
+idxc_status idxc_schedule_source(const idxc_schedule* s, int layer, int* src_layer) {
+    if (!s || !src_layer || layer < 0 || layer >= static_cast<int>(s->src.size())) return IDXC_ERR_INVALID_ARG;
+    *src_layer = s->src[layer];
+    return IDXC_OK;
+}
+
+idxc_status idxc_schedule_stats(const idxc_schedule* s, int* n_full, int* n_shared, int64_t* indexer_calls) {
+    if (!s) return IDXC_ERR_INVALID_ARG;
+    if (n_full) *n_full = s->n_full;
+    if (n_shared) *n_shared = s->n_shared;
+    if (indexer_calls) *indexer_calls = s->indexer_calls;
+    return IDXC_OK;
+}
+
+}  // extern "C"
+
+namespace {
+
+// Shared tail of the two *_layer calls: S layers hand back the cached tensor.
+idxc_status shared_layer(idxc_schedule* s, int layer, int64_t rows, int k_top, int32_t* topk_buf, uint32_t flags,
+                         cudaStream_t stream, const int32_t** topk_result) {
+    if (s->cache_layer != s->src[layer] || !s->cache_ptr) return IDXC_ERR_PATTERN;
+    if (rows != s->cache_rows || k_top != s->cache_k_top) return IDXC_ERR_INVALID_ARG;
+    if (flags & IDXC_FLAG_COPY_SHARED) {
+        if (!topk_buf) return IDXC_ERR_INVALID_ARG;
+        if (topk_buf != s->cache_ptr &&
+            cudaMemcpyAsync(topk_buf, s->cache_ptr, static_cast<size_t>(rows) * k_top * sizeof(int32_t),
+                            cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+            return IDXC_ERR_CUDA;
+        *topk_result = topk_buf;
+    } else {
+        *topk_result = s->cache_ptr;
+    }
+    return IDXC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+idxc_status idxc_schedule_prefill_layer(idxc_schedule* s, int layer, const void* q, const void* k, const float* w,
+                                        const float* q_scale, const float* k_scale, int64_t q_begin, int64_t q_len,
+                                        int64_t L_k, int H_I, int d_I, int k_top, idxc_dtype dt, float* scores_out,
+                                        int64_t ld_scores, int32_t* topk_buf, void* workspace, size_t workspace_bytes,
+                                        uint32_t flags, void* cuda_stream, const int32_t** topk_result) {
+    if (!s || !topk_result || layer < 0 || layer >= static_cast<int>(s->src.size())) return IDXC_ERR_INVALID_ARG;
+    *topk_result = nullptr;
+    if (s->pattern[layer] == 'S')
+        return shared_layer(s, layer, q_len, k_top, topk_buf, flags, static_cast<cudaStream_t>(cuda_stream), topk_result);
+    if (!topk_buf) return IDXC_ERR_INVALID_ARG;
+    idxc_status st = idxc_indexer_prefill(q, k, w, q_scale, k_scale, q_begin, q_len, L_k, H_I, d_I, k_top, dt,
+                                          scores_out, ld_scores, topk_buf, workspace, workspace_bytes,
+                                          flags & ~IDXC_FLAG_COPY_SHARED, cuda_stream);
+    if (st != IDXC_OK) return st;
+    s->indexer_calls += 1;
+    s->cache_layer = layer;
+    s->cache_ptr = topk_buf;
+    s->cache_rows = q_len;
+    s->cache_k_top = k_top;
+    *topk_result = topk_buf;
+    return IDXC_OK;
+}
+
+idxc_status idxc_schedule_decode_layer(idxc_schedule* s, int layer, const void* q_step, const void* k_cache,
+                                       int64_t cache_rows, const float* w, const float* q_scale, const float* k_scale,
+                                       const int64_t* k_offsets, const int32_t* lens, int B, int64_t max_len, int H_I,
+                                       int d_I, int k_top, idxc_dtype dt, float* scores_out, int64_t ld_scores,
+                                       int32_t* topk_buf, void* workspace, size_t workspace_bytes, uint32_t flags,
+                                       void* cuda_stream, const int32_t** topk_result) {
+    if (!s || !topk_result || layer < 0 || layer >= static_cast<int>(s->src.size())) return IDXC_ERR_INVALID_ARG;
+    *topk_result = nullptr;
+    if (s->pattern[layer] == 'S')
+        return shared_layer(s, layer, B, k_top, topk_buf, flags, static_cast<cudaStream_t>(cuda_stream), topk_result);
+    if (!topk_buf) return IDXC_ERR_INVALID_ARG;
+    idxc_status st = idxc_indexer_decode(q_step, k_cache, cache_rows, w, q_scale, k_scale, k_offsets, lens, B, max_len,
+                                         H_I, d_I, k_top, dt, scores_out, ld_scores, topk_buf, workspace,
+                                         workspace_bytes, flags & ~IDXC_FLAG_COPY_SHARED, cuda_stream);
+    if (st != IDXC_OK) return st;
+    s->indexer_calls += 1;
+    s->cache_layer = layer;
+    s->cache_ptr = topk_buf;
+    s->cache_rows = B;
+    s->cache_k_top = k_top;
+    *topk_result = topk_buf;
+    return IDXC_OK;
+}
+
+idxc_status idxc_poll_device_status(void* cuda_stream) {
+    if (!device_info().ok) return IDXC_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return IDXC_ERR_CUDA;
+    unsigned int v = 0;
+    if (cudaMemcpyFromSymbol(&v, g_device_status, sizeof(v)) != cudaSuccess) return IDXC_ERR_CUDA;
+    if (v != 0) {
+        const unsigned int zero = 0;
+        if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(zero)) != cudaSuccess) return IDXC_ERR_CUDA;
+        return IDXC_ERR_DEVICE_TIMEOUT;
+    }
+    return IDXC_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,48 @@
+// Internal launch interface between the C-ABI layer (api.cu) and the kernel files.
+// Every launcher enqueues on `stream` and returns the CUDA error of the launch.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace idxc {
+
+// Row-wise top-k select (topk.cu). Row r has length lens[r] (device) if lens != nullptr,
+// else first_len + r * len_step, clamped to [0, ld].
+cudaError_t launch_topk_rows(const float* scores, int64_t ld, int64_t n_rows, int64_t first_len,
+                             int64_t len_step, const int32_t* lens, int k_top, int32_t* out,
+                             cudaStream_t stream);
+
+// Arguments shared by the scorers. A "row" is one query vector set [H, d].
+struct ScoreArgs {
+    const void* q;          // [n_rows, H, d]
+    const void* k;          // [k_rows, d]
+    const float* w;         // [n_rows, H]
+    const float* q_scale;   // [n_rows] or nullptr
+    const float* k_scale;   // [k_rows] or nullptr
+    const int64_t* k_offsets;  // decode: [n_rows] first key row of each sequence; prefill: nullptr
+    const int32_t* lens;       // decode: [n_rows] keys per sequence; prefill: nullptr
+    int64_t q_begin;        // prefill: position of row 0 (row r sees keys 0 .. q_begin + r)
+    int64_t n_rows;
+    int64_t k_rows;         // rows of k that may be addressed
+    int64_t max_len;        // decode: host bound on lens
+    int H, d;
+    int fp8;                // 0: bf16, 1: e4m3 codes with scales
+    float* scores;          // [n_rows, ld]
+    int64_t ld;
+};
+
+// Plain CUDA-core scorer (scorer_simt.cu): debugging aid and cross-check.
+cudaError_t launch_score_simt(const ScoreArgs& a, cudaStream_t stream);
+
+// tcgen05 scorers (scorer_tc.cu). `status` is the device status word. The tensor maps are
+// encoded by the caller: q as [n_rows*H, d] and k as [k_rows, d], 128-byte swizzle, inner
+// box 128 bytes, box rows 256 (q) and 128 (k) for prefill; box rows H (q) for decode.
+cudaError_t launch_score_prefill_tc(const ScoreArgs& a, const CUtensorMap& q_map, const CUtensorMap& k_map,
+                                    unsigned int* status, int sm_count, cudaStream_t stream);
+cudaError_t launch_score_decode_tc(const ScoreArgs& a, const CUtensorMap& q_map, const CUtensorMap& k_map,
+                                   unsigned int* status, int sm_count, cudaStream_t stream);
+bool score_tc_supported(int H, int d, int fp8);
+
+}  // namespace idxc

@@ -1,0 +1,665 @@
+// tcgen05 / TMEM indexer scorers for sm_100a.
+//
+// Score (Sec. 2.1): I[t,s] = sum_h w[t,h] * max(q[t,h,:] . k[s,:], 0), s <= t.
+// The dot products are one dense contraction [keys, d] x [d, (query, head)]. It is laid
+// out with KEYS ON THE MMA's M axis (TMEM lanes) and (query, head) ON N (TMEM columns):
+// an epilogue thread then owns one key and walks the heads of a query along its own
+// TMEM lane, so the gate, the w-weighted head sum and the final score are plain register
+// arithmetic with w broadcast from shared memory -- no cross-thread reduction.
+//
+// Prefill kernel (persistent, one CTA per SM, warp-specialised):
+//   warp 0      TMA producer: a block of 2*256/H queries (two 256-column B tiles) is loaded
+//               once per work item and stays in shared memory; 128-key A tiles stream
+//               through a ring of stages. Per-CTA loads only (no multicast).
+//   warp 1      MMA issuer: per key tile, one 128 x 256 x d UMMA chain into each of the two
+//               256-column TMEM accumulators, so accumulator A is drained while B is filled.
+//   warps 4-11  epilogue: tcgen05.ld, ReLU, w-FMA, causal predicate, coalesced score store.
+// Causal structure: a work item only visits key tiles up to its last query's position;
+// items are handed out longest first in a boustrophedon order over the CTAs.
+//
+// Decode kernel: work item = (sequence, run of key tiles); the sequence's H x d query tile
+// is the B operand (N = H), key tiles stream from HBM through a deep TMA ring.
+#include "kernels.h"
+#include "ptx_sm100.cuh"
+
+namespace idxc {
+namespace {
+
+constexpr int kTileKeys = 128;          // UMMA M
+constexpr int kTileCols = 256;          // UMMA N (prefill)
+constexpr int kChunkBytes = 128;        // one swizzle row: 64 bf16 or 128 fp8 elements
+constexpr int kQRegionBytes = kTileCols * kChunkBytes;   // 32 KB
+constexpr int kKRegionBytes = kTileKeys * kChunkBytes;   // 16 KB
+constexpr int kPrefillThreads = 384;    // 12 warps
+constexpr int kEpilogueWarp0 = 4;
+constexpr int kNumEpilogueWarps = 8;
+
+template <int NKH>
+struct PrefillCfg {
+    static constexpr int kStages = NKH == 2 ? 2 : 4;
+    static constexpr int kQBytes = 2 * NKH * kQRegionBytes;
+    static constexpr int kKBytes = kStages * NKH * kKRegionBytes;
+    static constexpr int kWBytes = kNumEpilogueWarps * 256 * 4;
+    static constexpr int kBarBytes = 256;
+    static constexpr int kSmemBytes = kQBytes + kKBytes + kWBytes + kBarBytes + 1024;   // + alignment slack
+};
+
+struct PrefillParams {
+    const float* w;
+    const float* q_scale;
+    const float* k_scale;
+    float* scores;
+    int64_t ld;
+    int64_t q_begin;
+    int64_t n_rows;
+    int64_t k_rows;
+    unsigned int* status;
+};
+
+__device__ __forceinline__ void give_up(volatile uint32_t* abort_flag, unsigned int* status, unsigned int code) {
+    *abort_flag = 1u;
+    atomicCAS(status, 0u, code);
+}
+
+// NKH: 128-byte chunks per operand row (d * element size / 128). H: indexer heads.
+template <int NKH, int H, bool FP8>
+__global__ void __launch_bounds__(kPrefillThreads, 1)
+score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
+                        const PrefillParams p) {
+    using Cfg = PrefillCfg<NKH>;
+    constexpr int kStages = Cfg::kStages;
+    constexpr int QPA = kTileCols / H;       // queries per accumulator
+    constexpr int QB = 2 * QPA;              // queries per work item
+    constexpr int kElemsPerChunk = FP8 ? 128 : 64;
+    constexpr uint32_t kIdesc = FP8 ? umma_idesc(0, 0, kTileKeys, kTileCols) : umma_idesc(1, 1, kTileKeys, kTileCols);
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    uint8_t* q_smem = smem;                                   // [2][NKH][256 x 128 B]
+    uint8_t* k_smem = q_smem + Cfg::kQBytes;                  // [kStages][NKH][128 x 128 B]
+    float* w_smem = reinterpret_cast<float*>(k_smem + Cfg::kKBytes);   // [8 warps][256]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(w_smem) + Cfg::kWBytes);
+    // barrier map
+    const uint32_t bar_q_full = smem_u32(bars + 0);           // [2]
+    const uint32_t bar_q_empty = smem_u32(bars + 2);          // [2]
+    const uint32_t bar_acc_full = smem_u32(bars + 4);         // [2]
+    const uint32_t bar_acc_empty = smem_u32(bars + 6);        // [2]
+    const uint32_t bar_k_full = smem_u32(bars + 8);           // [kStages]
+    const uint32_t bar_k_empty = smem_u32(bars + 8 + kStages);
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(bars + 8 + 2 * kStages);
+    volatile uint32_t* abort_flag = tmem_base_slot + 1;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar_q_full + 8 * i, 1);
+            mbar_init(bar_q_empty + 8 * i, 1);
+            mbar_init(bar_acc_full + 8 * i, 1);
+            mbar_init(bar_acc_empty + 8 * i, kNumEpilogueWarps);
+        }
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(bar_k_full + 8 * i, 1);
+            mbar_init(bar_k_empty + 8 * i, 1);
+        }
+        *abort_flag = 0u;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_base_slot), 512);
+        tmem_relinquish_alloc_permit();
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    tcgen05_fence_after_sync();
+    const uint32_t tmem_base = *tmem_base_slot;
+
+    const int64_t n_items = (p.n_rows + QB - 1) / QB;
+    const int G = gridDim.x;
+    const int cta = blockIdx.x;
+    // work item of this CTA in round `rho` (longest first, boustrophedon), or -1
+    auto item_of_round = [&](int64_t rho) -> int64_t {
+        const int64_t seq = rho * G + ((rho & 1) ? (G - 1 - cta) : cta);
+        return seq < n_items ? n_items - 1 - seq : -1;
+    };
+    auto key_tiles_of_item = [&](int64_t item) -> int {
+        int64_t last = item * QB + QB;
+        if (last > p.n_rows) last = p.n_rows;
+        return static_cast<int>((p.q_begin + last + kTileKeys - 1) / kTileKeys);   // positions 0 .. q_begin+last-1
+    };
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ------------------------------------------------------------ TMA producer
+            tma_prefetch_desc(&q_map);
+            tma_prefetch_desc(&k_map);
+            int stage = 0;
+            uint32_t k_phase = 0, q_phase = 0;
+            bool ok = true;
+            for (int64_t rho = 0; ok; ++rho) {
+                const int64_t item = item_of_round(rho);
+                if (item < 0) break;
+                const int nkt = key_tiles_of_item(item);
+                for (int half = 0; half < 2 && ok; ++half) {
+                    ok = mbar_wait(bar_q_empty + 8 * half, q_phase ^ 1u, abort_flag);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(bar_q_full + 8 * half, NKH * kQRegionBytes);
+                    const int row0 = static_cast<int>((item * QB + half * QPA) * H);
+                    for (int kh = 0; kh < NKH; ++kh)
+                        tma_load_2d(smem_u32(q_smem + (half * NKH + kh) * kQRegionBytes), &q_map, bar_q_full + 8 * half,
+                                    kh * kElemsPerChunk, row0);
+                }
+                for (int kt = 0; kt < nkt && ok; ++kt) {
+                    ok = mbar_wait(bar_k_empty + 8 * stage, k_phase ^ 1u, abort_flag);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(bar_k_full + 8 * stage, NKH * kKRegionBytes);
+                    for (int kh = 0; kh < NKH; ++kh)
+                        tma_load_2d(smem_u32(k_smem + (stage * NKH + kh) * kKRegionBytes), &k_map, bar_k_full + 8 * stage,
+                                    kh * kElemsPerChunk, kt * kTileKeys);
+                    if (++stage == kStages) { stage = 0; k_phase ^= 1u; }
+                }
+                q_phase ^= 1u;
+            }
+            if (!ok) give_up(abort_flag, p.status, DEV_TIMEOUT_PRODUCER);
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ------------------------------------------------------------ MMA issuer
+            int stage = 0;
+            uint32_t k_phase = 0, q_phase = 0;
+            uint32_t acc_phase[2] = {0u, 0u};
+            bool ok = true;
+            for (int64_t rho = 0; ok; ++rho) {
+                const int64_t item = item_of_round(rho);
+                if (item < 0) break;
+                const int nkt = key_tiles_of_item(item);
+                for (int kt = 0; kt < nkt && ok; ++kt) {
+                    ok = mbar_wait(bar_k_full + 8 * stage, k_phase, abort_flag);
+                    if (!ok) break;
+                    for (int half = 0; half < 2; ++half) {
+                        if (kt == 0) {
+                            ok = mbar_wait(bar_q_full + 8 * half, q_phase, abort_flag);
+                            if (!ok) break;
+                        }
+                        ok = mbar_wait(bar_acc_empty + 8 * half, acc_phase[half] ^ 1u, abort_flag);
+                        if (!ok) break;
+                        acc_phase[half] ^= 1u;
+                        tcgen05_fence_after_sync();
+                        const uint32_t d_tmem = tmem_base + half * kTileCols;
+#pragma unroll
+                        for (int kh = 0; kh < NKH; ++kh) {
+                            const uint32_t a_base = smem_u32(k_smem + (stage * NKH + kh) * kKRegionBytes);
+                            const uint32_t b_base = smem_u32(q_smem + (half * NKH + kh) * kQRegionBytes);
+#pragma unroll
+                            for (int ks = 0; ks < 4; ++ks) {   // 32 bytes of K per MMA: 16 bf16 or 32 fp8
+                                const uint64_t a_desc = umma_smem_desc_sw128(a_base + ks * 32);
+                                const uint64_t b_desc = umma_smem_desc_sw128(b_base + ks * 32);
+                                if constexpr (FP8) umma_f8(d_tmem, a_desc, b_desc, kIdesc, (kh | ks) != 0);
+                                else umma_f16(d_tmem, a_desc, b_desc, kIdesc, (kh | ks) != 0);
+                            }
+                        }
+                        umma_commit(bar_acc_full + 8 * half);
+                        if (kt == nkt - 1) umma_commit(bar_q_empty + 8 * half);
+                    }
+                    if (!ok) break;
+                    umma_commit(bar_k_empty + 8 * stage);
+                    if (++stage == kStages) { stage = 0; k_phase ^= 1u; }
+                }
+                q_phase ^= 1u;
+            }
+            if (!ok) give_up(abort_flag, p.status, DEV_TIMEOUT_MMA);
+        }
+    } else if (warp >= kEpilogueWarp0) {
+        // ---------------------------------------------------------------- epilogue
+        constexpr int QPW = 128 / H;                 // queries per warp per accumulator
+        const int ew = warp - kEpilogueWarp0;
+        const int quarter = warp & 3;                // TMEM lane quarter this warp may read
+        const int colhalf = ew >> 2;                 // which 128 columns of the accumulator
+        const int key_in_tile = quarter * 32 + lane;
+        float* my_w = w_smem + ew * 256;             // [half][128]: w (times q_scale) of this warp's queries
+        uint32_t acc_phase[2] = {0u, 0u};
+        bool ok = true;
+        for (int64_t rho = 0; ok; ++rho) {
+            const int64_t item = item_of_round(rho);
+            if (item < 0) break;
+            const int nkt = key_tiles_of_item(item);
+            const int64_t row_base = item * QB;
+            __syncwarp();
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                // 128 consecutive floats of w: rows row_base + half*QPA + colhalf*QPW .. +QPW-1
+                const int64_t row = row_base + half * QPA + colhalf * QPW + (lane * 4) / H;
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (row < p.n_rows) {
+                    v = __ldg(reinterpret_cast<const float4*>(p.w + row * H + (lane * 4) % H));
+                    if constexpr (FP8) {
+                        const float qs = __ldg(p.q_scale + row);
+                        v.x *= qs; v.y *= qs; v.z *= qs; v.w *= qs;
+                    }
+                }
+                reinterpret_cast<float4*>(my_w + half * 128)[lane] = v;
+            }
+            __syncwarp();
+            for (int kt = 0; kt < nkt && ok; ++kt) {
+                const int64_t s = static_cast<int64_t>(kt) * kTileKeys + key_in_tile;
+                float ksc = 1.f;
+                if constexpr (FP8) ksc = s < p.k_rows ? __ldg(p.k_scale + s) : 0.f;
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_acc_full + 8 * half, acc_phase[half], abort_flag));   // warp-uniform
+                    if (!ok) break;
+                    acc_phase[half] ^= 1u;
+                    tcgen05_fence_after_sync();
+                    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
+                                           static_cast<uint32_t>(half * kTileCols + colhalf * 128);
+                    const float4* w4 = reinterpret_cast<const float4*>(my_w + half * 128);
+                    float acc[QPW];
+#pragma unroll
+                    for (int i = 0; i < QPW; ++i) acc[i] = 0.f;
+                    uint32_t ra[32], rb[32];
+                    tmem_ld_32x32b_x32(taddr, ra);
+                    tmem_ld_wait(ra);
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {          // 4 chunks of 32 columns
+                        uint32_t (&cur)[32] = (c & 1) ? rb : ra;
+                        uint32_t (&nxt)[32] = (c & 1) ? ra : rb;
+                        if (c + 1 < 4) tmem_ld_32x32b_x32(taddr + (c + 1) * 32, nxt);
+#pragma unroll
+                        for (int j4 = 0; j4 < 8; ++j4) {
+                            const float4 wv = w4[c * 8 + j4];
+                            const int col = c * 32 + j4 * 4;        // column within this warp's 128
+                            float& a = acc[col / H];                // 4 consecutive columns share a query (H % 4 == 0)
+                            a = fmaf(fmaxf(__uint_as_float(cur[j4 * 4 + 0]), 0.f), wv.x, a);
+                            a = fmaf(fmaxf(__uint_as_float(cur[j4 * 4 + 1]), 0.f), wv.y, a);
+                            a = fmaf(fmaxf(__uint_as_float(cur[j4 * 4 + 2]), 0.f), wv.z, a);
+                            a = fmaf(fmaxf(__uint_as_float(cur[j4 * 4 + 3]), 0.f), wv.w, a);
+                        }
+                        if (c + 1 < 4) tmem_ld_wait(nxt);
+                    }
+                    // this warp's TMEM reads of the accumulator are complete
+                    tcgen05_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_acc_empty + 8 * half);
+#pragma unroll
+                    for (int i = 0; i < QPW; ++i) {
+                        const int64_t row = row_base + half * QPA + colhalf * QPW + i;
+                        const int64_t t = p.q_begin + row;
+                        if (row < p.n_rows && s <= t) {
+                            float val = acc[i];
+                            if constexpr (FP8) val *= ksc;
+                            p.scores[row * p.ld + s] = val;
+                        }
+                    }
+                }
+            }
+        }
+        if (!ok && lane == 0) give_up(abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
+    }
+
+    // ------------------------------------------------------------------- teardown
+    __syncwarp();
+    if (*abort_flag) {
+        // a role gave up: give copies that may still be in flight time to land before
+        // shared memory and TMEM are released (bounded: about a millisecond)
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) __nanosleep(1000);
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tcgen05_fence_after_sync();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+template <int NKH, int H, bool FP8>
+cudaError_t launch_prefill_instance(const ScoreArgs& a, const CUtensorMap& q_map, const CUtensorMap& k_map,
+                                    unsigned int* status, int sm_count, cudaStream_t stream) {
+    using Cfg = PrefillCfg<NKH>;
+    auto kern = score_prefill_tc_kernel<NKH, H, FP8>;
+    static bool attr_done = false;   // per instantiation; the attribute is per function, setting it twice is harmless
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    constexpr int QB = 2 * (kTileCols / H);
+    const int64_t n_items = (a.n_rows + QB - 1) / QB;
+    const int grid = static_cast<int>(n_items < sm_count ? n_items : sm_count);
+    PrefillParams p{a.w, a.q_scale, a.k_scale, a.scores, a.ld, a.q_begin, a.n_rows, a.k_rows, status};
+    kern<<<grid, kPrefillThreads, Cfg::kSmemBytes, stream>>>(q_map, k_map, p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+bool score_tc_supported(int H, int d, int fp8) {
+    if (H != 16 && H != 32 && H != 64) return false;
+    if (fp8) return d == 128;
+    return d == 64 || d == 128;
+}
+
+cudaError_t launch_score_prefill_tc(const ScoreArgs& a, const CUtensorMap& q_map, const CUtensorMap& k_map,
+                                    unsigned int* status, int sm_count, cudaStream_t stream) {
+    if (a.n_rows <= 0) return cudaSuccess;
+#define IDXC_DISPATCH_H(NKH, FP8)                                                                              \
+    switch (a.H) {                                                                                             \
+        case 16: return launch_prefill_instance<NKH, 16, FP8>(a, q_map, k_map, status, sm_count, stream);      \
+        case 32: return launch_prefill_instance<NKH, 32, FP8>(a, q_map, k_map, status, sm_count, stream);      \
+        case 64: return launch_prefill_instance<NKH, 64, FP8>(a, q_map, k_map, status, sm_count, stream);      \
+        default: return cudaErrorInvalidValue;                                                                 \
+    }
+    if (a.fp8) {
+        if (a.d == 128) { IDXC_DISPATCH_H(1, true) }
+        return cudaErrorInvalidValue;
+    }
+    if (a.d == 64) { IDXC_DISPATCH_H(1, false) }
+    if (a.d == 128) { IDXC_DISPATCH_H(2, false) }
+#undef IDXC_DISPATCH_H
+    return cudaErrorInvalidValue;
+}
+
+// ===================================================================== decode
+namespace {
+
+constexpr int kDecodeThreads = 192;      // warp 0 producer, warp 1 MMA, warps 2-5 epilogue
+constexpr int kDecodeChunkTiles = 8;     // key tiles (of 128 keys) per work item
+constexpr int kDecodeAccSlots = 4;       // TMEM accumulators in flight (64 columns apart)
+
+template <int NKH, int H>
+struct DecodeCfg {
+    static constexpr int kStages = NKH == 2 ? 5 : 8;
+    static constexpr int kQRegion = H * kChunkBytes;                  // one 128-byte chunk of the query tile
+    static constexpr int kQBytes = 2 * NKH * kQRegion;                // double buffered
+    static constexpr int kKBytes = kStages * NKH * kKRegionBytes;
+    static constexpr int kWBytes = 4 * 64 * 4;
+    static constexpr int kBarBytes = 512;
+    static constexpr int kSmemBytes = kQBytes + kKBytes + kWBytes + kBarBytes + 1024;
+};
+
+struct DecodeParams {
+    const float* w;
+    const float* q_scale;
+    const float* k_scale;
+    const int64_t* k_offsets;
+    const int32_t* lens;
+    float* scores;
+    int64_t ld;
+    int64_t max_len;
+    int B;
+    unsigned int* status;
+};
+
+// Walks the (sequence, chunk) work items of one CTA: items are numbered sequence-major,
+// sequence b having ceil(len_b / (128 * kDecodeChunkTiles)) of them; CTA c takes items
+// c, c + G, c + 2G, ...
+struct DecodeItemWalker {
+    const int32_t* lens;
+    int64_t max_len;
+    int B, G;
+    int64_t next;        // next item number of this CTA
+    int b;               // sequence the cursor is in
+    int64_t base;        // first item number of sequence b
+    __device__ DecodeItemWalker(const DecodeParams& p, int cta, int grid)
+        : lens(p.lens), max_len(p.max_len), B(p.B), G(grid), next(cta), b(0), base(0) {}
+    __device__ int len_of(int bb) const {
+        int64_t l = lens[bb];
+        l = l < 0 ? 0 : (l > max_len ? max_len : l);
+        return static_cast<int>(l);
+    }
+    // Fetches the next item: sequence, first key tile, number of key tiles, sequence length.
+    __device__ bool pop(int& seq, int& tile0, int& ntiles, int& len) {
+        while (b < B) {
+            const int l = len_of(b);
+            const int tiles = (l + kTileKeys - 1) / kTileKeys;
+            const int chunks = (tiles + kDecodeChunkTiles - 1) / kDecodeChunkTiles;
+            if (next < base + chunks) {
+                const int c = static_cast<int>(next - base);
+                seq = b;
+                tile0 = c * kDecodeChunkTiles;
+                ntiles = tiles - tile0 < kDecodeChunkTiles ? tiles - tile0 : kDecodeChunkTiles;
+                len = l;
+                next += G;
+                return true;
+            }
+            base += chunks;
+            ++b;
+        }
+        return false;
+    }
+};
+
+template <int NKH, int H, bool FP8>
+__global__ void __launch_bounds__(kDecodeThreads, 1)
+score_decode_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
+                       const DecodeParams p) {
+    using Cfg = DecodeCfg<NKH, H>;
+    constexpr int kStages = Cfg::kStages;
+    constexpr int kElemsPerChunk = FP8 ? 128 : 64;
+    constexpr uint32_t kIdesc = FP8 ? umma_idesc(0, 0, kTileKeys, H) : umma_idesc(1, 1, kTileKeys, H);
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    uint8_t* k_smem = smem;                                  // [kStages][NKH][128 x 128 B]
+    uint8_t* q_smem = k_smem + Cfg::kKBytes;                 // [2][NKH][H x 128 B]
+    float* w_smem = reinterpret_cast<float*>(q_smem + Cfg::kQBytes);   // [4 warps][64]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(w_smem) + Cfg::kWBytes);
+    const uint32_t bar_q_full = smem_u32(bars + 0);          // [2]
+    const uint32_t bar_q_empty = smem_u32(bars + 2);         // [2]
+    const uint32_t bar_acc_full = smem_u32(bars + 4);        // [4]
+    const uint32_t bar_acc_empty = smem_u32(bars + 8);       // [4]
+    const uint32_t bar_k_full = smem_u32(bars + 12);         // [kStages]
+    const uint32_t bar_k_empty = smem_u32(bars + 12 + kStages);
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(bars + 12 + 2 * kStages);
+    volatile uint32_t* abort_flag = tmem_base_slot + 1;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar_q_full + 8 * i, 1);
+            mbar_init(bar_q_empty + 8 * i, 1);
+        }
+        for (int i = 0; i < kDecodeAccSlots; ++i) {
+            mbar_init(bar_acc_full + 8 * i, 1);
+            mbar_init(bar_acc_empty + 8 * i, 4);
+        }
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(bar_k_full + 8 * i, 1);
+            mbar_init(bar_k_empty + 8 * i, 1);
+        }
+        *abort_flag = 0u;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_base_slot), 256);
+        tmem_relinquish_alloc_permit();
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    tcgen05_fence_after_sync();
+    const uint32_t tmem_base = *tmem_base_slot;
+
+    DecodeItemWalker walk(p, blockIdx.x, gridDim.x);
+    int seq, tile0, ntiles, len;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            tma_prefetch_desc(&q_map);
+            tma_prefetch_desc(&k_map);
+            int stage = 0, qbuf = 0;
+            uint32_t k_phase = 0, q_phase[2] = {0u, 0u};
+            bool ok = true;
+            while (ok && walk.pop(seq, tile0, ntiles, len)) {
+                ok = mbar_wait(bar_q_empty + 8 * qbuf, q_phase[qbuf] ^ 1u, abort_flag);
+                if (!ok) break;
+                q_phase[qbuf] ^= 1u;
+                mbar_arrive_expect_tx(bar_q_full + 8 * qbuf, NKH * Cfg::kQRegion);
+                for (int kh = 0; kh < NKH; ++kh)
+                    tma_load_2d(smem_u32(q_smem + (qbuf * NKH + kh) * Cfg::kQRegion), &q_map, bar_q_full + 8 * qbuf,
+                                kh * kElemsPerChunk, seq * H);
+                const int64_t row0 = p.k_offsets[seq] + static_cast<int64_t>(tile0) * kTileKeys;
+                for (int kt = 0; kt < ntiles && ok; ++kt) {
+                    ok = mbar_wait(bar_k_empty + 8 * stage, k_phase ^ 1u, abort_flag);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(bar_k_full + 8 * stage, NKH * kKRegionBytes);
+                    for (int kh = 0; kh < NKH; ++kh)
+                        tma_load_2d(smem_u32(k_smem + (stage * NKH + kh) * kKRegionBytes), &k_map, bar_k_full + 8 * stage,
+                                    kh * kElemsPerChunk, static_cast<int>(row0 + kt * kTileKeys));
+                    if (++stage == kStages) { stage = 0; k_phase ^= 1u; }
+                }
+                qbuf ^= 1;
+            }
+            if (!ok) give_up(abort_flag, p.status, DEV_TIMEOUT_PRODUCER);
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            int stage = 0, qbuf = 0, slot = 0;
+            uint32_t k_phase = 0, q_phase[2] = {0u, 0u}, acc_phase[kDecodeAccSlots] = {0u, 0u, 0u, 0u};
+            bool ok = true;
+            while (ok && walk.pop(seq, tile0, ntiles, len)) {
+                ok = mbar_wait(bar_q_full + 8 * qbuf, q_phase[qbuf], abort_flag);
+                if (!ok) break;
+                q_phase[qbuf] ^= 1u;
+                for (int kt = 0; kt < ntiles && ok; ++kt) {
+                    ok = mbar_wait(bar_k_full + 8 * stage, k_phase, abort_flag);
+                    if (!ok) break;
+                    ok = mbar_wait(bar_acc_empty + 8 * slot, acc_phase[slot] ^ 1u, abort_flag);
+                    if (!ok) break;
+                    acc_phase[slot] ^= 1u;
+                    tcgen05_fence_after_sync();
+                    const uint32_t d_tmem = tmem_base + slot * 64;
+#pragma unroll
+                    for (int kh = 0; kh < NKH; ++kh) {
+                        const uint32_t a_base = smem_u32(k_smem + (stage * NKH + kh) * kKRegionBytes);
+                        const uint32_t b_base = smem_u32(q_smem + (qbuf * NKH + kh) * Cfg::kQRegion);
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) {
+                            const uint64_t a_desc = umma_smem_desc_sw128(a_base + ks * 32);
+                            const uint64_t b_desc = umma_smem_desc_sw128(b_base + ks * 32);
+                            if constexpr (FP8) umma_f8(d_tmem, a_desc, b_desc, kIdesc, (kh | ks) != 0);
+                            else umma_f16(d_tmem, a_desc, b_desc, kIdesc, (kh | ks) != 0);
+                        }
+                    }
+                    umma_commit(bar_acc_full + 8 * slot);
+                    umma_commit(bar_k_empty + 8 * stage);
+                    if (kt == ntiles - 1) umma_commit(bar_q_empty + 8 * qbuf);
+                    if (++stage == kStages) { stage = 0; k_phase ^= 1u; }
+                    slot = (slot + 1) & (kDecodeAccSlots - 1);
+                }
+                qbuf ^= 1;
+            }
+            if (!ok) give_up(abort_flag, p.status, DEV_TIMEOUT_MMA);
+        }
+    } else {
+        const int quarter = warp & 3;
+        const int key_in_tile = quarter * 32 + lane;
+        float* my_w = w_smem + (warp - 2) * 64;
+        int slot = 0;
+        uint32_t acc_phase[kDecodeAccSlots] = {0u, 0u, 0u, 0u};
+        bool ok = true;
+        while (ok && walk.pop(seq, tile0, ntiles, len)) {
+            __syncwarp();
+            for (int h = lane; h < H; h += 32) {
+                float v = __ldg(p.w + static_cast<int64_t>(seq) * H + h);
+                if constexpr (FP8) v *= __ldg(p.q_scale + seq);
+                my_w[h] = v;
+            }
+            __syncwarp();
+            const int64_t krow0 = p.k_offsets[seq];
+            for (int kt = 0; kt < ntiles && ok; ++kt) {
+                const int s = (tile0 + kt) * kTileKeys + key_in_tile;
+                float ksc = 1.f;
+                if constexpr (FP8) ksc = s < len ? __ldg(p.k_scale + krow0 + s) : 0.f;
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_acc_full + 8 * slot, acc_phase[slot], abort_flag));   // warp-uniform
+                if (!ok) break;
+                acc_phase[slot] ^= 1u;
+                tcgen05_fence_after_sync();
+                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(slot * 64);
+                float acc = 0.f;
+                if constexpr (H == 16) {
+                    uint32_t r[16];
+                    tmem_ld_32x32b_x16(taddr, r);
+                    tmem_ld_wait(r);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) acc = fmaf(fmaxf(__uint_as_float(r[j]), 0.f), my_w[j], acc);
+                } else {
+#pragma unroll
+                    for (int c = 0; c < H / 32; ++c) {
+                        uint32_t r[32];
+                        tmem_ld_32x32b_x32(taddr + c * 32, r);
+                        tmem_ld_wait(r);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) acc = fmaf(fmaxf(__uint_as_float(r[j]), 0.f), my_w[c * 32 + j], acc);
+                    }
+                }
+                tcgen05_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_acc_empty + 8 * slot);
+                if (s < len) {
+                    if constexpr (FP8) acc *= ksc;
+                    p.scores[static_cast<int64_t>(seq) * p.ld + s] = acc;
+                }
+                slot = (slot + 1) & (kDecodeAccSlots - 1);
+            }
+        }
+        if (!ok && lane == 0) give_up(abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
+    }
+
+    __syncwarp();
+    if (*abort_flag) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) __nanosleep(1000);
+    }
+    tcgen05_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tcgen05_fence_after_sync();
+        tmem_dealloc(tmem_base, 256);
+    }
+}
+
+template <int NKH, int H, bool FP8>
+cudaError_t launch_decode_instance(const ScoreArgs& a, const CUtensorMap& q_map, const CUtensorMap& k_map,
+                                   unsigned int* status, int sm_count, cudaStream_t stream) {
+    using Cfg = DecodeCfg<NKH, H>;
+    auto kern = score_decode_tc_kernel<NKH, H, FP8>;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    const int64_t tiles = (a.max_len + kTileKeys - 1) / kTileKeys;
+    const int64_t items = a.n_rows * ((tiles + kDecodeChunkTiles - 1) / kDecodeChunkTiles);
+    if (items <= 0) return cudaSuccess;
+    const int grid = static_cast<int>(items < sm_count ? items : sm_count);
+    DecodeParams p{a.w, a.q_scale, a.k_scale, a.k_offsets, a.lens, a.scores, a.ld, a.max_len, static_cast<int>(a.n_rows), status};
+    kern<<<grid, kDecodeThreads, Cfg::kSmemBytes, stream>>>(q_map, k_map, p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_score_decode_tc(const ScoreArgs& a, const CUtensorMap& q_map, const CUtensorMap& k_map,
+                                   unsigned int* status, int sm_count, cudaStream_t stream) {
+    if (a.n_rows <= 0 || a.max_len <= 0) return cudaSuccess;
+#define IDXC_DISPATCH_H(NKH, FP8)                                                                             \
+    switch (a.H) {                                                                                            \
+        case 16: return launch_decode_instance<NKH, 16, FP8>(a, q_map, k_map, status, sm_count, stream);      \
+        case 32: return launch_decode_instance<NKH, 32, FP8>(a, q_map, k_map, status, sm_count, stream);      \
+        case 64: return launch_decode_instance<NKH, 64, FP8>(a, q_map, k_map, status, sm_count, stream);      \
+        default: return cudaErrorInvalidValue;                                                                \
+    }
+    if (a.fp8) {
+        if (a.d == 128) { IDXC_DISPATCH_H(1, true) }
+        return cudaErrorInvalidValue;
+    }
+    if (a.d == 64) { IDXC_DISPATCH_H(1, false) }
+    if (a.d == 128) { IDXC_DISPATCH_H(2, false) }
+#undef IDXC_DISPATCH_H
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace idxc

@@ -1,0 +1,98 @@
+"""No-GPU checks of the boundary: the shared library loads, exports every symbol the
+header declares, validates arguments before touching the device, and its host-side
+schedule logic agrees with the schedule oracle and the patterns the paper prints."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from oracle import schedule as oracle_schedule
+from tests.test_oracle_schedule import printed_patterns
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def idxc():
+    from paper_2603_12201_b200 import build
+    build.build()
+    from paper_2603_12201_b200 import binding
+    return binding
+
+
+def test_library_exports_every_declared_symbol(idxc):
+    header = open(os.path.join(ROOT, "include", "idxc.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = sorted(set(re.findall(r"\b(idxc_[a-z_]+)\s*\(", header)))
+    assert declared == sorted(idxc.EXPORTED_SYMBOLS)
+    L = idxc.lib()
+    for name in declared:
+        assert hasattr(L, name), name
+
+
+def test_status_strings(idxc):
+    seen = {idxc.status_string(s) for s in range(7)}
+    assert len(seen) == 7 and "ok" in seen
+
+
+def test_schedule_host_logic_matches_oracle_and_printed_patterns(idxc):
+    pats = [p for _, _, _, p in printed_patterns()] + ["F", "FFFF", "FSSSFSSSFSSS"]
+    for pat in pats:
+        sch = idxc.Schedule(pat)
+        want = oracle_schedule.source_layers(pat)
+        assert [sch.source(l) for l in range(len(pat))] == want
+        assert sch.stats() == (pat.count("F"), pat.count("S"), 0)
+        with pytest.raises(idxc.IdxcError):
+            sch.source(len(pat))
+        sch.close()
+
+
+@pytest.mark.parametrize("bad", ["", "SFF", "FXS", "fss"])
+def test_schedule_rejects_invalid_patterns(idxc, bad):
+    with pytest.raises(idxc.IdxcError) as e:
+        idxc.Schedule(bad)
+    assert e.value.status == idxc.ERR_PATTERN
+
+
+def test_argument_validation_happens_before_any_device_work(idxc):
+    L = idxc.lib()
+    one = ctypes.c_void_p(16)      # never dereferenced: the calls must fail on the sizes first
+    # k_top out of range
+    assert L.idxc_indexer_prefill(one, one, one, None, None, 0, 8, 8, 16, 64, 0, idxc.BF16, None, 0, one, one, 1 << 20, 0, None) == idxc.ERR_INVALID_ARG
+    assert L.idxc_indexer_prefill(one, one, one, None, None, 0, 8, 8, 16, 64, 4096, idxc.BF16, None, 0, one, one, 1 << 20, 0, None) == idxc.ERR_INVALID_ARG
+    # head count / head dim without a tensor-core kernel
+    assert L.idxc_indexer_prefill(one, one, one, None, None, 0, 8, 8, 48, 64, 8, idxc.BF16, None, 0, one, one, 1 << 20, 0, None) == idxc.ERR_UNSUPPORTED
+    assert L.idxc_indexer_prefill(one, one, one, None, None, 0, 8, 8, 16, 96, 8, idxc.BF16, None, 0, one, one, 1 << 20, 0, None) == idxc.ERR_UNSUPPORTED
+    # K shorter than the last query position
+    assert L.idxc_indexer_prefill(one, one, one, None, None, 4, 8, 8, 16, 64, 8, idxc.BF16, None, 0, one, one, 1 << 20, 0, None) == idxc.ERR_INVALID_ARG
+    # unknown dtype / flag
+    assert L.idxc_indexer_prefill(one, one, one, None, None, 0, 8, 8, 16, 64, 8, 7, None, 0, one, one, 1 << 20, 0, None) == idxc.ERR_INVALID_ARG
+    assert L.idxc_indexer_prefill(one, one, one, None, None, 0, 8, 8, 16, 64, 8, idxc.BF16, None, 0, one, one, 1 << 20, 0x80, None) == idxc.ERR_INVALID_ARG
+    # fp8 without scales, null q, misaligned q
+    assert L.idxc_indexer_prefill(one, one, one, None, None, 0, 8, 8, 64, 128, 8, idxc.FP8_E4M3, None, 0, one, one, 1 << 20, 0, None) == idxc.ERR_INVALID_ARG
+    assert L.idxc_indexer_prefill(None, one, one, None, None, 0, 8, 8, 16, 64, 8, idxc.BF16, None, 0, one, one, 1 << 20, 0, None) == idxc.ERR_INVALID_ARG
+    assert L.idxc_indexer_prefill(ctypes.c_void_p(20), one, one, None, None, 0, 8, 8, 16, 64, 8, idxc.BF16, None, 0, one, one, 1 << 20, 0, None) == idxc.ERR_INVALID_ARG
+    # decode: negative batch, missing lens
+    assert L.idxc_indexer_decode(one, one, 100, one, None, None, one, one, -1, 10, 16, 64, 8, idxc.BF16, None, 0, one, one, 1 << 20, 0, None) == idxc.ERR_INVALID_ARG
+    assert L.idxc_indexer_decode(one, one, 100, one, None, None, one, None, 2, 10, 16, 64, 8, idxc.BF16, None, 0, one, one, 1 << 20, 0, None) == idxc.ERR_INVALID_ARG
+    # top-k: ld not a multiple of 4
+    assert L.idxc_topk_rows(one, 10, 2, 1, 1, None, 4, one, None) == idxc.ERR_INVALID_ARG
+
+
+def test_workspace_queries(idxc):
+    assert idxc.prefill_workspace_bytes(0, 0, 16, 64, 8) == 0
+    b = idxc.prefill_workspace_bytes(2048, 2048, 16, 64, 256)
+    assert b == 2048 * 2048 * 4
+    big = idxc.prefill_workspace_bytes(131072, 131072, 64, 128, 2048)
+    assert big <= 8 << 30 and big % (131072 * 4 * 32) == 0
+    assert idxc.decode_workspace_bytes(32, 131072, 64, 128, 2048) == 32 * 131072 * 4
+
+
+def test_binding_refuses_cpu_tensors(idxc):
+    import torch
+    q = torch.zeros(8, 16, 64, dtype=torch.bfloat16)
+    k = torch.zeros(8, 64, dtype=torch.bfloat16)
+    w = torch.zeros(8, 16)
+    with pytest.raises(ValueError):
+        idxc.indexer_prefill(q, k, w, 4, topk_out=torch.zeros(8, 4, dtype=torch.int32))

@@ -1,0 +1,333 @@
+"""GPU parity: the CUDA path, called through the C-ABI binding, against the FP64 oracle
+on the same seeded inputs, element by element. Sizes span several 128-key tiles, several
+work items and ragged tails; edge cases cover short rows, chunking, ties and empty input."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import schedule as oracle_schedule
+from paper_2603_12201_b200 import binding as idxc
+from paper_2603_12201_b200 import synth
+from tests.util import (RTOL_BF16, RTOL_FP8, assert_scores_close, assert_topk_valid, codes, f32)
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _to_dev(inp):
+    for name in ("q", "k", "w", "q_scale", "k_scale", "q_step", "k_cache", "k_offsets", "lens"):
+        if hasattr(inp, name) and getattr(inp, name) is not None:
+            setattr(inp, name, getattr(inp, name).to(DEV))
+    return inp
+
+
+def _oracle_prefill(inp, k_top, rows=None, q_begin=0, q_slice=None):
+    dt = oracle.FP8_E4M3 if inp.fp8 else oracle.BF16
+    q, w, qs = inp.q, inp.w, inp.q_scale
+    if q_slice is not None:
+        q, w = q[q_slice], w[q_slice]
+        qs = None if qs is None else qs[q_slice]
+    return oracle.indexer_prefill(codes(q), codes(inp.k), f32(w), k_top, dt, f32(qs), f32(inp.k_scale),
+                                  q_begin=q_begin, rows=rows)
+
+
+def _gpu_prefill(inp, k_top, flags=0, with_scores=True, q_begin=0, q_slice=None, workspace=None):
+    q, w, qs = inp.q, inp.w, inp.q_scale
+    if q_slice is not None:
+        q, w = q[q_slice].contiguous(), w[q_slice].contiguous()
+        qs = None if qs is None else qs[q_slice].contiguous()
+    q_len, L_k = q.shape[0], inp.k.shape[0]
+    ld = (L_k + 3) // 4 * 4
+    scores = torch.full((q_len, ld), float("nan"), device=DEV) if with_scores else None
+    topk = torch.full((q_len, k_top), -7, dtype=torch.int32, device=DEV)
+    if workspace is None and not with_scores:
+        workspace = idxc.alloc_workspace(idxc.prefill_workspace_bytes(q_len, L_k, q.shape[1], q.shape[2], k_top), DEV)
+    idxc.indexer_prefill(q, inp.k, w, k_top, qs, inp.k_scale, q_begin=q_begin, scores_out=scores, topk_out=topk,
+                         workspace=workspace, flags=flags)
+    idxc.poll_device_status()
+    return (None if scores is None else scores.cpu().numpy()), topk.cpu().numpy()
+
+
+def _check_prefill(inp, k_top, g_scores, g_topk, rtol, rows=None):
+    """All rows (or the listed ones) of a full prefill (q_begin = 0) against the oracle.
+    Returns the fraction of rows whose index set equals the oracle's exactly."""
+    o_scores, _ = _oracle_prefill(inp, k_top, rows=rows)
+    row_ids = range(g_topk.shape[0]) if rows is None else rows
+    exact = 0
+    for j, t in enumerate(row_ids):
+        o_row = o_scores[j, : t + 1]
+        if g_scores is not None:
+            assert_scores_close(g_scores[t, : t + 1], o_row, rtol, what=f"row {t}")
+        exact += assert_topk_valid(g_topk[t], o_row, k_top, rtol, what=f"row {t}")
+    return exact / max(len(row_ids), 1)
+
+
+def _own_topk_exact(g_scores, g_topk, k_top, q_begin=0):
+    """The selector alone: indices must be the exact top-k (lowest index on ties) of the GPU's own scores."""
+    for r in range(g_topk.shape[0]):
+        n = q_begin + r + 1
+        kk = min(k_top, n)
+        order = np.argsort(-g_scores[r, :n].astype(np.float64), kind="stable")
+        assert np.array_equal(np.sort(order[:kk]), g_topk[r, :kk]), f"row {r}"
+        assert np.all(g_topk[r, kk:] == -1)
+
+
+# ------------------------------------------------------------------------------ top-k alone
+@pytest.mark.parametrize("n,k_top", [(1, 1), (5, 8), (300, 64), (4096, 2048), (4100, 2048), (33000, 2048), (131072, 2048)])
+def test_topk_rows_matches_oracle(n, k_top):
+    g = torch.Generator().manual_seed(n)
+    rows = 6
+    ld = (n + 3) // 4 * 4
+    s = torch.randn(rows, ld, generator=g)
+    s[1] = torch.round(s[1] * 2) / 2                      # many exact ties
+    s[2] = 0.0                                            # all equal (threshold bucket overflows)
+    s[3] = torch.arange(ld, dtype=torch.float32)          # increasing: sliding window
+    s[4] = -torch.arange(ld, dtype=torch.float32)         # decreasing: sink
+    s[5, ::3] = -0.0
+    lens = torch.tensor([n, n, n, n, n, max(n - 3, 0)], dtype=torch.int32)
+    out = torch.full((rows, k_top), -7, dtype=torch.int32, device=DEV)
+    idxc.topk_rows(s.to(DEV), k_top, out, lens=lens.to(DEV))
+    out = out.cpu().numpy()
+    for r in range(rows):
+        want = oracle.topk(s[r, : int(lens[r])].to(torch.float64).numpy(), k_top)
+        assert np.array_equal(out[r], want), f"row {r}"
+
+
+def test_topk_rows_causal_lengths_and_empty():
+    g = torch.Generator().manual_seed(5)
+    n_rows, ld, k_top = 70, 72, 16
+    s = torch.randn(n_rows, ld, generator=g)
+    out = torch.full((n_rows, k_top), -7, dtype=torch.int32, device=DEV)
+    idxc.topk_rows(s.to(DEV), k_top, out, first_len=1, len_step=1)
+    out = out.cpu().numpy()
+    for r in range(n_rows):
+        assert np.array_equal(out[r], oracle.topk(s[r, : r + 1].to(torch.float64).numpy(), k_top))
+    empty = torch.empty((0, 8), device=DEV)
+    idxc.topk_rows(empty, 4, torch.empty((0, 4), dtype=torch.int32, device=DEV), first_len=1, len_step=1)
+
+
+# ------------------------------------------------------------------------------ prefill
+@pytest.mark.parametrize("L,H,d,k_top,fp8,flags", [
+    (200, 4, 32, 16, False, idxc.FLAG_SIMT_SCORER),
+    (200, 4, 32, 16, True, idxc.FLAG_SIMT_SCORER),
+    (300, 16, 64, 32, False, 0),
+    (517, 32, 64, 64, False, 0),
+    (1000, 64, 128, 128, False, 0),
+    (700, 32, 128, 64, False, 0),
+    (900, 64, 128, 100, True, 0),
+    (333, 16, 128, 40, True, 0),
+])
+def test_prefill_matches_oracle(L, H, d, k_top, fp8, flags):
+    inp = _to_dev(synth.prefill_inputs(L, H, d, seed=10 + L, fp8=fp8))
+    g_scores, g_topk = _gpu_prefill(inp, k_top, flags=flags)
+    rtol = RTOL_FP8 if fp8 else RTOL_BF16
+    _check_prefill(inp, k_top, g_scores, g_topk, rtol)
+    _own_topk_exact(g_scores, g_topk, k_top)
+    # entries above the diagonal are never written
+    iu = np.triu_indices(L, k=1)
+    assert np.all(np.isnan(g_scores[:, :L][iu]))
+
+
+def test_config1_full():
+    c = synth.CONFIGS["cfg1"]
+    inp = _to_dev(synth.prefill_inputs(c["L"], c["H"], c["d"], seed=c["seed"]))
+    g_scores, g_topk = _gpu_prefill(inp, c["k_top"])
+    frac = _check_prefill(inp, c["k_top"], g_scores, g_topk, RTOL_BF16)
+    _own_topk_exact(g_scores, g_topk, c["k_top"])
+    assert frac > 0.98          # near-ties inside the tolerance band are rare
+
+
+def test_prefill_chunked_workspace_and_scoreless_paths_agree():
+    L, H, d, k_top = 1100, 64, 128, 96
+    inp = _to_dev(synth.prefill_inputs(L, H, d, seed=77))
+    s_full, t_full = _gpu_prefill(inp, k_top)
+    # no score output: scores go through the workspace; a small workspace forces several chunks
+    ld = (L + 31) // 32 * 32
+    _, t_ws = _gpu_prefill(inp, k_top, with_scores=False)
+    _, t_small = _gpu_prefill(inp, k_top, with_scores=False, workspace=idxc.alloc_workspace(64 * ld * 4, DEV))
+    assert np.array_equal(t_ws, t_full) and np.array_equal(t_small, t_full)
+    # query chunks against the full K (chunked prefill) give the same rows
+    for q0, q1 in [(0, 256), (256, 700), (700, 1100)]:
+        s_c, t_c = _gpu_prefill(inp, k_top, q_begin=q0, q_slice=slice(q0, q1))
+        assert np.array_equal(t_c, t_full[q0:q1])
+        for r in range(q1 - q0):
+            assert np.array_equal(s_c[r, : q0 + r + 1], s_full[q0 + r, : q0 + r + 1])
+    with pytest.raises(idxc.IdxcError) as e:
+        _gpu_prefill(inp, k_top, with_scores=False, workspace=idxc.alloc_workspace(8 * ld * 4, DEV))
+    assert e.value.status == idxc.ERR_WORKSPACE
+
+
+def test_prefill_duplicate_keys_pick_lowest_index_and_gate():
+    L, H, d, k_top = 400, 16, 64, 8
+    inp = synth.prefill_inputs(L, H, d, seed=3)
+    inp.k[200:] = inp.k[:200]                       # every key appears twice: bit-identical scores
+    inp = _to_dev(inp)
+    g_scores, g_topk = _gpu_prefill(inp, k_top)
+    assert np.array_equal(g_scores[399, 200:400], g_scores[399, :200])
+    _own_topk_exact(g_scores, g_topk, k_top)
+    _check_prefill(inp, k_top, g_scores, g_topk, RTOL_BF16)
+    # all dot products <= 0: every score is exactly zero and the lowest positions win
+    inp2 = synth.prefill_inputs(L, H, d, seed=4)
+    inp2.q = inp2.q.abs()
+    inp2.k = -inp2.k.abs()
+    inp2 = _to_dev(inp2)
+    s2, t2 = _gpu_prefill(inp2, k_top)
+    for t in range(L):
+        assert np.all(s2[t, : t + 1] == 0.0)
+        kk = min(k_top, t + 1)
+        assert t2[t, :kk].tolist() == list(range(kk))
+
+
+def test_prefill_rejects_bad_arguments():
+    inp = _to_dev(synth.prefill_inputs(64, 16, 64, seed=1))
+    topk = torch.empty((64, 8), dtype=torch.int32, device=DEV)
+    ws = idxc.alloc_workspace(1 << 20, DEV)
+    with pytest.raises(idxc.IdxcError) as e:
+        idxc.indexer_prefill(inp.q, inp.k, inp.w, 8, q_begin=1, topk_out=topk, workspace=ws)      # L_k < q_begin + q_len
+    assert e.value.status == idxc.ERR_INVALID_ARG
+    with pytest.raises(idxc.IdxcError) as e:
+        idxc.indexer_prefill(inp.q, inp.k, inp.w, 8)                                              # no output at all
+    assert e.value.status == idxc.ERR_INVALID_ARG
+    with pytest.raises(idxc.IdxcError) as e:
+        idxc.indexer_prefill(inp.q, inp.k, inp.w, 8, topk_out=topk)                               # no workspace
+    assert e.value.status == idxc.ERR_WORKSPACE
+    with pytest.raises(ValueError):
+        idxc.indexer_prefill(inp.q.cpu(), inp.k, inp.w, 8, topk_out=topk, workspace=ws)           # no CPU path
+    # zero query rows: a no-op
+    idxc.indexer_prefill(inp.q[:0], inp.k, inp.w[:0], 8, topk_out=topk[:0], workspace=ws)
+
+
+# ------------------------------------------------------------------------------ decode
+@pytest.mark.parametrize("B,H,d,k_top,fp8,lens,flags", [
+    (3, 4, 32, 8, False, [5, 130, 77], idxc.FLAG_SIMT_SCORER),
+    (4, 64, 128, 64, False, [1, 127, 1500, 3000], 0),
+    (5, 16, 64, 32, False, [129, 2048, 31, 1025, 4000], 0),
+    (3, 32, 128, 48, True, [999, 2500, 50], 0),
+    (2, 64, 128, 2048, False, [2047, 5000], 0),
+])
+def test_decode_matches_oracle(B, H, d, k_top, fp8, lens, flags):
+    inp = _to_dev(synth.decode_inputs(B, H, d, 0, 0, seed=20 + B, fp8=fp8, lens=lens, row_align=8))
+    ld = (inp.max_len + 3) // 4 * 4
+    scores = torch.full((B, ld), float("nan"), device=DEV)
+    topk = torch.full((B, k_top), -7, dtype=torch.int32, device=DEV)
+    idxc.indexer_decode(inp.q_step, inp.k_cache, inp.w, inp.k_offsets, inp.lens, inp.max_len, k_top, inp.q_scale,
+                        inp.k_scale, scores_out=scores, topk_out=topk, flags=flags)
+    idxc.poll_device_status()
+    # without score output (workspace path) the indices are the same
+    topk2 = torch.full((B, k_top), -7, dtype=torch.int32, device=DEV)
+    ws = idxc.alloc_workspace(idxc.decode_workspace_bytes(B, inp.max_len, H, d, k_top), DEV)
+    idxc.indexer_decode(inp.q_step, inp.k_cache, inp.w, inp.k_offsets, inp.lens, inp.max_len, k_top, inp.q_scale,
+                        inp.k_scale, topk_out=topk2, workspace=ws, flags=flags)
+    assert torch.equal(topk, topk2)
+    dt = oracle.FP8_E4M3 if fp8 else oracle.BF16
+    o_scores, _ = oracle.indexer_decode(codes(inp.q_step), codes(inp.k_cache), f32(inp.w), inp.k_offsets.cpu().numpy(),
+                                        inp.lens.cpu().numpy(), k_top, dt, f32(inp.q_scale), f32(inp.k_scale))
+    g_scores, g_topk = scores.cpu().numpy(), topk.cpu().numpy()
+    rtol = RTOL_FP8 if fp8 else RTOL_BF16
+    for b in range(B):
+        n = lens[b]
+        assert_scores_close(g_scores[b, :n], o_scores[b, :n], rtol, what=f"seq {b}")
+        assert np.all(np.isnan(g_scores[b, n:]))
+        assert_topk_valid(g_topk[b], o_scores[b, :n], k_top, rtol, what=f"seq {b}")
+        order = np.argsort(-g_scores[b, :n].astype(np.float64), kind="stable")
+        kk = min(k_top, n)
+        assert np.array_equal(np.sort(order[:kk]), g_topk[b, :kk])
+
+
+def test_decode_equals_prefill_row():
+    L, H, d, k_top = 640, 64, 128, 50
+    inp = _to_dev(synth.prefill_inputs(L, H, d, seed=31))
+    s_p, t_p = _gpu_prefill(inp, k_top)
+    ts = [0, 127, 128, 300, 639]
+    lens = torch.tensor([t + 1 for t in ts], dtype=torch.int32, device=DEV)
+    offs = torch.zeros(len(ts), dtype=torch.int64, device=DEV)
+    ld = 640
+    scores = torch.full((len(ts), ld), float("nan"), device=DEV)
+    topk = torch.empty((len(ts), k_top), dtype=torch.int32, device=DEV)
+    idxc.indexer_decode(inp.q[ts].contiguous(), inp.k, inp.w[ts].contiguous(), offs, lens, L, k_top,
+                        scores_out=scores, topk_out=topk)
+    idxc.poll_device_status()
+    sc = scores.cpu().numpy()
+    for j, t in enumerate(ts):
+        assert np.allclose(sc[j, : t + 1], s_p[t, : t + 1], rtol=1e-5, atol=1e-4)   # same products, other tile shape
+        o_row = _oracle_prefill(inp, k_top, rows=[t])[0][0, : t + 1]
+        assert_topk_valid(topk[j].cpu().numpy(), o_row, k_top, RTOL_BF16)
+
+
+# ------------------------------------------------------------------------------ schedule
+def test_schedule_prefill_shares_bit_for_bit():
+    pattern = "FSSFSFSS"
+    L, H, d, k_top = 384, 16, 64, 24
+    layers = [_to_dev(synth.prefill_inputs(L, H, d, seed=5, layer=l)) for l in range(len(pattern))]
+    ws = idxc.alloc_workspace(idxc.prefill_workspace_bytes(L, L, H, d, k_top), DEV)
+    bufs = [torch.full((L, k_top), -9, dtype=torch.int32, device=DEV) for _ in pattern]
+    sch = idxc.Schedule(pattern)
+    for copy_flag in (0, idxc.FLAG_COPY_SHARED):
+        sch.begin_pass()
+        before = sch.stats()[2]
+        launches0 = idxc.launch_count()
+        outs = []
+        for l, ch in enumerate(pattern):
+            x = layers[l]
+            if ch == "F":
+                t = sch.prefill_layer(l, x.q, x.k, x.w, k_top, topk_buf=bufs[l], workspace=ws, flags=copy_flag)
+            else:   # S layers get no inputs at all: proves they are never read
+                t = sch.prefill_layer(l, k_top=k_top, q_len=L, topk_buf=bufs[l] if copy_flag else None, flags=copy_flag)
+            outs.append(t)
+        idxc.poll_device_status()
+        nf, ns, calls = sch.stats()
+        assert (nf, ns) == (3, 5) and calls - before == 3
+        assert idxc.launch_count() - launches0 == 2 * 3            # scorer + top-k per F layer, nothing on S layers
+        src = oracle_schedule.source_layers(pattern)
+        for l in range(len(pattern)):
+            assert sch.source(l) == src[l]
+            assert torch.equal(outs[l], outs[src[l]])
+            if copy_flag:
+                assert outs[l].data_ptr() == bufs[l].data_ptr()
+            else:
+                assert outs[l].data_ptr() == bufs[src[l]].data_ptr()   # alias of the F layer's buffer
+        # against the oracle's loop, F layers checked with the band criterion
+        def oracle_layer(l):
+            return _oracle_prefill(layers[l], k_top)[0]
+        for l in [0, 3, 5]:
+            o_scores = oracle_layer(l)
+            g = outs[l].cpu().numpy()
+            for t in range(L):
+                assert_topk_valid(g[t], o_scores[t, : t + 1], k_top, RTOL_BF16)
+    # visiting an S layer before its F layer ran in this pass is an error
+    sch.begin_pass()
+    with pytest.raises(idxc.IdxcError) as e:
+        sch.prefill_layer(1, k_top=k_top, q_len=L)
+    assert e.value.status == idxc.ERR_PATTERN
+    sch.close()
+
+
+def test_schedule_decode_layers():
+    pattern = "FSFS"
+    B, H, d, k_top = 3, 64, 128, 32
+    lens = [300, 1000, 129]
+    layers = [_to_dev(synth.decode_inputs(B, H, d, 0, 0, seed=8, layer=l, lens=lens)) for l in range(4)]
+    sch = idxc.Schedule(pattern)
+    sch.begin_pass()
+    ws = idxc.alloc_workspace(idxc.decode_workspace_bytes(B, 1000, H, d, k_top), DEV)
+    bufs = [torch.empty((B, k_top), dtype=torch.int32, device=DEV) for _ in pattern]
+    outs = []
+    for l, ch in enumerate(pattern):
+        x = layers[l]
+        if ch == "F":
+            outs.append(sch.decode_layer(l, x.q_step, x.k_cache, x.w, x.k_offsets, x.lens, x.max_len, k_top,
+                                         topk_buf=bufs[l], workspace=ws))
+        else:
+            outs.append(sch.decode_layer(l, B=B, k_top=k_top))
+    idxc.poll_device_status()
+    assert torch.equal(outs[1], outs[0]) and torch.equal(outs[3], outs[2]) and not torch.equal(outs[0], outs[2])
+    assert sch.stats() == (2, 2, 2)
+    for l in (0, 2):
+        x = layers[l]
+        o_scores, _ = oracle.indexer_decode(codes(x.q_step), codes(x.k_cache), f32(x.w), x.k_offsets.cpu().numpy(),
+                                            x.lens.cpu().numpy(), k_top)
+        g = outs[l].cpu().numpy()
+        for b in range(B):
+            assert_topk_valid(g[b], o_scores[b, : lens[b]], k_top, RTOL_BF16)
+    sch.close()
