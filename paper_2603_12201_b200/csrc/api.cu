@@ -143,8 +143,8 @@ idxc_status idxc_indexer_prefill(const void* q, const void* k, const float* w, c
     idxc_status st = check_common(H_I, d_I, k_top, dt, flags);
     if (st != IDXC_OK) return st;
     if (q_begin < 0 || q_len < 0 || L_k < q_begin + q_len || L_k > (int64_t(1) << 30)) return IDXC_ERR_INVALID_ARG;
-    if (!scores_out && !topk_out) return IDXC_ERR_INVALID_ARG;
     if (q_len == 0) return IDXC_OK;
+    if (!scores_out && !topk_out) return IDXC_ERR_INVALID_ARG;
     if (!q || !k || !w || !aligned(q, 16) || !aligned(k, 16) || !aligned(w, 16)) return IDXC_ERR_INVALID_ARG;
     const bool fp8 = dt == IDXC_FP8_E4M3;
     if (fp8 && (!q_scale || !k_scale)) return IDXC_ERR_INVALID_ARG;
@@ -206,8 +206,8 @@ idxc_status idxc_indexer_decode(const void* q_step, const void* k_cache, int64_t
     if (st != IDXC_OK) return st;
     if (B < 0 || max_len < 0 || max_len > (int64_t(1) << 30) || cache_rows < 0 || cache_rows > (int64_t(1) << 31) - 256)
         return IDXC_ERR_INVALID_ARG;
-    if (!scores_out && !topk_out) return IDXC_ERR_INVALID_ARG;
     if (B == 0) return IDXC_OK;
+    if (!scores_out && !topk_out) return IDXC_ERR_INVALID_ARG;
     if (!q_step || !k_cache || !w || !k_offsets || !lens) return IDXC_ERR_INVALID_ARG;
     if (!aligned(q_step, 16) || !aligned(k_cache, 16) || !aligned(k_offsets, 8) || !aligned(lens, 4)) return IDXC_ERR_INVALID_ARG;
     const bool fp8 = dt == IDXC_FP8_E4M3;
