@@ -1,0 +1,423 @@
+#!/usr/bin/env python
+"""Benchmark of the lightning-indexer hot path on B200.
+
+One "step" = one Full layer of the indexer on the config-2 workload (L = 32768, H_I = 64,
+d_I = 128, k = 2048, clustered keys): the scoring kernel followed by the top-k kernel,
+called through the C-ABI binding. The headline `value` is causal (query, key) pairs scored
+and selected per second, inputs resident in HBM. The same JSON line also carries
+  roofline      the dominant kernel (tcgen05 scorer) against the measured BF16 peak
+  e2e           the same step with host buffers (pinned H2D of q/k/w, D2H of the indices)
+  cpu_baseline  the FP64 oracle timed on the machine's host cores on a bounded row sample
+  decode        config 3 (B = 32, 16K-128K cached keys): microseconds per decode step vs HBM
+  schedule      IndexCache 1-in-4 Full pattern vs all-Full on config-2-shaped layers
+`--impl reference` times the CPU oracle instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+METRIC = "indexer+top-k Gpairs/s (prefill)"
+UNIT = "Gpairs/s"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per scorer launch on this workload, from the
+# ncu capture summarised in profiles/ (None until a capture exists).
+SCORER_DRAM_TRAFFIC_BYTES = None
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as fh:
+            d = json.load(fh)
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"],
+                    bf16_tflops_sustained=d.get("bf16_tflops_sustained", d["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while a region runs."""
+
+    def __init__(self, device_index: int, period_s: float = 0.005):
+        self.period = period_s
+        self.samples = []
+        self.reasons = set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            try:
+                uuid = torch.cuda.get_device_properties(device_index).uuid
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + str(uuid)).encode())
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._h = None
+
+    _NAMES = {
+        0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x10: "sync_boost",
+        0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown",
+        0x100: "display_clock_setting",
+    }
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                for bit, name in self._NAMES.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["unavailable"]}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz, "samples": len(self.samples),
+                "reasons": sorted(self.reasons)}
+
+
+def dist_setup(n_gpus):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    return rank, world, local
+
+
+def max_over_ranks(x: float, world: int, device) -> float:
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def causal_pairs(L: int) -> int:
+    return L * (L + 1) // 2
+
+
+def sample_rows(L: int, n: int, offset: int = 0):
+    """Deterministic bounded sample of whole rows: evenly spaced, plus the edges."""
+    stride = max(1, L // n)
+    rows = sorted(set([0, L - 1] + [min(L - 1, offset % stride + i * stride) for i in range(n)]))
+    return rows
+
+
+def oracle_sample_rate(inp, k_top, rows):
+    """Times the oracle (as it stands) on the listed rows; returns (pairs/s, seconds, index rows)."""
+    import oracle
+    from tests.util import codes, f32
+    dt = oracle.FP8_E4M3 if inp.fp8 else oracle.BF16
+    q, k, w = codes(inp.q), codes(inp.k), f32(inp.w)
+    qs, ks = f32(inp.q_scale), f32(inp.k_scale)
+    t0 = time.perf_counter()
+    _, tk = oracle.indexer_prefill(q, k, w, k_top, dt, qs, ks, rows=rows, want_scores=False)
+    sec = time.perf_counter() - t0
+    pairs = sum(r + 1 for r in rows)
+    return pairs / sec, sec, tk
+
+
+def run_reference(args, rank):
+    """--impl reference: the CPU oracle on bounded row samples of the same workload."""
+    if rank != 0:
+        return
+    import oracle
+    from paper_2603_12201_b200 import synth
+    c = synth.CONFIGS[args.workload]
+    L, H, d, k_top = c["L"], c["H"], c["d"], c["k_top"]
+    inp = synth.prefill_inputs(L, H, d, seed=c["seed"], device="cpu", fp8=c["fp8"], clustered=c["clustered"])
+    n_rows = args.ref_rows
+    for i in range(args.warmup):
+        oracle_sample_rate(inp, k_top, sample_rows(L, max(8, n_rows // 8), offset=i))
+    total_pairs, total_sec = 0, 0.0
+    for i in range(args.steps):
+        rows = sample_rows(L, n_rows, offset=7 * i + 3)
+        rate, sec, _ = oracle_sample_rate(inp, k_top, rows)
+        total_pairs += sum(r + 1 for r in rows)
+        total_sec += sec
+    value = total_pairs / total_sec / 1e9
+    sample = f"{n_rows} evenly spaced whole rows of the L={L} workload per step (all s <= t), {args.steps} steps"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * total_sec / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: prefill L={L} H_I={H} d_I={d} k_top={k_top} (bounded row sample)"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def time_decode(idxc, synth, dev, peaks, steps, warmup):
+    c = synth.CONFIGS["cfg3"]
+    x = synth.decode_inputs(c["B"], c["H"], c["d"], c["len_lo"], c["len_hi"], seed=c["seed"], device=dev)
+    B, k_top = c["B"], c["k_top"]
+    topk = torch.empty((B, k_top), dtype=torch.int32, device=dev)
+    ws = idxc.alloc_workspace(idxc.decode_workspace_bytes(B, x.max_len, c["H"], c["d"], k_top), dev)
+    ld = (x.max_len + 31) // 32 * 32
+    scores = ws[: B * ld * 4].view(torch.float32).view(B, ld)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3 * steps)]
+    for i in range(warmup + steps):
+        j = i - warmup
+        if j >= 0:
+            ev[3 * j].record()
+        idxc.indexer_decode(x.q_step, x.k_cache, x.w, x.k_offsets, x.lens, x.max_len, k_top, scores_out=scores)
+        if j >= 0:
+            ev[3 * j + 1].record()
+        idxc.topk_rows(scores, k_top, topk, lens=x.lens)
+        if j >= 0:
+            ev[3 * j + 2].record()
+    torch.cuda.synchronize()
+    idxc.poll_device_status()
+    t_score = [ev[3 * j].elapsed_time(ev[3 * j + 1]) * 1e3 for j in range(steps)]
+    t_total = [ev[3 * j].elapsed_time(ev[3 * j + 2]) * 1e3 for j in range(steps)]
+    keys = int(x.lens.sum().item())
+    bytes_k = keys * c["d"] * 2
+    us_score, us_total = statistics.median(t_score), statistics.median(t_total)
+    gbs = bytes_k / (us_score * 1e-6) / 1e9
+    return {
+        "workload": f"cfg3: decode B={B} H_I={c['H']} d_I={c['d']} k_top={k_top}, sum(lens)={keys}",
+        "us_per_step": us_total, "us_scorer": us_score, "us_topk": us_total - us_score,
+        "k_cache_bytes": bytes_k,
+        "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": gbs / peaks["hbm_gbs"], "traffic": None, "kernel": "score_decode_tc_kernel",
+                     "of": peaks["source"]},
+        "frac_step_vs_hbm": bytes_k / (us_total * 1e-6) / 1e9 / peaks["hbm_gbs"],
+    }
+
+
+def time_schedule(idxc, synth, dev, L, H, d, k_top, n_layers, every, seed, reps):
+    """1-in-`every` Full pattern vs all-Full on the same per-layer inputs (config-4 shape, fewer layers by default)."""
+    layers = [synth.prefill_inputs(L, H, d, seed=seed, device=dev, layer=l) for l in range(n_layers)]
+    ws = idxc.alloc_workspace(idxc.prefill_workspace_bytes(L, L, H, d, k_top), dev)
+    bufs = [torch.empty((L, k_top), dtype=torch.int32, device=dev) for _ in range(n_layers)]
+
+    def run(pattern):
+        sch = idxc.Schedule(pattern)
+        times = []
+        for _ in range(reps + 1):
+            sch.begin_pass()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for l, ch in enumerate(pattern):
+                x = layers[l]
+                if ch == "F":
+                    sch.prefill_layer(l, x.q, x.k, x.w, k_top, topk_buf=bufs[l], workspace=ws)
+                else:
+                    sch.prefill_layer(l, k_top=k_top, q_len=L)
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        calls = sch.stats()[2]
+        sch.close()
+        return statistics.median(times[1:]), calls // (reps + 1)
+
+    pat = synth.uniform_pattern(n_layers, every)
+    t_sched, calls_sched = run(pat)
+    t_full, calls_full = run("F" * n_layers)
+    idxc.poll_device_status()
+    return {"workload": f"cfg4-shaped: N={n_layers} layers, L={L}, H_I={H}, d_I={d}, k_top={k_top}, F every {every}",
+            "ms_scheduled": t_sched, "ms_all_full": t_full, "ratio": t_full / t_sched,
+            "indexer_calls": [calls_sched, calls_full]}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2"])
+    ap.add_argument("--ref-rows", type=int, default=128, help="rows per step of the reference (oracle) arm")
+    ap.add_argument("--cpu-rows", type=int, default=1024, help="rows of the cpu_baseline sample")
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-extras", action="store_true", help="skip the decode and schedule sections")
+    ap.add_argument("--schedule-layers", type=int, default=8)
+    ap.add_argument("--schedule-L", type=int, default=32768)
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+
+    if args.impl == "reference":
+        rank = int(os.environ.get("RANK", "0"))
+        run_reference(args, rank)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the indexer has no CPU path (use --impl reference for the oracle)")
+    rank, world, local = dist_setup(args.gpus)
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    from paper_2603_12201_b200 import binding as idxc
+    from paper_2603_12201_b200 import synth
+    idxc.lib()
+    peaks = load_peaks()
+
+    c = synth.CONFIGS[args.workload]
+    L, H, d, k_top = c["L"], c["H"], c["d"], c["k_top"]
+    # independent problem per rank (weak scaling): same shape, rank-specific seed
+    inp = synth.prefill_inputs(L, H, d, seed=c["seed"] + 1000 * rank, device=dev, fp8=c["fp8"], clustered=c["clustered"])
+    ld = (L + 31) // 32 * 32
+    scores = torch.empty((L, ld), dtype=torch.float32, device=dev)
+    topk = torch.empty((L, k_top), dtype=torch.int32, device=dev)
+    pairs = causal_pairs(L)
+    K, W = args.steps, args.warmup
+
+    def step(evs=None):
+        if evs:
+            evs[0].record()
+        idxc.indexer_prefill(inp.q, inp.k, inp.w, k_top, inp.q_scale, inp.k_scale, scores_out=scores)   # scorer launch
+        if evs:
+            evs[1].record()
+        idxc.topk_rows(scores, k_top, topk, first_len=1, len_step=1)                                    # top-k launch
+        if evs:
+            evs[2].record()
+
+    for _ in range(W):
+        step()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    torch.cuda.synchronize()
+    barrier(world)
+    launches0 = idxc.launch_count()
+    with ClockSampler(local) as clk:
+        t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t_start.record()
+        for i in range(K):
+            step(evs[i])
+        t_end.record()
+        torch.cuda.synchronize()
+    barrier(world)
+    launches = idxc.launch_count() - launches0
+    idxc.poll_device_status()
+    total_ms = max_over_ranks(t_start.elapsed_time(t_end), world, dev)
+    ms_per_step = total_ms / K
+    value = world * pairs * K / (total_ms * 1e-3) / 1e9
+    scorer_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
+    topk_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
+    flops = 2.0 * H * d * pairs
+    achieved_tf = flops / (scorer_ms * 1e-3) / 1e12
+    roofline = {
+        "bound": "tensor", "achieved": achieved_tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+        "frac": achieved_tf / peaks["bf16_tflops"], "traffic": SCORER_DRAM_TRAFFIC_BYTES,
+        "kernel": "score_prefill_tc_kernel", "ms_per_launch": scorer_ms, "of": peaks["source"] + " burst peak",
+        "frac_of_sustained": achieved_tf / peaks["bf16_tflops_sustained"],
+        "algorithmic_flops_per_launch": flops,
+        "topk_kernel": {"ms_per_launch": topk_ms, "bound": "hbm",
+                        "achieved": (4.0 * pairs + 4.0 * L * k_top) / (topk_ms * 1e-3) / 1e9,
+                        "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                        "frac": (4.0 * pairs + 4.0 * L * k_top) / (topk_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+    }
+
+    # ---- e2e: host buffers, H2D of the step's inputs and D2H of its result inside the timed region
+    hq = torch.empty(inp.q.shape, dtype=inp.q.dtype, pin_memory=True).copy_(inp.q)
+    hk = torch.empty(inp.k.shape, dtype=inp.k.dtype, pin_memory=True).copy_(inp.k)
+    hw = torch.empty(inp.w.shape, dtype=inp.w.dtype, pin_memory=True).copy_(inp.w)
+    hout = torch.empty(topk.shape, dtype=topk.dtype, pin_memory=True)
+    dq, dk, dw = torch.empty_like(inp.q), torch.empty_like(inp.k), torch.empty_like(inp.w)
+    ws = scores.view(torch.uint8).view(-1)
+
+    def e2e_step():
+        dq.copy_(hq, non_blocking=True)
+        dk.copy_(hk, non_blocking=True)
+        dw.copy_(hw, non_blocking=True)
+        idxc.indexer_prefill(dq, dk, dw, k_top, topk_out=topk, workspace=ws)    # the call a user makes
+        hout.copy_(topk, non_blocking=True)
+
+    e2e_step()
+    torch.cuda.synchronize()
+    barrier(world)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.e2e_steps):
+        e2e_step()
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
+    h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hw))
+    d2h = hout.numel() * hout.element_size()
+    e2e = {"value": world * pairs * args.e2e_steps / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.e2e_steps, "steps": args.e2e_steps}
+    assert torch.equal(hout.to(dev), topk)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "fp8_e4m3" if c["fp8"] else "bf16", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: single-layer indexer prefill, batch 1, L={L}, H_I={H}, d_I={d}, "
+                               f"k_top={k_top}, causal, seed {c['seed']}" + (", clustered keys" if c["clustered"] else ""),
+                   "parallelism": f"independent problem per GPU x{world}",
+                   "l2": f"inputs {(inp.q.numel() * inp.q.element_size()) >> 20} MiB and scores "
+                         f"{scores.numel() * 4 >> 20} MiB per step exceed the 126 MB L2; no flush needed"},
+        "roofline": roofline, "e2e": e2e, "gpu_launches": launches, "clocks": clk.summary(),
+        "kernel_ms": {"scorer": scorer_ms, "topk": topk_ms},
+    }
+
+    if rank == 0 and world == 1:
+        # ---- the oracle on this machine's host cores, bounded sample of the same workload; doubles as a parity spot check
+        host = synth.PrefillInputs(inp.q.cpu(), inp.k.cpu(), inp.w.cpu(),
+                                   None if inp.q_scale is None else inp.q_scale.cpu(),
+                                   None if inp.k_scale is None else inp.k_scale.cpu(), inp.fp8)
+        rows = sample_rows(L, args.cpu_rows)
+        import oracle
+        rate, sec, o_tk = oracle_sample_rate(host, k_top, rows)
+        g_tk = topk[rows].cpu().numpy()
+        same = sum(int((g_tk[j] == o_tk[j]).all()) for j in range(len(rows)))
+        line["cpu_baseline"] = {
+            "value": rate / 1e9, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "sample": f"{len(rows)} evenly spaced whole rows (all s <= t) of the same inputs, {sec:.1f} s",
+            "rows_with_identical_index_set": f"{same}/{len(rows)}"}
+        if not args.no_extras:
+            line["decode"] = time_decode(idxc, synth, dev, peaks, steps=max(K, 10), warmup=W)
+            line["schedule"] = time_schedule(idxc, synth, dev, args.schedule_L, H, d, k_top, args.schedule_layers, 4,
+                                             seed=3, reps=2)
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
