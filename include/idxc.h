@@ -116,6 +116,33 @@ idxc_status idxc_indexer_decode(const void* q_step, const void* k_cache, int64_t
                                 void* cuda_stream);
 
 /* ---------------------------------------------------------------------------
+ * Decode without caller-provided scratch. (The paper has no counterpart: this entry point
+ * exists for hosts that cannot allocate device memory where they decode, e.g. a serving
+ * process whose KV-cache pool already owns all free HBM, or a decode loop that cannot
+ * afford the device-wide stall of cudaMalloc / cudaFree.)
+ * Same operation, arguments and rules as idxc_indexer_decode with scores_out == NULL, but the
+ * fp32 score scratch lives in an array built into the library (IDXC_NOALLOC_SCRATCH_BYTES on
+ * every GPU that loads the library, until the process exits) instead of a workspace. The call
+ * allocates nothing on host or device. Limits and behaviour:
+ *   - B * round_up(max_len, 32) * 4 bytes must not exceed IDXC_NOALLOC_SCRATCH_BYTES (e.g.
+ *     B = 32 sequences of up to 131072 keys); larger requests return IDXC_ERR_WORKSPACE and
+ *     launch nothing. topk_out is required.
+ *   - The first call on each device looks up the array's device address (that device must be
+ *     current); make that first call before starting any stream capture.
+ *   - Every call shares the one array. Calls whose kernels can overlap on the GPU (different
+ *     streams without an ordering between them) race and return unspecified indices; calls on
+ *     one stream, or ordered by events, are safe. The array keeps the previous call's scores
+ *     and needs no clearing: each call writes every score it later reads.
+ * ------------------------------------------------------------------------- */
+#define IDXC_NOALLOC_SCRATCH_BYTES (16u << 20)
+
+idxc_status idxc_indexer_decode_noalloc(const void* q_step, const void* k_cache, int64_t cache_rows,
+                                        const float* w, const float* q_scale, const float* k_scale,
+                                        const int64_t* k_offsets, const int32_t* lens,
+                                        int B, int64_t max_len, int H_I, int d_I, int k_top, idxc_dtype dt,
+                                        int32_t* topk_out, uint32_t flags, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------
  * Top-k alone (Sec. 3 "Notation"), for rows of fp32 scores already in memory.
  * Row r has length lens[r] if lens != NULL (device int32), else
  * first_len + r * len_step (len_step = 1: causal rows; 0: equal rows), clamped to

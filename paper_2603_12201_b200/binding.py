@@ -24,8 +24,9 @@ EXPORTED_SYMBOLS = [
     "idxc_status_string", "idxc_prefill_workspace_bytes", "idxc_indexer_prefill", "idxc_decode_workspace_bytes",
     "idxc_indexer_decode", "idxc_topk_rows", "idxc_schedule_create", "idxc_schedule_destroy",
     "idxc_schedule_begin_pass", "idxc_schedule_source", "idxc_schedule_stats", "idxc_schedule_prefill_layer",
-    "idxc_schedule_decode_layer", "idxc_poll_device_status", "idxc_launch_count",
+    "idxc_schedule_decode_layer", "idxc_poll_device_status", "idxc_launch_count", "idxc_indexer_decode_noalloc",
 ]
+NOALLOC_SCRATCH_BYTES = 16 << 20
 
 
 class IdxcError(RuntimeError):
@@ -59,6 +60,8 @@ def lib() -> ctypes.CDLL:
         L.idxc_indexer_prefill.argtypes = prefill_args
         L.idxc_indexer_decode.restype = i32
         L.idxc_indexer_decode.argtypes = decode_args
+        L.idxc_indexer_decode_noalloc.restype = i32
+        L.idxc_indexer_decode_noalloc.argtypes = [vp, vp, i64, vp, vp, vp, vp, vp, i32, i64, i32, i32, i32, i32, vp, u32, vp]
         L.idxc_topk_rows.restype = i32
         L.idxc_topk_rows.argtypes = [vp, i64, i64, i64, i64, vp, i32, vp, vp]
         L.idxc_schedule_create.restype = i32
@@ -196,6 +199,19 @@ def indexer_decode(q_step, k_cache, w, k_offsets, lens, max_len, k_top, q_scale=
     args = _decode_marshal(q_step, k_cache, w, q_scale, k_scale, k_offsets, lens, max_len, k_top, scores_out,
                            topk_out, workspace, flags, stream)
     _check(lib().idxc_indexer_decode(*args), "idxc_indexer_decode")
+
+
+def indexer_decode_noalloc(q_step, k_cache, w, k_offsets, lens, max_len, k_top, topk_out, q_scale=None, k_scale=None,
+                           flags=0, stream=None):
+    """idxc_indexer_decode_noalloc: the decode step with the score scratch kept in an array
+    built into the library, for hosts that cannot hand over (or allocate) a workspace. The
+    step's scores, B * round_up(max_len, 32) * 4 bytes, must fit NOALLOC_SCRATCH_BYTES;
+    calls that may overlap on the GPU share that array and race."""
+    a = _decode_marshal(q_step, k_cache, w, q_scale, k_scale, k_offsets, lens, max_len, k_top, None, topk_out,
+                        None, flags, stream)
+    # same leading arguments as idxc_indexer_decode, without scores_out/ld and workspace/size
+    args = a[:14] + [a[16], a[19], a[20]]
+    _check(lib().idxc_indexer_decode_noalloc(*args), "idxc_indexer_decode_noalloc")
 
 
 def topk_rows(scores, k_top, topk_out, first_len=0, len_step=0, lens=None, stream=None):
