@@ -276,6 +276,8 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the decode and schedule sections")
     ap.add_argument("--schedule-layers", type=int, default=8)
     ap.add_argument("--schedule-L", type=int, default=32768)
+    ap.add_argument("--L", type=int, default=0, help="override the workload's sequence length (small profiling cases)")
+    ap.add_argument("--only-decode", action="store_true", help="run only the decode section (profiling)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -295,7 +297,13 @@ def main():
     idxc.lib()
     peaks = load_peaks()
 
-    c = synth.CONFIGS[args.workload]
+    if args.only_decode:
+        print(json.dumps({"decode": time_decode(idxc, synth, dev, peaks, steps=max(args.steps, 1), warmup=args.warmup)}),
+              flush=True)
+        return
+    c = dict(synth.CONFIGS[args.workload])
+    if args.L:
+        c["L"] = args.L
     L, H, d, k_top = c["L"], c["H"], c["d"], c["k_top"]
     # independent problem per rank (weak scaling): same shape, rank-specific seed
     inp = synth.prefill_inputs(L, H, d, seed=c["seed"] + 1000 * rank, device=dev, fp8=c["fp8"], clustered=c["clustered"])
