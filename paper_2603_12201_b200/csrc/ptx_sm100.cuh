@@ -138,6 +138,19 @@ __device__ __forceinline__ void tmem_ld_32x32b_x16(uint32_t taddr, uint32_t (&r)
         : "r"(taddr)
         : "memory");
 }
+// 16 lanes x 32 consecutive fp32 columns -> 16 registers per thread. With j = lane % 4 and
+// g = lane / 4, register 4i+e (e = 0, 1) holds (TMEM lane g, column 8i + 2j + e) and register
+// 4i+2+e holds (TMEM lane g + 8, same column), for i = 0..3 (the m16n8 accumulator fragment,
+// repeated along the columns). The lane field of taddr selects the first of the 16 lanes.
+__device__ __forceinline__ void tmem_ld_16x256b_x4(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
 // Wait for this thread's outstanding TMEM loads. The loaded registers are passed through
 // as in/out operands so that no use of them can be scheduled ahead of the wait.
 __device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {

@@ -3,9 +3,9 @@
 // Score (Sec. 2.1): I[t,s] = sum_h w[t,h] * max(q[t,h,:] . k[s,:], 0), s <= t.
 // The dot products are one dense contraction [keys, d] x [d, (query, head)]. It is laid
 // out with KEYS ON THE MMA's M axis (TMEM lanes) and (query, head) ON N (TMEM columns):
-// an epilogue thread then owns one key and walks the heads of a query along its own
-// TMEM lane, so the gate, the w-weighted head sum and the final score are plain register
-// arithmetic with w broadcast from shared memory -- no cross-thread reduction.
+// an epilogue thread then owns a few keys and a quarter of the (query, head) columns, so
+// the gate and the w-weighted head sum are register arithmetic with w held in registers,
+// finished by a two-step shuffle across the four threads that share a key.
 //
 // Prefill kernel (persistent, one CTA per SM, warp-specialised):
 //   warp 0      TMA producer: a block of 2*256/H queries (two 256-column B tiles) is loaded
@@ -13,7 +13,8 @@
 //               through a ring of stages. Per-CTA loads only (no multicast).
 //   warp 1      MMA issuer: per key tile, one 128 x 256 x d UMMA chain into each of the two
 //               256-column TMEM accumulators, so accumulator A is drained while B is filled.
-//   warps 4-11  epilogue: tcgen05.ld, ReLU, w-FMA, causal predicate, coalesced score store.
+//   warps 4-11  epilogue: tcgen05.ld (16x256b), ReLU, FMA with w held in registers, two shuffles per
+//               score to join the four threads of a key, causal predicate, coalesced score store.
 // Causal structure: a work item only visits key tiles up to its last query's position;
 // items are handed out longest first in a boustrophedon order over the CTAs.
 //
@@ -39,9 +40,8 @@ struct PrefillCfg {
     static constexpr int kStages = NKH == 2 ? 2 : 4;
     static constexpr int kQBytes = 2 * NKH * kQRegionBytes;
     static constexpr int kKBytes = kStages * NKH * kKRegionBytes;
-    static constexpr int kWBytes = kNumEpilogueWarps * 256 * 4;
     static constexpr int kBarBytes = 256;
-    static constexpr int kSmemBytes = kQBytes + kKBytes + kWBytes + kBarBytes + 1024;   // + alignment slack
+    static constexpr int kSmemBytes = kQBytes + kKBytes + kBarBytes + 1024;   // + alignment slack
 };
 
 struct PrefillParams {
@@ -77,8 +77,7 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint8_t* q_smem = smem;                                   // [2][NKH][256 x 128 B]
     uint8_t* k_smem = q_smem + Cfg::kQBytes;                  // [kStages][NKH][128 x 128 B]
-    float* w_smem = reinterpret_cast<float*>(k_smem + Cfg::kKBytes);   // [8 warps][256]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(w_smem) + Cfg::kWBytes);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(k_smem + Cfg::kKBytes);
     // barrier map
     const uint32_t bar_q_full = smem_u32(bars + 0);           // [2]
     const uint32_t bar_q_empty = smem_u32(bars + 2);          // [2]
@@ -212,12 +211,18 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
         }
     } else if (warp >= kEpilogueWarp0) {
         // ---------------------------------------------------------------- epilogue
+        // TMEM is read with the 16x256b shape: a thread owns 4 keys (TMEM lanes g, g+8, g+16, g+24 of
+        // its warp's lane quarter, g = lane/4) and the columns 8i + 2j + {0,1} (j = lane%4) of every
+        // 8-column group. Its share of w (64 values per work item) therefore lives in registers and
+        // the gate/FMA loop issues no shared-memory loads; the four threads of a group add their
+        // partial head sums with two shuffles per score at the end.
         constexpr int QPW = 128 / H;                 // queries per warp per accumulator
+        constexpr int ES = H >= 32 ? 2 : 1;          // independent partial sums per (key, query)
         const int ew = warp - kEpilogueWarp0;
         const int quarter = warp & 3;                // TMEM lane quarter this warp may read
         const int colhalf = ew >> 2;                 // which 128 columns of the accumulator
-        const int key_in_tile = quarter * 32 + lane;
-        float* my_w = w_smem + ew * 256;             // [half][128]: w (times q_scale) of this warp's queries
+        const int j = lane & 3, g = lane >> 2;
+        const int key_written = quarter * 32 + g + 8 * j;    // the key (of the thread's four) this thread stores
         uint32_t acc_phase[2] = {0u, 0u};
         bool ok = true;
         for (int64_t rho = 0; ok; ++rho) {
@@ -225,24 +230,27 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
             if (item < 0) break;
             const int nkt = key_tiles_of_item(item);
             const int64_t row_base = item * QB;
-            __syncwarp();
+            float wreg[2][16][2];
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
-                // 128 consecutive floats of w: rows row_base + half*QPA + colhalf*QPW .. +QPW-1
-                const int64_t row = row_base + half * QPA + colhalf * QPW + (lane * 4) / H;
-                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (row < p.n_rows) {
-                    v = __ldg(reinterpret_cast<const float4*>(p.w + row * H + (lane * 4) % H));
-                    if constexpr (FP8) {
-                        const float qs = __ldg(p.q_scale + row);
-                        v.x *= qs; v.y *= qs; v.z *= qs; v.w *= qs;
+#pragma unroll
+                for (int grp = 0; grp < 16; ++grp) {
+                    const int col = 8 * grp + 2 * j;                       // column within this warp's 128
+                    const int64_t row = row_base + half * QPA + colhalf * QPW + (8 * grp) / H;
+                    float2 v = make_float2(0.f, 0.f);
+                    if (row < p.n_rows) {
+                        v = __ldg(reinterpret_cast<const float2*>(p.w + row * H + col % H));
+                        if constexpr (FP8) {
+                            const float qs = __ldg(p.q_scale + row);
+                            v.x *= qs; v.y *= qs;
+                        }
                     }
+                    wreg[half][grp][0] = v.x;
+                    wreg[half][grp][1] = v.y;
                 }
-                reinterpret_cast<float4*>(my_w + half * 128)[lane] = v;
             }
-            __syncwarp();
             for (int kt = 0; kt < nkt && ok; ++kt) {
-                const int64_t s = static_cast<int64_t>(kt) * kTileKeys + key_in_tile;
+                const int64_t s = static_cast<int64_t>(kt) * kTileKeys + key_written;
                 float ksc = 1.f;
                 if constexpr (FP8) ksc = s < p.k_rows ? __ldg(p.k_scale + s) : 0.f;
 #pragma unroll
@@ -253,29 +261,38 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
                     tcgen05_fence_after_sync();
                     const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                            static_cast<uint32_t>(half * kTileCols + colhalf * 128);
-                    const float4* w4 = reinterpret_cast<const float4*>(my_w + half * 128);
-                    float acc[QPW];
+                    float acc[4][QPW][ES];
 #pragma unroll
-                    for (int i = 0; i < QPW; ++i) acc[i] = 0.f;
-                    uint32_t ra[32], rb[32];
-                    tmem_ld_32x32b_x32(taddr, ra);
+                    for (int r = 0; r < 4; ++r)
+#pragma unroll
+                        for (int i = 0; i < QPW; ++i)
+#pragma unroll
+                            for (int e = 0; e < ES; ++e) acc[r][i][e] = 0.f;
+                    uint32_t ra[16], rb[16];
+                    tmem_ld_16x256b_x4(taddr, ra);
                     tmem_ld_wait(ra);
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {          // 4 chunks of 32 columns
-                        uint32_t (&cur)[32] = (c & 1) ? rb : ra;
-                        uint32_t (&nxt)[32] = (c & 1) ? ra : rb;
-                        if (c + 1 < 4) tmem_ld_32x32b_x32(taddr + (c + 1) * 32, nxt);
+                    for (int n = 0; n < 8; ++n) {          // n = lane half (16 TMEM lanes) * 4 + 32-column chunk
+                        uint32_t (&cur)[16] = (n & 1) ? rb : ra;
+                        uint32_t (&nxt)[16] = (n & 1) ? ra : rb;
+                        if (n + 1 < 8)
+                            tmem_ld_16x256b_x4(taddr + (static_cast<uint32_t>(((n + 1) >> 2) * 16) << 16) + ((n + 1) & 3) * 32, nxt);
+                        const int lh = n >> 2, c = n & 3;
 #pragma unroll
-                        for (int j4 = 0; j4 < 8; ++j4) {
-                            const float4 wv = w4[c * 8 + j4];
-                            const int col = c * 32 + j4 * 4;        // column within this warp's 128
-                            float& a = acc[col / H];                // 4 consecutive columns share a query (H % 4 == 0)
-                            a = fmaf(fmaxf(__uint_as_float(cur[j4 * 4 + 0]), 0.f), wv.x, a);
-                            a = fmaf(fmaxf(__uint_as_float(cur[j4 * 4 + 1]), 0.f), wv.y, a);
-                            a = fmaf(fmaxf(__uint_as_float(cur[j4 * 4 + 2]), 0.f), wv.z, a);
-                            a = fmaf(fmaxf(__uint_as_float(cur[j4 * 4 + 3]), 0.f), wv.w, a);
+                        for (int i = 0; i < 4; ++i) {
+                            const int grp = 4 * c + i;
+                            const int qi = (8 * grp) / H;
+                            const float w0 = wreg[half][grp][0], w1 = wreg[half][grp][1];
+                            float& a0 = acc[2 * lh][qi][0];
+                            float& a1 = acc[2 * lh][qi][ES - 1];
+                            float& b0 = acc[2 * lh + 1][qi][0];
+                            float& b1 = acc[2 * lh + 1][qi][ES - 1];
+                            a0 = fmaf(fmaxf(__uint_as_float(cur[4 * i + 0]), 0.f), w0, a0);
+                            a1 = fmaf(fmaxf(__uint_as_float(cur[4 * i + 1]), 0.f), w1, a1);
+                            b0 = fmaf(fmaxf(__uint_as_float(cur[4 * i + 2]), 0.f), w0, b0);
+                            b1 = fmaf(fmaxf(__uint_as_float(cur[4 * i + 3]), 0.f), w1, b1);
                         }
-                        if (c + 1 < 4) tmem_ld_wait(nxt);
+                        if (n + 1 < 8) tmem_ld_wait(nxt);
                     }
                     // this warp's TMEM reads of the accumulator are complete
                     tcgen05_fence_before_sync();
@@ -283,12 +300,20 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
                     if (lane == 0) mbar_arrive(bar_acc_empty + 8 * half);
 #pragma unroll
                     for (int i = 0; i < QPW; ++i) {
+                        float mine = 0.f;
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) {
+                            float v = acc[r][i][0];
+                            if constexpr (ES == 2) v += acc[r][i][1];
+                            v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
+                            v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
+                            if (r == j) mine = v;                      // thread j of the group stores key g + 8j
+                        }
                         const int64_t row = row_base + half * QPA + colhalf * QPW + i;
                         const int64_t t = p.q_begin + row;
                         if (row < p.n_rows && s <= t) {
-                            float val = acc[i];
-                            if constexpr (FP8) val *= ksc;
-                            p.scores[row * p.ld + s] = val;
+                            if constexpr (FP8) mine *= ksc;
+                            p.scores[row * p.ld + s] = mine;
                         }
                     }
                 }
