@@ -1,49 +1,48 @@
 // Row-wise top-k select (Sec. 3 "Notation": T_t = Top-k(I_t)).
 //
-// One 512-thread CTA per row; each of its 16 warps owns one contiguous segment of the row.
-// The k-th largest score is found exactly by a radix select on order-preserving 32-bit keys
-// (12 + 10 + 10 bits, most significant first), in two sweeps over the row:
+// One CTA per row, many rows in flight per SM (256 threads and <= 48 registers per thread when
+// there are many rows; 512 threads when there are only a few long rows, as in decode). Each warp
+// owns one contiguous segment of the row. Scores are compared through order-preserving 32-bit
+// keys (larger score <=> larger key, -0 == +0); the k-th largest is found exactly by a radix
+// select, 12 + 10 + 10 key bits, most significant first:
 //   sweep 1 (the HBM read)  4096-bin shared-memory histogram of the top 12 key bits; a suffix
-//                           scan finds the threshold bucket b1 holding the k-th largest score;
-//   sweep 2 (L2)            scores above bucket b1 are certainly selected: their positions are
-//                           marked in a shared-memory selection map (4 flag bits per byte, one
-//                           byte per 128-bit load). Scores inside bucket b1 (typically < 1 % of the
-//                           row) are kept with their index; digits 2 and 3 run on those only and
-//                           give the exact threshold T, after which the kept scores above T, and
-//                           the lowest-index ones equal to T until k are reached, are marked too.
-//   emission                a block-wide prefix popcount over the map ranks every marked position,
-//                           so the indices come out ascending, with a deterministic tie-break and no
-//                           atomics on the output.
-// Sweep 2 compares floats against the bucket bounds, which orders exactly like the keys
-// (-0 == +0). If the threshold bucket holds more scores than the shared buffer (many near-equal
-// scores, e.g. a constant row), or the row is longer than the selection map, the remaining digits
-// are histogrammed over the whole row and the emission uses block-wide prefix sums over the row
-// instead; same result, slower.
+//                           scan finds the threshold bucket b1 holding the k-th largest score.
+//   sweep 2 (L2)            scores above bucket b1 are certainly selected, scores inside it
+//                           (typically < 2 % of the row) are candidates: both are flagged in a
+//                           shared-memory map (one byte per 128-bit load: low nibble "selected",
+//                           high nibble "candidate").
+//   candidates              gathered with key and position by walking the high nibbles (slots by
+//                           prefix popcount, no atomics); digits 2 and 3 on those only give the
+//                           exact threshold T; candidates above T, and the lowest-position ones
+//                           equal to T until k are reached, are flagged as selected.
+//   emission                a block-wide prefix popcount over the low nibbles ranks every selected
+//                           position: ascending indices, deterministic tie-break, no atomics on
+//                           the output.
+// Sweep 2 compares floats against the bucket bounds, which orders exactly like the keys. If the
+// threshold bucket holds more scores than the candidate buffer (many near-equal scores, e.g. a
+// constant row), or the row is longer than the map, digits 2 and 3 are histogrammed over the whole
+// row and the emission uses block-wide prefix sums over the row instead; same result, slower.
 #include "kernels.h"
 
 namespace idxc {
 namespace {
 
-constexpr int TK_THREADS = 512;
-constexpr int TK_WARPS = TK_THREADS / 32;
-constexpr int TK_BINS1 = 4096;   // top 12 bits
-constexpr int TK_BINS23 = 1024;  // next 10 and last 10 bits
-constexpr int TK_CAP = 4096;     // candidate keys kept in shared memory
-constexpr int TK_UNROLL = 8;     // 128-bit loads in flight per lane in each sweep
-
-struct TopkSmem {
-    uint32_t hist[TK_BINS1];
-    uint32_t warp_sums[2][TK_WARPS];
-    uint32_t sel_bucket;
-    uint32_t sel_above;
-    uint32_t cand_count;
-};
-// Dynamic shared memory: cand_low[TK_CAP] (low 20 key bits of the kept scores), cand_idx[TK_CAP]
-// (their positions), then the selection map (one byte per 4 scores).
-constexpr int TK_DYN_FIXED_BYTES = 2 * TK_CAP * 4;
+constexpr int TK_BINS1 = 4096;   // top 12 key bits
+constexpr int TK_BINS23 = 1024;  // 10-bit digits
+// The candidate buffers live in the upper three quarters of the 4096-bin histogram, which is
+// only needed as a whole until the threshold bucket is known: 1536 keys + 1536 positions.
+constexpr int TK_CAP = (TK_BINS1 - TK_BINS23) / 2;
+constexpr int TK_UNROLL = 4;     // 128-bit loads in flight per lane in a sweep
 constexpr int TK_MAP_MAX_BYTES = 128 * 1024;      // rows up to 524288 scores use the map
 
-// Larger float <=> larger key; -0 and +0 share a key.
+template <int WARPS>
+struct TopkSmem {
+    uint32_t hist[TK_BINS1];
+    uint32_t warp_sums[2][WARPS];
+    uint32_t sel_bucket;
+    uint32_t sel_above;
+};
+
 __device__ __forceinline__ uint32_t score_key(float x) {
     uint32_t u = __float_as_uint(x);
     if ((u << 1) == 0u) u = 0u;
@@ -60,7 +59,8 @@ __device__ __forceinline__ uint32_t score_digit1(float x) {
 
 // Exclusive prefix sum of `v` over the block in thread order; `total` = block sum.
 // `slot` alternates between calls so one barrier per call is enough.
-__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, TopkSmem& sm, int& slot, uint32_t& total) {
+template <int WARPS>
+__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, TopkSmem<WARPS>& sm, int& slot, uint32_t& total) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     uint32_t inc = v;
 #pragma unroll
@@ -70,25 +70,25 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, TopkSmem& sm, in
     }
     if (lane == 31) sm.warp_sums[slot][wid] = inc;
     __syncthreads();
-    uint32_t ws = lane < TK_WARPS ? sm.warp_sums[slot][lane] : 0u;
+    uint32_t ws = lane < WARPS ? sm.warp_sums[slot][lane] : 0u;
     uint32_t winc = ws;
 #pragma unroll
-    for (int o = 1; o < TK_WARPS; o <<= 1) {
+    for (int o = 1; o < WARPS; o <<= 1) {
         uint32_t y = __shfl_up_sync(0xFFFFFFFFu, winc, o);
         if (lane >= o) winc += y;
     }
-    uint32_t base = __shfl_sync(0xFFFFFFFFu, winc - ws, wid);
-    total = __shfl_sync(0xFFFFFFFFu, winc, TK_WARPS - 1);
+    const uint32_t base = __shfl_sync(0xFFFFFFFFu, winc - ws, wid);
+    total = __shfl_sync(0xFFFFFFFFu, winc, WARPS - 1);
     slot ^= 1;
     return base + inc - v;
 }
 
-// Calls f(score, index) for every element of the row, 128-bit loads where possible.
-template <typename F>
+// Calls f(score, index) for every element of the row (thread-strided), 128-bit loads.
+template <int THREADS, typename F>
 __device__ __forceinline__ void for_each_score(const float* __restrict__ src, int n, F f) {
     const int nvec = n >> 2;
     const float4* src4 = reinterpret_cast<const float4*>(src);
-    for (int v = threadIdx.x; v < nvec; v += TK_THREADS) {
+    for (int v = threadIdx.x; v < nvec; v += THREADS) {
         float4 x = __ldg(src4 + v);
         f(x.x, 4 * v);
         f(x.y, 4 * v + 1);
@@ -99,12 +99,11 @@ __device__ __forceinline__ void for_each_score(const float* __restrict__ src, in
     if (threadIdx.x < 4 && i < n) f(__ldg(src + i), i);
 }
 
-// Visits this warp's segment [seg_begin, seg_end) of a row of n scores in index order, 128
-// scores per step (lane l holds the 4 scores at step_base + 4l). U steps are loaded before any
-// is processed, so U 128-bit loads per lane are in flight. f(x, base) gets the lane's float4
-// and the index of its first score; scores at index >= n are padding (the row pitch is a
+// Visits this warp's segment [seg_begin, seg_end) of a row of n scores in index order, one
+// 128-score block per step (lane l holds the 4 scores at block_base + 4l). U steps are loaded
+// before any is processed, so U 128-bit loads per lane are in flight. f(x, base) gets the lane's
+// float4 and the index of its first score; scores at index >= n are padding (the row pitch is a
 // multiple of 4, so the load itself stays inside the row) and must be ignored by f.
-// The step condition is warp-uniform, so f may use warp collectives.
 template <int U, typename F>
 __device__ __forceinline__ void sweep_segment(const float* __restrict__ src, int n, int seg_begin, int seg_end, int lane, F f) {
     for (int cb = seg_begin; cb < seg_end; cb += 128 * U) {
@@ -112,7 +111,8 @@ __device__ __forceinline__ void sweep_segment(const float* __restrict__ src, int
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int base = cb + 128 * u + 4 * lane;
-            x[u] = base < n ? __ldg(reinterpret_cast<const float4*>(src + base)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            x[u] = (cb + 128 * u < seg_end && base < n) ? __ldg(reinterpret_cast<const float4*>(src + base))
+                                                        : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -124,16 +124,26 @@ __device__ __forceinline__ void sweep_segment(const float* __restrict__ src, int
 // hist[0..NB) holds counts per digit value. Finds the digit value `bucket` holding the
 // need-th largest element (1-based): above < need <= above + hist[bucket], where `above`
 // counts the elements in larger buckets. Requires sum(hist) >= need. Ends with a barrier.
-template <int NB>
-__device__ __forceinline__ void select_bucket(TopkSmem& sm, uint32_t need, int& slot, uint32_t& bucket, uint32_t& above) {
-    constexpr int PER = NB / TK_THREADS;
+template <int NB, int THREADS>
+__device__ __forceinline__ void select_bucket(TopkSmem<THREADS / 32>& sm, uint32_t need, int& slot, uint32_t& bucket,
+                                              uint32_t& above) {
+    constexpr int PER = NB / THREADS;
     uint32_t loc[PER];
     uint32_t sum = 0;
-    const int top = NB - 1 - static_cast<int>(threadIdx.x) * PER;   // my largest bin
+    const int top = NB - static_cast<int>(threadIdx.x) * PER;       // one past my largest bin
+    if constexpr (PER % 4 == 0) {
 #pragma unroll
-    for (int j = 0; j < PER; ++j) {
-        loc[j] = sm.hist[top - j];
-        sum += loc[j];
+        for (int j4 = 0; j4 < PER / 4; ++j4) {
+            const uint4 v = *reinterpret_cast<const uint4*>(&sm.hist[top - 4 * (j4 + 1)]);
+            loc[4 * j4 + 0] = v.w; loc[4 * j4 + 1] = v.z; loc[4 * j4 + 2] = v.y; loc[4 * j4 + 3] = v.x;   // descending bins
+            sum += v.x + v.y + v.z + v.w;
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            loc[j] = sm.hist[top - 1 - j];
+            sum += loc[j];
+        }
     }
     uint32_t total;
     uint32_t run = block_excl_scan(sum, sm, slot, total);
@@ -141,7 +151,7 @@ __device__ __forceinline__ void select_bucket(TopkSmem& sm, uint32_t need, int& 
 #pragma unroll
         for (int j = 0; j < PER; ++j) {
             if (need <= run + loc[j]) {
-                sm.sel_bucket = static_cast<uint32_t>(top - j);
+                sm.sel_bucket = static_cast<uint32_t>(top - 1 - j);
                 sm.sel_above = run;
                 break;
             }
@@ -153,21 +163,29 @@ __device__ __forceinline__ void select_bucket(TopkSmem& sm, uint32_t need, int& 
     above = sm.sel_above;
 }
 
-__device__ __forceinline__ void zero_hist(TopkSmem& sm, int nb) {
-    for (int i = threadIdx.x; i < nb; i += TK_THREADS) sm.hist[i] = 0u;
+template <int THREADS>
+__device__ __forceinline__ void zero_hist(TopkSmem<THREADS / 32>& sm, int nb) {
+    uint4* h4 = reinterpret_cast<uint4*>(sm.hist);
+    for (int i = threadIdx.x; i < nb / 4; i += THREADS) h4[i] = make_uint4(0u, 0u, 0u, 0u);
 }
 
-__global__ void __launch_bounds__(TK_THREADS, 2)
+// CAP_DYN = 0: the candidate buffers alias the histogram (TK_CAP entries). CAP_DYN > 0: they hold
+// CAP_DYN entries and live in dynamic shared memory behind the map (for launches with few, long rows,
+// whose threshold bucket holds more scores).
+template <int THREADS, int MIN_BLOCKS, int CAP_DYN>
+__global__ void __launch_bounds__(THREADS, MIN_BLOCKS)
 topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int64_t n_rows, int64_t first_len, int64_t len_step,
                  const int32_t* __restrict__ lens, int k_top, int32_t* __restrict__ out, int map_scores) {
-    __shared__ TopkSmem sm;
-    extern __shared__ uint32_t dyn[];
-    uint32_t* cand_low = dyn;
-    uint32_t* cand_idx = dyn + TK_CAP;
-    uint32_t* sel_map = dyn + 2 * TK_CAP;                        // map_scores / 16 words
+    constexpr int WARPS = THREADS / 32;
+    __shared__ __align__(16) TopkSmem<WARPS> sm;
+    extern __shared__ uint32_t sel_map[];                        // map_scores / 16 words
     uint8_t* sel_bytes = reinterpret_cast<uint8_t*>(sel_map);
+    constexpr int CAP = CAP_DYN > 0 ? CAP_DYN : TK_CAP;
+    uint32_t* cand_key = CAP_DYN > 0 ? sel_map + map_scores / 16 : sm.hist + TK_BINS23;   // aliased: valid once b1 is known
+    uint32_t* cand_idx = cand_key + CAP;
     int slot = 0;
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const uint32_t k = static_cast<uint32_t>(k_top);
     // longest rows first when lengths grow with the row number
     for (int64_t blk = blockIdx.x; blk < n_rows; blk += gridDim.x) {
         const int64_t row = n_rows - 1 - blk;
@@ -176,92 +194,101 @@ topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int64_t n_rows, i
         const int n = static_cast<int>(len);
         int32_t* out_row = out + row * static_cast<int64_t>(k_top);
         if (n <= k_top) {   // fewer candidates than k: all of them, then padding
-            for (int j = threadIdx.x; j < k_top; j += TK_THREADS) out_row[j] = j < n ? j : -1;
+            for (int j = threadIdx.x; j < k_top; j += THREADS) out_row[j] = j < n ? j : -1;
             continue;
         }
         const float* src = scores + row * ld;
         // this warp's segment: a multiple of 128 scores, so every lane loads aligned float4s
-        const int seg = (((n + TK_WARPS - 1) / TK_WARPS) + 127) & ~127;
+        const int seg = (((n + WARPS - 1) / WARPS) + 127) & ~127;
         const int seg_begin = wid * seg < n ? wid * seg : n;
         const int seg_end = seg_begin + seg < n ? seg_begin + seg : n;
 
-        // ---- sweep 1: histogram of digit 1 (key bits 31..20) over the whole row
-        __syncthreads();   // previous row's readers of sm are done
-        zero_hist(sm, TK_BINS1);
-        if (threadIdx.x == 0) sm.cand_count = 0u;
+        // ---- sweep 1: histogram of the top 12 key bits over the whole row
+        __syncthreads();   // earlier readers of sm are done
+        zero_hist<THREADS>(sm, TK_BINS1);
         __syncthreads();
         sweep_segment<TK_UNROLL>(src, n, seg_begin, seg_end, lane, [&](const float4& x, int base) {
-            if (base + 3 < n) {
-                atomicAdd(&sm.hist[score_digit1(x.x)], 1u);
-                atomicAdd(&sm.hist[score_digit1(x.y)], 1u);
-                atomicAdd(&sm.hist[score_digit1(x.z)], 1u);
-                atomicAdd(&sm.hist[score_digit1(x.w)], 1u);
-            } else {
-                const float xs[4] = {x.x, x.y, x.z, x.w};
+            const float xs[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (base + e < n) atomicAdd(&sm.hist[score_digit1(xs[e])], 1u);
-            }
+            for (int e = 0; e < 4; ++e)
+                if (base + e < n) atomicAdd(&sm.hist[score_digit1(xs[e])], 1u);
         });
         __syncthreads();
         uint32_t b1, above1;
-        select_bucket<TK_BINS1>(sm, static_cast<uint32_t>(k_top), slot, b1, above1);
+        select_bucket<TK_BINS1, THREADS>(sm, k, slot, b1, above1);
         const uint32_t c1 = sm.hist[b1];
-        uint32_t need = static_cast<uint32_t>(k_top) - above1;   // rank inside bucket b1, 1-based
-        uint32_t b2, above2, b3, above3;
-        __syncthreads();   // everyone has read hist[b1]
+        uint32_t need = k - above1;          // rank inside bucket b1, 1-based
+        uint32_t b2, b3, above;
+        __syncthreads();                     // everyone has read hist[b1]: the candidate buffers may now overwrite the bins
 
-        if (c1 <= static_cast<uint32_t>(TK_CAP) && n <= map_scores) {
-            // ---- sweep 2: mark the scores above bucket b1, keep the scores inside it
+        if (c1 <= static_cast<uint32_t>(CAP) && n <= map_scores) {
+            // ---- sweep 2: flag the scores above bucket b1 (selected) and inside it (candidates)
             const float lo = key_to_score(b1 << 20);                       // smallest score of bucket b1
             const bool has_above = b1 < TK_BINS1 - 1;
             const float hi = key_to_score(has_above ? ((b1 + 1) << 20) : 0xFFFFFFFFu);   // smallest score above it
             sweep_segment<TK_UNROLL>(src, n, seg_begin, seg_end, lane, [&](const float4& x4, int base) {
                 const float x[4] = {x4.x, x4.y, x4.z, x4.w};
-                uint32_t nib = 0;
+                uint32_t flags = 0;
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     if (base + e >= n || !(x[e] >= lo)) continue;
-                    if (has_above && x[e] >= hi) {
-                        nib |= 1u << e;
-                    } else {
-                        const uint32_t slot_i = atomicAdd(&sm.cand_count, 1u);
-                        if (slot_i < TK_CAP) {
-                            cand_low[slot_i] = score_key(x[e]) & 0xFFFFFu;
-                            cand_idx[slot_i] = static_cast<uint32_t>(base + e);
+                    flags |= (has_above && x[e] >= hi) ? (1u << e) : (16u << e);
+                }
+                sel_bytes[base >> 2] = static_cast<uint8_t>(flags);        // lanes past the end of the row write 0
+            });
+            __syncthreads();
+            // ---- gather the candidates (high nibbles) with their keys; slots by prefix popcount
+            const int words = (n + 15) >> 4;
+            const int wpt = (words + THREADS - 1) / THREADS;
+            const int w0 = static_cast<int>(threadIdx.x) * wpt < words ? static_cast<int>(threadIdx.x) * wpt : words;
+            const int w1 = w0 + wpt < words ? w0 + wpt : words;
+            {
+                uint32_t cnt = 0;
+                for (int w = w0; w < w1; ++w) cnt += __popc(sel_map[w] & 0xF0F0F0F0u);
+                uint32_t total;
+                uint32_t pos = block_excl_scan(cnt, sm, slot, total);
+                for (int w = w0; w < w1; ++w) {
+                    uint32_t m = sel_map[w] & 0xF0F0F0F0u;
+                    while (m) {
+                        const int b = __ffs(m) - 1;
+                        m &= m - 1;
+                        const int idx = 16 * w + 4 * (b >> 3) + (b & 7) - 4;
+                        if (pos < static_cast<uint32_t>(CAP)) {
+                            cand_key[pos] = score_key(__ldg(src + idx)) & 0xFFFFFu;
+                            cand_idx[pos] = static_cast<uint32_t>(idx);
                         }
+                        ++pos;
                     }
                 }
-                sel_bytes[base >> 2] = static_cast<uint8_t>(nib);      // lanes past the end of the row write 0
-            });
-            zero_hist(sm, TK_BINS23);
+            }
+            // ---- digits 2 and 3 on the candidates
+            zero_hist<THREADS>(sm, TK_BINS23);
             __syncthreads();
-            // ---- digits 2 and 3 on the kept scores
-            for (uint32_t i = threadIdx.x; i < c1; i += TK_THREADS) atomicAdd(&sm.hist[(cand_low[i] >> 10) & 1023u], 1u);
+            for (uint32_t i = threadIdx.x; i < c1; i += THREADS) atomicAdd(&sm.hist[cand_key[i] >> 10], 1u);
             __syncthreads();
-            select_bucket<TK_BINS23>(sm, need, slot, b2, above2);
-            need -= above2;
-            zero_hist(sm, TK_BINS23);
+            select_bucket<TK_BINS23, THREADS>(sm, need, slot, b2, above);
+            need -= above;
+            zero_hist<THREADS>(sm, TK_BINS23);
             __syncthreads();
-            for (uint32_t i = threadIdx.x; i < c1; i += TK_THREADS) {
-                const uint32_t c = cand_low[i];
+            for (uint32_t i = threadIdx.x; i < c1; i += THREADS) {
+                const uint32_t c = cand_key[i];
                 if ((c >> 10) == b2) atomicAdd(&sm.hist[c & 1023u], 1u);
             }
             __syncthreads();
-            select_bucket<TK_BINS23>(sm, need, slot, b3, above3);
-            need -= above3;
+            select_bucket<TK_BINS23, THREADS>(sm, need, slot, b3, above);
+            need -= above;
             const uint32_t t_low = (b2 << 10) | b3;              // low 20 key bits of the k-th largest score
             const uint32_t need_eq = need;                       // how many scores equal to it are taken (>= 1)
             const uint32_t m_eq = sm.hist[b3];                   // how many there are
-            // ---- mark the kept scores that are selected
-            for (uint32_t i = threadIdx.x; i < c1; i += TK_THREADS) {
-                const uint32_t low = cand_low[i];
-                bool take = low > t_low;
-                if (low == t_low) {
+            // ---- flag the selected candidates
+            for (uint32_t i = threadIdx.x; i < c1; i += THREADS) {
+                const uint32_t c = cand_key[i];
+                bool take = c > t_low;
+                if (c == t_low) {
                     take = true;
                     if (m_eq != need_eq) {                       // ties compete: the lowest positions win
                         uint32_t before = 0;
-                        for (uint32_t i2 = 0; i2 < c1; ++i2) before += (cand_low[i2] == t_low) & (cand_idx[i2] < cand_idx[i]);
+                        for (uint32_t i2 = 0; i2 < c1; ++i2) before += (cand_key[i2] == t_low) & (cand_idx[i2] < cand_idx[i]);
                         take = before < need_eq;
                     }
                 }
@@ -271,75 +298,70 @@ topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int64_t n_rows, i
                 }
             }
             __syncthreads();
-            // ---- emission: rank the marked positions by a prefix popcount over the map
-            const int words = (n + 15) >> 4;
-            const int wpt = (words + TK_THREADS - 1) / TK_THREADS;
-            const int w0 = static_cast<int>(threadIdx.x) * wpt < words ? static_cast<int>(threadIdx.x) * wpt : words;
-            const int w1 = w0 + wpt < words ? w0 + wpt : words;
+            // ---- emission: rank the selected positions by a prefix popcount over the low nibbles
             uint32_t cnt = 0;
-            for (int w = w0; w < w1; ++w) cnt += __popc(sel_map[w]);
+            for (int w = w0; w < w1; ++w) cnt += __popc(sel_map[w] & 0x0F0F0F0Fu);
             uint32_t total;
             uint32_t rank = block_excl_scan(cnt, sm, slot, total);
             for (int w = w0; w < w1; ++w) {
-                uint32_t m = sel_map[w];
+                uint32_t m = sel_map[w] & 0x0F0F0F0Fu;
                 while (m) {
                     const int b = __ffs(m) - 1;
                     m &= m - 1;
-                    if (rank < static_cast<uint32_t>(k_top)) out_row[rank] = 16 * w + 4 * (b >> 3) + (b & 7);
+                    if (rank < k) out_row[rank] = 16 * w + 4 * (b >> 3) + (b & 7);
                     ++rank;
                 }
             }
             continue;
         }
 
-        // ---- crowded threshold bucket: digits 2 and 3 over the row, block-scan emission
-        zero_hist(sm, TK_BINS23);
+        // ---- slow path: digits 2 and 3 over the whole row, then block-scan emission
+        zero_hist<THREADS>(sm, TK_BINS23);
         __syncthreads();
-        for_each_score(src, n, [&](float x, int) {
+        for_each_score<THREADS>(src, n, [&](float x, int) {
             const uint32_t key = score_key(x);
             if ((key >> 20) == b1) atomicAdd(&sm.hist[(key >> 10) & 1023u], 1u);
         });
         __syncthreads();
-        select_bucket<TK_BINS23>(sm, need, slot, b2, above2);
-        need -= above2;
-        zero_hist(sm, TK_BINS23);
+        select_bucket<TK_BINS23, THREADS>(sm, need, slot, b2, above);
+        need -= above;
+        zero_hist<THREADS>(sm, TK_BINS23);
         __syncthreads();
         const uint32_t p2 = (b1 << 10) | b2;
-        for_each_score(src, n, [&](float x, int) {
+        for_each_score<THREADS>(src, n, [&](float x, int) {
             const uint32_t key = score_key(x);
             if ((key >> 10) == p2) atomicAdd(&sm.hist[key & 1023u], 1u);
         });
         __syncthreads();
-        select_bucket<TK_BINS23>(sm, need, slot, b3, above3);
-        need -= above3;
-        const uint32_t T = (b1 << 20) | (b2 << 10) | b3;   // key of the k-th largest score
+        select_bucket<TK_BINS23, THREADS>(sm, need, slot, b3, above);
+        need -= above;
+        const uint32_t T = (p2 << 10) | b3;   // key of the k-th largest score
         const uint32_t need_eq = need;
-        const uint32_t n_gt = static_cast<uint32_t>(k_top) - need_eq;
+        const uint32_t n_gt = k - need_eq;
         uint32_t gt_base = 0, eq_base = 0;
-        for (int v0 = 0; 4 * v0 < n; v0 += TK_THREADS) {
+        for (int v0 = 0; 4 * v0 < n; v0 += THREADS) {
             const int base = 4 * (v0 + static_cast<int>(threadIdx.x));
             float x[4] = {0.f, 0.f, 0.f, 0.f};
-            bool valid[4];
             if (base < n) {
                 const float4 v4 = __ldg(reinterpret_cast<const float4*>(src + base));
                 x[0] = v4.x; x[1] = v4.y; x[2] = v4.z; x[3] = v4.w;
             }
-#pragma unroll
-            for (int e = 0; e < 4; ++e) valid[e] = base + e < n;
             uint32_t key[4];
             uint32_t cg = 0, ce = 0;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                key[e] = valid[e] ? score_key(x[e]) : 0u;
-                if (valid[e]) { cg += key[e] > T; ce += key[e] == T; }
+                const bool valid = base + e < n;
+                key[e] = valid ? score_key(x[e]) : 0u;
+                if (valid) { cg += key[e] > T; ce += key[e] == T; }
             }
-            uint32_t total;
-            const uint32_t excl = block_excl_scan(cg | (ce << 16), sm, slot, total);
-            uint32_t my_gt = gt_base + (excl & 0xFFFFu);
-            uint32_t my_eq = eq_base + (excl >> 16);
+            uint32_t tot_g, tot_e;
+            const uint32_t ex_g = block_excl_scan(cg, sm, slot, tot_g);
+            const uint32_t ex_e = block_excl_scan(ce, sm, slot, tot_e);
+            uint32_t my_gt = gt_base + ex_g;
+            uint32_t my_eq = eq_base + ex_e;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                if (!valid[e]) continue;
+                if (base + e >= n) continue;
                 if (key[e] > T) {
                     out_row[my_gt + (my_eq < need_eq ? my_eq : need_eq)] = base + e;
                     ++my_gt;
@@ -348,11 +370,27 @@ topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int64_t n_rows, i
                     ++my_eq;
                 }
             }
-            gt_base += total & 0xFFFFu;
-            eq_base += total >> 16;
+            gt_base += tot_g;
+            eq_base += tot_e;
             if (gt_base == n_gt && eq_base >= need_eq) break;   // all k found (uniform across the block)
         }
     }
+}
+
+template <int THREADS, int MIN_BLOCKS, int CAP_DYN>
+cudaError_t launch_instance(const float* scores, int64_t ld, int64_t n_rows, int64_t first_len, int64_t len_step,
+                            const int32_t* lens, int k_top, int32_t* out, int map_bytes, cudaStream_t stream) {
+    auto kern = topk_rows_kernel<THREADS, MIN_BLOCKS, CAP_DYN>;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TK_MAP_MAX_BYTES + 8 * CAP_DYN);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    const int64_t max_grid = 1 << 20;
+    const unsigned grid = static_cast<unsigned>(n_rows < max_grid ? n_rows : max_grid);
+    kern<<<grid, THREADS, map_bytes + 8 * CAP_DYN, stream>>>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, map_bytes * 4);
+    return cudaGetLastError();
 }
 
 }  // namespace
@@ -360,25 +398,16 @@ topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int64_t n_rows, i
 cudaError_t launch_topk_rows(const float* scores, int64_t ld, int64_t n_rows, int64_t first_len, int64_t len_step,
                              const int32_t* lens, int k_top, int32_t* out, cudaStream_t stream) {
     if (n_rows <= 0) return cudaSuccess;
-    // the selection map covers the longest row of this launch, rounded up to a whole sweep step
+    // the selection map covers the longest row of this launch, rounded up to a whole 128-score block
     int64_t longest = lens ? ld : first_len + (n_rows - 1) * len_step;
     if (longest > ld) longest = ld;
     if (longest < 0) longest = 0;
     int64_t map_bytes = (longest + 127) / 128 * 32;
     if (map_bytes > TK_MAP_MAX_BYTES) map_bytes = TK_MAP_MAX_BYTES;
-    const int dyn_bytes = TK_DYN_FIXED_BYTES + static_cast<int>(map_bytes);
-    static int attr_bytes = 0;
-    if (dyn_bytes > attr_bytes) {
-        cudaError_t e = cudaFuncSetAttribute(topk_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             TK_DYN_FIXED_BYTES + TK_MAP_MAX_BYTES);
-        if (e != cudaSuccess) return e;
-        attr_bytes = TK_DYN_FIXED_BYTES + TK_MAP_MAX_BYTES;
-    }
-    const int64_t max_grid = 1 << 20;
-    const unsigned grid = static_cast<unsigned>(n_rows < max_grid ? n_rows : max_grid);
-    topk_rows_kernel<<<grid, TK_THREADS, dyn_bytes, stream>>>(scores, ld, n_rows, first_len, len_step, lens, k_top, out,
-                                                              static_cast<int>(map_bytes * 4));
-    return cudaGetLastError();
+    // many rows: small CTAs, many per SM; few rows: more threads per row
+    if (n_rows >= 1024)
+        return launch_instance<256, 6, 0>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, static_cast<int>(map_bytes), stream);
+    return launch_instance<512, 2, 8192>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, static_cast<int>(map_bytes), stream);
 }
 
 }  // namespace idxc
