@@ -107,32 +107,6 @@ class ClockSampler:
                 "reasons": sorted(self.reasons)}
 
 
-def dist_setup(n_gpus):
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if world > 1:
-        import torch.distributed as dist
-        torch.cuda.set_device(local)
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    return rank, world, local
-
-
-def max_over_ranks(x: float, world: int, device) -> float:
-    if world == 1:
-        return x
-    import torch.distributed as dist
-    t = torch.tensor([x], dtype=torch.float64, device=device)
-    dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    return float(t.item())
-
-
-def barrier(world):
-    if world > 1:
-        import torch.distributed as dist
-        dist.barrier()
-
-
 def causal_pairs(L: int) -> int:
     return L * (L + 1) // 2
 
@@ -289,9 +263,12 @@ def main():
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the indexer has no CPU path (use --impl reference for the oracle)")
-    rank, world, local = dist_setup(args.gpus)
+    from paper_2603_12201_b200 import dist as pdist
+    _, _, local = pdist.env_rank_world()
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
+    rank, world = pdist.init("nccl", dev)
+    barrier, max_over_ranks = pdist.barrier, pdist.max_over_ranks
     from paper_2603_12201_b200 import binding as idxc
     from paper_2603_12201_b200 import synth
     idxc.lib()
@@ -306,7 +283,7 @@ def main():
         c["L"] = args.L
     L, H, d, k_top = c["L"], c["H"], c["d"], c["k_top"]
     # independent problem per rank (weak scaling): same shape, rank-specific seed
-    inp = synth.prefill_inputs(L, H, d, seed=c["seed"] + 1000 * rank, device=dev, fp8=c["fp8"], clustered=c["clustered"])
+    inp = synth.prefill_inputs(L, H, d, seed=pdist.rank_seed(c["seed"], rank), device=dev, fp8=c["fp8"], clustered=c["clustered"])
     ld = (L + 31) // 32 * 32
     scores = torch.empty((L, ld), dtype=torch.float32, device=dev)
     topk = torch.empty((L, k_top), dtype=torch.int32, device=dev)
@@ -341,7 +318,7 @@ def main():
     idxc.poll_device_status()
     total_ms = max_over_ranks(t_start.elapsed_time(t_end), world, dev)
     ms_per_step = total_ms / K
-    value = world * pairs * K / (total_ms * 1e-3) / 1e9
+    value = pdist.whole_job_rate(pairs, K, total_ms, world) / 1e9
     scorer_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
     topk_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
     flops = 2.0 * H * d * pairs
@@ -385,7 +362,7 @@ def main():
     e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
     h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hw))
     d2h = hout.numel() * hout.element_size()
-    e2e = {"value": world * pairs * args.e2e_steps / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+    e2e = {"value": pdist.whole_job_rate(pairs, args.e2e_steps, e2e_ms, world) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.e2e_steps, "steps": args.e2e_steps}
     assert torch.equal(hout.to(dev), topk)
 
@@ -422,9 +399,7 @@ def main():
                                              seed=3, reps=2)
     if rank == 0:
         print(json.dumps(line), flush=True)
-    if world > 1:
-        import torch.distributed as dist
-        dist.destroy_process_group()
+    pdist.shutdown(world)
 
 
 if __name__ == "__main__":
