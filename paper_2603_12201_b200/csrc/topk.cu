@@ -407,7 +407,7 @@ cudaError_t launch_topk_rows(const float* scores, int64_t ld, int64_t n_rows, in
     // many rows: small CTAs, many per SM; few rows: more threads per row
     if (n_rows >= 1024)
         return launch_instance<256, 6, 0>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, static_cast<int>(map_bytes), stream);
-    return launch_instance<512, 2, 8192>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, static_cast<int>(map_bytes), stream);
+    return launch_instance<1024, 1, 8192>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, static_cast<int>(map_bytes), stream);
 }
 
 }  // namespace idxc
