@@ -203,7 +203,8 @@ def time_decode(idxc, synth, dev, peaks, steps, warmup):
 
 
 def time_schedule(idxc, synth, dev, L, H, d, k_top, n_layers, every, seed, reps):
-    """1-in-`every` Full pattern vs all-Full on the same per-layer inputs (config-4 shape, fewer layers by default)."""
+    """1-in-`every` Full pattern vs all-Full on the same per-layer inputs (config-4 shape; N = 48 and
+    L = 65536 with --full, fewer and shorter layers by default)."""
     layers = [synth.prefill_inputs(L, H, d, seed=seed, device=dev, layer=l) for l in range(n_layers)]
     ws = idxc.alloc_workspace(idxc.prefill_workspace_bytes(L, L, H, d, k_top), dev)
     bufs = [torch.empty((L, k_top), dtype=torch.int32, device=dev) for _ in range(n_layers)]
@@ -232,9 +233,83 @@ def time_schedule(idxc, synth, dev, L, H, d, k_top, n_layers, every, seed, reps)
     t_sched, calls_sched = run(pat)
     t_full, calls_full = run("F" * n_layers)
     idxc.poll_device_status()
+    pairs = causal_pairs(L)
     return {"workload": f"cfg4-shaped: N={n_layers} layers, L={L}, H_I={H}, d_I={d}, k_top={k_top}, F every {every}",
             "ms_scheduled": t_sched, "ms_all_full": t_full, "ratio": t_full / t_sched,
-            "indexer_calls": [calls_sched, calls_full]}
+            "indexer_calls": [calls_sched, calls_full],
+            "gpairs_per_s_full_layers": pairs * calls_full / (t_full * 1e-3) / 1e9}
+
+
+def time_fp8_chunked(idxc, synth, dev, peaks, L, chunk, H, d, k_top, seed, decode_B):
+    """Config-5 shape: one Full layer of FP8 (e4m3 + per-token scales) chunked prefill, query chunks of
+    `chunk` rows against the full causal K, then one decode step at batch `decode_B` on caches of length L."""
+    inp = synth.prefill_inputs(L, H, d, seed=seed, device=dev, fp8=True)
+    topk = torch.empty((L, k_top), dtype=torch.int32, device=dev)
+    ws = idxc.alloc_workspace(idxc.prefill_workspace_bytes(chunk, L, H, d, k_top, idxc.FP8_E4M3), dev)
+    ld = (L + 31) // 32 * 32
+    scores = ws[: chunk * ld * 4].view(torch.float32).view(chunk, ld)
+
+    def layer(split):
+        t_sc = t_tk = 0.0
+        evs = []
+        for q0 in range(0, L, chunk):
+            sl = slice(q0, q0 + chunk)
+            if split:
+                e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+                e[0].record()
+                idxc.indexer_prefill(inp.q[sl], inp.k, inp.w[sl], k_top, inp.q_scale[sl], inp.k_scale, q_begin=q0,
+                                     scores_out=scores)
+                e[1].record()
+                idxc.topk_rows(scores, k_top, topk[sl], first_len=q0 + 1, len_step=1)
+                e[2].record()
+                evs.append(e)
+            else:
+                idxc.indexer_prefill(inp.q[sl], inp.k, inp.w[sl], k_top, inp.q_scale[sl], inp.k_scale, q_begin=q0,
+                                     topk_out=topk[sl], workspace=ws)
+        torch.cuda.synchronize()
+        for e in evs:
+            t_sc += e[0].elapsed_time(e[1])
+            t_tk += e[1].elapsed_time(e[2])
+        return t_sc, t_tk
+
+    layer(False)                                        # warm-up
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    layer(False)
+    e1.record()
+    torch.cuda.synchronize()
+    ms_layer = e0.elapsed_time(e1)
+    t_sc, t_tk = layer(True)
+    idxc.poll_device_status()
+    pairs = causal_pairs(L)
+    flops = 2.0 * H * d * pairs
+    out = {"workload": f"cfg5-shaped: L={L} in {L // chunk} chunks of {chunk}, e4m3 + per-token scales, H_I={H}, d_I={d}, "
+                       f"k_top={k_top}, one Full layer",
+           "ms_per_layer": ms_layer, "gpairs_per_s": pairs / (ms_layer * 1e-3) / 1e9,
+           "ms_scorer": t_sc, "ms_topk": t_tk, "scorer_tflops": flops / (t_sc * 1e-3) / 1e12,
+           "scorer_frac_of_2x_bf16_peak": flops / (t_sc * 1e-3) / 1e12 / (2 * peaks["bf16_tflops"]),
+           "fp8_peak_note": "no measured FP8 peak on this pool: 2 x measured bf16 burst peak (nominal ratio)"}
+    # decode step on caches of length L
+    x = synth.decode_inputs(decode_B, H, d, L, L, seed=seed, device=dev, layer=1, fp8=True, lens=[L] * decode_B)
+    x.k_cache[:L] = inp.k
+    x.k_scale[:L] = inp.k_scale
+    dtop = torch.empty((decode_B, k_top), dtype=torch.int32, device=dev)
+    dws = idxc.alloc_workspace(idxc.decode_workspace_bytes(decode_B, L, H, d, k_top, idxc.FP8_E4M3), dev)
+    times = []
+    for i in range(13):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        idxc.indexer_decode(x.q_step, x.k_cache, x.w, x.k_offsets, x.lens, L, k_top, x.q_scale, x.k_scale, topk_out=dtop,
+                            workspace=dws)
+        b.record()
+        torch.cuda.synchronize()
+        times.append(a.elapsed_time(b) * 1e3)
+    us = statistics.median(times[3:])
+    nbytes = decode_B * L * (d + 4)
+    out["decode"] = {"B": decode_B, "us_per_step": us, "bytes": nbytes,
+                     "frac_of_hbm": nbytes / (us * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                     "note": "138 MB of keys nearly fit the 126 MB L2; repeated steps re-read part of them from L2"}
+    return out
 
 
 def main():
@@ -250,6 +325,7 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the decode and schedule sections")
     ap.add_argument("--schedule-layers", type=int, default=8)
     ap.add_argument("--schedule-L", type=int, default=32768)
+    ap.add_argument("--full", action="store_true", help="extras at full size: config 4 with N=48, L=65536; config 5 with L=131072")
     ap.add_argument("--L", type=int, default=0, help="override the workload's sequence length (small profiling cases)")
     ap.add_argument("--only-decode", action="store_true", help="run only the decode section (profiling)")
     args = ap.parse_args()
@@ -395,8 +471,16 @@ def main():
             "rows_with_identical_index_set": f"{same}/{len(rows)}"}
         if not args.no_extras:
             line["decode"] = time_decode(idxc, synth, dev, peaks, steps=max(K, 10), warmup=W)
-            line["schedule"] = time_schedule(idxc, synth, dev, args.schedule_L, H, d, k_top, args.schedule_layers, 4,
-                                             seed=3, reps=2)
+            del hq, hk, hw, dq, dk, dw, inp, host
+            torch.cuda.empty_cache()
+            c4, c5 = synth.CONFIGS["cfg4"], synth.CONFIGS["cfg5"]
+            n_layers, sched_L = (c4["N"], c4["L"]) if args.full else (args.schedule_layers, args.schedule_L)
+            line["schedule"] = time_schedule(idxc, synth, dev, sched_L, c4["H"], c4["d"], c4["k_top"], n_layers, c4["every"],
+                                             seed=c4["seed"], reps=1 if args.full else 2)
+            torch.cuda.empty_cache()
+            fp8_L = c5["L"] if args.full else 32768
+            line["fp8_chunked"] = time_fp8_chunked(idxc, synth, dev, peaks, fp8_L, c5["chunk"], c5["H"], c5["d"], c5["k_top"],
+                                                   c5["seed"], c5["decode_B"])
     if rank == 0:
         print(json.dumps(line), flush=True)
     pdist.shutdown(world)
