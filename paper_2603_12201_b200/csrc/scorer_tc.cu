@@ -217,7 +217,6 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
         // the gate/FMA loop issues no shared-memory loads; the four threads of a group add their
         // partial head sums with two shuffles per score at the end.
         constexpr int QPW = 128 / H;                 // queries per warp per accumulator
-        constexpr int ES = H >= 32 ? 2 : 1;          // independent partial sums per (key, query)
         const int ew = warp - kEpilogueWarp0;
         const int quarter = warp & 3;                // TMEM lane quarter this warp may read
         const int colhalf = ew >> 2;                 // which 128 columns of the accumulator
@@ -230,7 +229,7 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
             if (item < 0) break;
             const int nkt = key_tiles_of_item(item);
             const int64_t row_base = item * QB;
-            float wreg[2][16][2];
+            uint64_t wreg[2][16];                      // (w of column 8g+2j, w of column 8g+2j+1), packed
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
 #pragma unroll
@@ -245,8 +244,7 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
                             v.x *= qs; v.y *= qs;
                         }
                     }
-                    wreg[half][grp][0] = v.x;
-                    wreg[half][grp][1] = v.y;
+                    wreg[half][grp] = pack_f32x2(v.x, v.y);
                 }
             }
             for (int kt = 0; kt < nkt && ok; ++kt) {
@@ -261,13 +259,12 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
                     tcgen05_fence_after_sync();
                     const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                            static_cast<uint32_t>(half * kTileCols + colhalf * 128);
-                    float acc[4][QPW][ES];
+                    // acc[r][i]: partial sums of (key slot r, query i) over this thread's even / odd columns
+                    uint64_t acc[4][QPW];
 #pragma unroll
                     for (int r = 0; r < 4; ++r)
 #pragma unroll
-                        for (int i = 0; i < QPW; ++i)
-#pragma unroll
-                            for (int e = 0; e < ES; ++e) acc[r][i][e] = 0.f;
+                        for (int i = 0; i < QPW; ++i) acc[r][i] = 0ull;
                     uint32_t ra[16], rb[16];
                     tmem_ld_16x256b_x4(taddr, ra);
                     tmem_ld_wait(ra);
@@ -282,15 +279,13 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
                         for (int i = 0; i < 4; ++i) {
                             const int grp = 4 * c + i;
                             const int qi = (8 * grp) / H;
-                            const float w0 = wreg[half][grp][0], w1 = wreg[half][grp][1];
-                            float& a0 = acc[2 * lh][qi][0];
-                            float& a1 = acc[2 * lh][qi][ES - 1];
-                            float& b0 = acc[2 * lh + 1][qi][0];
-                            float& b1 = acc[2 * lh + 1][qi][ES - 1];
-                            a0 = fmaf(fmaxf(__uint_as_float(cur[4 * i + 0]), 0.f), w0, a0);
-                            a1 = fmaf(fmaxf(__uint_as_float(cur[4 * i + 1]), 0.f), w1, a1);
-                            b0 = fmaf(fmaxf(__uint_as_float(cur[4 * i + 2]), 0.f), w0, b0);
-                            b1 = fmaf(fmaxf(__uint_as_float(cur[4 * i + 3]), 0.f), w1, b1);
+                            // gate, then one packed FMA per key slot: (even column, odd column) * (w_even, w_odd)
+                            const uint64_t xa = pack_f32x2(fmaxf(__uint_as_float(cur[4 * i + 0]), 0.f),
+                                                           fmaxf(__uint_as_float(cur[4 * i + 1]), 0.f));
+                            const uint64_t xb = pack_f32x2(fmaxf(__uint_as_float(cur[4 * i + 2]), 0.f),
+                                                           fmaxf(__uint_as_float(cur[4 * i + 3]), 0.f));
+                            acc[2 * lh][qi] = fma_f32x2(xa, wreg[half][grp], acc[2 * lh][qi]);
+                            acc[2 * lh + 1][qi] = fma_f32x2(xb, wreg[half][grp], acc[2 * lh + 1][qi]);
                         }
                         if (n + 1 < 8) tmem_ld_wait(nxt);
                     }
@@ -303,8 +298,9 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
                         float mine = 0.f;
 #pragma unroll
                         for (int r = 0; r < 4; ++r) {
-                            float v = acc[r][i][0];
-                            if constexpr (ES == 2) v += acc[r][i][1];
+                            float v, v_odd;
+                            unpack_f32x2(acc[r][i], v, v_odd);
+                            v += v_odd;
                             v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
                             v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
                             if (r == j) mine = v;                      // thread j of the group stores key g + 8j
