@@ -31,13 +31,21 @@ constexpr int kTileCols = 256;          // UMMA N (prefill)
 constexpr int kChunkBytes = 128;        // one swizzle row: 64 bf16 or 128 fp8 elements
 constexpr int kQRegionBytes = kTileCols * kChunkBytes;   // 32 KB
 constexpr int kKRegionBytes = kTileKeys * kChunkBytes;   // 16 KB
-constexpr int kPrefillThreads = 384;    // 12 warps
+// 8 epilogue warps measured faster than 16 on B200 (6.5 ms vs 6.9 ms on config 2): the kernel runs at the
+// board's power limit, and the extra warps cost more than the latency they hide.
+#ifndef IDXC_EPI_WARPS
+#define IDXC_EPI_WARPS 8
+#endif
 constexpr int kEpilogueWarp0 = 4;
-constexpr int kNumEpilogueWarps = 8;
+constexpr int kNumEpilogueWarps = IDXC_EPI_WARPS;       // 8 or 16: 2 or 4 per TMEM lane quarter
+constexpr int kPrefillThreads = (kEpilogueWarp0 + kNumEpilogueWarps) * 32;
+constexpr int kColsPerEpiWarp = kTileCols / (kNumEpilogueWarps / 4);   // 128 or 64 accumulator columns per warp
+constexpr int kGroupsPerEpiWarp = kColsPerEpiWarp / 8;               // 8-column groups per warp
+constexpr int kChunksPerEpiWarp = kColsPerEpiWarp / 32;              // 32-column TMEM loads per 16 lanes
 
 template <int NKH>
 struct PrefillCfg {
-    static constexpr int kStages = NKH == 2 ? 2 : 4;
+    static constexpr int kStages = NKH == 2 ? 3 : 4;
     static constexpr int kQBytes = 2 * NKH * kQRegionBytes;
     static constexpr int kKBytes = kStages * NKH * kKRegionBytes;
     static constexpr int kBarBytes = 256;
@@ -216,10 +224,11 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
         // 8-column group. Its share of w (64 values per work item) therefore lives in registers and
         // the gate/FMA loop issues no shared-memory loads; the four threads of a group add their
         // partial head sums with two shuffles per score at the end.
-        constexpr int QPW = 128 / H;                 // queries per warp per accumulator
+        constexpr int QPW = kColsPerEpiWarp / H;     // queries per warp per accumulator
+        static_assert(QPW >= 1, "an epilogue warp must cover at least one query");
         const int ew = warp - kEpilogueWarp0;
         const int quarter = warp & 3;                // TMEM lane quarter this warp may read
-        const int colhalf = ew >> 2;                 // which 128 columns of the accumulator
+        const int colhalf = ew >> 2;                 // which slice of kColsPerEpiWarp columns of the accumulator
         const int j = lane & 3, g = lane >> 2;
         const int key_written = quarter * 32 + g + 8 * j;    // the key (of the thread's four) this thread stores
         uint32_t acc_phase[2] = {0u, 0u};
@@ -229,12 +238,12 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
             if (item < 0) break;
             const int nkt = key_tiles_of_item(item);
             const int64_t row_base = item * QB;
-            uint64_t wreg[2][16];                      // (w of column 8g+2j, w of column 8g+2j+1), packed
+            uint64_t wreg[2][kGroupsPerEpiWarp];       // (w of column 8g+2j, w of column 8g+2j+1), packed
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
 #pragma unroll
-                for (int grp = 0; grp < 16; ++grp) {
-                    const int col = 8 * grp + 2 * j;                       // column within this warp's 128
+                for (int grp = 0; grp < kGroupsPerEpiWarp; ++grp) {
+                    const int col = 8 * grp + 2 * j;                       // column within this warp's slice
                     const int64_t row = row_base + half * QPA + colhalf * QPW + (8 * grp) / H;
                     float2 v = make_float2(0.f, 0.f);
                     if (row < p.n_rows) {
@@ -258,7 +267,7 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
                     acc_phase[half] ^= 1u;
                     tcgen05_fence_after_sync();
                     const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
-                                           static_cast<uint32_t>(half * kTileCols + colhalf * 128);
+                                           static_cast<uint32_t>(half * kTileCols + colhalf * kColsPerEpiWarp);
                     // acc[r][i]: partial sums of (key slot r, query i) over this thread's even / odd columns
                     uint64_t acc[4][QPW];
 #pragma unroll
@@ -268,13 +277,15 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
                     uint32_t ra[16], rb[16];
                     tmem_ld_16x256b_x4(taddr, ra);
                     tmem_ld_wait(ra);
+                    constexpr int NL = 2 * kChunksPerEpiWarp;
 #pragma unroll
-                    for (int n = 0; n < 8; ++n) {          // n = lane half (16 TMEM lanes) * 4 + 32-column chunk
+                    for (int n = 0; n < NL; ++n) {         // n = lane half (16 TMEM lanes) * chunks + 32-column chunk
                         uint32_t (&cur)[16] = (n & 1) ? rb : ra;
                         uint32_t (&nxt)[16] = (n & 1) ? ra : rb;
-                        if (n + 1 < 8)
-                            tmem_ld_16x256b_x4(taddr + (static_cast<uint32_t>(((n + 1) >> 2) * 16) << 16) + ((n + 1) & 3) * 32, nxt);
-                        const int lh = n >> 2, c = n & 3;
+                        if (n + 1 < NL)
+                            tmem_ld_16x256b_x4(taddr + (static_cast<uint32_t>(((n + 1) / kChunksPerEpiWarp) * 16) << 16) +
+                                                   ((n + 1) % kChunksPerEpiWarp) * 32, nxt);
+                        const int lh = n / kChunksPerEpiWarp, c = n % kChunksPerEpiWarp;
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
                             const int grp = 4 * c + i;
@@ -287,7 +298,7 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
                             acc[2 * lh][qi] = fma_f32x2(xa, wreg[half][grp], acc[2 * lh][qi]);
                             acc[2 * lh + 1][qi] = fma_f32x2(xb, wreg[half][grp], acc[2 * lh + 1][qi]);
                         }
-                        if (n + 1 < 8) tmem_ld_wait(nxt);
+                        if (n + 1 < NL) tmem_ld_wait(nxt);
                     }
                     // this warp's TMEM reads of the accumulator are complete
                     tcgen05_fence_before_sync();
