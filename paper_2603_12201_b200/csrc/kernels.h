@@ -14,6 +14,13 @@ cudaError_t launch_topk_rows(const float* scores, int64_t ld, int64_t n_rows, in
                              int64_t len_step, const int32_t* lens, int k_top, int32_t* out,
                              cudaStream_t stream);
 
+// Cluster variant for a few long rows (topk_cluster.cu): 8 CTAs per row exchanging through
+// distributed shared memory. `longest` = longest row of the launch.
+bool topk_cluster_applicable(int64_t n_rows, int64_t longest);
+cudaError_t launch_topk_rows_cluster(const float* scores, int64_t ld, int64_t n_rows, int64_t first_len,
+                                     int64_t len_step, const int32_t* lens, int k_top, int32_t* out,
+                                     int64_t longest, cudaStream_t stream);
+
 // Arguments shared by the scorers. A "row" is one query vector set [H, d].
 struct ScoreArgs {
     const void* q;          // [n_rows, H, d]
