@@ -31,9 +31,10 @@ import torch  # noqa: E402
 METRIC = "indexer+top-k Gpairs/s (prefill)"
 UNIT = "Gpairs/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum per scorer launch on this workload, from the
-# ncu capture summarised in profiles/ (None until a capture exists).
-SCORER_DRAM_TRAFFIC_BYTES = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the full-size ncu captures summarised
+# in profiles/score_prefill_tc_L8192.txt and profiles/score_decode_tc_cfg3.txt (None for other sizes).
+SCORER_DRAM_TRAFFIC_BYTES = {32768: 613146880 + 2114112000}
+DECODE_SCORER_DRAM_TRAFFIC_BYTES = 767080960 + 14429952
 
 
 def load_peaks():
@@ -196,7 +197,8 @@ def time_decode(idxc, synth, dev, peaks, steps, warmup):
         "us_per_step": us_total, "us_scorer": us_score, "us_topk": us_total - us_score,
         "k_cache_bytes": bytes_k,
         "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": gbs / peaks["hbm_gbs"], "traffic": None, "kernel": "score_decode_tc_kernel",
+                     "frac": gbs / peaks["hbm_gbs"], "traffic": DECODE_SCORER_DRAM_TRAFFIC_BYTES,
+                     "algorithmic_bytes": bytes_k, "kernel": "score_decode_tc_kernel",
                      "of": peaks["source"]},
         "frac_step_vs_hbm": bytes_k / (us_total * 1e-6) / 1e9 / peaks["hbm_gbs"],
     }
@@ -401,7 +403,9 @@ def main():
     achieved_tf = flops / (scorer_ms * 1e-3) / 1e12
     roofline = {
         "bound": "tensor", "achieved": achieved_tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-        "frac": achieved_tf / peaks["bf16_tflops"], "traffic": SCORER_DRAM_TRAFFIC_BYTES,
+        "frac": achieved_tf / peaks["bf16_tflops"],
+        "traffic": SCORER_DRAM_TRAFFIC_BYTES.get(L) if args.workload == "cfg2" else None,
+        "algorithmic_bytes": inp.q.numel() * inp.q.element_size() + inp.k.numel() * inp.k.element_size() + inp.w.numel() * 4 + 4 * pairs,
         "kernel": "score_prefill_tc_kernel", "ms_per_launch": scorer_ms, "of": peaks["source"] + " burst peak",
         "frac_of_sustained": achieved_tf / peaks["bf16_tflops_sustained"],
         "algorithmic_flops_per_launch": flops,
