@@ -108,6 +108,11 @@ class ClockSampler:
                 "reasons": sorted(self.reasons)}
 
 
+def workload_name(name: str, c: dict) -> str:
+    return (f"{name}: single-layer indexer prefill, batch 1, L={c['L']}, H_I={c['H']}, d_I={c['d']}, k_top={c['k_top']}, "
+            f"causal, seed {c['seed']}" + (", clustered keys" if c["clustered"] else ""))
+
+
 def causal_pairs(L: int) -> int:
     return L * (L + 1) // 2
 
@@ -157,7 +162,7 @@ def run_reference(args, rank):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * total_sec / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{args.workload}: prefill L={L} H_I={H} d_I={d} k_top={k_top} (bounded row sample)"},
+        "config": {"workload": workload_name(args.workload, c)},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -450,8 +455,7 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "fp8_e4m3" if c["fp8"] else "bf16", "data": "synthetic",
-        "config": {"workload": f"{args.workload}: single-layer indexer prefill, batch 1, L={L}, H_I={H}, d_I={d}, "
-                               f"k_top={k_top}, causal, seed {c['seed']}" + (", clustered keys" if c["clustered"] else ""),
+        "config": {"workload": workload_name(args.workload, c),
                    "parallelism": f"independent problem per GPU x{world}",
                    "l2": f"inputs {(inp.q.numel() * inp.q.element_size()) >> 20} MiB and scores "
                          f"{scores.numel() * 4 >> 20} MiB per step exceed the 126 MB L2; no flush needed"},
