@@ -328,7 +328,7 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2"])
     ap.add_argument("--ref-rows", type=int, default=128, help="rows per step of the reference (oracle) arm")
     ap.add_argument("--cpu-rows", type=int, default=1024, help="rows of the cpu_baseline sample")
-    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--e2e-steps", type=int, default=8)
     ap.add_argument("--no-extras", action="store_true", help="skip the decode and schedule sections")
     ap.add_argument("--schedule-layers", type=int, default=8)
     ap.add_argument("--schedule-L", type=int, default=32768)
@@ -420,36 +420,68 @@ def main():
                         "frac": (4.0 * pairs + 4.0 * L * k_top) / (topk_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
     }
 
-    # ---- e2e: host buffers, H2D of the step's inputs and D2H of its result inside the timed region
+    # ---- e2e: host buffers; every step copies its inputs H2D (pinned) and its result D2H inside the timed
+    # region. Steps are software-pipelined over three streams with double-buffered device inputs and outputs
+    # (copy-in of step i+1 and copy-out of step i-1 overlap the kernels of step i), as a serving loop would.
     hq = torch.empty(inp.q.shape, dtype=inp.q.dtype, pin_memory=True).copy_(inp.q)
     hk = torch.empty(inp.k.shape, dtype=inp.k.dtype, pin_memory=True).copy_(inp.k)
     hw = torch.empty(inp.w.shape, dtype=inp.w.dtype, pin_memory=True).copy_(inp.w)
-    hout = torch.empty(topk.shape, dtype=topk.dtype, pin_memory=True)
-    dq, dk, dw = torch.empty_like(inp.q), torch.empty_like(inp.k), torch.empty_like(inp.w)
+    hout = [torch.empty(topk.shape, dtype=topk.dtype, pin_memory=True) for _ in range(2)]
+    dq = [torch.empty_like(inp.q) for _ in range(2)]
+    dk = [torch.empty_like(inp.k) for _ in range(2)]
+    dw = [torch.empty_like(inp.w) for _ in range(2)]
+    dtop = [topk, torch.empty_like(topk)]
     ws = scores.view(torch.uint8).view(-1)
+    s_in, s_run, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev), torch.cuda.Stream(dev)
 
-    def e2e_step():
-        dq.copy_(hq, non_blocking=True)
-        dk.copy_(hk, non_blocking=True)
-        dw.copy_(hw, non_blocking=True)
-        idxc.indexer_prefill(dq, dk, dw, k_top, topk_out=topk, workspace=ws)    # the call a user makes
-        hout.copy_(topk, non_blocking=True)
+    def e2e_run(n_steps):
+        in_done = [None, None]      # event: inputs of the step using buffer b have landed
+        run_done = [None, None]     # event: kernels of the step using buffer b have finished
+        out_done = [None, None]     # event: result of the step using buffer b has been copied out
+        for i in range(n_steps):
+            b = i & 1
+            with torch.cuda.stream(s_in):
+                if run_done[b] is not None:
+                    s_in.wait_event(run_done[b])             # the kernels that read this input buffer are done
+                dq[b].copy_(hq, non_blocking=True)
+                dk[b].copy_(hk, non_blocking=True)
+                dw[b].copy_(hw, non_blocking=True)
+                in_done[b] = s_in.record_event()
+            with torch.cuda.stream(s_run):
+                s_run.wait_event(in_done[b])
+                if out_done[b] is not None:
+                    s_run.wait_event(out_done[b])            # the previous result in this buffer has left
+                idxc.indexer_prefill(dq[b], dk[b], dw[b], k_top, topk_out=dtop[b], workspace=ws, stream=s_run)   # the user's call
+                run_done[b] = s_run.record_event()
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(run_done[b])
+                hout[b].copy_(dtop[b], non_blocking=True)
+                out_done[b] = s_out.record_event()
+        for st in (s_in, s_run, s_out):
+            torch.cuda.current_stream().wait_stream(st)
 
-    e2e_step()
+    torch.cuda.synchronize()
+    e2e_run(2)
     torch.cuda.synchronize()
     barrier(world)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    for _ in range(args.e2e_steps):
-        e2e_step()
+    for st in (s_in, s_run, s_out):
+        st.wait_event(e0)
+    e2e_run(args.e2e_steps)
     e1.record()
     torch.cuda.synchronize()
     e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
     h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hw))
-    d2h = hout.numel() * hout.element_size()
+    d2h = hout[0].numel() * hout[0].element_size()
     e2e = {"value": pdist.whole_job_rate(pairs, args.e2e_steps, e2e_ms, world) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
-           "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.e2e_steps, "steps": args.e2e_steps}
-    assert torch.equal(hout.to(dev), topk)
+           "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.e2e_steps, "steps": args.e2e_steps,
+           "pipelined": "3 streams, double-buffered inputs and results"}
+    ref_top = torch.empty_like(topk)
+    idxc.indexer_prefill(inp.q, inp.k, inp.w, k_top, inp.q_scale, inp.k_scale, topk_out=ref_top, workspace=ws)
+    torch.cuda.synchronize()
+    assert torch.equal(hout[0].to(dev), ref_top) and torch.equal(hout[1].to(dev), ref_top)
+    topk.copy_(ref_top)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
@@ -479,7 +511,7 @@ def main():
             "rows_with_identical_index_set": f"{same}/{len(rows)}"}
         if not args.no_extras:
             line["decode"] = time_decode(idxc, synth, dev, peaks, steps=max(K, 10), warmup=W)
-            del hq, hk, hw, dq, dk, dw, inp, host
+            del hq, hk, hw, dq, dk, dw, dtop, hout, inp, host
             torch.cuda.empty_cache()
             c4, c5 = synth.CONFIGS["cfg4"], synth.CONFIGS["cfg5"]
             n_layers, sched_L = (c4["N"], c4["L"]) if args.full else (args.schedule_layers, args.schedule_L)
