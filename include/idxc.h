@@ -204,6 +204,14 @@ idxc_status idxc_schedule_decode_layer(idxc_schedule* s, int layer,
  * ran out since the last poll (the record is cleared). */
 idxc_status idxc_poll_device_status(void* cuda_stream);
 
+/* Self-test of the bounded device waits (no counterpart in the paper). Every spin-wait in this library's
+ * kernels gives up after a cycle budget, records a code in a device status word and lets the kernel return,
+ * so that a lost signal shows up as IDXC_ERR_DEVICE_TIMEOUT instead of a hung GPU. This call enqueues a
+ * one-warp kernel whose only wait can never be satisfied, with a budget of wait_cycles SM cycles (clamped to
+ * 1e8, about 50 ms); the next idxc_poll_device_status on the stream then returns IDXC_ERR_DEVICE_TIMEOUT
+ * once, and IDXC_OK afterwards. Nothing traps or faults. */
+idxc_status idxc_selftest_bounded_wait(uint32_t wait_cycles, void* cuda_stream);
+
 /* Number of kernel launches this library has made in this process (all streams). */
 int64_t idxc_launch_count(void);
 

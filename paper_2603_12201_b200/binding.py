@@ -25,6 +25,7 @@ EXPORTED_SYMBOLS = [
     "idxc_indexer_decode", "idxc_topk_rows", "idxc_schedule_create", "idxc_schedule_destroy",
     "idxc_schedule_begin_pass", "idxc_schedule_source", "idxc_schedule_stats", "idxc_schedule_prefill_layer",
     "idxc_schedule_decode_layer", "idxc_poll_device_status", "idxc_launch_count", "idxc_indexer_decode_noalloc",
+    "idxc_selftest_bounded_wait",
 ]
 NOALLOC_SCRATCH_BYTES = 16 << 20
 
@@ -78,6 +79,8 @@ def lib() -> ctypes.CDLL:
         L.idxc_schedule_prefill_layer.argtypes = [vp, i32] + prefill_args + [ctypes.POINTER(vp)]
         L.idxc_schedule_decode_layer.restype = i32
         L.idxc_schedule_decode_layer.argtypes = [vp, i32] + decode_args + [ctypes.POINTER(vp)]
+        L.idxc_selftest_bounded_wait.restype = i32
+        L.idxc_selftest_bounded_wait.argtypes = [u32, vp]
         L.idxc_poll_device_status.restype = i32
         L.idxc_poll_device_status.argtypes = [vp]
         _lib = L
@@ -222,6 +225,12 @@ def topk_rows(scores, k_top, topk_out, first_len=0, len_step=0, lens=None, strea
         raise ValueError("topk_out must be [n_rows, k_top]")
     _check(lib().idxc_topk_rows(_ptr(scores), ld, n_rows, int(first_len), int(len_step), _ptr(lens), int(k_top),
                                 _ptr(topk_out), _stream(stream)), "idxc_topk_rows")
+
+
+def selftest_bounded_wait(wait_cycles: int = 1_000_000, stream=None):
+    """idxc_selftest_bounded_wait: enqueue a kernel whose wait can never be satisfied; the next
+    poll_device_status() must raise IdxcError(ERR_DEVICE_TIMEOUT)."""
+    _check(lib().idxc_selftest_bounded_wait(int(wait_cycles), _stream(stream)), "idxc_selftest_bounded_wait")
 
 
 def poll_device_status(stream=None):

@@ -373,6 +373,14 @@ idxc_status idxc_schedule_decode_layer(idxc_schedule* s, int layer, const void* 
     return IDXC_OK;
 }
 
+idxc_status idxc_selftest_bounded_wait(uint32_t wait_cycles, void* cuda_stream) {
+    if (!device_info().ok) return IDXC_ERR_CUDA;
+    const long long budget = wait_cycles > 100000000u ? 100000000LL : static_cast<long long>(wait_cycles);
+    g_launches += 1;
+    return launch_selftest_bounded_wait(device_info().status_ptr, budget, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+               ? IDXC_OK : IDXC_ERR_CUDA;
+}
+
 idxc_status idxc_poll_device_status(void* cuda_stream) {
     if (!device_info().ok) return IDXC_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);

@@ -52,4 +52,8 @@ cudaError_t launch_score_decode_tc(const ScoreArgs& a, const CUtensorMap& q_map,
                                    unsigned int* status, int sm_count, cudaStream_t stream);
 bool score_tc_supported(int H, int d, int fp8);
 
+// selftest.cu: one tiny kernel whose only wait can never be satisfied; it must record a time-out in
+// `status` after `budget_cycles` and return.
+cudaError_t launch_selftest_bounded_wait(unsigned int* status, long long budget_cycles, cudaStream_t stream);
+
 }  // namespace idxc

@@ -16,6 +16,7 @@ enum : unsigned int {
     DEV_TIMEOUT_PRODUCER = 0x101,
     DEV_TIMEOUT_MMA = 0x102,
     DEV_TIMEOUT_EPILOGUE = 0x103,
+    DEV_TIMEOUT_SELFTEST = 0x1FF,
 };
 
 // ~1 s at the 1.9 GHz boost clock; legitimate waits in these kernels are < 1 ms.
@@ -51,14 +52,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait. `abort_flag` is a shared-memory word any role sets when it gives up;
 // polling it lets the other roles leave at once instead of each running out its own budget.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          long long budget = kWaitCycleBudget) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 63u) == 0) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitCycleBudget) return false;
+            if (clock64() - t0 > budget) return false;
         }
     }
     return true;

@@ -331,3 +331,18 @@ def test_schedule_decode_layers():
         for b in range(B):
             assert_topk_valid(g[b], o_scores[b, : lens[b]], k_top, RTOL_BF16)
     sch.close()
+
+
+# ------------------------------------------------------------------------------ failure detection
+def test_bounded_wait_reports_timeout_and_context_stays_usable():
+    """A device-side wait that nothing satisfies runs out (here after ~1e6 cycles), the kernel returns, the
+    host reads IDXC_ERR_DEVICE_TIMEOUT once, and the library keeps working afterwards."""
+    idxc.poll_device_status()
+    idxc.selftest_bounded_wait(1_000_000)
+    with pytest.raises(idxc.IdxcError) as e:
+        idxc.poll_device_status()
+    assert e.value.status == idxc.ERR_DEVICE_TIMEOUT
+    idxc.poll_device_status()                               # the record was cleared
+    inp = _to_dev(synth.prefill_inputs(256, 16, 64, seed=9))
+    g_scores, g_topk = _gpu_prefill(inp, 16)
+    _check_prefill(inp, 16, g_scores, g_topk, RTOL_BF16)
