@@ -62,6 +62,8 @@ def _load():
         lib.orc_topk.argtypes = [vp, i64, i32, vp]
         lib.orc_prefill.restype = ctypes.c_int
         lib.orc_prefill.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i32, i32, i32, i32, vp, i64, vp, i64, vp]
+        lib.orc_quantize_e4m3.restype = ctypes.c_int
+        lib.orc_quantize_e4m3.argtypes = [vp, i64, i64, vp, vp]
         lib.orc_decode.restype = ctypes.c_int
         lib.orc_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, i64, vp]
         _lib = lib
@@ -168,3 +170,18 @@ def indexer_decode(q_step, k_cache, w, k_offsets, lens, k_top, dtype=BF16, q_sca
     if rc:
         raise ValueError("orc_decode: bad arguments")
     return scores, tk
+
+
+def quantize_e4m3(x_bf16):
+    """Per-token e4m3 quantiser (Sec. 2.1, 'FP8 arithmetic'): x [n_tokens, ...] bf16 codes (uint16).
+    Returns (codes uint8 of the same shape, scale [n_tokens] fp32): scale = max(amax, 1e-12) / 448,
+    code = e4m3(x / scale), round to nearest even, saturating; all in binary32."""
+    x = _check(x_bf16, np.uint16, "x")
+    n = x.shape[0]
+    row = int(np.prod(x.shape[1:])) if x.ndim > 1 else 1
+    codes = np.empty(x.shape, dtype=np.uint8)
+    scale = np.empty((n,), dtype=np.float32)
+    rc = _load().orc_quantize_e4m3(_ptr(x), n, row, _ptr(codes), _ptr(scale))
+    if rc:
+        raise ValueError("orc_quantize_e4m3: bad arguments")
+    return codes, scale

@@ -24,7 +24,8 @@
 // reducing to a BLAS matrix product, rank-1 closed form, one-hot inputs,
 // all-negative gate, sliding-window / sink top-k closed forms, duplicate-key
 // tie-break, exhaustive number-format round trips against the format
-// definitions. No function here is "parity unpinned".
+// definitions; the quantiser against a library conversion and closed forms.
+// No function here is "parity unpinned".
 
 #include <algorithm>
 #include <cmath>
@@ -238,6 +239,30 @@ int orc_decode(const void* q_step, const void* k_cache, const float* w, const fl
             for (int64_t s = n; s < ld; ++s) o[s] = -std::numeric_limits<double>::infinity();
         }
         if (topk_out) topk_row(row.data(), n, k_top, topk_out + static_cast<int64_t>(b) * k_top);
+    }
+    return 0;
+}
+
+// Per-token FP8 quantiser, the step in front of the indexer (Sec. 2.1: the indexer runs in FP8
+// arithmetic). Reading taken: one fp32 scale per token, scale = max(amax, 1e-12) / 448 and
+// code = e4m3(x / scale) with round-to-nearest-even and saturation. The code is an integer decided by
+// floating point, so the decision is taken in the precision the kernel uses: IEEE binary32 for amax,
+// the two divisions and the rounding input. x: [n_tokens, row_elems] bf16 codes.
+int orc_quantize_e4m3(const uint16_t* x, int64_t n_tokens, int64_t row_elems, uint8_t* codes, float* scale) {
+    if (n_tokens < 0 || row_elems < 1) return 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < n_tokens; ++r) {
+        float amax = 0.0f;
+        for (int64_t i = 0; i < row_elems; ++i) {
+            float v = static_cast<float>(bf16_to_f64(x[r * row_elems + i]));
+            amax = std::fmax(amax, std::fabs(v));
+        }
+        const float sc = std::fmax(amax, 1e-12f) / 448.0f;
+        scale[r] = sc;
+        for (int64_t i = 0; i < row_elems; ++i) {
+            float v = static_cast<float>(bf16_to_f64(x[r * row_elems + i]));
+            codes[r * row_elems + i] = f32_to_e4m3(v / sc);
+        }
     }
     return 0;
 }
