@@ -319,6 +319,32 @@ def time_fp8_chunked(idxc, synth, dev, peaks, L, chunk, H, d, k_top, seed, decod
     return out
 
 
+def time_quantize(idxc, dev, peaks, n_tokens, H, d):
+    """NEXT-1: per-token bf16 -> e4m3 quantiser on query-shaped rows [n_tokens, H*d] and key-shaped rows
+    [16 * n_tokens, d] (both larger than L2). Algorithmic bytes: 2 read + 1 written per element + 4 per token."""
+    out = {}
+    for name, rows, row_elems in (("queries", n_tokens, H * d), ("keys", 16 * n_tokens, d)):
+        x = torch.randn((rows, row_elems), device=dev, dtype=torch.float32).to(torch.bfloat16)
+        codes_out = torch.empty((rows, row_elems), dtype=torch.uint8, device=dev)
+        scale_out = torch.empty((rows,), dtype=torch.float32, device=dev)
+        for _ in range(3):
+            idxc.quantize_e4m3(x, codes_out, scale_out)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(10):
+            idxc.quantize_e4m3(x, codes_out, scale_out)
+        b.record()
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / 10
+        nbytes = rows * row_elems * 3 + rows * 4
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        out[name] = {"rows": rows, "row_elems": row_elems, "ms": ms, "bytes": nbytes,
+                     "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                  "frac": gbs / peaks["hbm_gbs"], "of": peaks["source"]}}
+        del x, codes_out, scale_out
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -530,6 +556,7 @@ def main():
             line["schedule"] = time_schedule(idxc, synth, dev, sched_L, c4["H"], c4["d"], c4["k_top"], n_layers, c4["every"],
                                              seed=c4["seed"], reps=1 if args.full else 2)
             torch.cuda.empty_cache()
+            line["quantize_e4m3"] = time_quantize(idxc, dev, peaks, 32768, c5["H"], c5["d"])
             fp8_L = c5["L"] if args.full else 32768
             line["fp8_chunked"] = time_fp8_chunked(idxc, synth, dev, peaks, fp8_L, c5["chunk"], c5["H"], c5["d"], c5["k_top"],
                                                    c5["seed"], c5["decode_B"])

@@ -154,6 +154,22 @@ idxc_status idxc_topk_rows(const float* scores, int64_t ld, int64_t n_rows,
                            int k_top, int32_t* topk_out, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------
+ * Per-token FP8 quantiser with optional K-cache append: the step in front of the indexer
+ * (Sec. 2.1: the lightning indexer uses FP8 arithmetic). For token r:
+ *     scale[r]  = max(max_i |x[r, i]|, 1e-12) / 448                    (fp32)
+ *     code[r,i] = e4m3(x[r, i] / scale[r])      round to nearest even, saturating at +-448
+ * exactly the format idxc_indexer_prefill / idxc_indexer_decode read with IDXC_FP8_E4M3.
+ *   x          [n_tokens, row_elems] bf16, 16-byte aligned; row_elems = d_I for keys, H_I * d_I for
+ *              queries: a multiple of 8, at most 8192
+ *   codes_out  [rows, row_elems] uint8 (8-byte aligned), scale_out [rows] fp32
+ *   dst_rows   NULL: token r is written at row r. Otherwise a device array [n_tokens] int64: token r is
+ *              written at row dst_rows[r] of codes_out / scale_out (appending new keys to an indexer K
+ *              cache). The caller guarantees the rows are in range and distinct.
+ * ------------------------------------------------------------------------- */
+idxc_status idxc_quantize_e4m3(const void* x, int64_t n_tokens, int row_elems, void* codes_out, float* scale_out,
+                               const int64_t* dst_rows, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------
  * IndexCache layer schedule (Sec. 3 "Overview", Figure 2(b)).
  * pattern c_0 .. c_{N-1} over {'F','S'}: an F (Full) layer runs its indexer and its
  * result becomes the cached index tensor; an S (Shared) layer returns the cached

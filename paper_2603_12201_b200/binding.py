@@ -25,7 +25,7 @@ EXPORTED_SYMBOLS = [
     "idxc_indexer_decode", "idxc_topk_rows", "idxc_schedule_create", "idxc_schedule_destroy",
     "idxc_schedule_begin_pass", "idxc_schedule_source", "idxc_schedule_stats", "idxc_schedule_prefill_layer",
     "idxc_schedule_decode_layer", "idxc_poll_device_status", "idxc_launch_count", "idxc_indexer_decode_noalloc",
-    "idxc_selftest_bounded_wait",
+    "idxc_selftest_bounded_wait", "idxc_quantize_e4m3",
 ]
 NOALLOC_SCRATCH_BYTES = 16 << 20
 
@@ -79,6 +79,8 @@ def lib() -> ctypes.CDLL:
         L.idxc_schedule_prefill_layer.argtypes = [vp, i32] + prefill_args + [ctypes.POINTER(vp)]
         L.idxc_schedule_decode_layer.restype = i32
         L.idxc_schedule_decode_layer.argtypes = [vp, i32] + decode_args + [ctypes.POINTER(vp)]
+        L.idxc_quantize_e4m3.restype = i32
+        L.idxc_quantize_e4m3.argtypes = [vp, i64, i32, vp, vp, vp, vp]
         L.idxc_selftest_bounded_wait.restype = i32
         L.idxc_selftest_bounded_wait.argtypes = [u32, vp]
         L.idxc_poll_device_status.restype = i32
@@ -225,6 +227,23 @@ def topk_rows(scores, k_top, topk_out, first_len=0, len_step=0, lens=None, strea
         raise ValueError("topk_out must be [n_rows, k_top]")
     _check(lib().idxc_topk_rows(_ptr(scores), ld, n_rows, int(first_len), int(len_step), _ptr(lens), int(k_top),
                                 _ptr(topk_out), _stream(stream)), "idxc_topk_rows")
+
+
+def quantize_e4m3(x, codes_out, scale_out, dst_rows=None, stream=None):
+    """idxc_quantize_e4m3: x [n_tokens, ...] bf16 -> e4m3 codes (float8_e4m3fn or uint8 tensor with the same
+    trailing shape) and one fp32 scale per token, written at row r or at row dst_rows[r]."""
+    _dev(x, "x", torch.bfloat16); _dev(codes_out, "codes_out"); _dev(scale_out, "scale_out", torch.float32)
+    _dev(dst_rows, "dst_rows", torch.int64)
+    if codes_out.element_size() != 1:
+        raise TypeError("codes_out must be an 8-bit tensor")
+    n = x.shape[0]
+    row = x.numel() // n if n else int(torch.tensor(x.shape[1:]).prod())
+    if codes_out.numel() // max(codes_out.shape[0], 1) != row or scale_out.shape[0] != codes_out.shape[0]:
+        raise ValueError("codes_out / scale_out rows do not match x")
+    if dst_rows is None and codes_out.shape[0] < n:
+        raise ValueError("codes_out has fewer rows than x")
+    _check(lib().idxc_quantize_e4m3(_ptr(x), n, row, _ptr(codes_out), _ptr(scale_out), _ptr(dst_rows), _stream(stream)),
+           "idxc_quantize_e4m3")
 
 
 def selftest_bounded_wait(wait_cycles: int = 1_000_000, stream=None):

@@ -373,6 +373,18 @@ idxc_status idxc_schedule_decode_layer(idxc_schedule* s, int layer, const void* 
     return IDXC_OK;
 }
 
+idxc_status idxc_quantize_e4m3(const void* x, int64_t n_tokens, int row_elems, void* codes_out, float* scale_out,
+                               const int64_t* dst_rows, void* cuda_stream) {
+    if (n_tokens < 0 || row_elems < 8 || (row_elems & 7) || row_elems > 8192) return IDXC_ERR_INVALID_ARG;
+    if (n_tokens == 0) return IDXC_OK;
+    if (!x || !codes_out || !scale_out || !aligned(x, 16) || !aligned(codes_out, 8) || !aligned(scale_out, 4))
+        return IDXC_ERR_INVALID_ARG;
+    if (dst_rows && !aligned(dst_rows, 8)) return IDXC_ERR_INVALID_ARG;
+    g_launches += 1;
+    return launch_quantize_e4m3(x, n_tokens, row_elems, codes_out, scale_out, dst_rows,
+                                static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? IDXC_OK : IDXC_ERR_CUDA;
+}
+
 idxc_status idxc_selftest_bounded_wait(uint32_t wait_cycles, void* cuda_stream) {
     if (!device_info().ok) return IDXC_ERR_CUDA;
     const long long budget = wait_cycles > 100000000u ? 100000000LL : static_cast<long long>(wait_cycles);

@@ -52,6 +52,10 @@ cudaError_t launch_score_decode_tc(const ScoreArgs& a, const CUtensorMap& q_map,
                                    unsigned int* status, int sm_count, cudaStream_t stream);
 bool score_tc_supported(int H, int d, int fp8);
 
+// quantize.cu: per-token e4m3 quantiser (row_elems a multiple of 8, at most 8192), optional row scatter.
+cudaError_t launch_quantize_e4m3(const void* x, int64_t n_tokens, int row_elems, void* codes, float* scale,
+                                 const int64_t* dst_rows, cudaStream_t stream);
+
 // selftest.cu: one tiny kernel whose only wait can never be satisfied; it must record a time-out in
 // `status` after `budget_cycles` and return.
 cudaError_t launch_selftest_bounded_wait(unsigned int* status, long long budget_cycles, cudaStream_t stream);

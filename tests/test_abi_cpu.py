@@ -24,7 +24,7 @@ def idxc():
 def test_library_exports_every_declared_symbol(idxc):
     header = open(os.path.join(ROOT, "include", "idxc.h")).read()
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
-    declared = sorted(set(re.findall(r"\b(idxc_[a-z_]+)\s*\(", header)))
+    declared = sorted(set(re.findall(r"\b(idxc_[a-z0-9_]+)\s*\(", header)))
     assert declared == sorted(idxc.EXPORTED_SYMBOLS)
     L = idxc.lib()
     for name in declared:

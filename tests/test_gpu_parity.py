@@ -346,3 +346,50 @@ def test_bounded_wait_reports_timeout_and_context_stays_usable():
     inp = _to_dev(synth.prefill_inputs(256, 16, 64, seed=9))
     g_scores, g_topk = _gpu_prefill(inp, 16)
     _check_prefill(inp, 16, g_scores, g_topk, RTOL_BF16)
+
+
+# ------------------------------------------------------------------------------ FP8 quantiser (step before the indexer)
+@pytest.mark.parametrize("n,shape", [(1, (128,)), (1000, (128,)), (777, (64,)), (300, (256,)), (65, (64, 128)), (33, (16, 64)),
+                                    (40, (8, 40)), (5, (8,))])
+def test_quantize_e4m3_bit_exact(n, shape):
+    g = torch.Generator().manual_seed(n)
+    x = (torch.randn((n,) + shape, generator=g) * torch.logspace(-3, 3, n)[(...,) + (None,) * len(shape)]).to(torch.bfloat16)
+    if n > 2:
+        x[1] = 0                                           # an all-zero token: scale floor, codes 0
+    xd = x.to(DEV)
+    codes_out = torch.full((n,) + shape, 0x55, dtype=torch.uint8, device=DEV)
+    scale_out = torch.full((n,), -1.0, device=DEV)
+    idxc.quantize_e4m3(xd, codes_out, scale_out)
+    o_codes, o_scale = oracle.quantize_e4m3(codes(x))
+    g_codes = codes_out.cpu().numpy()
+    assert np.array_equal(scale_out.cpu().numpy(), o_scale)
+    nz = (o_codes & 0x7F) != 0
+    assert np.array_equal(g_codes & 0x7F, o_codes & 0x7F) and np.array_equal(g_codes[nz], o_codes[nz])
+
+
+def test_quantize_e4m3_appends_to_a_k_cache_that_the_indexer_reads():
+    # new keys of three sequences are appended at the end of their cache rows, then one decode step reads the cache
+    B, H, d, k_top = 3, 64, 128, 32
+    lens_before = [200, 511, 64]
+    n_new = 1
+    base = synth.decode_inputs(B, H, d, 0, 0, seed=50, fp8=True, lens=[l + n_new for l in lens_before], row_align=128)
+    base = _to_dev(base)
+    g = torch.Generator().manual_seed(51)
+    new_keys = torch.randn(B, d, generator=g).to(torch.bfloat16).to(DEV)
+    dst = (base.k_offsets + torch.tensor(lens_before, device=DEV)).to(torch.int64)
+    idxc.quantize_e4m3(new_keys, base.k_cache.view(torch.uint8), base.k_scale, dst_rows=dst)
+    o_codes, o_scale = oracle.quantize_e4m3(codes(new_keys))
+    kc = base.k_cache.view(torch.uint8).cpu().numpy()
+    for b in range(B):
+        row = int(dst[b])
+        assert np.array_equal(kc[row] & 0x7F, o_codes[b] & 0x7F)
+        assert base.k_scale[row].item() == o_scale[b]
+    topk = torch.empty((B, k_top), dtype=torch.int32, device=DEV)
+    ws = idxc.alloc_workspace(idxc.decode_workspace_bytes(B, base.max_len, H, d, k_top, idxc.FP8_E4M3), DEV)
+    idxc.indexer_decode(base.q_step, base.k_cache, base.w, base.k_offsets, base.lens, base.max_len, k_top, base.q_scale,
+                        base.k_scale, topk_out=topk, workspace=ws)
+    idxc.poll_device_status()
+    o_sc, _ = oracle.indexer_decode(codes(base.q_step), codes(base.k_cache), f32(base.w), base.k_offsets.cpu().numpy(),
+                                    base.lens.cpu().numpy(), k_top, oracle.FP8_E4M3, f32(base.q_scale), f32(base.k_scale))
+    for b in range(B):
+        assert_topk_valid(topk[b].cpu().numpy(), o_sc[b, : lens_before[b] + n_new], k_top, RTOL_FP8)
