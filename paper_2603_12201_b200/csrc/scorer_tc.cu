@@ -19,7 +19,8 @@
 // items are handed out longest first in a boustrophedon order over the CTAs.
 //
 // Decode kernel: work item = (sequence, run of key tiles); the sequence's H x d query tile
-// is the B operand (N = H), key tiles stream from HBM through a deep TMA ring.
+// is the B operand (N = H), key tiles stream from HBM through a deep TMA ring; two groups of four
+// epilogue warps drain alternate TMEM accumulator slots.
 #include "kernels.h"
 #include "ptx_sm100.cuh"
 
@@ -395,7 +396,8 @@ cudaError_t launch_score_prefill_tc(const ScoreArgs& a, const CUtensorMap& q_map
 // ===================================================================== decode
 namespace {
 
-constexpr int kDecodeThreads = 192;      // warp 0 producer, warp 1 MMA, warps 2-5 epilogue
+constexpr int kDecodeEpiWarps = 8;       // two groups of 4 (one warp per TMEM lane quarter); group g drains slots g, g+2
+constexpr int kDecodeThreads = (2 + kDecodeEpiWarps) * 32;   // warp 0 producer, warp 1 MMA, warps 2-9 epilogue
 // Key tiles (of 128 keys) per work item. Measured on B200 (B = 32, 16K-128K keys per sequence): 16 tiles
 // stream at 6.1 TB/s; 6-8 tiles per item lose 20 % (all CTAs then walk HBM with the same 192-256 KB stride).
 constexpr int kDecodeChunkTiles = 16;
@@ -407,7 +409,7 @@ struct DecodeCfg {
     static constexpr int kQRegion = H * kChunkBytes;                  // one 128-byte chunk of the query tile
     static constexpr int kQBytes = 2 * NKH * kQRegion;                // double buffered
     static constexpr int kKBytes = kStages * NKH * kKRegionBytes;
-    static constexpr int kWBytes = 4 * 64 * 4;
+    static constexpr int kWBytes = kDecodeEpiWarps * (64 + kDecodeChunkTiles * 32) * 4;   // per warp: w, and the key scales of one item
     static constexpr int kBarBytes = 512;
     static constexpr int kSmemBytes = kQBytes + kKBytes + kWBytes + kBarBytes + 1024;
 };
@@ -588,8 +590,10 @@ score_decode_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
         }
     } else {
         const int quarter = warp & 3;
+        const int grp = (warp - 2) >> 2;                 // which accumulator slots this warp drains
         const int key_in_tile = quarter * 32 + lane;
-        float* my_w = w_smem + (warp - 2) * 64;
+        float* my_w = w_smem + (warp - 2) * (64 + kDecodeChunkTiles * 32);
+        float* my_ksc = my_w + 64;                       // FP8: k_scale of my key in every tile of the item
         int slot = 0;
         uint32_t acc_phase[kDecodeAccSlots] = {0u, 0u, 0u, 0u};
         bool ok = true;
@@ -600,42 +604,72 @@ score_decode_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                 if constexpr (FP8) v *= __ldg(p.q_scale + seq);
                 my_w[h] = v;
             }
-            __syncwarp();
             const int64_t krow0 = p.k_offsets[seq];
-            for (int kt = 0; kt < ntiles && ok; ++kt) {
+            if constexpr (FP8) {
+                // all key scales of the item at once: independent loads in flight instead of one exposed
+                // memory latency per tile
+#pragma unroll 4
+                for (int kt = 0; kt < ntiles; ++kt) {
+                    const int s2 = (tile0 + kt) * kTileKeys + key_in_tile;
+                    my_ksc[kt * 32 + lane] = s2 < len ? __ldg(p.k_scale + krow0 + s2) : 0.f;
+                }
+            }
+            __syncwarp();
+            const float4* w4 = reinterpret_cast<const float4*>(my_w);
+            for (int kt = 0; kt < ntiles && ok; ++kt, slot = (slot + 1) & (kDecodeAccSlots - 1)) {
+                if ((slot & 1) != grp) continue;         // the other group's tile
                 const int s = (tile0 + kt) * kTileKeys + key_in_tile;
-                float ksc = 1.f;
-                if constexpr (FP8) ksc = s < len ? __ldg(p.k_scale + krow0 + s) : 0.f;
                 ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_acc_full + 8 * slot, acc_phase[slot], abort_flag));   // warp-uniform
                 if (!ok) break;
                 acc_phase[slot] ^= 1u;
                 tcgen05_fence_after_sync();
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(slot * 64);
-                float acc = 0.f;
+                float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;    // four independent partial sums over the heads
                 if constexpr (H == 16) {
                     uint32_t r[16];
                     tmem_ld_32x32b_x16(taddr, r);
                     tmem_ld_wait(r);
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) acc = fmaf(fmaxf(__uint_as_float(r[j]), 0.f), my_w[j], acc);
+                    for (int j4 = 0; j4 < 4; ++j4) {
+                        const float4 wv = w4[j4];
+                        a0 = fmaf(fmaxf(__uint_as_float(r[4 * j4 + 0]), 0.f), wv.x, a0);
+                        a1 = fmaf(fmaxf(__uint_as_float(r[4 * j4 + 1]), 0.f), wv.y, a1);
+                        a2 = fmaf(fmaxf(__uint_as_float(r[4 * j4 + 2]), 0.f), wv.z, a2);
+                        a3 = fmaf(fmaxf(__uint_as_float(r[4 * j4 + 3]), 0.f), wv.w, a3);
+                    }
                 } else {
+                    uint32_t ra[32], rb[32];
+                    tmem_ld_32x32b_x32(taddr, ra);
+                    if constexpr (H == 64) tmem_ld_32x32b_x32(taddr + 32, rb);
+                    tmem_ld_wait(ra);                    // waits for every load issued so far
+                    if constexpr (H == 64) tmem_ld_wait(rb);
 #pragma unroll
-                    for (int c = 0; c < H / 32; ++c) {
-                        uint32_t r[32];
-                        tmem_ld_32x32b_x32(taddr + c * 32, r);
-                        tmem_ld_wait(r);
+                    for (int j4 = 0; j4 < 8; ++j4) {
+                        const float4 wv = w4[j4];
+                        a0 = fmaf(fmaxf(__uint_as_float(ra[4 * j4 + 0]), 0.f), wv.x, a0);
+                        a1 = fmaf(fmaxf(__uint_as_float(ra[4 * j4 + 1]), 0.f), wv.y, a1);
+                        a2 = fmaf(fmaxf(__uint_as_float(ra[4 * j4 + 2]), 0.f), wv.z, a2);
+                        a3 = fmaf(fmaxf(__uint_as_float(ra[4 * j4 + 3]), 0.f), wv.w, a3);
+                    }
+                    if constexpr (H == 64) {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) acc = fmaf(fmaxf(__uint_as_float(r[j]), 0.f), my_w[c * 32 + j], acc);
+                        for (int j4 = 0; j4 < 8; ++j4) {
+                            const float4 wv = w4[8 + j4];
+                            a0 = fmaf(fmaxf(__uint_as_float(rb[4 * j4 + 0]), 0.f), wv.x, a0);
+                            a1 = fmaf(fmaxf(__uint_as_float(rb[4 * j4 + 1]), 0.f), wv.y, a1);
+                            a2 = fmaf(fmaxf(__uint_as_float(rb[4 * j4 + 2]), 0.f), wv.z, a2);
+                            a3 = fmaf(fmaxf(__uint_as_float(rb[4 * j4 + 3]), 0.f), wv.w, a3);
+                        }
                     }
                 }
                 tcgen05_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_acc_empty + 8 * slot);
                 if (s < len) {
-                    if constexpr (FP8) acc *= ksc;
+                    float acc = (a0 + a1) + (a2 + a3);
+                    if constexpr (FP8) acc *= my_ksc[kt * 32 + lane];
                     p.scores[static_cast<int64_t>(seq) * p.ld + s] = acc;
                 }
-                slot = (slot + 1) & (kDecodeAccSlots - 1);
             }
         }
         if (!ok && lane == 0) give_up(abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
