@@ -13,7 +13,7 @@
 //               through a ring of stages. Per-CTA loads only (no multicast).
 //   warp 1      MMA issuer: per key tile, one 128 x 256 x d UMMA chain into each of the two
 //               256-column TMEM accumulators, so accumulator A is drained while B is filled.
-//   warps 4-11  epilogue: tcgen05.ld (16x256b), ReLU, FMA with w held in registers, two shuffles per
+//   warps 2-9   epilogue: tcgen05.ld (16x256b), ReLU, FMA with w held in registers, two shuffles per
 //               score to join the four threads of a key, causal predicate, coalesced score store.
 // Causal structure: a work item only visits key tiles up to its last query's position;
 // items are handed out longest first in a boustrophedon order over the CTAs.
@@ -37,7 +37,8 @@ constexpr int kKRegionBytes = kTileKeys * kChunkBytes;   // 16 KB
 #ifndef IDXC_EPI_WARPS
 #define IDXC_EPI_WARPS 8
 #endif
-constexpr int kEpilogueWarp0 = 4;
+constexpr int kEpilogueWarp0 = 2;       // warps 0, 1: TMA producer, MMA issuer; no idle warps, so that the
+                                        // registers left on the SM can host a top-k CTA next to this kernel
 constexpr int kNumEpilogueWarps = IDXC_EPI_WARPS;       // 8 or 16: 2 or 4 per TMEM lane quarter
 constexpr int kPrefillThreads = (kEpilogueWarp0 + kNumEpilogueWarps) * 32;
 constexpr int kColsPerEpiWarp = kTileCols / (kNumEpilogueWarps / 4);   // 128 or 64 accumulator columns per warp
