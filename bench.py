@@ -345,6 +345,30 @@ def time_quantize(idxc, dev, peaks, n_tokens, H, d):
     return out
 
 
+def time_overlap(idxc, dev, peaks, rows, k_top, n_layers):
+    """NEXT-3: pairwise top-k index overlap (Appendix A) over n_layers index tensors [rows, k_top] in one launch.
+    Algorithmic bytes: each pair reads both tensors once (2 * rows * k_top * 4)."""
+    g = torch.Generator(device=dev).manual_seed(11)
+    tops = []
+    for l in range(n_layers):       # sorted random subsets of [0, 8 * k_top): valid ascending index rows
+        t = torch.rand((rows, 8 * k_top), generator=g, device=dev).topk(k_top, dim=1).indices.to(torch.int32)
+        tops.append(torch.sort(t, dim=1).values.contiguous())
+    idxc.topk_overlap(tops)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(5):
+        mean = idxc.topk_overlap(tops)
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / 5
+    n_pairs = n_layers * (n_layers - 1) // 2
+    nbytes = n_pairs * 2 * rows * k_top * 4
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"layers": n_layers, "pairs": n_pairs, "rows": rows, "k_top": k_top, "ms": ms, "mean_overlap": float(mean.mean()),
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                         "of": peaks["source"], "note": "every tensor is read n_layers-1 times; repeats may hit L2"}}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -556,6 +580,7 @@ def main():
             line["schedule"] = time_schedule(idxc, synth, dev, sched_L, c4["H"], c4["d"], c4["k_top"], n_layers, c4["every"],
                                              seed=c4["seed"], reps=1 if args.full else 2)
             torch.cuda.empty_cache()
+            line["topk_overlap"] = time_overlap(idxc, dev, peaks, 8192, c5["k_top"], 6)
             line["quantize_e4m3"] = time_quantize(idxc, dev, peaks, 32768, c5["H"], c5["d"])
             fp8_L = c5["L"] if args.full else 32768
             line["fp8_chunked"] = time_fp8_chunked(idxc, synth, dev, peaks, fp8_L, c5["chunk"], c5["H"], c5["d"], c5["k_top"],

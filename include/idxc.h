@@ -215,6 +215,37 @@ idxc_status idxc_schedule_decode_layer(idxc_schedule* s, int layer,
                                        void* workspace, size_t workspace_bytes, uint32_t flags,
                                        void* cuda_stream, const int32_t** topk_result);
 
+/* ---------------------------------------------------------------------------
+ * Pattern tooling on index tensors.
+ *
+ * idxc_topk_overlap -- the cross-layer top-k index overlap of Appendix A: for a pair of index tensors
+ * T_a, T_b ([rows, k_top] int32, ascending, -1 padded, as produced above) the per-row ratio
+ * |T_a[r] n T_b[r]| / (valid entries of T_a[r]) and its sum over the rows.
+ *   layers   DEVICE array of device pointers to the index tensors
+ *   pairs    DEVICE int32 [2 * n_pairs]: pair p compares layers[pairs[2p]] with layers[pairs[2p+1]]
+ *   sums_out DEVICE double [n_pairs]: sum over rows of the ratio (divide by rows for the mean); zeroed by the call
+ *   row_out  NULL, or DEVICE float [rows] (only with n_pairs == 1): the per-row ratios
+ * One launch covers all pairs (n_pairs <= 65535).
+ *
+ * idxc_pattern_search_dp -- the similarity-based search of Appendix C (HOST only, no GPU work): S is a HOST
+ * row-major [N, N] matrix, S[l*N + j] (j < l) = how well layer j's indices serve layer l. Writes to
+ * pattern_out (HOST, N chars, not terminated) a pattern with exactly M Full layers, the first layer Full, that
+ * maximises the sum over Shared layers l of S[l, f(l)], and that maximum to value_out (HOST, may be NULL).
+ *
+ * idxc_pattern_search_greedy -- Algorithm 1 (HOST driver): starting from all-Full, K times flip to Shared the
+ * remaining layer (never layer 0) whose flip gives the lowest eval_loss(pattern, N, user); ties go to the
+ * lowest layer. eval_loss receives a NUL-terminated pattern. order_out (HOST, K ints, may be NULL) gets the
+ * flipped layers in order, evaluations_out (HOST, may be NULL) the number of loss evaluations
+ * (N(N-1)/2 for K = N-1).
+ * ------------------------------------------------------------------------- */
+typedef double (*idxc_eval_loss_fn)(const char* pattern, int N, void* user);
+
+idxc_status idxc_topk_overlap(const int32_t* const* layers, const int32_t* pairs, int n_pairs, int64_t rows, int k_top,
+                              double* sums_out, float* row_out, void* cuda_stream);
+idxc_status idxc_pattern_search_dp(const double* S, int N, int M, char* pattern_out, double* value_out);
+idxc_status idxc_pattern_search_greedy(int N, int K, idxc_eval_loss_fn eval_loss, void* user, char* pattern_out,
+                                       int* order_out, int64_t* evaluations_out);
+
 /* Synchronises the stream, then returns IDXC_OK, IDXC_ERR_CUDA, or
  * IDXC_ERR_DEVICE_TIMEOUT if any kernel of this library recorded a bounded wait that
  * ran out since the last poll (the record is cleared). */

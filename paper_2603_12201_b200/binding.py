@@ -25,9 +25,13 @@ EXPORTED_SYMBOLS = [
     "idxc_indexer_decode", "idxc_topk_rows", "idxc_schedule_create", "idxc_schedule_destroy",
     "idxc_schedule_begin_pass", "idxc_schedule_source", "idxc_schedule_stats", "idxc_schedule_prefill_layer",
     "idxc_schedule_decode_layer", "idxc_poll_device_status", "idxc_launch_count", "idxc_indexer_decode_noalloc",
-    "idxc_selftest_bounded_wait", "idxc_quantize_e4m3",
+    "idxc_selftest_bounded_wait", "idxc_quantize_e4m3", "idxc_topk_overlap", "idxc_pattern_search_dp",
+    "idxc_pattern_search_greedy",
 ]
 NOALLOC_SCRATCH_BYTES = 16 << 20
+
+
+EVAL_LOSS_FN = ctypes.CFUNCTYPE(ctypes.c_double, ctypes.c_char_p, ctypes.c_int, ctypes.c_void_p)
 
 
 class IdxcError(RuntimeError):
@@ -79,6 +83,13 @@ def lib() -> ctypes.CDLL:
         L.idxc_schedule_prefill_layer.argtypes = [vp, i32] + prefill_args + [ctypes.POINTER(vp)]
         L.idxc_schedule_decode_layer.restype = i32
         L.idxc_schedule_decode_layer.argtypes = [vp, i32] + decode_args + [ctypes.POINTER(vp)]
+        L.idxc_topk_overlap.restype = i32
+        L.idxc_topk_overlap.argtypes = [vp, vp, i32, i64, i32, vp, vp, vp]
+        L.idxc_pattern_search_dp.restype = i32
+        L.idxc_pattern_search_dp.argtypes = [vp, i32, i32, ctypes.c_char_p, ctypes.POINTER(ctypes.c_double)]
+        L.idxc_pattern_search_greedy.restype = i32
+        L.idxc_pattern_search_greedy.argtypes = [i32, i32, EVAL_LOSS_FN, vp, ctypes.c_char_p, ctypes.POINTER(i32),
+                                                 ctypes.POINTER(i64)]
         L.idxc_quantize_e4m3.restype = i32
         L.idxc_quantize_e4m3.argtypes = [vp, i64, i32, vp, vp, vp, vp]
         L.idxc_selftest_bounded_wait.restype = i32
@@ -244,6 +255,49 @@ def quantize_e4m3(x, codes_out, scale_out, dst_rows=None, stream=None):
         raise ValueError("codes_out has fewer rows than x")
     _check(lib().idxc_quantize_e4m3(_ptr(x), n, row, _ptr(codes_out), _ptr(scale_out), _ptr(dst_rows), _stream(stream)),
            "idxc_quantize_e4m3")
+
+
+def topk_overlap(layers, pairs=None, want_rows=False, stream=None):
+    """idxc_topk_overlap. layers: list of [rows, k_top] int32 index tensors; pairs: list of (a, b) layer
+    indices (default: every pair a < b). Returns a [n_pairs] float64 tensor of MEAN row ratios (and, with
+    want_rows and a single pair, the per-row ratios)."""
+    for t in layers:
+        _dev(t, "layer", torch.int32)
+    rows, k_top = layers[0].shape
+    if pairs is None:
+        pairs = [(a, b) for a in range(len(layers)) for b in range(a + 1, len(layers))]
+    dev = layers[0].device
+    ptrs = torch.tensor([t.data_ptr() for t in layers], dtype=torch.int64, device=dev)
+    pr = torch.tensor(pairs, dtype=torch.int32, device=dev).reshape(-1)
+    sums = torch.empty((len(pairs),), dtype=torch.float64, device=dev)
+    row_out = torch.empty((rows,), dtype=torch.float32, device=dev) if want_rows else None
+    _check(lib().idxc_topk_overlap(_ptr(ptrs), _ptr(pr), len(pairs), rows, k_top, _ptr(sums), _ptr(row_out), _stream(stream)),
+           "idxc_topk_overlap")
+    mean = sums / max(rows, 1)
+    return (mean, row_out) if want_rows else mean
+
+
+def pattern_search_dp(S, M: int):
+    """idxc_pattern_search_dp on a host [N, N] similarity matrix. Returns (pattern, value)."""
+    import numpy as np
+    S = np.ascontiguousarray(S, dtype=np.float64)
+    N = S.shape[0]
+    buf = ctypes.create_string_buffer(N)
+    val = ctypes.c_double()
+    _check(lib().idxc_pattern_search_dp(S.ctypes.data_as(ctypes.c_void_p), N, int(M), buf, ctypes.byref(val)),
+           "idxc_pattern_search_dp")
+    return buf.raw[:N].decode(), val.value
+
+
+def pattern_search_greedy(N: int, K: int, eval_loss):
+    """idxc_pattern_search_greedy (Algorithm 1). eval_loss(pattern: str) -> float.
+    Returns (pattern, order of flipped layers, number of evaluations)."""
+    cb = EVAL_LOSS_FN(lambda p, n, user: float(eval_loss(p[:n].decode())))
+    buf = ctypes.create_string_buffer(N)
+    order = (ctypes.c_int * max(K, 1))()
+    evals = ctypes.c_int64()
+    _check(lib().idxc_pattern_search_greedy(N, K, cb, None, buf, order, ctypes.byref(evals)), "idxc_pattern_search_greedy")
+    return buf.raw[:N].decode(), list(order)[:K], evals.value
 
 
 def selftest_bounded_wait(wait_cycles: int = 1_000_000, stream=None):

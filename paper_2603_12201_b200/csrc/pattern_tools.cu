@@ -1,0 +1,174 @@
+// Pattern tooling on index tensors (the paper's Appendix A, Appendix C and Algorithm 1).
+//   * overlap kernel: per query row |T_a n T_b| / (valid entries of T_a), for one pair of index tensors or
+//     for every pair of N layers in one launch. Both rows are ascending, so each element of one row is
+//     looked up in the other by binary search in shared memory. HBM-bound: 2 * 4 * k bytes per row pair.
+//   * similarity DP (host): the exact pattern with M Full layers that maximises the summed similarity of
+//     the Shared layers to their source layers.
+//   * greedy layer selection (host): Algorithm 1 with the caller's loss function.
+#include <vector>
+
+#include "../../include/idxc.h"
+#include "kernels.h"
+
+namespace idxc {
+namespace {
+
+constexpr int OV_THREADS = 256;
+
+// grid.x: row blocks (grid-stride), grid.y: pair index. pairs[2p], pairs[2p+1]: layer indices of pair p.
+// sums[p] accumulates the row ratios (double, atomicAdd); row_out (optional, single pair) gets each ratio.
+__global__ void __launch_bounds__(OV_THREADS)
+overlap_kernel(const int32_t* const* __restrict__ layers, const int* __restrict__ pairs, int64_t rows, int k_top,
+               double* __restrict__ sums, float* __restrict__ row_out) {
+    extern __shared__ int32_t sh[];                 // row of T_b, k_top entries
+    __shared__ int warp_cnt[OV_THREADS / 32];
+    __shared__ int valid_b_s;
+    const int p = blockIdx.y;
+    const int32_t* Ta = layers[pairs[2 * p]];
+    const int32_t* Tb = layers[pairs[2 * p + 1]];
+    double local_sum = 0.0;
+    for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
+        const int32_t* a = Ta + r * k_top;
+        const int32_t* b = Tb + r * k_top;
+        __syncthreads();
+        if (threadIdx.x == 0) valid_b_s = 0;
+        __syncthreads();
+        int nb_local = 0;
+        for (int i = threadIdx.x; i < k_top; i += OV_THREADS) {
+            const int32_t v = __ldg(b + i);
+            sh[i] = v;
+            nb_local += v >= 0;
+        }
+        if (nb_local) atomicAdd(&valid_b_s, nb_local);
+        __syncthreads();
+        const int nb = valid_b_s;                   // valid entries come first (padding is at the end)
+        int hits = 0, valid_a = 0;
+        for (int i = threadIdx.x; i < k_top; i += OV_THREADS) {
+            const int32_t v = __ldg(a + i);
+            if (v < 0) continue;
+            ++valid_a;
+            int lo = 0, hi = nb;                    // first position with sh[pos] >= v
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (sh[mid] < v) lo = mid + 1; else hi = mid;
+            }
+            hits += (lo < nb && sh[lo] == v);
+        }
+        int packed = hits | (valid_a << 16);        // both <= 2048
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) packed += __shfl_xor_sync(0xFFFFFFFFu, packed, o);
+        if ((threadIdx.x & 31) == 0) warp_cnt[threadIdx.x >> 5] = packed;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int tot = 0;
+            for (int w = 0; w < OV_THREADS / 32; ++w) tot += warp_cnt[w];
+            const int h = tot & 0xFFFF, va = tot >> 16;
+            const double ratio = va ? static_cast<double>(h) / va : 0.0;
+            local_sum += ratio;
+            if (row_out) row_out[r] = static_cast<float>(ratio);
+        }
+    }
+    if (threadIdx.x == 0) atomicAdd(&sums[p], local_sum);
+}
+
+}  // namespace
+
+cudaError_t launch_overlap(const int32_t* const* layers_dev, const int* pairs_dev, int n_pairs, int64_t rows, int k_top,
+                           double* sums_dev, float* row_out, cudaStream_t stream) {
+    if (n_pairs <= 0 || rows <= 0) return cudaSuccess;
+    const unsigned gx = static_cast<unsigned>(rows < 4096 ? rows : 4096);
+    dim3 grid(gx, static_cast<unsigned>(n_pairs));
+    overlap_kernel<<<grid, OV_THREADS, k_top * sizeof(int32_t), stream>>>(layers_dev, pairs_dev, rows, k_top, sums_dev, row_out);
+    return cudaGetLastError();
+}
+
+}  // namespace idxc
+
+using namespace idxc;
+
+extern "C" {
+
+idxc_status idxc_topk_overlap(const int32_t* const* layers, const int32_t* pairs, int n_pairs, int64_t rows, int k_top,
+                              double* sums_out, float* row_out, void* cuda_stream) {
+    if (n_pairs < 0 || rows < 0 || k_top < 1 || k_top > IDXC_MAX_K_TOP) return IDXC_ERR_INVALID_ARG;
+    if (n_pairs == 0 || rows == 0) return IDXC_OK;
+    if (!layers || !pairs || !sums_out) return IDXC_ERR_INVALID_ARG;
+    if (row_out && n_pairs != 1) return IDXC_ERR_INVALID_ARG;
+    if (n_pairs > 65535) return IDXC_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemsetAsync(sums_out, 0, sizeof(double) * n_pairs, stream) != cudaSuccess) return IDXC_ERR_CUDA;
+    return launch_overlap(layers, pairs, n_pairs, rows, k_top, sums_out, row_out, stream) == cudaSuccess ? IDXC_OK
+                                                                                                          : IDXC_ERR_CUDA;
+}
+
+// Appendix C: dp[i][m] = best total similarity of layers 0..i with m Full layers, layer i Full.
+idxc_status idxc_pattern_search_dp(const double* S, int N, int M, char* pattern_out, double* value_out) {
+    if (!S || !pattern_out || N < 1 || M < 1 || M > N) return IDXC_ERR_INVALID_ARG;
+    const double NEG = -1e300;
+    // seg[j][i] = sum_{t=j+1}^{i-1} S[t][j]: the Shared layers between Full layers j and i (i == N: to the end)
+    std::vector<std::vector<double>> seg(N, std::vector<double>(N + 1, 0.0));
+    for (int j = 0; j < N; ++j) {
+        double run = 0.0;
+        for (int i = j + 1; i <= N; ++i) {
+            seg[j][i] = run;
+            if (i < N) run += S[static_cast<size_t>(i) * N + j];
+        }
+    }
+    std::vector<std::vector<double>> dp(N, std::vector<double>(M + 1, NEG));
+    std::vector<std::vector<int>> prev(N, std::vector<int>(M + 1, -1));
+    dp[0][1] = 0.0;                                  // the first layer is always Full
+    for (int i = 1; i < N; ++i)
+        for (int m = 2; m <= M && m <= i + 1; ++m)
+            for (int j = m - 2; j < i; ++j) {
+                if (dp[j][m - 1] <= NEG) continue;
+                const double v = dp[j][m - 1] + seg[j][i];
+                if (v > dp[i][m]) { dp[i][m] = v; prev[i][m] = j; }
+            }
+    double best = NEG;
+    int last = -1;
+    for (int i = M - 1; i < N; ++i) {
+        if (dp[i][M] <= NEG) continue;
+        const double v = dp[i][M] + seg[i][N];
+        if (v > best) { best = v; last = i; }
+    }
+    if (last < 0) return IDXC_ERR_INVALID_ARG;
+    for (int l = 0; l < N; ++l) pattern_out[l] = 'S';
+    for (int i = last, m = M; i >= 0 && m >= 1; i = prev[i][m], --m) {
+        pattern_out[i] = 'F';
+        if (prev[i][m] < 0) break;
+    }
+    if (value_out) *value_out = best;
+    return IDXC_OK;
+}
+
+// Algorithm 1. Ties go to the lowest layer.
+idxc_status idxc_pattern_search_greedy(int N, int K, idxc_eval_loss_fn eval_loss, void* user, char* pattern_out,
+                                       int* order_out, int64_t* evaluations_out) {
+    if (N < 1 || K < 0 || K > N - 1 || !eval_loss || !pattern_out) return IDXC_ERR_INVALID_ARG;
+    std::vector<char> c(N + 1, 'F');
+    c[N] = '\0';
+    std::vector<int> remaining;
+    for (int l = 1; l < N; ++l) remaining.push_back(l);
+    int64_t evals = 0;
+    for (int step = 0; step < K; ++step) {
+        int best_pos = -1;
+        double best_loss = 0.0;
+        for (size_t pos = 0; pos < remaining.size(); ++pos) {
+            const int l = remaining[pos];
+            c[l] = 'S';
+            const double loss = eval_loss(c.data(), N, user);
+            c[l] = 'F';
+            ++evals;
+            if (best_pos < 0 || loss < best_loss) { best_pos = static_cast<int>(pos); best_loss = loss; }
+        }
+        const int l = remaining[best_pos];
+        c[l] = 'S';
+        remaining.erase(remaining.begin() + best_pos);
+        if (order_out) order_out[step] = l;
+    }
+    for (int l = 0; l < N; ++l) pattern_out[l] = c[l];
+    if (evaluations_out) *evaluations_out = evals;
+    return IDXC_OK;
+}
+
+}  // extern "C"

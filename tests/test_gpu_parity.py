@@ -393,3 +393,28 @@ def test_quantize_e4m3_appends_to_a_k_cache_that_the_indexer_reads():
                                     base.lens.cpu().numpy(), k_top, oracle.FP8_E4M3, f32(base.q_scale), f32(base.k_scale))
     for b in range(B):
         assert_topk_valid(topk[b].cpu().numpy(), o_sc[b, : lens_before[b] + n_new], k_top, RTOL_FP8)
+
+
+# ------------------------------------------------------------------------------ pattern tooling: top-k overlap (Appendix A)
+def test_topk_overlap_matches_oracle():
+    from oracle import pattern as opat
+    L, H, d, k_top = 700, 16, 64, 64
+    n_layers = 4
+    tops = []
+    ws = idxc.alloc_workspace(idxc.prefill_workspace_bytes(L, L, H, d, k_top), DEV)
+    for l in range(n_layers):
+        inp = synth.prefill_inputs(L, H, d, seed=60, layer=l // 2)       # layers 0,1 and 2,3 share inputs
+        if l % 2 == 1:
+            inp.w = inp.w * (1.0 + 0.5 * torch.randn(inp.w.shape, generator=torch.Generator().manual_seed(l)))
+        inp = _to_dev(inp)
+        t = torch.empty((L, k_top), dtype=torch.int32, device=DEV)
+        idxc.indexer_prefill(inp.q, inp.k, inp.w, k_top, topk_out=t, workspace=ws)
+        tops.append(t)
+    mean = idxc.topk_overlap(tops).cpu().numpy()
+    pairs = [(a, b) for a in range(n_layers) for b in range(a + 1, n_layers)]
+    host = [t.cpu().numpy() for t in tops]
+    for p, (a, b) in enumerate(pairs):
+        assert mean[p] == pytest.approx(opat.overlap(host[a], host[b]), abs=1e-9)
+    m1, rows = idxc.topk_overlap(tops, pairs=[(1, 0)], want_rows=True)
+    assert np.allclose(rows.cpu().numpy(), opat.overlap_rows(host[1], host[0]), atol=1e-6)
+    assert idxc.topk_overlap([tops[0], tops[0]]).item() == 1.0          # identical tensors overlap fully
