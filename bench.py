@@ -369,6 +369,31 @@ def time_overlap(idxc, dev, peaks, rows, k_top, n_layers):
                          "of": peaks["source"], "note": "every tensor is read n_layers-1 times; repeats may hit L2"}}
 
 
+def time_distill(idxc, dev, peaks, L, n_targets):
+    """NEXT-4: forward value of the multi-layer distillation loss (Eq. 1) on causal rows of length t+1.
+    Algorithmic bytes: 4 * (1 + n_targets) per causal pair (the scores' second read comes from L2)."""
+    g = torch.Generator(device=dev).manual_seed(13)
+    scores = torch.randn((L, L), generator=g, device=dev)
+    targets = []
+    for _ in range(n_targets):
+        p = torch.rand((L, L), generator=g, device=dev).tril_()
+        p /= p.sum(dim=1, keepdim=True)
+        targets.append(p)
+    idxc.distill_kl(scores, targets)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(5):
+        loss = idxc.distill_kl(scores, targets)
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / 5
+    nbytes = causal_pairs(L) * 4 * (1 + n_targets)
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"rows": L, "targets": n_targets, "ms": ms, "loss": float(loss.item()),
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                         "of": peaks["source"]}}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -579,6 +604,8 @@ def main():
             n_layers, sched_L = (c4["N"], c4["L"]) if args.full else (args.schedule_layers, args.schedule_L)
             line["schedule"] = time_schedule(idxc, synth, dev, sched_L, c4["H"], c4["d"], c4["k_top"], n_layers, c4["every"],
                                              seed=c4["seed"], reps=1 if args.full else 2)
+            torch.cuda.empty_cache()
+            line["distill_kl"] = time_distill(idxc, dev, peaks, 16384, 2)
             torch.cuda.empty_cache()
             line["topk_overlap"] = time_overlap(idxc, dev, peaks, 8192, c5["k_top"], 6)
             line["quantize_e4m3"] = time_quantize(idxc, dev, peaks, 32768, c5["H"], c5["d"])

@@ -246,6 +246,22 @@ idxc_status idxc_pattern_search_dp(const double* S, int N, int M, char* pattern_
 idxc_status idxc_pattern_search_greedy(int N, int K, idxc_eval_loss_fn eval_loss, void* user, char* pattern_out,
                                        int* order_out, int64_t* evaluations_out);
 
+/* ---------------------------------------------------------------------------
+ * Multi-layer distillation loss of training-aware IndexCache, forward value (Eq. 1):
+ *     L_multi = sum_{j=0..m} 1/(m+1) sum_t KL( p_t^(l+j) || Softmax(I_t) )
+ * I = indexer scores of the Full layer l, p^(l+j) = target distributions of the layers it serves.
+ *   scores   [rows, ld] fp32 (without topk: 16-byte aligned, ld a multiple of 4, targets too); row r covers
+ *            positions [0, first_len + r * len_step) (causal: 1, 1)
+ *   targets  HOST array of n_targets (= m + 1, at most 16) DEVICE pointers to [rows, ld] fp32 distributions
+ *   topk     NULL, or [rows, k_top] int32 (ascending, -1 padded): the sparse-training form, the KL is taken
+ *            over these positions only, with the target renormalised over them
+ *   loss_out DEVICE double[1] (zeroed by the call); row_loss_out NULL or DEVICE float [rows]
+ * Entries with p = 0 contribute 0.
+ * ------------------------------------------------------------------------- */
+idxc_status idxc_distill_kl(const float* scores, int64_t ld, int64_t rows, int64_t first_len, int64_t len_step,
+                            const float* const* targets, int n_targets, const int32_t* topk, int k_top,
+                            double* loss_out, float* row_loss_out, void* cuda_stream);
+
 /* Synchronises the stream, then returns IDXC_OK, IDXC_ERR_CUDA, or
  * IDXC_ERR_DEVICE_TIMEOUT if any kernel of this library recorded a bounded wait that
  * ran out since the last poll (the record is cleared). */

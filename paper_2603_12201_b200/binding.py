@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = [
     "idxc_schedule_begin_pass", "idxc_schedule_source", "idxc_schedule_stats", "idxc_schedule_prefill_layer",
     "idxc_schedule_decode_layer", "idxc_poll_device_status", "idxc_launch_count", "idxc_indexer_decode_noalloc",
     "idxc_selftest_bounded_wait", "idxc_quantize_e4m3", "idxc_topk_overlap", "idxc_pattern_search_dp",
-    "idxc_pattern_search_greedy",
+    "idxc_pattern_search_greedy", "idxc_distill_kl",
 ]
 NOALLOC_SCRATCH_BYTES = 16 << 20
 
@@ -90,6 +90,8 @@ def lib() -> ctypes.CDLL:
         L.idxc_pattern_search_greedy.restype = i32
         L.idxc_pattern_search_greedy.argtypes = [i32, i32, EVAL_LOSS_FN, vp, ctypes.c_char_p, ctypes.POINTER(i32),
                                                  ctypes.POINTER(i64)]
+        L.idxc_distill_kl.restype = i32
+        L.idxc_distill_kl.argtypes = [vp, i64, i64, i64, i64, ctypes.POINTER(vp), i32, vp, i32, vp, vp, vp]
         L.idxc_quantize_e4m3.restype = i32
         L.idxc_quantize_e4m3.argtypes = [vp, i64, i32, vp, vp, vp, vp]
         L.idxc_selftest_bounded_wait.restype = i32
@@ -298,6 +300,25 @@ def pattern_search_greedy(N: int, K: int, eval_loss):
     evals = ctypes.c_int64()
     _check(lib().idxc_pattern_search_greedy(N, K, cb, None, buf, order, ctypes.byref(evals)), "idxc_pattern_search_greedy")
     return buf.raw[:N].decode(), list(order)[:K], evals.value
+
+
+def distill_kl(scores, targets, first_len=1, len_step=1, topk=None, want_rows=False, stream=None):
+    """idxc_distill_kl: the multi-layer distillation loss (Eq. 1). scores [rows, ld] fp32; targets: list of
+    [rows, ld] fp32 distributions; topk: optional [rows, k] int32. Returns the loss as a 1-element float64 device
+    tensor (and the per-row values with want_rows)."""
+    _dev(scores, "scores", torch.float32); _dev(topk, "topk", torch.int32)
+    rows, ld = scores.shape
+    for t in targets:
+        _dev(t, "target", torch.float32)
+        if tuple(t.shape) != (rows, ld):
+            raise ValueError("targets must have the shape of scores")
+    ptrs = (ctypes.c_void_p * len(targets))(*[t.data_ptr() for t in targets])
+    loss = torch.empty((1,), dtype=torch.float64, device=scores.device)
+    row_out = torch.empty((rows,), dtype=torch.float32, device=scores.device) if want_rows else None
+    k_top = 0 if topk is None else topk.shape[1]
+    _check(lib().idxc_distill_kl(_ptr(scores), ld, rows, int(first_len), int(len_step), ptrs, len(targets), _ptr(topk), k_top,
+                                 _ptr(loss), _ptr(row_out), _stream(stream)), "idxc_distill_kl")
+    return (loss, row_out) if want_rows else loss
 
 
 def selftest_bounded_wait(wait_cycles: int = 1_000_000, stream=None):

@@ -418,3 +418,32 @@ def test_topk_overlap_matches_oracle():
     m1, rows = idxc.topk_overlap(tops, pairs=[(1, 0)], want_rows=True)
     assert np.allclose(rows.cpu().numpy(), opat.overlap_rows(host[1], host[0]), atol=1e-6)
     assert idxc.topk_overlap([tops[0], tops[0]]).item() == 1.0          # identical tensors overlap fully
+
+
+# ------------------------------------------------------------------------------ multi-layer distillation loss (Eq. 1)
+def test_distill_kl_matches_oracle():
+    from oracle import distill as odist
+    L, H, d, k_top = 300, 16, 64, 32
+    inp = _to_dev(synth.prefill_inputs(L, H, d, seed=70))
+    g_scores, g_topk = _gpu_prefill(inp, k_top)
+    scores = torch.nan_to_num(torch.from_numpy(g_scores), nan=0.0).to(DEV).contiguous()      # entries above the diagonal are unused
+    gen = torch.Generator().manual_seed(71)
+    targets = []
+    for j in range(3):
+        p = torch.rand((L, scores.shape[1]), generator=gen) * torch.tril(torch.ones(L, scores.shape[1]))
+        p[:, 5] = 0.0                                           # exact zeros in a target contribute nothing
+        p[5, 5] = 1.0
+        targets.append((p / p.sum(dim=1, keepdim=True)).to(DEV).contiguous())
+    loss, rows = idxc.distill_kl(scores, targets, want_rows=True)
+    want, want_rows = odist.multi_layer_loss(scores.cpu().numpy(), [t.cpu().numpy() for t in targets])
+    assert loss.item() == pytest.approx(want, rel=2e-5)
+    assert np.allclose(rows.cpu().numpy(), want_rows, rtol=1e-4, atol=1e-6)
+    # sparse-training form on the indices the top-k kernel selected
+    tk = torch.from_numpy(g_topk).to(DEV)
+    loss_k, rows_k = idxc.distill_kl(scores, targets, topk=tk, want_rows=True)
+    want_k, want_rows_k = odist.multi_layer_loss(scores.cpu().numpy(), [t.cpu().numpy() for t in targets], topk=g_topk)
+    assert loss_k.item() == pytest.approx(want_k, rel=2e-5)
+    assert np.allclose(rows_k.cpu().numpy(), want_rows_k, rtol=1e-4, atol=1e-6)
+    # the loss of the Softmax of the scores against itself is zero
+    q = torch.softmax(scores.masked_fill(torch.triu(torch.ones_like(scores, dtype=torch.bool), diagonal=1), float("-inf")), dim=1)
+    assert abs(idxc.distill_kl(scores, [q.contiguous()]).item()) < 1e-3 * L
