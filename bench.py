@@ -423,10 +423,16 @@ def main():
         raise SystemExit("bench.py needs a CUDA device: the indexer has no CPU path (use --impl reference for the oracle)")
     from paper_2603_12201_b200 import dist as pdist
     _, _, local = pdist.env_rank_world()
-    dev = torch.device("cuda", local)
+    # IDXC_BENCH_BACKEND=gloo is a functional smoke path for boxes with fewer GPUs than ranks: the ranks then
+    # share the visible GPUs and the (host-side) timing reduction goes through gloo. Numbers from it mean nothing.
+    backend = os.environ.get("IDXC_BENCH_BACKEND", "nccl")
+    dev = torch.device("cuda", local % torch.cuda.device_count() if backend == "gloo" else local)
     torch.cuda.set_device(dev)
-    rank, world = pdist.init("nccl", dev)
-    barrier, max_over_ranks = pdist.barrier, pdist.max_over_ranks
+    rank, world = pdist.init(backend, dev)
+    barrier = pdist.barrier
+
+    def max_over_ranks(x, w, device):
+        return pdist.max_over_ranks(x, w, "cpu" if backend == "gloo" else device)
     from paper_2603_12201_b200 import binding as idxc
     from paper_2603_12201_b200 import synth
     idxc.lib()
