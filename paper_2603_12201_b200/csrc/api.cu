@@ -2,8 +2,10 @@
 // host-side IndexCache schedule object. No device memory is allocated here.
 #include <atomic>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
+#include <utility>
 #include <vector>
 
 #include "../../include/idxc.h"
@@ -25,15 +27,23 @@ struct DeviceInfo {
     decltype(&cuTensorMapEncodeTiled) encode = nullptr;
 };
 
+constexpr int kMaxDevices = 64;
+std::mutex g_info_mutex;
+
+// Per-device facts (SM count, address of this device's status word), looked up once per device
+// under a mutex: a process may drive several devices and call from several threads.
 DeviceInfo& device_info() {
-    static DeviceInfo info;
+    static DeviceInfo infos[kMaxDevices];
+    static DeviceInfo bad;            // ok == false: no current device, or an index beyond the table
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return bad;
+    std::lock_guard<std::mutex> lock(g_info_mutex);
+    DeviceInfo& info = infos[dev];
     if (!info.ready) {
         info.ready = true;
-        int dev = 0;
         void* fn = nullptr;
         cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&info.sm_count, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
+        if (cudaDeviceGetAttribute(&info.sm_count, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
             cudaGetSymbolAddress(reinterpret_cast<void**>(&info.status_ptr), g_device_status) == cudaSuccess &&
             cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
             qres == cudaDriverEntryPointSuccess && fn != nullptr) {
@@ -90,6 +100,22 @@ idxc_status launch_scorer(const ScoreArgs& a, bool decode, uint32_t flags, cudaS
 }
 
 }  // namespace
+
+// Function attributes are per device: remember which (kernel, device) pairs have been raised.
+cudaError_t ensure_max_dynamic_smem(const void* kernel, int bytes) {
+    static std::mutex mu;
+    static std::vector<std::pair<const void*, int>> done;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(mu);
+    for (const auto& p : done)
+        if (p.first == kernel && p.second == dev) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) done.emplace_back(kernel, dev);
+    return e;
+}
+
 }  // namespace idxc
 
 using namespace idxc;

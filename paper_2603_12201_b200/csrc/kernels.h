@@ -8,6 +8,9 @@
 
 namespace idxc {
 
+// Raises a kernel's dynamic shared-memory limit to `bytes` once per (kernel, device); thread-safe (api.cu).
+cudaError_t ensure_max_dynamic_smem(const void* kernel, int bytes);
+
 // Row-wise top-k select (topk.cu). Row r has length lens[r] (device) if lens != nullptr,
 // else first_len + r * len_step, clamped to [0, ld].
 cudaError_t launch_topk_rows(const float* scores, int64_t ld, int64_t n_rows, int64_t first_len,

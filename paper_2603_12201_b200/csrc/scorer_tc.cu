@@ -352,12 +352,7 @@ cudaError_t launch_prefill_instance(const ScoreArgs& a, const CUtensorMap& q_map
                                     unsigned int* status, int sm_count, cudaStream_t stream) {
     using Cfg = PrefillCfg<NKH>;
     auto kern = score_prefill_tc_kernel<NKH, H, FP8>;
-    static bool attr_done = false;   // per instantiation; the attribute is per function, setting it twice is harmless
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    if (cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(kern), Cfg::kSmemBytes); e != cudaSuccess) return e;
     constexpr int QB = 2 * (kTileCols / H);
     const int64_t n_items = (a.n_rows + QB - 1) / QB;
     const int grid = static_cast<int>(n_items < sm_count ? n_items : sm_count);
@@ -694,12 +689,7 @@ cudaError_t launch_decode_instance(const ScoreArgs& a, const CUtensorMap& q_map,
                                    unsigned int* status, int sm_count, cudaStream_t stream) {
     using Cfg = DecodeCfg<NKH, H>;
     auto kern = score_decode_tc_kernel<NKH, H, FP8>;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    if (cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(kern), Cfg::kSmemBytes); e != cudaSuccess) return e;
     const int64_t tiles = (a.max_len + kTileKeys - 1) / kTileKeys;
     const int64_t items = a.n_rows * ((tiles + kDecodeChunkTiles - 1) / kDecodeChunkTiles);
     if (items <= 0) return cudaSuccess;

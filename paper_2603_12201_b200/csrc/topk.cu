@@ -173,12 +173,7 @@ template <int THREADS, int MIN_BLOCKS, int CAP_DYN>
 cudaError_t launch_instance(const float* scores, int64_t ld, int64_t n_rows, int64_t first_len, int64_t len_step,
                             const int32_t* lens, int k_top, int32_t* out, int map_bytes, cudaStream_t stream) {
     auto kern = topk_rows_kernel<THREADS, MIN_BLOCKS, CAP_DYN>;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TK_MAP_MAX_BYTES + 8 * CAP_DYN);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    if (cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(kern), TK_MAP_MAX_BYTES + 8 * CAP_DYN); e != cudaSuccess) return e;
     const int64_t max_grid = 1 << 20;
     const unsigned grid = static_cast<unsigned>(n_rows < max_grid ? n_rows : max_grid);
     kern<<<grid, THREADS, map_bytes + 8 * CAP_DYN, stream>>>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, map_bytes * 4);

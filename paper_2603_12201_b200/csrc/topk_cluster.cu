@@ -240,13 +240,7 @@ cudaError_t launch_topk_rows_cluster(const float* scores, int64_t ld, int64_t n_
     const int64_t part = (((longest + CL_SIZE - 1) / CL_SIZE) + 127) & ~int64_t(127);
     const int map_bytes = static_cast<int>(part / 4);
     const int dyn_bytes = map_bytes + 2 * CL_CAP * 4;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(topk_rows_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             CL_MAX_PART / 4 + 2 * CL_CAP * 4);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    if (cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(topk_rows_cluster_kernel), CL_MAX_PART / 4 + 2 * CL_CAP * 4); e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(n_rows * CL_SIZE));
     cfg.blockDim = dim3(CL_THREADS);
