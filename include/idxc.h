@@ -262,6 +262,35 @@ idxc_status idxc_distill_kl(const float* scores, int64_t ld, int64_t rows, int64
                             const float* const* targets, int n_targets, const int32_t* topk, int k_top,
                             double* loss_out, float* row_loss_out, void* cuda_stream);
 
+/* ---------------------------------------------------------------------------
+ * Sparse core attention over the selected positions (Sec. 2.1 "DeepSeek Sparse Attention": "the main attention
+ * is computed only over this sparse subset"; Fig. 2: X <- SparseAttn_l(X, T^(l))). The paper runs it under
+ * Multi-head Latent Attention and prints no shapes; this entry point takes the multi-query form latent
+ * attention is served in: all heads of a query attend the same row per token, whose leading d_v columns are
+ * also the value:
+ *     s[t,h,j]   = scale * < q[t,h,:], kv[kv_base[t] + topk[t,j], 0:d_qk] >      for usable entries
+ *     out[t,h,:] = sum_j Softmax_j(s[t,h,:])[j] * kv[kv_base[t] + topk[t,j], 0:d_v]
+ *     lse[t,h]   = log sum_j exp(s[t,h,j])                                        (natural logarithm)
+ * An entry is usable when topk[t,j] >= 0 and the row it names lies inside [0, n_kv); other entries are
+ * skipped (they may sit anywhere in the row, order is free, duplicates count twice). A query without usable
+ * entries gets out = 0 and lse = -inf.
+ *   q        DEVICE bf16 [n_q, H, d_qk], 16-byte aligned      kv  DEVICE bf16 [n_kv, d_qk], 16-byte aligned
+ *   topk     DEVICE int32 [n_q, k_top] (k_top >= 1)            kv_base  NULL or DEVICE int64 [n_q] (decode: the
+ *            first cache row of the query's sequence; prefill: NULL)
+ *   out      DEVICE bf16 [n_q, H, d_v], 16-byte aligned        lse  NULL or DEVICE fp32 [n_q, H]
+ *   workspace DEVICE, idxc_sparse_attention_workspace_bytes(n_q) bytes, 16-byte aligned; caller-owned
+ * Supported shape: 1 <= H <= 128, d_qk = 576, d_v = 512 (tcgen05 path); anything else IDXC_ERR_UNSUPPORTED.
+ * Arithmetic: bf16 products with fp32 accumulation, fp32 softmax with the probabilities rounded to bf16 for
+ * the second product, bf16 output. Unselected rows are never read, except that row 0 of kv stands in for
+ * skipped entries with weight 0 and must therefore hold finite numbers. Enqueues 2 kernels; nothing is
+ * allocated. Errors: IDXC_ERR_INVALID_ARG (null or misaligned pointer, sizes out of range),
+ * IDXC_ERR_WORKSPACE, IDXC_ERR_UNSUPPORTED, IDXC_ERR_CUDA.
+ * ------------------------------------------------------------------------- */
+size_t idxc_sparse_attention_workspace_bytes(int64_t n_q);
+idxc_status idxc_sparse_attention(const void* q, const void* kv, const int32_t* topk, const int64_t* kv_base,
+                                  int64_t n_q, int64_t n_kv, int H, int d_qk, int d_v, int k_top, float scale,
+                                  void* out, float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* Synchronises the stream, then returns IDXC_OK, IDXC_ERR_CUDA, or
  * IDXC_ERR_DEVICE_TIMEOUT if any kernel of this library recorded a bounded wait that
  * ran out since the last poll (the record is cleared). */

@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = [
     "idxc_schedule_begin_pass", "idxc_schedule_source", "idxc_schedule_stats", "idxc_schedule_prefill_layer",
     "idxc_schedule_decode_layer", "idxc_poll_device_status", "idxc_launch_count", "idxc_indexer_decode_noalloc",
     "idxc_selftest_bounded_wait", "idxc_quantize_e4m3", "idxc_topk_overlap", "idxc_pattern_search_dp",
-    "idxc_pattern_search_greedy", "idxc_distill_kl",
+    "idxc_pattern_search_greedy", "idxc_distill_kl", "idxc_sparse_attention_workspace_bytes", "idxc_sparse_attention",
 ]
 NOALLOC_SCRATCH_BYTES = 16 << 20
 
@@ -92,6 +92,10 @@ def lib() -> ctypes.CDLL:
                                                  ctypes.POINTER(i64)]
         L.idxc_distill_kl.restype = i32
         L.idxc_distill_kl.argtypes = [vp, i64, i64, i64, i64, ctypes.POINTER(vp), i32, vp, i32, vp, vp, vp]
+        L.idxc_sparse_attention_workspace_bytes.restype = sz
+        L.idxc_sparse_attention_workspace_bytes.argtypes = [i64]
+        L.idxc_sparse_attention.restype = i32
+        L.idxc_sparse_attention.argtypes = [vp, vp, vp, vp, i64, i64, i32, i32, i32, i32, ctypes.c_float, vp, vp, vp, sz, vp]
         L.idxc_quantize_e4m3.restype = i32
         L.idxc_quantize_e4m3.argtypes = [vp, i64, i32, vp, vp, vp, vp]
         L.idxc_selftest_bounded_wait.restype = i32
@@ -319,6 +323,28 @@ def distill_kl(scores, targets, first_len=1, len_step=1, topk=None, want_rows=Fa
     _check(lib().idxc_distill_kl(_ptr(scores), ld, rows, int(first_len), int(len_step), ptrs, len(targets), _ptr(topk), k_top,
                                  _ptr(loss), _ptr(row_out), _stream(stream)), "idxc_distill_kl")
     return (loss, row_out) if want_rows else loss
+
+
+def sparse_attention(q, kv, topk, d_v, scale, kv_base=None, want_lse=True, out=None, workspace=None, stream=None):
+    """idxc_sparse_attention: attention of q [n_q, H, d_qk] bf16 over the rows of kv [n_kv, d_qk] bf16 named by
+    topk [n_q, k_top] int32 (entries < 0 skipped); values are the leading d_v columns of the same rows.
+    Returns (out [n_q, H, d_v] bf16, lse [n_q, H] fp32 or None)."""
+    _dev(q, "q", torch.bfloat16); _dev(kv, "kv", torch.bfloat16); _dev(topk, "topk", torch.int32)
+    _dev(kv_base, "kv_base", torch.int64)
+    n_q, H, d_qk = q.shape
+    n_kv = kv.shape[0]
+    if kv.shape[1] != d_qk or topk.shape[0] != n_q:
+        raise ValueError("kv must be [n_kv, d_qk] and topk [n_q, k_top]")
+    if out is None:
+        out = torch.empty((n_q, H, d_v), dtype=torch.bfloat16, device=q.device)
+    lse = torch.empty((n_q, H), dtype=torch.float32, device=q.device) if want_lse else None
+    need = int(lib().idxc_sparse_attention_workspace_bytes(n_q))
+    if workspace is None:
+        workspace = alloc_workspace(max(need, 256), q.device)
+    _check(lib().idxc_sparse_attention(_ptr(q), _ptr(kv), _ptr(topk), _ptr(kv_base), n_q, n_kv, H, d_qk, int(d_v), topk.shape[1],
+                                       ctypes.c_float(scale), _ptr(out), _ptr(lse), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                       _stream(stream)), "idxc_sparse_attention")
+    return out, lse
 
 
 def selftest_bounded_wait(wait_cycles: int = 1_000_000, stream=None):

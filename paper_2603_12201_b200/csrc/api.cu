@@ -411,6 +411,32 @@ idxc_status idxc_quantize_e4m3(const void* x, int64_t n_tokens, int row_elems, v
                                 static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? IDXC_OK : IDXC_ERR_CUDA;
 }
 
+size_t idxc_sparse_attention_workspace_bytes(int64_t n_q) {
+    return n_q > 0 ? static_cast<size_t>(round_up(n_q * 4, 256)) : 0;
+}
+
+idxc_status idxc_sparse_attention(const void* q, const void* kv, const int32_t* topk, const int64_t* kv_base, int64_t n_q,
+                                  int64_t n_kv, int H, int d_qk, int d_v, int k_top, float scale, void* out, float* lse,
+                                  void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (n_q < 0 || n_kv < 0 || H < 1 || d_qk < 1 || d_v < 1 || d_v > d_qk || k_top < 1) return IDXC_ERR_INVALID_ARG;
+    if (!sparse_attn_supported(H, d_qk, d_v)) return IDXC_ERR_UNSUPPORTED;
+    if (n_q == 0) return IDXC_OK;
+    if (n_q * H >= (int64_t(1) << 31)) return IDXC_ERR_INVALID_ARG;
+    if (!q || !topk || !out || (n_kv > 0 && !kv)) return IDXC_ERR_INVALID_ARG;
+    if (!aligned(q, 16) || !aligned(kv, 16) || !aligned(out, 16) || !aligned(topk, 4) || (kv_base && !aligned(kv_base, 8)) ||
+        (lse && !aligned(lse, 4)))
+        return IDXC_ERR_INVALID_ARG;
+    if (!workspace || !aligned(workspace, 16) || workspace_bytes < idxc_sparse_attention_workspace_bytes(n_q)) return IDXC_ERR_WORKSPACE;
+    DeviceInfo& di = device_info();
+    if (!di.ok) return IDXC_ERR_CUDA;
+    CUtensorMap q_map;
+    if (!encode_operand_map(&q_map, q, n_q * H, d_qk, false, H)) return IDXC_ERR_CUDA;
+    g_launches += 2;
+    return launch_sparse_attn(kv, topk, kv_base, n_q, n_kv, H, k_top, scale, out, lse, static_cast<int32_t*>(workspace), q_map,
+                              di.status_ptr, di.sm_count, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+               ? IDXC_OK : IDXC_ERR_CUDA;
+}
+
 idxc_status idxc_selftest_bounded_wait(uint32_t wait_cycles, void* cuda_stream) {
     if (!device_info().ok) return IDXC_ERR_CUDA;
     const long long budget = wait_cycles > 100000000u ? 100000000LL : static_cast<long long>(wait_cycles);

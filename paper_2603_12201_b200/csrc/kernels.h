@@ -59,6 +59,13 @@ bool score_tc_supported(int H, int d, int fp8);
 cudaError_t launch_quantize_e4m3(const void* x, int64_t n_tokens, int row_elems, void* codes, float* scale,
                                  const int64_t* dst_rows, cudaStream_t stream);
 
+// sparse_attn.cu: attention over the selected rows. q_map: q as [n_q * H, 576] bf16, 128-byte swizzle, box
+// 64 columns x H rows. n_eff: [n_q] int32 scratch.
+bool sparse_attn_supported(int H, int d_qk, int d_v);
+cudaError_t launch_sparse_attn(const void* kv, const int32_t* topk, const int64_t* kv_base, int64_t n_q, int64_t n_kv, int H,
+                               int k_top, float scale, void* out, float* lse, int32_t* n_eff, const CUtensorMap& q_map,
+                               unsigned int* status, int sm_count, cudaStream_t stream);
+
 // selftest.cu: one tiny kernel whose only wait can never be satisfied; it must record a time-out in
 // `status` after `budget_cycles` and return.
 cudaError_t launch_selftest_bounded_wait(unsigned int* status, long long budget_cycles, cudaStream_t stream);

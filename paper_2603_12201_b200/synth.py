@@ -27,7 +27,7 @@ import torch
 
 E4M3_MAX = 448.0
 
-_TENSOR_IDS = {"q": 1, "k": 2, "w": 3, "centers": 4, "ids": 5, "lens": 6}
+_TENSOR_IDS = {"q": 1, "k": 2, "w": 3, "centers": 4, "ids": 5, "lens": 6, "attn_q": 7, "attn_kv": 8, "sel": 9}
 
 
 def _gen(seed: int, layer: int, name: str, device) -> torch.Generator:
@@ -139,6 +139,50 @@ def decode_inputs(B: int, H: int, d: int, len_lo: int, len_hi: int, seed: int, d
     w = _randn((B, H), _gen(seed, layer, "w", dev), dev) * (1.0 / math.sqrt(H))
     return DecodeInputs(q_step, k_cache, w.contiguous(), q_scale, k_scale, offs.to(dev), lens_t.to(torch.int32).to(dev),
                         int(lens_t.max().item()) if B else 0, fp8)
+
+
+@dataclass
+class AttnInputs:
+    q: torch.Tensor                 # [n_q, H, d_qk] bf16: attention queries
+    kv: torch.Tensor                # [n_kv, d_qk] bf16: one shared latent row per token (values = leading columns)
+
+
+def attention_inputs(n_q: int, n_kv: int, H: int, d_qk: int, seed: int, device="cpu", layer: int = 0) -> AttnInputs:
+    """Inputs of the sparse core attention: q, kv ~ N(0, 1) rounded to bf16 (latent rows of a normalised
+    cache have unit RMS). No trained weights are involved: the rows are synthetic."""
+    dev = torch.device(device)
+    gq = _gen(seed, layer, "attn_q", dev)
+    q = torch.empty((n_q, H, d_qk), dtype=torch.bfloat16, device=dev)
+    slab = max(1, min(n_q, (1 << 28) // (H * d_qk))) if n_q else 1
+    for r0 in range(0, n_q, slab):
+        r1 = min(n_q, r0 + slab)
+        q[r0:r1] = _randn((r1 - r0, H, d_qk), gq, dev).to(torch.bfloat16)
+    kv = _randn((n_kv, d_qk), _gen(seed, layer, "attn_kv", dev), dev).to(torch.bfloat16)
+    return AttnInputs(q, kv)
+
+
+def random_selection(positions, k_top: int, seed: int, device="cpu", layer: int = 0) -> torch.Tensor:
+    """A stand-in for an indexer's output: for each query position t in ``positions`` a uniformly random set of
+    min(k_top, t + 1) distinct causal positions from [0, t], ascending, padded with -1. [len(positions), k_top] int32."""
+    dev = torch.device(device)
+    pos = torch.as_tensor(positions, dtype=torch.int64, device=dev)
+    n = int(pos.max().item()) + 1 if pos.numel() else 0
+    g = _gen(seed, layer, "sel", dev)
+    out = torch.full((pos.numel(), k_top), -1, dtype=torch.int32, device=dev)
+    step = max(1, (1 << 26) // max(n, 1))
+    ar = torch.arange(n, device=dev)
+    for r0 in range(0, pos.numel(), step):
+        p = pos[r0:r0 + step]
+        key = torch.rand((p.numel(), n), generator=g, device=dev)
+        key.masked_fill_(ar[None, :] > p[:, None], 2.0)                  # not causal: never drawn
+        kk = min(k_top, n)
+        val, idx = torch.topk(key, kk, dim=1, largest=False)
+        idx = torch.where(val <= 1.0, idx, torch.full_like(idx, n + 1))  # fewer than k_top causal positions
+        idx, _ = torch.sort(idx, dim=1)
+        idx = torch.where(idx > n, torch.full_like(idx, -1), idx)
+        # ascending with the -1 padding at the end
+        out[r0:r0 + step, :kk] = idx.to(torch.int32)
+    return out
 
 
 def uniform_pattern(n_layers: int, every: int) -> str:

@@ -1,0 +1,129 @@
+"""Parity of idxc_sparse_attention with the oracle (Sec. 2.1: attention over the selected subset; Fig. 2 SparseAttn).
+
+Tolerance. Scores are exact bf16 products summed in fp32 (error ~1e-6 of the operand norms, negligible). The
+probabilities are rounded to bf16 before the second product: independent relative errors, uniform within 2^-9,
+standard deviation 2^-9 / sqrt(3) = 1.1e-3, so the output moves by about 1.1e-3 * sqrt(sum_j p_j^2 v_j^2), which is
+also the scale of the output row itself (its rms). The output is then rounded to bf16: up to 2^-9 = 2e-3 relative.
+Together about 1.6e-3 * rms per output as a standard deviation; the cases below compare several million outputs,
+whose largest deviation sits near 5.5 sigma = 9e-3 * rms. The bound used is
+|gpu - oracle| <= 1.5e-2 * max(|oracle|, rms of that (query, head) output row), about 9 sigma; an indexing or
+masking mistake moves outputs by the order of rms itself. lse is compared to 2e-3 absolute.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import sparse_attn as osa
+from paper_2603_12201_b200 import binding, synth
+from tests.util import codes
+
+pytestmark = pytest.mark.gpu
+
+RTOL_ATTN = 1.5e-2
+ATOL_LSE = 2e-3
+H, D_QK, D_V = 128, 576, 512
+
+
+def _check(out, lse, o_out, o_lse, rows, what):
+    g = out.float().cpu().numpy()[rows].astype(np.float64)
+    rms = np.sqrt(np.mean(np.square(o_out), axis=-1, keepdims=True))
+    bound = RTOL_ATTN * np.maximum(np.abs(o_out), rms)
+    err = np.abs(g - o_out)
+    bad = err > bound
+    assert not bad.any(), f"{what}: {int(bad.sum())} outputs off, worst {float((err / np.maximum(bound, 1e-300)).max()):.2f}x the bound at {np.argwhere(bad)[0]}"
+    if lse is not None:
+        gl = lse.cpu().numpy()[rows].astype(np.float64)
+        fin = np.isfinite(o_lse)
+        assert np.array_equal(np.isneginf(gl), np.isneginf(o_lse)), f"{what}: lse -inf pattern"
+        assert np.all(np.abs(gl[fin] - o_lse[fin]) <= ATOL_LSE), f"{what}: lse off by {np.abs(gl[fin] - o_lse[fin]).max()}"
+    return float((err / np.maximum(bound, 1e-300)).max())
+
+
+def _run(inp, topk, scale, kv_base=None, rows=None, h=H, what=""):
+    out, lse = binding.sparse_attention(inp.q, inp.kv, topk, D_V, scale, kv_base=kv_base)
+    binding.poll_device_status()
+    rows = np.arange(inp.q.shape[0]) if rows is None else np.asarray(rows)
+    o_out, o_lse = osa.sparse_attention(codes(inp.q), codes(inp.kv), topk.cpu().numpy(), D_V, scale,
+                                        kv_base=None if kv_base is None else kv_base.cpu().numpy(), rows=rows)
+    return _check(out, lse, o_out, o_lse, rows, what)
+
+
+def test_prefill_ragged_rows_flat_and_peaked_softmax():
+    # positions chosen so that rows hold 1, 63, 64, 65, 127..129, 2047, 2048 entries: several tiles and ragged tails
+    pos = [0, 62, 63, 64, 126, 127, 128, 1000, 2046, 2047, 2048, 2500, 2999]
+    n_kv = 3000
+    inp = synth.attention_inputs(len(pos), n_kv, H, D_QK, seed=11, device="cuda")
+    topk = synth.random_selection(pos, 2048, seed=11, device="cuda")
+    assert int((topk[3] >= 0).sum()) == 65 and int((topk[-1] >= 0).sum()) == 2048
+    _run(inp, topk, 1.0 / np.sqrt(D_QK), what="flat")
+    # a large scale makes the softmax peaked: the running reference maximum has to move and O be rescaled
+    _run(inp, topk, 0.3, what="peaked")
+
+
+def test_many_queries_span_all_ctas():
+    n_q, n_kv = 400, 4096                      # more queries than SMs: every CTA walks several queries
+    pos = torch.randint(0, n_kv, (n_q,), generator=torch.Generator().manual_seed(5)).tolist()
+    inp = synth.attention_inputs(n_q, n_kv, H, D_QK, seed=12, device="cuda")
+    topk = synth.random_selection(pos, 512, seed=12, device="cuda")
+    rows = list(range(0, n_q, 9)) + [n_q - 1]
+    _run(inp, topk, 0.08, rows=rows, what="many")
+
+
+def test_skipped_entries_anywhere_out_of_range_and_empty_rows():
+    n_q, n_kv, k_top = 6, 500, 300
+    inp = synth.attention_inputs(n_q, n_kv, H, D_QK, seed=13, device="cuda")
+    topk = synth.random_selection([499] * n_q, k_top, seed=13, device="cuda")
+    g = torch.Generator().manual_seed(1)
+    holes = torch.rand((k_top,), generator=g) < 0.3
+    topk[0, holes.cuda()] = -1                               # holes anywhere
+    topk[1, 64:128] = -1                                     # one whole tile of holes
+    topk[2, :] = -1                                          # nothing selected
+    topk[3, 10:20] = 100000                                  # outside the cache: skipped
+    topk[4] = topk[4].flip(0)                                # order is free
+    topk[5, 1:] = -1                                         # a single entry: out = its value row
+    out, lse = binding.sparse_attention(inp.q, inp.kv, topk, D_V, 0.1)
+    binding.poll_device_status()
+    ref_topk = topk.cpu().numpy().copy()
+    ref_topk[ref_topk >= n_kv] = -1
+    o_out, o_lse = osa.sparse_attention(codes(inp.q), codes(inp.kv), ref_topk, D_V, 0.1)
+    _check(out, lse, o_out, o_lse, np.arange(n_q), "holes")
+    assert torch.all(out[2] == 0) and torch.all(torch.isneginf(lse[2]))
+    only = int(topk[5, 0])
+    assert torch.equal(out[5], inp.kv[only, :D_V].expand(H, D_V))
+
+
+def test_fewer_heads_and_decode_style_base_offsets():
+    h, B = 16, 5
+    lens = [700, 64, 2100, 1, 300]
+    offs = np.concatenate([[0], np.cumsum([((n + 127) // 128) * 128 for n in lens])[:-1]])
+    n_kv = int(offs[-1] + lens[-1])
+    inp = synth.attention_inputs(B, n_kv, h, D_QK, seed=14, device="cuda")
+    topk = synth.random_selection([n - 1 for n in lens], 2048, seed=14, device="cuda")       # relative to the sequence
+    base = torch.as_tensor(offs, dtype=torch.int64, device="cuda")
+    _run(inp, topk, 0.06, kv_base=base, h=h, what="decode")
+
+
+def test_indices_from_the_indexer_chain():
+    # the real chain: indexer scores -> top-k -> attention over those rows
+    L, k_top = 1536, 256
+    pin = synth.prefill_inputs(L, 64, 128, seed=15, device="cuda", clustered=True)
+    topk = torch.empty((L, k_top), dtype=torch.int32, device="cuda")
+    ws = binding.alloc_workspace(binding.prefill_workspace_bytes(L, L, 64, 128, k_top), "cuda")
+    binding.indexer_prefill(pin.q, pin.k, pin.w, k_top, topk_out=topk, workspace=ws)
+    inp = synth.attention_inputs(L, L, H, D_QK, seed=15, device="cuda")
+    rows = [0, 1, 63, 255, 256, 257, 777, L - 1]
+    _run(inp, topk, 1.0 / np.sqrt(D_QK), rows=rows, what="chain")
+
+
+def test_argument_errors():
+    inp = synth.attention_inputs(2, 10, H, D_QK, seed=1, device="cuda")
+    topk = torch.zeros((2, 8), dtype=torch.int32, device="cuda")
+    with pytest.raises(binding.IdxcError) as e:
+        binding.sparse_attention(inp.q[:, :, :512].contiguous(), inp.kv[:, :512].contiguous(), topk, 256, 1.0)
+    assert e.value.status == binding.ERR_UNSUPPORTED
+    with pytest.raises(binding.IdxcError) as e:
+        binding.sparse_attention(inp.q, inp.kv, topk, D_V, 1.0, workspace=torch.empty(4, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == binding.ERR_WORKSPACE
+    # zero queries: nothing to do
+    out, _ = binding.sparse_attention(inp.q[:0], inp.kv, topk[:0], D_V, 1.0)
+    assert out.shape == (0, H, D_V)
