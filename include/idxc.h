@@ -278,7 +278,9 @@ idxc_status idxc_distill_kl(const float* scores, int64_t ld, int64_t rows, int64
  *   topk     DEVICE int32 [n_q, k_top] (k_top >= 1)            kv_base  NULL or DEVICE int64 [n_q] (decode: the
  *            first cache row of the query's sequence; prefill: NULL)
  *   out      DEVICE bf16 [n_q, H, d_v], 16-byte aligned        lse  NULL or DEVICE fp32 [n_q, H]
- *   workspace DEVICE, idxc_sparse_attention_workspace_bytes(n_q) bytes, 16-byte aligned; caller-owned
+ *   workspace DEVICE, idxc_sparse_attention_workspace_bytes(n_q, k_top) bytes, 16-byte aligned; caller-owned.
+ *            It holds per-query entry counts and, per resident CTA, a query's probabilities between its two
+ *            passes over the selected rows (about 0.5 MB per CTA at k_top = 2048)
  * Supported shape: 1 <= H <= 128, d_qk = 576, d_v = 512 (tcgen05 path); anything else IDXC_ERR_UNSUPPORTED.
  * Arithmetic: bf16 products with fp32 accumulation, fp32 softmax with the probabilities rounded to bf16 for
  * the second product, bf16 output. Unselected rows are never read, except that row 0 of kv stands in for
@@ -286,7 +288,7 @@ idxc_status idxc_distill_kl(const float* scores, int64_t ld, int64_t rows, int64
  * allocated. Errors: IDXC_ERR_INVALID_ARG (null or misaligned pointer, sizes out of range),
  * IDXC_ERR_WORKSPACE, IDXC_ERR_UNSUPPORTED, IDXC_ERR_CUDA.
  * ------------------------------------------------------------------------- */
-size_t idxc_sparse_attention_workspace_bytes(int64_t n_q);
+size_t idxc_sparse_attention_workspace_bytes(int64_t n_q, int k_top);
 idxc_status idxc_sparse_attention(const void* q, const void* kv, const int32_t* topk, const int64_t* kv_base,
                                   int64_t n_q, int64_t n_kv, int H, int d_qk, int d_v, int k_top, float scale,
                                   void* out, float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream);

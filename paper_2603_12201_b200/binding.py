@@ -93,7 +93,7 @@ def lib() -> ctypes.CDLL:
         L.idxc_distill_kl.restype = i32
         L.idxc_distill_kl.argtypes = [vp, i64, i64, i64, i64, ctypes.POINTER(vp), i32, vp, i32, vp, vp, vp]
         L.idxc_sparse_attention_workspace_bytes.restype = sz
-        L.idxc_sparse_attention_workspace_bytes.argtypes = [i64]
+        L.idxc_sparse_attention_workspace_bytes.argtypes = [i64, i32]
         L.idxc_sparse_attention.restype = i32
         L.idxc_sparse_attention.argtypes = [vp, vp, vp, vp, i64, i64, i32, i32, i32, i32, ctypes.c_float, vp, vp, vp, sz, vp]
         L.idxc_quantize_e4m3.restype = i32
@@ -338,7 +338,7 @@ def sparse_attention(q, kv, topk, d_v, scale, kv_base=None, want_lse=True, out=N
     if out is None:
         out = torch.empty((n_q, H, d_v), dtype=torch.bfloat16, device=q.device)
     lse = torch.empty((n_q, H), dtype=torch.float32, device=q.device) if want_lse else None
-    need = int(lib().idxc_sparse_attention_workspace_bytes(n_q))
+    need = int(lib().idxc_sparse_attention_workspace_bytes(n_q, topk.shape[1]))
     if workspace is None:
         workspace = alloc_workspace(max(need, 256), q.device)
     _check(lib().idxc_sparse_attention(_ptr(q), _ptr(kv), _ptr(topk), _ptr(kv_base), n_q, n_kv, H, d_qk, int(d_v), topk.shape[1],

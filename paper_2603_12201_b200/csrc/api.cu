@@ -411,8 +411,9 @@ idxc_status idxc_quantize_e4m3(const void* x, int64_t n_tokens, int row_elems, v
                                 static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? IDXC_OK : IDXC_ERR_CUDA;
 }
 
-size_t idxc_sparse_attention_workspace_bytes(int64_t n_q) {
-    return n_q > 0 ? static_cast<size_t>(round_up(n_q * 4, 256)) : 0;
+size_t idxc_sparse_attention_workspace_bytes(int64_t n_q, int k_top) {
+    if (n_q <= 0 || k_top < 1) return 0;
+    return static_cast<size_t>(round_up(n_q * 4, 256)) + sparse_attn_scratch_bytes(n_q, k_top);
 }
 
 idxc_status idxc_sparse_attention(const void* q, const void* kv, const int32_t* topk, const int64_t* kv_base, int64_t n_q,
@@ -426,14 +427,15 @@ idxc_status idxc_sparse_attention(const void* q, const void* kv, const int32_t* 
     if (!aligned(q, 16) || !aligned(kv, 16) || !aligned(out, 16) || !aligned(topk, 4) || (kv_base && !aligned(kv_base, 8)) ||
         (lse && !aligned(lse, 4)))
         return IDXC_ERR_INVALID_ARG;
-    if (!workspace || !aligned(workspace, 16) || workspace_bytes < idxc_sparse_attention_workspace_bytes(n_q)) return IDXC_ERR_WORKSPACE;
+    if (!workspace || !aligned(workspace, 16) || workspace_bytes < idxc_sparse_attention_workspace_bytes(n_q, k_top)) return IDXC_ERR_WORKSPACE;
     DeviceInfo& di = device_info();
     if (!di.ok) return IDXC_ERR_CUDA;
     CUtensorMap q_map;
     if (!encode_operand_map(&q_map, q, n_q * H, d_qk, false, H)) return IDXC_ERR_CUDA;
     g_launches += 2;
-    return launch_sparse_attn(kv, topk, kv_base, n_q, n_kv, H, k_top, scale, out, lse, static_cast<int32_t*>(workspace), q_map,
-                              di.status_ptr, di.sm_count, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+    void* scratch = static_cast<uint8_t*>(workspace) + round_up(n_q * 4, 256);
+    return launch_sparse_attn(kv, topk, kv_base, n_q, n_kv, H, k_top, scale, out, lse, static_cast<int32_t*>(workspace), scratch,
+                              q_map, di.status_ptr, di.sm_count, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
                ? IDXC_OK : IDXC_ERR_CUDA;
 }
 

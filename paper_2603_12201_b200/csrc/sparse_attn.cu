@@ -5,20 +5,30 @@
 //
 // One persistent CTA per SM walks queries. The 128 heads of a query are the M dimension of every UMMA, so a
 // thread of the softmax warps owns one head row (no cross-lane reductions). The output accumulator of a
-// query, 128 x 512 fp32, is all of tensor memory, so a query is processed in two passes over its selected
-// rows, one per 256-column half of d_v; each pass recomputes the scores.
-//   tensor memory (512 columns): O half [0,256) | S [256,320) | P as bf16 pairs [320,352) | 5 of the 9
-//     64-column blocks of Q as bf16 pairs [352,512) (the A operand of the score MMAs; the other 4 blocks of Q
-//     stay in shared memory: there is no room for both a resident Q and two tiles of gathered rows)
-//   shared memory: 2 stages x (64 gathered rows x 576 bf16, as 9 blocks of [64 rows x 128 B], 128-byte
-//     swizzle) | 4 blocks of Q [128 rows x 128 B]. A block of gathered rows is at once the K-major B operand
-//     of S = Q K^T (rows = keys) and the MN-major B operand of O += P V (64 contiguous value columns).
-//   warps: 0 MMA issuer, 1 Q loader (TMA), 2-5 row gather (16-byte cp.async into the swizzled layout),
-//     6-9 softmax: S from tensor memory, running reference maximum with a lazy rescale of O (only when the
-//     maximum grows by more than 2^8), P written back to tensor memory as the A operand of the PV MMAs.
+// query, 128 x 512 fp32, is all of tensor memory, so a query takes two passes over its selected rows, one per
+// 256-column half of d_v:
+//   pass 1  gathers whole rows (576 columns), S = Q K^T, softmax, O[:, 0:256] += P V; the bf16 probabilities P
+//           and the rescale factors of the running maximum also go to a per-CTA scratch area in global memory
+//   pass 2  gathers only columns 256..511 of the same rows, reads P back and does O[:, 256:512] += P V with the
+//           same sequence of rescales: no second score product, half the gather bytes.
+// Tensor memory (512 columns): O half [0,256) | S double-buffered [256,320), [320,384); P overwrites the first
+//   32 columns of its S buffer as bf16 pairs and is the A operand of the PV MMAs | Q blocks 0..3 (of 9 blocks of
+//   64 columns) as bf16 pairs [384,512), the A operand of their score MMAs; Q blocks 4..8 stay in shared memory.
+// Shared memory: 2 stages x 9 blocks of [64 gathered rows x 128 B] (128-byte swizzle) | 5 blocks of Q
+//   [128 rows x 128 B]. A block of gathered rows is at once the K-major B operand of S (rows = keys) and the
+//   MN-major B operand of P V (64 contiguous value columns). A stage is two slots with their own barriers:
+//   "V" = blocks 0..3 (needed until the PV product) and "E" = blocks 4..8 (free again once the scores are
+//   done), so the next tile's E part is gathered while this tile is still in its softmax. Pass 2 uses the four
+//   slots as a ring of four value tiles.
+// Warps: 0 MMA issuer (tile i+1's scores are issued before tile i's PV product, so the tensor pipe works
+//   while the softmax warps turn S(i) into P(i)), 1 Q loader (TMA), 2-9 row gather (16-byte cp.async into the
+//   swizzled layout; two warps per slot, each slot its own acquire/copy/publish stream), 10-13 softmax: running reference maximum with a lazy rescale of O (only when the maximum
+//   grows by more than 2^8).
 // Entries < 0 or pointing outside the cache are skipped; a query's tiles end at its last usable entry
 // (counted by a small kernel first).
 #include <cuda_bf16.h>
+
+#include <type_traits>
 
 #include "kernels.h"
 #include "ptx_sm100.cuh"
@@ -26,26 +36,31 @@
 namespace idxc {
 namespace {
 
-constexpr int kSaThreads = 320;
+constexpr int kSaGatherWarps = 8;          // warps 2 .. 9
+constexpr int kSaThreads = 32 * (2 + kSaGatherWarps + 4);
+static_assert(kSaGatherWarps == 8, "two gather warps per slot, four slots");
 constexpr int kSaBK = 64;                 // gathered rows per tile
 constexpr int kSaNB = 9;                  // 64-column blocks of d_qk = 576
 constexpr int kSaNVH = 4;                 // value blocks per pass (256 columns)
-constexpr int kSaQT = 5;                  // Q blocks held in tensor memory
-constexpr int kSaQS = kSaNB - kSaQT;      // Q blocks held in shared memory
+constexpr int kSaQT = 4;                  // Q blocks held in tensor memory (blocks 0..3)
+constexpr int kSaQS = kSaNB - kSaQT;      // Q blocks held in shared memory (blocks 4..8)
 constexpr uint32_t kSaQBlockBytes = 128 * 128;
 constexpr uint32_t kSaKBlockBytes = kSaBK * 128;
 constexpr uint32_t kSaStageBytes = kSaNB * kSaKBlockBytes;            // 73728
-constexpr uint32_t kSaQSmemBytes = kSaQS * kSaQBlockBytes;            // 65536
+constexpr uint32_t kSaQSmemBytes = kSaQS * kSaQBlockBytes;            // 81920
 constexpr uint32_t kSaSmemBytes = 2 * kSaStageBytes + kSaQSmemBytes + 256 + 1024;
 static_assert(kSaQT * kSaQBlockBytes <= 2 * kSaStageBytes, "the Q staging area lives in the tile stages");
-constexpr uint32_t kColO = 0, kColS = 256, kColP = 320, kColQ = 352;
+static_assert(kSaSmemBytes <= 232448, "shared memory budget of one CTA");
+constexpr uint32_t kColO = 0, kColS = 256, kColQ = 384;   // S buffer b at kColS + 64 b; P in its first 32 columns
 constexpr float kRescaleThreshold = 8.f;  // log2 units: P stays below 2^8
+constexpr uint32_t kSaScratchTileBytes = 128 * kSaBK * 2 + 128 * 4;   // P [128][64] bf16 + rescale factors [128] fp32
 
 struct SaParams {
     const uint8_t* kv;          // [n_kv, 576] bf16
     const int32_t* topk;        // [n_q, k_top]
     const int64_t* kv_base;     // [n_q] or nullptr
     const int32_t* n_eff;       // [n_q] entries to visit per query
+    uint8_t* scratch;           // [grid][tiles per query][kSaScratchTileBytes]
     int64_t n_q, n_kv;
     int H, k_top;
     float scale_log2;           // scale * log2(e)
@@ -89,21 +104,24 @@ __global__ void __launch_bounds__(kSaThreads, 1)
 sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    uint8_t* stage_smem = smem;                               // [2][9][64 x 128 B]; Q blocks 0..4 are staged here first
-    uint8_t* q_smem = smem + 2 * kSaStageBytes;               // [4][128 x 128 B]: Q blocks 5..8
+    uint8_t* stage_smem = smem;                               // [2][9][64 x 128 B]; Q blocks 0..3 are staged here first
+    uint8_t* q_smem = smem + 2 * kSaStageBytes;               // [5][128 x 128 B]: Q blocks 4..8
     uint64_t* bars = reinterpret_cast<uint64_t*>(q_smem + kSaQSmemBytes);
     const uint32_t bar_q_full = smem_u32(bars + 0);
-    const uint32_t bar_q_ready = smem_u32(bars + 1);          // Q blocks 0..4 copied to tensor memory, staging free
+    const uint32_t bar_q_ready = smem_u32(bars + 1);          // Q blocks 0..3 copied to tensor memory, staging free
     const uint32_t bar_q_empty = smem_u32(bars + 2);
-    const uint32_t bar_kv_full = smem_u32(bars + 3);          // [2]
-    const uint32_t bar_kv_empty = smem_u32(bars + 5);         // [2]
-    const uint32_t bar_s_full = smem_u32(bars + 7);
-    const uint32_t bar_p_ready = smem_u32(bars + 8);
-    const uint32_t bar_o_full = smem_u32(bars + 9);
-    const uint32_t bar_o_free = smem_u32(bars + 10);
-    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(bars + 11);
+    // slot = 2 * stage + group, group 0 = "V" (blocks 0..3), group 1 = "E" (blocks 4..8)
+    const uint32_t bar_slot_full = smem_u32(bars + 3);        // [4]
+    const uint32_t bar_slot_empty = smem_u32(bars + 7);       // [4]
+    const uint32_t bar_s_full = smem_u32(bars + 11);          // [2] S buffers
+    const uint32_t bar_p_ready = smem_u32(bars + 13);         // [4] pass 1 uses two (P in its S buffer), pass 2 a ring of four
+    const uint32_t bar_p_free = smem_u32(bars + 17);          // [4] pass 2: the PV product has read P buffer b
+    const uint32_t bar_o_full = smem_u32(bars + 21);
+    const uint32_t bar_o_free = smem_u32(bars + 22);
+    const uint32_t bar_pv_done = smem_u32(bars + 23);         // one phase per PV tile
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(bars + 24);
     volatile uint32_t* abort_flag = tmem_base_slot + 1;
-    volatile uint16_t* tile_mask = reinterpret_cast<volatile uint16_t*>(bars + 12);   // [2 stages][4 gather warps]
+    volatile uint32_t* tile_mask = reinterpret_cast<volatile uint32_t*>(bars + 25);   // [2 stages][2]: usable entries of the tile, rows 0..31 and 32..63
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -112,14 +130,18 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
         mbar_init(bar_q_full, 1);
         mbar_init(bar_q_ready, 4);
         mbar_init(bar_q_empty, 1);
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(bar_kv_full + 8 * i, 4);
-            mbar_init(bar_kv_empty + 8 * i, 1);
+        for (int i = 0; i < 4; ++i) {
+            mbar_init(bar_slot_full + 8 * i, 2);
+            mbar_init(bar_slot_empty + 8 * i, 1);
         }
-        mbar_init(bar_s_full, 1);
-        mbar_init(bar_p_ready, 4);
+        for (int i = 0; i < 2; ++i) mbar_init(bar_s_full + 8 * i, 1);
+        for (int i = 0; i < 4; ++i) {
+            mbar_init(bar_p_ready + 8 * i, 4);
+            mbar_init(bar_p_free + 8 * i, 1);
+        }
         mbar_init(bar_o_full, 1);
         mbar_init(bar_o_free, 4);
+        mbar_init(bar_pv_done, 1);
         *abort_flag = 0u;
         fence_mbar_init();
     }
@@ -133,68 +155,126 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
     const uint32_t tmem_base = *tmem_base_slot;
 
     auto tiles_of = [&](int64_t t) -> int { return (__ldg(p.n_eff + t) + kSaBK - 1) / kSaBK; };
+    // first block of a slot's data inside the stage area
+    auto slot_smem = [&](int slot) -> uint8_t* { return stage_smem + (slot >> 1) * kSaStageBytes + (slot & 1) * (kSaNVH * kSaKBlockBytes); };
+    const int tiles_per_query = (p.k_top + kSaBK - 1) / kSaBK;
+    uint8_t* scratch = p.scratch + static_cast<size_t>(blockIdx.x) * tiles_per_query * kSaScratchTileBytes;
 
     if (warp == 0) {
-        if (lane == 0) {
-            // ------------------------------------------------------------ MMA issuer
-            constexpr uint32_t kIdescS = umma_idesc(1, 1, 128, kSaBK);
-            constexpr uint32_t kIdescPV = umma_idesc(1, 1, 128, 64 * kSaNVH) | kUmmaBMajorMN;
-            uint32_t ph_q_full = 0, ph_q_ready = 0, ph_p_ready = 0, ph_o_free = 0;
-            uint32_t ph_kv_full[2] = {0u, 0u};
-            int stage = 0;
-            bool ok = true;
-            for (int64_t t = blockIdx.x; t < p.n_q && ok; t += gridDim.x) {
-                const int nt = tiles_of(t);
-                if (nt == 0) continue;
-                ok = mbar_wait(bar_q_full, ph_q_full, abort_flag) && mbar_wait(bar_q_ready, ph_q_ready, abort_flag);
-                if (!ok) break;
-                ph_q_full ^= 1u;
-                ph_q_ready ^= 1u;
-                for (int half = 0; half < 2 && ok; ++half) {
-                    ok = mbar_wait(bar_o_free, ph_o_free ^ 1u, abort_flag);    // the previous pass's O has been read out
-                    if (!ok) break;
-                    ph_o_free ^= 1u;
-                    for (int i = 0; i < nt; ++i) {
-                        ok = mbar_wait(bar_kv_full + 8 * stage, ph_kv_full[stage], abort_flag);
-                        if (!ok) break;
-                        ph_kv_full[stage] ^= 1u;
-                        tcgen05_fence_after_sync();
-                        const uint32_t tile = smem_u32(stage_smem + stage * kSaStageBytes);
-                        // S = Q K^T over the 9 column blocks
+        // ---------------------------------------------------------------- MMA issuer
+        // The whole warp runs this role with uniform control flow and one elected lane issues each MMA (see
+        // umma_f16_elect); descriptors are a per-tile base plus compile-time offsets in 16-byte units.
+        constexpr uint32_t kIdescS = umma_idesc(1, 1, 128, kSaBK);
+        constexpr uint32_t kIdescPV = umma_idesc(1, 1, 128, 64 * kSaNVH) | kUmmaBMajorMN;
+        uint32_t ph_q_full = 0, ph_q_ready = 0, ph_o_free = 0;
+        uint32_t ph_slot_full[4] = {0u, 0u, 0u, 0u}, ph_p_ready[4] = {0u, 0u, 0u, 0u};
+        int stage_s = 0, stage_pv = 0;      // pass 1: stage of the next tile to score / to multiply by V
+        bool ok = true;
+        const uint64_t q_desc0 = umma_smem_desc_sw128(smem_u32(q_smem));
+        auto wait_bar = [&](uint32_t bar, uint32_t parity) -> bool {
+            return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort_flag));
+        };
+        auto wait_slot = [&](int slot) -> bool {
+            if (!wait_bar(bar_slot_full + 8 * slot, ph_slot_full[slot])) return false;
+            ph_slot_full[slot] ^= 1u;
+            tcgen05_fence_after_sync();
+            return true;
+        };
+        // 16 gathered rows per MMA; P (bf16 pairs) starts at tensor-memory column p_col
+        auto issue_pv = [&](uint32_t v_blocks, uint32_t p_col, bool first_tile) {
+            const uint64_t v_desc0 = umma_smem_desc_sw128_mn(v_blocks, kSaKBlockBytes);
+            if (first_tile) umma_f16_ts_elect<false>(tmem_base + kColO, tmem_base + p_col, v_desc0, kIdescPV);
+            else umma_f16_ts_elect<true>(tmem_base + kColO, tmem_base + p_col, v_desc0, kIdescPV);
 #pragma unroll
-                        for (int b = 0; b < kSaNB; ++b) {
+            for (int ks = 1; ks < kSaBK / 16; ++ks)
+                umma_f16_ts_elect<true>(tmem_base + kColO, tmem_base + p_col + ks * 8, v_desc0 + (ks * 16 * 128) / 16, kIdescPV);
+        };
+        for (int64_t t = blockIdx.x; t < p.n_q && ok; t += gridDim.x) {
+            const int nt = tiles_of(t);
+            if (nt == 0) continue;
+            ok = wait_bar(bar_q_full, ph_q_full) && wait_bar(bar_q_ready, ph_q_ready);
+            if (!ok) break;
+            ph_q_full ^= 1u;
+            ph_q_ready ^= 1u;
+            // ---- pass 1: scores and the first half of the output
+            ok = wait_bar(bar_o_free, ph_o_free ^ 1u);        // the previous query's O has been read out
+            if (!ok) break;
+            ph_o_free ^= 1u;
+            // Issue order: S(i+1) blocks 4..8 | P(i) V(i) | S(i+1) blocks 0..3. The first part keeps the tensor pipe busy
+            // while the softmax warps turn S(i) into P(i); the PV product comes before the second part so that
+            // its value slot is free again (and refilled) well before the tile after next needs it.
+            auto issue_s_e = [&](int i) -> bool {            // blocks 4..8 against Q in shared memory
+                if (!wait_slot(2 * stage_s + 1)) return false;
+                const uint32_t s_tmem = tmem_base + kColS + (i & 1) * 64;
+                const uint64_t k_desc0 = umma_smem_desc_sw128(smem_u32(stage_smem + stage_s * kSaStageBytes));
 #pragma unroll
-                            for (int ks = 0; ks < 4; ++ks) {
-                                const uint64_t b_desc = umma_smem_desc_sw128(tile + b * kSaKBlockBytes + ks * 32);
-                                if (b < kSaQT)
-                                    umma_f16_ts(tmem_base + kColS, tmem_base + kColQ + b * 32 + ks * 8, b_desc, kIdescS, (b | ks) != 0);
-                                else
-                                    umma_f16(tmem_base + kColS,
-                                             umma_smem_desc_sw128(smem_u32(q_smem + (b - kSaQT) * kSaQBlockBytes) + ks * 32), b_desc,
-                                             kIdescS, 1u);
-                            }
-                        }
-                        umma_commit(bar_s_full);
-                        ok = mbar_wait(bar_p_ready, ph_p_ready, abort_flag);
-                        if (!ok) break;
-                        ph_p_ready ^= 1u;
-                        tcgen05_fence_after_sync();
-                        // O[:, 256 half .. +256] += P V: 16 gathered rows per MMA
+                for (int b = kSaQT; b < kSaNB; ++b) {
 #pragma unroll
-                        for (int ks = 0; ks < kSaBK / 16; ++ks) {
-                            const uint64_t v_desc = umma_smem_desc_sw128_mn(
-                                tile + (half * kSaNVH) * kSaKBlockBytes + ks * 16 * 128, kSaKBlockBytes);
-                            umma_f16_ts(tmem_base + kColO, tmem_base + kColP + ks * 8, v_desc, kIdescPV, (i | ks) != 0);
-                        }
-                        umma_commit(bar_kv_empty + 8 * stage);
-                        if (i == nt - 1) umma_commit(bar_o_full);
-                        stage ^= 1;
+                    for (int ks = 0; ks < 4; ++ks) {
+                        const uint64_t a_desc = q_desc0 + ((b - kSaQT) * kSaQBlockBytes + ks * 32) / 16;
+                        const uint64_t b_desc = k_desc0 + (b * kSaKBlockBytes + ks * 32) / 16;
+                        if (b == kSaQT && ks == 0) umma_f16_elect<false>(s_tmem, a_desc, b_desc, kIdescS);
+                        else umma_f16_elect<true>(s_tmem, a_desc, b_desc, kIdescS);
                     }
                 }
-                if (ok) umma_commit(bar_q_empty);
+                umma_commit_elect(bar_slot_empty + 8 * (2 * stage_s + 1));    // blocks 4..8 are not needed again
+                return true;
+            };
+            auto issue_s_v = [&](int i) -> bool {            // blocks 0..3 against Q in tensor memory
+                if (!wait_slot(2 * stage_s)) return false;
+                const uint32_t s_tmem = tmem_base + kColS + (i & 1) * 64;
+                const uint64_t k_desc0 = umma_smem_desc_sw128(smem_u32(stage_smem + stage_s * kSaStageBytes));
+#pragma unroll
+                for (int b = 0; b < kSaQT; ++b) {
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                        umma_f16_ts_elect<true>(s_tmem, tmem_base + kColQ + b * 32 + ks * 8,
+                                                k_desc0 + (b * kSaKBlockBytes + ks * 32) / 16, kIdescS);
+                }
+                umma_commit_elect(bar_s_full + 8 * (i & 1));
+                stage_s ^= 1;
+                return true;
+            };
+            ok = issue_s_e(0) && issue_s_v(0);
+            for (int i = 0; i < nt && ok; ++i) {
+                if (i + 1 < nt) {
+                    ok = issue_s_e(i + 1);
+                    if (!ok) break;
+                }
+                ok = wait_bar(bar_p_ready + 8 * (i & 1), ph_p_ready[i & 1]);
+                if (!ok) break;
+                ph_p_ready[i & 1] ^= 1u;
+                tcgen05_fence_after_sync();
+                issue_pv(smem_u32(stage_smem + stage_pv * kSaStageBytes), kColS + (i & 1) * 64, i == 0);
+                umma_commit_elect(bar_slot_empty + 8 * (2 * stage_pv));
+                umma_commit_elect(bar_pv_done);
+                if (i == nt - 1) umma_commit_elect(bar_o_full);
+                stage_pv ^= 1;
+                if (i + 1 < nt) {
+                    ok = issue_s_v(i + 1);
+                    if (!ok) break;
+                }
             }
-            if (!ok) sa_give_up(abort_flag, p.status, DEV_TIMEOUT_MMA);
+            if (!ok) break;
+            // ---- pass 2: the second half of the output from the saved P; the four slots are a ring of value tiles
+            ok = wait_bar(bar_o_free, ph_o_free ^ 1u);
+            if (!ok) break;
+            ph_o_free ^= 1u;
+            for (int i = 0; i < nt; ++i) {
+                const int slot = i & 3;
+                ok = wait_slot(slot) && wait_bar(bar_p_ready + 8 * slot, ph_p_ready[slot]);
+                if (!ok) break;
+                ph_p_ready[slot] ^= 1u;
+                tcgen05_fence_after_sync();
+                issue_pv(smem_u32(slot_smem(slot)), kColS + slot * 32, i == 0);
+                umma_commit_elect(bar_slot_empty + 8 * slot);
+                umma_commit_elect(bar_p_free + 8 * slot);
+                umma_commit_elect(bar_pv_done);
+                if (i == nt - 1) umma_commit_elect(bar_o_full);
+            }
+            if (ok) umma_commit_elect(bar_q_empty);
         }
+        if (!ok && lane == 0) sa_give_up(abort_flag, p.status, DEV_TIMEOUT_MMA);
     } else if (warp == 1) {
         if (lane == 0) {
             // ------------------------------------------------------------ Q loader
@@ -215,13 +295,17 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
             }
             if (!ok) sa_give_up(abort_flag, p.status, DEV_TIMEOUT_PRODUCER);
         }
-    } else if (warp < 6) {
+    } else if (warp < 2 + kSaGatherWarps) {
         // ---------------------------------------------------------------- row gather
-        const int gw = warp - 2;                      // rows 16 gw .. 16 gw + 15 of every tile
-        uint32_t ph_q_ready = 0;
-        uint32_t ph_kv_empty[2] = {0u, 0u};
-        int stage = 0;
+        // Two warps per slot (32 rows each): a pair only ever fills its own slot, so the four slots are four
+        // independent acquire -> copy -> publish streams and a tile's landing time overlaps other tiles' copies.
+        const int gw = warp - 2;
+        const int slot = gw >> 1;                     // 2 * stage + group
+        const int row0 = (gw & 1) * 32;               // this warp's rows of every tile it handles
+        uint32_t ph_q_ready = 0, ph_empty = 0;
+        uint32_t tile_seq = 0;                        // pass-1 tiles before the current query: tile i sits in stage (tile_seq + i) & 1
         bool ok = true;
+        uint8_t* const slot_base = slot_smem(slot);
         for (int64_t t = blockIdx.x; t < p.n_q && ok; t += gridDim.x) {
             const int nt = tiles_of(t);
             if (nt == 0) continue;
@@ -230,38 +314,89 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
             ph_q_ready ^= 1u;
             const int64_t base = p.kv_base ? __ldg(p.kv_base + t) : 0;
             const int32_t* row_idx = p.topk + t * p.k_top;
-            for (int half = 0; half < 2 && ok; ++half) {
-                for (int i = 0; i < nt; ++i) {
-                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_kv_empty + 8 * stage, ph_kv_empty[stage] ^ 1u, abort_flag));
-                    if (!ok) break;
-                    ph_kv_empty[stage] ^= 1u;
-                    // lanes 0..15 look up this warp's rows
-                    const int j = i * kSaBK + gw * 16 + (lane & 15);
-                    int64_t src_row = -1;
-                    if (j < p.k_top) {
-                        const int64_t idx = __ldg(row_idx + j);
-                        if (idx >= 0 && base + idx >= 0 && base + idx < p.n_kv) src_row = base + idx;
-                    }
-                    const uint32_t valid = __ballot_sync(0xFFFFFFFFu, src_row >= 0) & 0xFFFFu;
-                    if (src_row < 0) src_row = 0;             // skipped entries load row 0 and are masked later
-                    uint8_t* tile = stage_smem + stage * kSaStageBytes;
-#pragma unroll 4
-                    for (int rr = 0; rr < 16; ++rr) {
-                        const int64_t r_src = __shfl_sync(0xFFFFFFFFu, src_row, rr);
-                        const uint8_t* src = p.kv + r_src * (kSaNB * 128);
-                        const int r = gw * 16 + rr;
+            // lane l looks up row row0 + l of tile i; returns the mask of usable entries
+            auto lookup = [&](int i, int64_t& src_row) -> uint32_t {
+                const int j = i * kSaBK + row0 + lane;
+                src_row = -1;
+                if (j < p.k_top) {
+                    const int64_t idx = __ldg(row_idx + j);
+                    if (idx >= 0 && base + idx >= 0 && base + idx < p.n_kv) src_row = base + idx;
+                }
+                const uint32_t valid = __ballot_sync(0xFFFFFFFFu, src_row >= 0);
+                if (src_row < 0) src_row = 0;                 // skipped entries load row 0 and get weight 0
+                return valid;
+            };
+            // copies chunks [c0, c0 + N_CHUNKS) (16 bytes each) of this warp's 32 rows into the slot, 8 rows at a
+            // time: their addresses are formed first, so that the copies issue back to back
+            auto gather = [&](int64_t src_row, int c0, auto n_chunks_tag) {
+                constexpr int N_CHUNKS = decltype(n_chunks_tag)::value;
+                constexpr int PER_LANE = (N_CHUNKS + 31) / 32;
+                uint32_t dst[PER_LANE];
 #pragma unroll
-                        for (int c = lane; c < kSaNB * 8; c += 32) {      // 72 chunks of 16 bytes per row
-                            const int b = c >> 3, ch = c & 7;
-                            cp_async_16(smem_u32(tile + b * kSaKBlockBytes + r * 128 + ((ch ^ (r & 7)) << 4)), src + c * 16);
-                        }
+                for (int k = 0; k < PER_LANE; ++k) {
+                    const int c = lane + 32 * k;
+                    dst[k] = smem_u32(slot_base) + (c >> 3) * kSaKBlockBytes + row0 * 128 + ((c & 7) << 4);
+                }
+#pragma unroll
+                for (int bt = 0; bt < 4; ++bt) {
+                    const uint8_t* src[8];
+#pragma unroll
+                    for (int rr = 0; rr < 8; ++rr)
+                        src[rr] = p.kv + __shfl_sync(0xFFFFFFFFu, src_row, bt * 8 + rr) * (kSaNB * 128) + (c0 + lane) * 16;
+                    // row r = row0 + 8 bt + rr: r & 7 == rr, so the swizzle is an XOR of rr into the chunk index
+#pragma unroll
+                    for (int rr = 0; rr < 8; ++rr) {
+#pragma unroll
+                        for (int k = 0; k < PER_LANE; ++k)
+                            if (lane + 32 * k < N_CHUNKS)
+                                cp_async_16((dst[k] ^ (rr << 4)) + (bt * 8 + rr) * 128, src[rr] + k * 512);
                     }
-                    if (lane == 0) tile_mask[stage * 4 + gw] = static_cast<uint16_t>(valid);
-                    cp_async_wait_all();
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_kv_full + 8 * stage);
-                    stage ^= 1;
+                }
+            };
+            auto acquire = [&]() -> bool {
+                const bool got = __all_sync(0xFFFFFFFFu, mbar_wait(bar_slot_empty + 8 * slot, ph_empty ^ 1u, abort_flag));
+                ph_empty ^= 1u;
+                return got;
+            };
+            auto publish = [&]() {
+                cp_async_wait_all();
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_slot_full + 8 * slot);
+            };
+            // ---- pass 1: the tiles that sit in this slot's stage; group 1 = columns 256..575, group 0 = columns 0..255
+            {
+                int64_t src_row, src_next = 0;
+                uint32_t valid_next = 0;
+                const int first = ((slot >> 1) ^ static_cast<int>(tile_seq & 1u)) & 1;
+                uint32_t valid = first < nt ? lookup(first, src_row) : 0u;
+                for (int i = first; i < nt; i += 2) {
+                    if (i + 2 < nt) valid_next = lookup(i + 2, src_next);
+                    ok = acquire();
+                    if (!ok) break;
+                    if (slot & 1) {
+                        gather(src_row, kSaNVH * 8, std::integral_constant<int, (kSaNB - kSaNVH) * 8>{});
+                    } else {
+                        gather(src_row, 0, std::integral_constant<int, kSaNVH * 8>{});
+                        if (lane == 0) tile_mask[(slot >> 1) * 2 + (gw & 1)] = valid;
+                    }
+                    publish();
+                    src_row = src_next;
+                    valid = valid_next;
+                }
+                tile_seq += static_cast<uint32_t>(nt);
+            }
+            // ---- pass 2: columns 256..511 only; tile i sits in slot i & 3
+            if (ok) {
+                int64_t src_row, src_next = 0;
+                if (slot < nt) lookup(slot, src_row);
+                for (int i = slot; i < nt; i += 4) {
+                    if (i + 4 < nt) lookup(i + 4, src_next);
+                    ok = acquire();
+                    if (!ok) break;
+                    gather(src_row, kSaNVH * 8, std::integral_constant<int, kSaNVH * 8>{});
+                    publish();
+                    src_row = src_next;
                 }
             }
         }
@@ -272,9 +407,54 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
         const int quarter = warp & 3;                  // TMEM lane quarter this warp may access
         const int row = quarter * 32 + lane;           // head
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-        uint32_t ph_q_full = 0, ph_s_full = 0, ph_o_full = 0;
+        uint32_t ph_q_full = 0, ph_o_full = 0;
+        uint32_t ph_s_full[2] = {0u, 0u}, ph_p_free[4] = {0u, 0u, 0u, 0u};
+        uint32_t pv_tiles = 0;                         // PV tiles before the current one, over the whole kernel
         int stage = 0;
         bool ok = true;
+        uint8_t* my_p = scratch + row * (kSaBK * 2);                  // + tile * kSaScratchTileBytes: this row's P, 128 bytes
+        uint8_t* my_alpha = scratch + 128 * kSaBK * 2 + row * 4;      // + tile * kSaScratchTileBytes: this row's factor
+        // multiplies this thread's row of O by alpha (the caller has made sure that every earlier PV product is complete)
+        auto scale_o = [&](float alpha) {
+            tcgen05_fence_after_sync();
+#pragma unroll 1
+            for (int c = 0; c < 8; ++c) {
+                uint32_t o[32];
+                tmem_ld_32x32b_x32(lane_base + kColO + c * 32, o);
+                tmem_ld_wait(o);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+                tmem_st_32x32b_x32(lane_base + kColO + c * 32, o);
+            }
+        };
+        // normalises this thread's row of O and writes 256 output columns
+        auto write_out = [&](__nv_bfloat16* dst_row, float inv) -> bool {
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar_o_full, ph_o_full, abort_flag))) return false;
+            ph_o_full ^= 1u;
+            tcgen05_fence_after_sync();
+#pragma unroll 1
+            for (int c = 0; c < 8; ++c) {
+                uint32_t o[32];
+                tmem_ld_32x32b_x32(lane_base + kColO + c * 32, o);
+                tmem_ld_wait(o);
+                if (row < p.H) {
+                    uint4* dst = reinterpret_cast<uint4*>(dst_row + c * 32);
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        uint4 w;
+                        w.x = pack_bf16x2(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
+                        w.y = pack_bf16x2(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
+                        w.z = pack_bf16x2(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
+                        w.w = pack_bf16x2(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
+                        dst[v] = w;
+                    }
+                }
+            }
+            tcgen05_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_o_free);
+            return true;
+        };
         for (int64_t t = blockIdx.x; t < p.n_q && ok; t += gridDim.x) {
             const int nt = tiles_of(t);
             __nv_bfloat16* out_row = p.out + (t * p.H + row) * 512;
@@ -285,7 +465,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
                 }
                 continue;
             }
-            // ---- Q blocks 0..4: staging (swizzled rows) -> tensor memory, two bf16 per column
+            // ---- Q blocks 0..3: staging (swizzled rows) -> tensor memory, two bf16 per column
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_q_full, ph_q_full, abort_flag));
             if (!ok) break;
             ph_q_full ^= 1u;
@@ -305,101 +485,120 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_q_ready);
 
-            float lse_val = 0.f;
-            for (int half = 0; half < 2 && ok; ++half) {
-                float m_ref = -INFINITY, l = 0.f;
-                for (int i = 0; i < nt; ++i) {
-                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_s_full, ph_s_full, abort_flag));
-                    if (!ok) break;
-                    ph_s_full ^= 1u;
-                    tcgen05_fence_after_sync();
-                    uint32_t sa[32], sb[32];
-                    tmem_ld_32x32b_x32(lane_base + kColS, sa);
-                    tmem_ld_32x32b_x32(lane_base + kColS + 32, sb);
-                    tmem_ld_wait(sa);
-                    tmem_ld_wait(sb);
-                    const uint32_t mlo = static_cast<uint32_t>(tile_mask[stage * 4 + 0]) | (static_cast<uint32_t>(tile_mask[stage * 4 + 1]) << 16);
-                    const uint32_t mhi = static_cast<uint32_t>(tile_mask[stage * 4 + 2]) | (static_cast<uint32_t>(tile_mask[stage * 4 + 3]) << 16);
-                    float mt = -INFINITY;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const float xa = (mlo >> j) & 1u ? __uint_as_float(sa[j]) * p.scale_log2 : -INFINITY;
-                        const float xb = (mhi >> j) & 1u ? __uint_as_float(sb[j]) * p.scale_log2 : -INFINITY;
-                        sa[j] = __float_as_uint(xa);
-                        sb[j] = __float_as_uint(xb);
-                        mt = fmaxf(mt, fmaxf(xa, xb));
-                    }
-                    // lazy reference maximum: move it only when the row maximum outgrew it by 2^8
-                    const bool move = mt > m_ref + kRescaleThreshold;      // also true for the first usable score (m_ref = -inf)
-                    if (__any_sync(0xFFFFFFFFu, move)) {
-                        float alpha = 1.f;
-                        if (move) {
-                            alpha = m_ref == -INFINITY ? 0.f : fast_exp2(m_ref - mt);
-                            m_ref = mt;
-                            l *= alpha;
-                        }
-                        if (i > 0) {                                       // every earlier PV MMA is complete (S was committed after them)
-#pragma unroll 1
-                            for (int c = 0; c < 8; ++c) {
-                                uint32_t o[32];
-                                tmem_ld_32x32b_x32(lane_base + kColO + c * 32, o);
-                                tmem_ld_wait(o);
-#pragma unroll
-                                for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
-                                tmem_st_32x32b_x32(lane_base + kColO + c * 32, o);
-                            }
-                        }
-                    }
-                    const float m_sub = m_ref == -INFINITY ? 0.f : m_ref;   // no usable score yet: every P is exp2(-inf) = 0
-                    uint32_t pr[32];
-                    float sum = 0.f;
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const float p0 = fast_exp2(__uint_as_float(sa[2 * j]) - m_sub), p1 = fast_exp2(__uint_as_float(sa[2 * j + 1]) - m_sub);
-                        const float p2 = fast_exp2(__uint_as_float(sb[2 * j]) - m_sub), p3 = fast_exp2(__uint_as_float(sb[2 * j + 1]) - m_sub);
-                        sum += (p0 + p1) + (p2 + p3);
-                        pr[j] = pack_bf16x2(p0, p1);
-                        pr[16 + j] = pack_bf16x2(p2, p3);
-                    }
-                    l += sum;
-                    tmem_st_32x32b_x32(lane_base + kColP, pr);
-                    tmem_st_wait();
-                    tcgen05_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_p_ready);
-                    stage ^= 1;
-                }
+            // ---- pass 1
+            float m_ref = -INFINITY, l = 0.f;
+            for (int i = 0; i < nt; ++i) {
+                const int sbuf = i & 1;
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_s_full + 8 * sbuf, ph_s_full[sbuf], abort_flag));
                 if (!ok) break;
-                // ---- this pass's 256 output columns
-                ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_o_full, ph_o_full, abort_flag));
-                if (!ok) break;
-                ph_o_full ^= 1u;
+                ph_s_full[sbuf] ^= 1u;
                 tcgen05_fence_after_sync();
-                const float inv = l > 0.f ? 1.f / l : 0.f;
-#pragma unroll 1
-                for (int c = 0; c < 8; ++c) {
-                    uint32_t o[32];
-                    tmem_ld_32x32b_x32(lane_base + kColO + c * 32, o);
-                    tmem_ld_wait(o);
-                    if (row < p.H) {
-                        uint4* dst = reinterpret_cast<uint4*>(out_row + half * 256 + c * 32);
+                const uint32_t s_tmem = lane_base + kColS + sbuf * 64;
+                uint32_t sa[32], sb[32];
+                tmem_ld_32x32b_x32(s_tmem, sa);
+                tmem_ld_32x32b_x32(s_tmem + 32, sb);
+                tmem_ld_wait(sa);
+                tmem_ld_wait(sb);
+                const uint32_t mlo = tile_mask[stage * 2], mhi = tile_mask[stage * 2 + 1];
+                float mt = -INFINITY;
 #pragma unroll
-                        for (int v = 0; v < 4; ++v) {
-                            uint4 w;
-                            w.x = pack_bf16x2(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
-                            w.y = pack_bf16x2(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
-                            w.z = pack_bf16x2(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
-                            w.w = pack_bf16x2(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
-                            dst[v] = w;
-                        }
-                    }
+                for (int j = 0; j < 32; ++j) {
+                    const float xa = (mlo >> j) & 1u ? __uint_as_float(sa[j]) * p.scale_log2 : -INFINITY;
+                    const float xb = (mhi >> j) & 1u ? __uint_as_float(sb[j]) * p.scale_log2 : -INFINITY;
+                    sa[j] = __float_as_uint(xa);
+                    sb[j] = __float_as_uint(xb);
+                    mt = fmaxf(mt, fmaxf(xa, xb));
                 }
+                // lazy reference maximum: move it only when the row maximum outgrew it by 2^8
+                const bool move = mt > m_ref + kRescaleThreshold;      // also true for the first usable score (m_ref = -inf)
+                float alpha = 1.f;
+                if (move) {
+                    alpha = m_ref == -INFINITY ? 0.f : fast_exp2(m_ref - mt);
+                    m_ref = mt;
+                    l *= alpha;
+                }
+                if (i > 0 && __any_sync(0xFFFFFFFFu, move)) {
+                    // PV(i-1) was issued before the second part of S(i), whose completion this thread has seen; the wait
+                    // below (one phase per PV tile: the barrier is in phase pv_tiles-1 or pv_tiles) then passes at once
+                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_pv_done, (pv_tiles - 1u) & 1u, abort_flag));
+                    if (!ok) break;
+                    scale_o(alpha);
+                }
+                const float m_sub = m_ref == -INFINITY ? 0.f : m_ref;   // no usable score yet: every P is exp2(-inf) = 0
+                uint32_t pr[32];
+                float sum = 0.f;
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const float p0 = fast_exp2(__uint_as_float(sa[2 * j]) - m_sub), p1 = fast_exp2(__uint_as_float(sa[2 * j + 1]) - m_sub);
+                    const float p2 = fast_exp2(__uint_as_float(sb[2 * j]) - m_sub), p3 = fast_exp2(__uint_as_float(sb[2 * j + 1]) - m_sub);
+                    sum += (p0 + p1) + (p2 + p3);
+                    pr[j] = pack_bf16x2(p0, p1);
+                    pr[16 + j] = pack_bf16x2(p2, p3);
+                }
+                l += sum;
+                tmem_st_32x32b_x32(s_tmem, pr);                   // P(i) over the first half of S(i): this thread holds its row
+                tmem_st_wait();
                 tcgen05_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_o_free);
-                if (half == 0) lse_val = l > 0.f ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
+                if (lane == 0) mbar_arrive(bar_p_ready + 8 * sbuf);
+                // keep P(i) and the factor for pass 2 (read back by this same thread)
+                uint4* dst = reinterpret_cast<uint4*>(my_p + static_cast<size_t>(i) * kSaScratchTileBytes);
+#pragma unroll
+                for (int v = 0; v < 8; ++v) __stcg(dst + v, make_uint4(pr[4 * v], pr[4 * v + 1], pr[4 * v + 2], pr[4 * v + 3]));
+                __stcg(reinterpret_cast<float*>(my_alpha + static_cast<size_t>(i) * kSaScratchTileBytes), alpha);
+                ++pv_tiles;
+                stage ^= 1;
             }
-            if (ok && p.lse && row < p.H) p.lse[t * p.H + row] = lse_val;
+            if (!ok) break;
+            const float inv = l > 0.f ? 1.f / l : 0.f;
+            ok = write_out(out_row, inv);
+            if (!ok) break;
+            if (p.lse && row < p.H) p.lse[t * p.H + row] = l > 0.f ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
+
+            // ---- pass 2: P and the factors come back from the scratch area, two tiles ahead, into a ring of four
+            // P buffers (the 128 columns of the S buffers)
+            uint4 pa[8], pb[8];                                  // P of tiles i and i + 1
+            float alpha_a, alpha_b = 1.f;
+            auto load_p = [&](int i, uint4 (&dst)[8], float& alpha) {
+                const uint4* src = reinterpret_cast<const uint4*>(my_p + static_cast<size_t>(i) * kSaScratchTileBytes);
+#pragma unroll
+                for (int v = 0; v < 8; ++v) dst[v] = __ldcg(src + v);
+                alpha = __ldcg(reinterpret_cast<const float*>(my_alpha + static_cast<size_t>(i) * kSaScratchTileBytes));
+            };
+            load_p(0, pa, alpha_a);
+            if (nt > 1) load_p(1, pb, alpha_b);
+            for (int i = 0; i < nt; ++i) {
+                const int pbuf = i & 3;
+                uint32_t pr[32];
+#pragma unroll
+                for (int v = 0; v < 8; ++v) { pr[4 * v] = pa[v].x; pr[4 * v + 1] = pa[v].y; pr[4 * v + 2] = pa[v].z; pr[4 * v + 3] = pa[v].w; }
+                const float alpha = alpha_a;
+#pragma unroll
+                for (int v = 0; v < 8; ++v) pa[v] = pb[v];
+                alpha_a = alpha_b;
+                if (i + 2 < nt) load_p(i + 2, pb, alpha_b);
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_p_free + 8 * pbuf, ph_p_free[pbuf] ^ 1u, abort_flag));   // PV(i-4) has read this buffer
+                if (!ok) break;
+                ph_p_free[pbuf] ^= 1u;
+                if (i > 0 && __any_sync(0xFFFFFFFFu, alpha != 1.f)) {
+                    // The factor applies to the sum over the tiles before i: PV(i-1) must be complete. It arrives on the
+                    // p_free barrier of its buffer; the parity is the one this thread's next wait on that buffer will use
+                    // (no PV product from tile i on can have been issued, so the barrier cannot be further ahead).
+                    const int prev = (i - 1) & 3;
+                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_p_free + 8 * prev, ph_p_free[prev] ^ 1u, abort_flag));
+                    if (!ok) break;
+                    scale_o(alpha);
+                }
+                tcgen05_fence_after_sync();
+                tmem_st_32x32b_x32(lane_base + kColS + pbuf * 32, pr);
+                tmem_st_wait();
+                tcgen05_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_p_ready + 8 * pbuf);
+                ++pv_tiles;
+            }
+            if (!ok) break;
+            ok = write_out(out_row + 256, inv);
         }
         if (!ok && lane == 0) sa_give_up(abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
     }
@@ -422,18 +621,26 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
 
 bool sparse_attn_supported(int H, int d_qk, int d_v) { return H >= 1 && H <= 128 && d_qk == 64 * kSaNB && d_v == 128 * kSaNVH; }
 
+int sparse_attn_grid(int64_t n_q, int sm_count) {
+    const int cap = sm_count < kSparseAttnMaxGrid ? sm_count : kSparseAttnMaxGrid;
+    return static_cast<int>(n_q < cap ? n_q : cap);
+}
+size_t sparse_attn_scratch_bytes(int64_t n_q, int k_top) {
+    const int64_t ctas = n_q < kSparseAttnMaxGrid ? n_q : kSparseAttnMaxGrid;
+    return static_cast<size_t>(ctas) * ((k_top + kSaBK - 1) / kSaBK) * kSaScratchTileBytes;
+}
+
 cudaError_t launch_sparse_attn(const void* kv, const int32_t* topk, const int64_t* kv_base, int64_t n_q, int64_t n_kv, int H,
-                               int k_top, float scale, void* out, float* lse, int32_t* n_eff, const CUtensorMap& q_map,
-                               unsigned int* status, int sm_count, cudaStream_t stream) {
+                               int k_top, float scale, void* out, float* lse, int32_t* n_eff, void* scratch,
+                               const CUtensorMap& q_map, unsigned int* status, int sm_count, cudaStream_t stream) {
     if (n_q <= 0) return cudaSuccess;
     const int64_t count_blocks = (n_q * 32 + 255) / 256;
     sparse_attn_count_kernel<<<static_cast<unsigned>(count_blocks), 256, 0, stream>>>(topk, kv_base, n_q, n_kv, k_top, n_eff);
     if (cudaError_t e = cudaGetLastError(); e != cudaSuccess) return e;
     if (cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(sparse_attn_kernel), kSaSmemBytes); e != cudaSuccess) return e;
-    SaParams p{static_cast<const uint8_t*>(kv), topk, kv_base, n_eff, n_q, n_kv, H, k_top, scale * 1.4426950408889634f,
-               static_cast<__nv_bfloat16*>(out), lse, status};
-    const int grid = static_cast<int>(n_q < sm_count ? n_q : sm_count);
-    sparse_attn_kernel<<<grid, kSaThreads, kSaSmemBytes, stream>>>(q_map, p);
+    SaParams p{static_cast<const uint8_t*>(kv), topk, kv_base, n_eff, static_cast<uint8_t*>(scratch), n_q, n_kv, H, k_top,
+               scale * 1.4426950408889634f, static_cast<__nv_bfloat16*>(out), lse, status};
+    sparse_attn_kernel<<<sparse_attn_grid(n_q, sm_count), kSaThreads, kSaSmemBytes, stream>>>(q_map, p);
     return cudaGetLastError();
 }
 
