@@ -60,14 +60,15 @@ cudaError_t launch_quantize_e4m3(const void* x, int64_t n_tokens, int row_elems,
                                  const int64_t* dst_rows, cudaStream_t stream);
 
 // sparse_attn.cu: attention over the selected rows. q_map: q as [n_q * H, 576] bf16, 128-byte swizzle, box
-// 64 columns x H rows. n_eff: [n_q] int32 scratch; scratch: sparse_attn_scratch_bytes(n_q, k_top) bytes, 16-byte
+// 64 columns x H rows; kv_map: kv as [n_kv, 576] bf16, 128-byte swizzle, box 64 columns x 1 row (gather form). n_eff: [n_q] int32 scratch; scratch: sparse_attn_scratch_bytes(n_q, k_top) bytes, 16-byte
 // aligned (the probabilities of a query between its two passes, per CTA). At most kSparseAttnMaxGrid CTAs run.
 constexpr int kSparseAttnMaxGrid = 160;
 bool sparse_attn_supported(int H, int d_qk, int d_v);
 size_t sparse_attn_scratch_bytes(int64_t n_q, int k_top);
 cudaError_t launch_sparse_attn(const void* kv, const int32_t* topk, const int64_t* kv_base, int64_t n_q, int64_t n_kv, int H,
                                int k_top, float scale, void* out, float* lse, int32_t* n_eff, void* scratch,
-                               const CUtensorMap& q_map, unsigned int* status, int sm_count, cudaStream_t stream);
+                               const CUtensorMap& q_map, const CUtensorMap& kv_map, unsigned int* status, int sm_count,
+                               cudaStream_t stream);
 
 // selftest.cu: one tiny kernel whose only wait can never be satisfied; it must record a time-out in
 // `status` after `budget_cycles` and return.

@@ -21,8 +21,9 @@
 //   done), so the next tile's E part is gathered while this tile is still in its softmax. Pass 2 uses the four
 //   slots as a ring of four value tiles.
 // Warps: 0 MMA issuer (tile i+1's scores are issued before tile i's PV product, so the tensor pipe works
-//   while the softmax warps turn S(i) into P(i)), 1 Q loader (TMA), 2-9 row gather (16-byte cp.async into the
-//   swizzled layout; two warps per slot, each slot its own acquire/copy/publish stream), 10-13 softmax: running reference maximum with a lazy rescale of O (only when the maximum
+//   while the softmax warps turn S(i) into P(i)), 1 Q loader (TMA), 2-9 row gather (TMA gather4: four rows of
+//   one 64-column block per instruction, which keeps the load/store unit free for the other warps' barrier and
+//   tensor-memory traffic; two warps per slot, each slot its own acquire/copy stream), 10-13 softmax: running reference maximum with a lazy rescale of O (only when the maximum
 //   grows by more than 2^8).
 // Entries < 0 or pointing outside the cache are skipped; a query's tiles end at its last usable entry
 // (counted by a small kernel first).
@@ -101,7 +102,7 @@ __global__ void sparse_attn_count_kernel(const int32_t* __restrict__ topk, const
 }
 
 __global__ void __launch_bounds__(kSaThreads, 1)
-sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) {
+sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap kv_map, const SaParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint8_t* stage_smem = smem;                               // [2][9][64 x 128 B]; Q blocks 0..3 are staged here first
@@ -131,7 +132,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
         mbar_init(bar_q_ready, 4);
         mbar_init(bar_q_empty, 1);
         for (int i = 0; i < 4; ++i) {
-            mbar_init(bar_slot_full + 8 * i, 2);
+            mbar_init(bar_slot_full + 8 * i, 2);         // one arrive (with its byte count) per gather warp of the slot
             mbar_init(bar_slot_empty + 8 * i, 1);
         }
         for (int i = 0; i < 2; ++i) mbar_init(bar_s_full + 8 * i, 1);
@@ -183,11 +184,10 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
         // 16 gathered rows per MMA; P (bf16 pairs) starts at tensor-memory column p_col
         auto issue_pv = [&](uint32_t v_blocks, uint32_t p_col, bool first_tile) {
             const uint64_t v_desc0 = umma_smem_desc_sw128_mn(v_blocks, kSaKBlockBytes);
-            if (first_tile) umma_f16_ts_elect<false>(tmem_base + kColO, tmem_base + p_col, v_desc0, kIdescPV);
-            else umma_f16_ts_elect<true>(tmem_base + kColO, tmem_base + p_col, v_desc0, kIdescPV);
 #pragma unroll
-            for (int ks = 1; ks < kSaBK / 16; ++ks)
-                umma_f16_ts_elect<true>(tmem_base + kColO, tmem_base + p_col + ks * 8, v_desc0 + (ks * 16 * 128) / 16, kIdescPV);
+            for (int ks = 0; ks < kSaBK / 16; ++ks)
+                umma_f16_ts_elect_acc(tmem_base + kColO, tmem_base + p_col + ks * 8, v_desc0 + (ks * 16 * 128) / 16, kIdescPV,
+                                      (first_tile && ks == 0) ? 0u : 1u);
         };
         for (int64_t t = blockIdx.x; t < p.n_q && ok; t += gridDim.x) {
             const int nt = tiles_of(t);
@@ -207,15 +207,15 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
                 if (!wait_slot(2 * stage_s + 1)) return false;
                 const uint32_t s_tmem = tmem_base + kColS + (i & 1) * 64;
                 const uint64_t k_desc0 = umma_smem_desc_sw128(smem_u32(stage_smem + stage_s * kSaStageBytes));
-#pragma unroll
+                // rolled over the blocks: the instruction footprint of the issuing warp stays small
+                uint64_t a_desc = q_desc0, b_desc = k_desc0 + (kSaQT * kSaKBlockBytes) / 16;
+#pragma unroll 1
                 for (int b = kSaQT; b < kSaNB; ++b) {
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {
-                        const uint64_t a_desc = q_desc0 + ((b - kSaQT) * kSaQBlockBytes + ks * 32) / 16;
-                        const uint64_t b_desc = k_desc0 + (b * kSaKBlockBytes + ks * 32) / 16;
-                        if (b == kSaQT && ks == 0) umma_f16_elect<false>(s_tmem, a_desc, b_desc, kIdescS);
-                        else umma_f16_elect<true>(s_tmem, a_desc, b_desc, kIdescS);
-                    }
+                    for (int ks = 0; ks < 4; ++ks)
+                        umma_f16_elect_acc(s_tmem, a_desc + (ks * 32) / 16, b_desc + (ks * 32) / 16, kIdescS, (b != kSaQT || ks != 0) ? 1u : 0u);
+                    a_desc += kSaQBlockBytes / 16;
+                    b_desc += kSaKBlockBytes / 16;
                 }
                 umma_commit_elect(bar_slot_empty + 8 * (2 * stage_s + 1));    // blocks 4..8 are not needed again
                 return true;
@@ -224,12 +224,15 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
                 if (!wait_slot(2 * stage_s)) return false;
                 const uint32_t s_tmem = tmem_base + kColS + (i & 1) * 64;
                 const uint64_t k_desc0 = umma_smem_desc_sw128(smem_u32(stage_smem + stage_s * kSaStageBytes));
-#pragma unroll
+                uint64_t b_desc = k_desc0;
+                uint32_t a_tmem = tmem_base + kColQ;
+#pragma unroll 1
                 for (int b = 0; b < kSaQT; ++b) {
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)
-                        umma_f16_ts_elect<true>(s_tmem, tmem_base + kColQ + b * 32 + ks * 8,
-                                                k_desc0 + (b * kSaKBlockBytes + ks * 32) / 16, kIdescS);
+                        umma_f16_ts_elect_acc(s_tmem, a_tmem + ks * 8, b_desc + (ks * 32) / 16, kIdescS, 1u);
+                    a_tmem += 32;
+                    b_desc += kSaKBlockBytes / 16;
                 }
                 umma_commit_elect(bar_s_full + 8 * (i & 1));
                 stage_s ^= 1;
@@ -279,11 +282,12 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
         if (lane == 0) {
             // ------------------------------------------------------------ Q loader
             tma_prefetch_desc(&q_map);
+            tma_prefetch_desc(&kv_map);
             uint32_t ph_q_empty = 0;
             bool ok = true;
             for (int64_t t = blockIdx.x; t < p.n_q; t += gridDim.x) {
                 if (tiles_of(t) == 0) continue;
-                ok = mbar_wait(bar_q_empty, ph_q_empty ^ 1u, abort_flag);   // every MMA of the previous query is done
+                ok = mbar_wait(bar_q_empty, ph_q_empty ^ 1u, abort_flag, kWaitCycleBudget, 500);   // every MMA of the previous query is done
                 if (!ok) break;
                 ph_q_empty ^= 1u;
                 mbar_arrive_expect_tx(bar_q_full, static_cast<uint32_t>(kSaNB * p.H * 128));
@@ -309,64 +313,47 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
         for (int64_t t = blockIdx.x; t < p.n_q && ok; t += gridDim.x) {
             const int nt = tiles_of(t);
             if (nt == 0) continue;
-            ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_q_ready, ph_q_ready, abort_flag));   // the staging area is free again
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_q_ready, ph_q_ready, abort_flag, kWaitCycleBudget, 200));   // the staging area is free again
             if (!ok) break;
             ph_q_ready ^= 1u;
             const int64_t base = p.kv_base ? __ldg(p.kv_base + t) : 0;
             const int32_t* row_idx = p.topk + t * p.k_top;
             // lane l looks up row row0 + l of tile i; returns the mask of usable entries
-            auto lookup = [&](int i, int64_t& src_row) -> uint32_t {
+            auto lookup = [&](int i, int& src_row) -> uint32_t {
                 const int j = i * kSaBK + row0 + lane;
                 src_row = -1;
                 if (j < p.k_top) {
                     const int64_t idx = __ldg(row_idx + j);
-                    if (idx >= 0 && base + idx >= 0 && base + idx < p.n_kv) src_row = base + idx;
+                    if (idx >= 0 && base + idx >= 0 && base + idx < p.n_kv) src_row = static_cast<int>(base + idx);
                 }
                 const uint32_t valid = __ballot_sync(0xFFFFFFFFu, src_row >= 0);
                 if (src_row < 0) src_row = 0;                 // skipped entries load row 0 and get weight 0
                 return valid;
             };
-            // copies chunks [c0, c0 + N_CHUNKS) (16 bytes each) of this warp's 32 rows into the slot, 8 rows at a
-            // time: their addresses are formed first, so that the copies issue back to back
-            auto gather = [&](int64_t src_row, int c0, auto n_chunks_tag) {
-                constexpr int N_CHUNKS = decltype(n_chunks_tag)::value;
-                constexpr int PER_LANE = (N_CHUNKS + 31) / 32;
-                uint32_t dst[PER_LANE];
-#pragma unroll
-                for (int k = 0; k < PER_LANE; ++k) {
-                    const int c = lane + 32 * k;
-                    dst[k] = smem_u32(slot_base) + (c >> 3) * kSaKBlockBytes + row0 * 128 + ((c & 7) << 4);
-                }
-#pragma unroll
-                for (int bt = 0; bt < 4; ++bt) {
-                    const uint8_t* src[8];
-#pragma unroll
-                    for (int rr = 0; rr < 8; ++rr)
-                        src[rr] = p.kv + __shfl_sync(0xFFFFFFFFu, src_row, bt * 8 + rr) * (kSaNB * 128) + (c0 + lane) * 16;
-                    // row r = row0 + 8 bt + rr: r & 7 == rr, so the swizzle is an XOR of rr into the chunk index
-#pragma unroll
-                    for (int rr = 0; rr < 8; ++rr) {
-#pragma unroll
-                        for (int k = 0; k < PER_LANE; ++k)
-                            if (lane + 32 * k < N_CHUNKS)
-                                cp_async_16((dst[k] ^ (rr << 4)) + (bt * 8 + rr) * 128, src[rr] + k * 512);
+            // TMA gather of column blocks [cb0, cb0 + n_blocks) of this warp's 32 rows into the slot's blocks 0..n_blocks-1:
+            // four rows per instruction, issued by lane 0, completion counted in bytes on the slot's barrier
+            auto gather = [&](int src_row, int cb0, int n_blocks) {
+                if (lane == 0) mbar_arrive_expect_tx(bar_slot_full + 8 * slot, static_cast<uint32_t>(32 * 128 * n_blocks));
+#pragma unroll 1
+                for (int g = 0; g < 8; ++g) {
+                    const int r0 = __shfl_sync(0xFFFFFFFFu, src_row, 4 * g), r1 = __shfl_sync(0xFFFFFFFFu, src_row, 4 * g + 1);
+                    const int r2 = __shfl_sync(0xFFFFFFFFu, src_row, 4 * g + 2), r3 = __shfl_sync(0xFFFFFFFFu, src_row, 4 * g + 3);
+                    if (lane == 0) {
+                        const uint32_t dst = smem_u32(slot_base) + (row0 + 4 * g) * 128;
+                        for (int b = 0; b < n_blocks; ++b)
+                            tma_gather4_2d(dst + b * kSaKBlockBytes, &kv_map, bar_slot_full + 8 * slot, (cb0 + b) * 64, r0, r1, r2, r3);
                     }
                 }
+                __syncwarp();
             };
             auto acquire = [&]() -> bool {
-                const bool got = __all_sync(0xFFFFFFFFu, mbar_wait(bar_slot_empty + 8 * slot, ph_empty ^ 1u, abort_flag));
+                const bool got = __all_sync(0xFFFFFFFFu, mbar_wait(bar_slot_empty + 8 * slot, ph_empty ^ 1u, abort_flag, kWaitCycleBudget, 100));
                 ph_empty ^= 1u;
                 return got;
             };
-            auto publish = [&]() {
-                cp_async_wait_all();
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_slot_full + 8 * slot);
-            };
             // ---- pass 1: the tiles that sit in this slot's stage; group 1 = columns 256..575, group 0 = columns 0..255
             {
-                int64_t src_row, src_next = 0;
+                int src_row = 0, src_next = 0;
                 uint32_t valid_next = 0;
                 const int first = ((slot >> 1) ^ static_cast<int>(tile_seq & 1u)) & 1;
                 uint32_t valid = first < nt ? lookup(first, src_row) : 0u;
@@ -375,12 +362,11 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
                     ok = acquire();
                     if (!ok) break;
                     if (slot & 1) {
-                        gather(src_row, kSaNVH * 8, std::integral_constant<int, (kSaNB - kSaNVH) * 8>{});
+                        gather(src_row, kSaNVH, kSaNB - kSaNVH);
                     } else {
-                        gather(src_row, 0, std::integral_constant<int, kSaNVH * 8>{});
                         if (lane == 0) tile_mask[(slot >> 1) * 2 + (gw & 1)] = valid;
+                        gather(src_row, 0, kSaNVH);
                     }
-                    publish();
                     src_row = src_next;
                     valid = valid_next;
                 }
@@ -388,19 +374,17 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
             }
             // ---- pass 2: columns 256..511 only; tile i sits in slot i & 3
             if (ok) {
-                int64_t src_row, src_next = 0;
+                int src_row = 0, src_next = 0;
                 if (slot < nt) lookup(slot, src_row);
                 for (int i = slot; i < nt; i += 4) {
                     if (i + 4 < nt) lookup(i + 4, src_next);
                     ok = acquire();
                     if (!ok) break;
-                    gather(src_row, kSaNVH * 8, std::integral_constant<int, kSaNVH * 8>{});
-                    publish();
+                    gather(src_row, kSaNVH, kSaNVH);
                     src_row = src_next;
                 }
             }
         }
-        cp_async_wait_all();
         if (!ok && lane == 0) sa_give_up(abort_flag, p.status, DEV_TIMEOUT_GATHER);
     } else {
         // ---------------------------------------------------------------- softmax and output
@@ -494,20 +478,29 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
                 ph_s_full[sbuf] ^= 1u;
                 tcgen05_fence_after_sync();
                 const uint32_t s_tmem = lane_base + kColS + sbuf * 64;
-                uint32_t sa[32], sb[32];
-                tmem_ld_32x32b_x32(s_tmem, sa);
-                tmem_ld_32x32b_x32(s_tmem + 32, sb);
-                tmem_ld_wait(sa);
-                tmem_ld_wait(sb);
                 const uint32_t mlo = tile_mask[stage * 2], mhi = tile_mask[stage * 2 + 1];
+                // Both sweeps over the 64 scores are rolled loops over 16-column chunks, read from tensor memory
+                // twice: the instruction footprint of the hot loop stays small.
+                // (the load of the next chunk is in flight while a chunk is processed: a tensor-memory load takes ~200 cycles)
                 float mt = -INFINITY;
+                auto max16 = [&](const uint32_t (&r)[16], uint32_t m16) {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const float xa = (mlo >> j) & 1u ? __uint_as_float(sa[j]) * p.scale_log2 : -INFINITY;
-                    const float xb = (mhi >> j) & 1u ? __uint_as_float(sb[j]) * p.scale_log2 : -INFINITY;
-                    sa[j] = __float_as_uint(xa);
-                    sb[j] = __float_as_uint(xb);
-                    mt = fmaxf(mt, fmaxf(xa, xb));
+                    for (int j = 0; j < 16; ++j)
+                        mt = fmaxf(mt, (m16 >> j) & 1u ? __uint_as_float(r[j]) * p.scale_log2 : -INFINITY);
+                };
+                {
+                    uint32_t ra[16], rb[16];
+                    tmem_ld_32x32b_x16(s_tmem, ra);
+#pragma unroll 1
+                    for (int h = 0; h < 2; ++h) {
+                        const uint32_t m32 = h ? mhi : mlo;
+                        tmem_ld_wait(ra);
+                        tmem_ld_32x32b_x16(s_tmem + 32 * h + 16, rb);
+                        max16(ra, m32);
+                        tmem_ld_wait(rb);
+                        if (h == 0) tmem_ld_32x32b_x16(s_tmem + 32, ra);
+                        max16(rb, m32 >> 16);
+                    }
                 }
                 // lazy reference maximum: move it only when the row maximum outgrew it by 2^8
                 const bool move = mt > m_ref + kRescaleThreshold;      // also true for the first usable score (m_ref = -inf)
@@ -525,26 +518,43 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
                     scale_o(alpha);
                 }
                 const float m_sub = m_ref == -INFINITY ? 0.f : m_ref;   // no usable score yet: every P is exp2(-inf) = 0
-                uint32_t pr[32];
+                // P(i) goes over the first half of S(i) chunk by chunk (columns 8c..8c+7 hold scores this thread has
+                // already read) and, with the factor, to the scratch area for pass 2 (read back by this same thread)
+                uint4* dst = reinterpret_cast<uint4*>(my_p + static_cast<size_t>(i) * kSaScratchTileBytes);
                 float sum = 0.f;
+                auto exp16 = [&](const uint32_t (&r)[16], uint32_t m16, int c) {
+                    uint32_t pr[8];
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const float p0 = fast_exp2(__uint_as_float(sa[2 * j]) - m_sub), p1 = fast_exp2(__uint_as_float(sa[2 * j + 1]) - m_sub);
-                    const float p2 = fast_exp2(__uint_as_float(sb[2 * j]) - m_sub), p3 = fast_exp2(__uint_as_float(sb[2 * j + 1]) - m_sub);
-                    sum += (p0 + p1) + (p2 + p3);
-                    pr[j] = pack_bf16x2(p0, p1);
-                    pr[16 + j] = pack_bf16x2(p2, p3);
+                    for (int j = 0; j < 8; ++j) {
+                        const float x0 = (m16 >> (2 * j)) & 1u ? __uint_as_float(r[2 * j]) * p.scale_log2 : -INFINITY;
+                        const float x1 = (m16 >> (2 * j + 1)) & 1u ? __uint_as_float(r[2 * j + 1]) * p.scale_log2 : -INFINITY;
+                        const float p0 = fast_exp2(x0 - m_sub), p1 = fast_exp2(x1 - m_sub);
+                        sum += p0 + p1;
+                        pr[j] = pack_bf16x2(p0, p1);
+                    }
+                    tmem_st_32x32b_x8(s_tmem + 8 * c, pr);
+                    __stcg(dst + 2 * c, make_uint4(pr[0], pr[1], pr[2], pr[3]));
+                    __stcg(dst + 2 * c + 1, make_uint4(pr[4], pr[5], pr[6], pr[7]));
+                };
+                {
+                    uint32_t ra[16], rb[16];
+                    tmem_ld_32x32b_x16(s_tmem, ra);
+#pragma unroll 1
+                    for (int h = 0; h < 2; ++h) {
+                        const uint32_t m32 = h ? mhi : mlo;
+                        tmem_ld_wait(ra);
+                        tmem_ld_32x32b_x16(s_tmem + 32 * h + 16, rb);
+                        exp16(ra, m32, 2 * h);
+                        tmem_ld_wait(rb);
+                        if (h == 0) tmem_ld_32x32b_x16(s_tmem + 32, ra);   // columns 32..47: beyond the P columns written so far
+                        exp16(rb, m32 >> 16, 2 * h + 1);
+                    }
                 }
                 l += sum;
-                tmem_st_32x32b_x32(s_tmem, pr);                   // P(i) over the first half of S(i): this thread holds its row
                 tmem_st_wait();
                 tcgen05_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_p_ready + 8 * sbuf);
-                // keep P(i) and the factor for pass 2 (read back by this same thread)
-                uint4* dst = reinterpret_cast<uint4*>(my_p + static_cast<size_t>(i) * kSaScratchTileBytes);
-#pragma unroll
-                for (int v = 0; v < 8; ++v) __stcg(dst + v, make_uint4(pr[4 * v], pr[4 * v + 1], pr[4 * v + 2], pr[4 * v + 3]));
                 __stcg(reinterpret_cast<float*>(my_alpha + static_cast<size_t>(i) * kSaScratchTileBytes), alpha);
                 ++pv_tiles;
                 stage ^= 1;
@@ -565,6 +575,11 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
                 for (int v = 0; v < 8; ++v) dst[v] = __ldcg(src + v);
                 alpha = __ldcg(reinterpret_cast<const float*>(my_alpha + static_cast<size_t>(i) * kSaScratchTileBytes));
             };
+            // the scratch area has usually left the L2 by now: pull this thread's lines back in well ahead of their use
+            auto prefetch_p = [&](int i) {
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(my_p + static_cast<size_t>(i) * kSaScratchTileBytes));
+            };
+            for (int i = 0; i < 8 && i < nt; ++i) prefetch_p(i);
             load_p(0, pa, alpha_a);
             if (nt > 1) load_p(1, pb, alpha_b);
             for (int i = 0; i < nt; ++i) {
@@ -577,6 +592,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
                 for (int v = 0; v < 8; ++v) pa[v] = pb[v];
                 alpha_a = alpha_b;
                 if (i + 2 < nt) load_p(i + 2, pb, alpha_b);
+                if (i + 8 < nt) prefetch_p(i + 8);
                 ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_p_free + 8 * pbuf, ph_p_free[pbuf] ^ 1u, abort_flag));   // PV(i-4) has read this buffer
                 if (!ok) break;
                 ph_p_free[pbuf] ^= 1u;
@@ -632,7 +648,7 @@ size_t sparse_attn_scratch_bytes(int64_t n_q, int k_top) {
 
 cudaError_t launch_sparse_attn(const void* kv, const int32_t* topk, const int64_t* kv_base, int64_t n_q, int64_t n_kv, int H,
                                int k_top, float scale, void* out, float* lse, int32_t* n_eff, void* scratch,
-                               const CUtensorMap& q_map, unsigned int* status, int sm_count, cudaStream_t stream) {
+                               const CUtensorMap& q_map, const CUtensorMap& kv_map, unsigned int* status, int sm_count, cudaStream_t stream) {
     if (n_q <= 0) return cudaSuccess;
     const int64_t count_blocks = (n_q * 32 + 255) / 256;
     sparse_attn_count_kernel<<<static_cast<unsigned>(count_blocks), 256, 0, stream>>>(topk, kv_base, n_q, n_kv, k_top, n_eff);
@@ -640,7 +656,7 @@ cudaError_t launch_sparse_attn(const void* kv, const int32_t* topk, const int64_
     if (cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(sparse_attn_kernel), kSaSmemBytes); e != cudaSuccess) return e;
     SaParams p{static_cast<const uint8_t*>(kv), topk, kv_base, n_eff, static_cast<uint8_t*>(scratch), n_q, n_kv, H, k_top,
                scale * 1.4426950408889634f, static_cast<__nv_bfloat16*>(out), lse, status};
-    sparse_attn_kernel<<<sparse_attn_grid(n_q, sm_count), kSaThreads, kSaSmemBytes, stream>>>(q_map, p);
+    sparse_attn_kernel<<<sparse_attn_grid(n_q, sm_count), kSaThreads, kSaSmemBytes, stream>>>(q_map, kv_map, p);
     return cudaGetLastError();
 }
 
