@@ -16,6 +16,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import sys
@@ -394,6 +395,44 @@ def time_distill(idxc, dev, peaks, L, n_targets):
                          "of": peaks["source"]}}
 
 
+def time_sparse_attention(idxc, synth, dev, peaks, L, n_q, k_top, seed, steps=3):
+    """NEXT-2: the consumer of the indices (Sec. 2.1): attention of the last n_q queries of an L-token prefill over the
+    k_top rows the indexer picked for them (the real chain: indexer scores -> top-k -> attention), 128 heads over a
+    shared latent row of 576 columns whose leading 512 are the value. Useful work: 2 * H * (d_qk + d_v) flops per
+    (query, selected row); the kernel also recomputes nothing (scores once, P V in two halves)."""
+    H_a, d_qk, d_v, H_i, d_i = 128, 576, 512, 64, 128
+    pin = synth.prefill_inputs(L, H_i, d_i, seed=seed, device=dev, clustered=True)
+    q0 = L - n_q
+    topk = torch.empty((n_q, k_top), dtype=torch.int32, device=dev)
+    ws = idxc.alloc_workspace(idxc.prefill_workspace_bytes(n_q, L, H_i, d_i, k_top), dev)
+    idxc.indexer_prefill(pin.q[q0:], pin.k, pin.w[q0:], k_top, q_begin=q0, topk_out=topk, workspace=ws)
+    del pin, ws
+    inp = synth.attention_inputs(n_q, L, H_a, d_qk, seed=seed, device=dev)
+    out = torch.empty((n_q, H_a, d_v), dtype=torch.bfloat16, device=dev)
+    ws = idxc.alloc_workspace(idxc.lib().idxc_sparse_attention_workspace_bytes(n_q, k_top), dev)
+    scale = 1.0 / math.sqrt(d_qk)
+    for _ in range(2):
+        idxc.sparse_attention(inp.q, inp.kv, topk, d_v, scale, out=out, workspace=ws, want_lse=False)
+    idxc.poll_device_status()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(steps):
+        idxc.sparse_attention(inp.q, inp.kv, topk, d_v, scale, out=out, workspace=ws, want_lse=False)
+    b.record()
+    torch.cuda.synchronize()
+    idxc.poll_device_status()
+    ms = a.elapsed_time(b) / steps
+    selected = int((topk >= 0).sum().item())
+    flops = 2.0 * H_a * (d_qk + d_v) * selected
+    tf = flops / (ms * 1e-3) / 1e12
+    gather_bytes = selected * (d_qk + d_v // 2) * 2
+    return {"workload": f"last {n_q} queries of an L={L} prefill, H=128, d_qk=576, d_v=512, k_top={k_top}, indices from the indexer",
+            "ms": ms, "queries_per_s": n_q / (ms * 1e-3), "selected_rows": selected,
+            "gathered_bytes": gather_bytes,
+            "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                         "frac": tf / peaks["bf16_tflops"], "of": peaks["source"] + " burst peak", "traffic": None}}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -410,6 +449,8 @@ def main():
     ap.add_argument("--full", action="store_true", help="extras at full size: config 4 with N=48, L=65536; config 5 with L=131072")
     ap.add_argument("--L", type=int, default=0, help="override the workload's sequence length (small profiling cases)")
     ap.add_argument("--only-decode", action="store_true", help="run only the decode section (profiling)")
+    ap.add_argument("--only-sparse-attention", action="store_true", help="run only the sparse-attention section (profiling)")
+    ap.add_argument("--sa-queries", type=int, default=8192, help="queries of the sparse-attention section")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -441,6 +482,10 @@ def main():
     if args.only_decode:
         print(json.dumps({"decode": time_decode(idxc, synth, dev, peaks, steps=max(args.steps, 1), warmup=args.warmup)}),
               flush=True)
+        return
+    if args.only_sparse_attention:
+        print(json.dumps({"sparse_attention": time_sparse_attention(idxc, synth, dev, peaks, args.L or 32768, args.sa_queries, 2048,
+                                                                     seed=7, steps=max(args.steps, 1))}), flush=True)
         return
     c = dict(synth.CONFIGS[args.workload])
     if args.L:
@@ -610,6 +655,8 @@ def main():
             n_layers, sched_L = (c4["N"], c4["L"]) if args.full else (args.schedule_layers, args.schedule_L)
             line["schedule"] = time_schedule(idxc, synth, dev, sched_L, c4["H"], c4["d"], c4["k_top"], n_layers, c4["every"],
                                              seed=c4["seed"], reps=1 if args.full else 2)
+            torch.cuda.empty_cache()
+            line["sparse_attention"] = time_sparse_attention(idxc, synth, dev, peaks, 32768, args.sa_queries, c4["k_top"], seed=7)
             torch.cuda.empty_cache()
             line["distill_kl"] = time_distill(idxc, dev, peaks, 16384, 2)
             torch.cuda.empty_cache()

@@ -127,3 +127,26 @@ def test_argument_errors():
     # zero queries: nothing to do
     out, _ = binding.sparse_attention(inp.q[:0], inp.kv, topk[:0], D_V, 1.0)
     assert out.shape == (0, H, D_V)
+
+
+def test_bench_size_chain_sampled_queries():
+    # the launch configuration of bench.py's sparse-attention section: the last 8192 queries of an L = 32768 prefill,
+    # k_top = 2048, indices from the indexer; the oracle checks a sample of whole queries, the rest is checked for
+    # finiteness and against the convex-hull property (|out| cannot exceed the largest selected |value|)
+    L, n_q, k_top = 32768, 8192, 2048
+    q0 = L - n_q
+    pin = synth.prefill_inputs(L, 64, 128, seed=7, device="cuda", clustered=True)
+    topk = torch.empty((n_q, k_top), dtype=torch.int32, device="cuda")
+    ws = binding.alloc_workspace(binding.prefill_workspace_bytes(n_q, L, 64, 128, k_top), "cuda")
+    binding.indexer_prefill(pin.q[q0:], pin.k, pin.w[q0:], k_top, q_begin=q0, topk_out=topk, workspace=ws)
+    del pin, ws
+    inp = synth.attention_inputs(n_q, L, H, D_QK, seed=7, device="cuda")
+    scale = 1.0 / np.sqrt(D_QK)
+    out, lse = binding.sparse_attention(inp.q, inp.kv, topk, D_V, scale)
+    binding.poll_device_status()
+    assert bool(torch.isfinite(out.float()).all()) and bool(torch.isfinite(lse).all())
+    vmax = float(inp.kv[:, :D_V].float().abs().max())
+    assert float(out.float().abs().max()) <= vmax * (1 + 2 ** -7)
+    rows = [0, 1, 147, 148, 2047, 4096, n_q - 149, n_q - 1]
+    o_out, o_lse = osa.sparse_attention(codes(inp.q[rows]), codes(inp.kv), topk[rows].cpu().numpy(), D_V, scale)
+    _check(out, lse, o_out, o_lse, np.asarray(rows), "bench size")
