@@ -21,9 +21,8 @@
 //   done), so the next tile's E part is gathered while this tile is still in its softmax. Pass 2 uses the four
 //   slots as a ring of four value tiles.
 // Warps: 0 MMA issuer (tile i+1's scores are issued before tile i's PV product, so the tensor pipe works
-//   while the softmax warps turn S(i) into P(i)), 1 Q loader (TMA), 2-9 row gather (TMA gather4: four rows of
-//   one 64-column block per instruction, which keeps the load/store unit free for the other warps' barrier and
-//   tensor-memory traffic; two warps per slot, each slot its own acquire/copy stream), 10-13 softmax: running reference maximum with a lazy rescale of O (only when the maximum
+//   while the softmax warps turn S(i) into P(i)), 1 Q loader (TMA), 2-9 row gather (16-byte cp.async into the
+//   swizzled layout; two warps per slot, each slot its own acquire/copy/publish stream), 10-13 softmax: running reference maximum with a lazy rescale of O (only when the maximum
 //   grows by more than 2^8).
 // Entries < 0 or pointing outside the cache are skipped; a query's tiles end at its last usable entry
 // (counted by a small kernel first).
@@ -132,7 +131,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         mbar_init(bar_q_ready, 4);
         mbar_init(bar_q_empty, 1);
         for (int i = 0; i < 4; ++i) {
-            mbar_init(bar_slot_full + 8 * i, 2);         // one arrive (with its byte count) per gather warp of the slot
+            mbar_init(bar_slot_full + 8 * i, 2);         // one arrive per gather warp of the slot
             mbar_init(bar_slot_empty + 8 * i, 1);
         }
         for (int i = 0; i < 2; ++i) mbar_init(bar_s_full + 8 * i, 1);
@@ -330,21 +329,33 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 if (src_row < 0) src_row = 0;                 // skipped entries load row 0 and get weight 0
                 return valid;
             };
-            // TMA gather of column blocks [cb0, cb0 + n_blocks) of this warp's 32 rows into the slot's blocks 0..n_blocks-1:
-            // four rows per instruction, issued by lane 0, completion counted in bytes on the slot's barrier
+            // Copies column blocks [cb0, cb0 + n_blocks) of this warp's 32 rows into the slot's blocks 0..n_blocks-1 with
+            // 16-byte cp.async into the swizzled layout: a warp instruction moves 512 contiguous bytes of one row. Eight
+            // rows' addresses are formed before their copies issue. (TMA gather4 was measured too: one instruction per
+            // four rows and block, about 22 cycles each at the TMA unit, 2.4x slower than this for the same bytes.)
             auto gather = [&](int src_row, int cb0, int n_blocks) {
-                if (lane == 0) mbar_arrive_expect_tx(bar_slot_full + 8 * slot, static_cast<uint32_t>(32 * 128 * n_blocks));
+                const uint32_t dst0 = smem_u32(slot_base) + (lane >> 3) * kSaKBlockBytes + row0 * 128 + ((lane & 7) << 4);
+                const uint32_t dst1 = dst0 + 4 * kSaKBlockBytes;        // chunk lane + 32 lies four blocks further
+                const bool second = lane + 32 < n_blocks * 8;
 #pragma unroll 1
-                for (int g = 0; g < 8; ++g) {
-                    const int r0 = __shfl_sync(0xFFFFFFFFu, src_row, 4 * g), r1 = __shfl_sync(0xFFFFFFFFu, src_row, 4 * g + 1);
-                    const int r2 = __shfl_sync(0xFFFFFFFFu, src_row, 4 * g + 2), r3 = __shfl_sync(0xFFFFFFFFu, src_row, 4 * g + 3);
-                    if (lane == 0) {
-                        const uint32_t dst = smem_u32(slot_base) + (row0 + 4 * g) * 128;
-                        for (int b = 0; b < n_blocks; ++b)
-                            tma_gather4_2d(dst + b * kSaKBlockBytes, &kv_map, bar_slot_full + 8 * slot, (cb0 + b) * 64, r0, r1, r2, r3);
+                for (int bt = 0; bt < 4; ++bt) {
+                    const uint8_t* src[8];
+#pragma unroll
+                    for (int rr = 0; rr < 8; ++rr)
+                        src[rr] = p.kv + static_cast<int64_t>(__shfl_sync(0xFFFFFFFFu, src_row, bt * 8 + rr)) * (kSaNB * 128) +
+                                  (cb0 * 8 + lane) * 16;
+                    // row r = row0 + 8 bt + rr: r & 7 == rr, so the swizzle is an XOR of rr into the chunk index
+#pragma unroll
+                    for (int rr = 0; rr < 8; ++rr) {
+                        const uint32_t off = (bt * 8 + rr) * 128;
+                        cp_async_16((dst0 ^ (rr << 4)) + off, src[rr]);
+                        if (second) cp_async_16((dst1 ^ (rr << 4)) + off, src[rr] + 512);
                     }
                 }
+                cp_async_wait_all();
+                fence_proxy_async_smem();
                 __syncwarp();
+                if (lane == 0) mbar_arrive(bar_slot_full + 8 * slot);
             };
             auto acquire = [&]() -> bool {
                 const bool got = __all_sync(0xFFFFFFFFu, mbar_wait(bar_slot_empty + 8 * slot, ph_empty ^ 1u, abort_flag, kWaitCycleBudget, 100));
