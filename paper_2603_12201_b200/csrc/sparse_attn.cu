@@ -578,8 +578,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 
             // ---- pass 2: P and the factors come back from the scratch area, two tiles ahead, into a ring of four
             // P buffers (the 128 columns of the S buffers)
-            uint4 pa[8], pb[8];                                  // P of tiles i and i + 1
-            float alpha_a, alpha_b = 1.f;
+            uint4 pa[8], pb[8];                                  // P of an even and of an odd tile, loaded two tiles ahead
+            float alpha_a = 1.f, alpha_b = 1.f;
             auto load_p = [&](int i, uint4 (&dst)[8], float& alpha) {
                 const uint4* src = reinterpret_cast<const uint4*>(my_p + static_cast<size_t>(i) * kSaScratchTileBytes);
 #pragma unroll
@@ -590,32 +590,22 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             auto prefetch_p = [&](int i) {
                 asm volatile("prefetch.global.L2 [%0];" ::"l"(my_p + static_cast<size_t>(i) * kSaScratchTileBytes));
             };
-            for (int i = 0; i < 8 && i < nt; ++i) prefetch_p(i);
-            load_p(0, pa, alpha_a);
-            if (nt > 1) load_p(1, pb, alpha_b);
-            for (int i = 0; i < nt; ++i) {
+            // hands P(i) to the MMA warp: wait for its ring buffer, replay the rescale of pass 1, store, signal
+            auto hand_over = [&](int i, const uint4 (&src)[8], float alpha) -> bool {
                 const int pbuf = i & 3;
-                uint32_t pr[32];
-#pragma unroll
-                for (int v = 0; v < 8; ++v) { pr[4 * v] = pa[v].x; pr[4 * v + 1] = pa[v].y; pr[4 * v + 2] = pa[v].z; pr[4 * v + 3] = pa[v].w; }
-                const float alpha = alpha_a;
-#pragma unroll
-                for (int v = 0; v < 8; ++v) pa[v] = pb[v];
-                alpha_a = alpha_b;
-                if (i + 2 < nt) load_p(i + 2, pb, alpha_b);
-                if (i + 8 < nt) prefetch_p(i + 8);
-                ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_p_free + 8 * pbuf, ph_p_free[pbuf] ^ 1u, abort_flag));   // PV(i-4) has read this buffer
-                if (!ok) break;
+                if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar_p_free + 8 * pbuf, ph_p_free[pbuf] ^ 1u, abort_flag))) return false;   // PV(i-4) has read this buffer
                 ph_p_free[pbuf] ^= 1u;
                 if (i > 0 && __any_sync(0xFFFFFFFFu, alpha != 1.f)) {
                     // The factor applies to the sum over the tiles before i: PV(i-1) must be complete. It arrives on the
                     // p_free barrier of its buffer; the parity is the one this thread's next wait on that buffer will use
                     // (no PV product from tile i on can have been issued, so the barrier cannot be further ahead).
                     const int prev = (i - 1) & 3;
-                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_p_free + 8 * prev, ph_p_free[prev] ^ 1u, abort_flag));
-                    if (!ok) break;
+                    if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar_p_free + 8 * prev, ph_p_free[prev] ^ 1u, abort_flag))) return false;
                     scale_o(alpha);
                 }
+                uint32_t pr[32];
+#pragma unroll
+                for (int v = 0; v < 8; ++v) { pr[4 * v] = src[v].x; pr[4 * v + 1] = src[v].y; pr[4 * v + 2] = src[v].z; pr[4 * v + 3] = src[v].w; }
                 tcgen05_fence_after_sync();
                 tmem_st_32x32b_x32(lane_base + kColS + pbuf * 32, pr);
                 tmem_st_wait();
@@ -623,6 +613,23 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_p_ready + 8 * pbuf);
                 ++pv_tiles;
+                return true;
+            };
+            for (int i = 0; i < 8 && i < nt; ++i) prefetch_p(i);
+            load_p(0, pa, alpha_a);
+            if (nt > 1) load_p(1, pb, alpha_b);
+#pragma unroll 1
+            for (int i = 0; i < nt && ok; i += 2) {
+                ok = hand_over(i, pa, alpha_a);
+                if (!ok) break;
+                if (i + 2 < nt) load_p(i + 2, pa, alpha_a);
+                if (i + 8 < nt) prefetch_p(i + 8);
+                if (i + 1 < nt) {
+                    ok = hand_over(i + 1, pb, alpha_b);
+                    if (!ok) break;
+                    if (i + 3 < nt) load_p(i + 3, pb, alpha_b);
+                    if (i + 9 < nt) prefetch_p(i + 9);
+                }
             }
             if (!ok) break;
             ok = write_out(out_row + 256, inv);
