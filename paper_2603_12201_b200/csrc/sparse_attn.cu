@@ -578,17 +578,26 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 
             // ---- pass 2: P and the factors come back from the scratch area, two tiles ahead, into a ring of four
             // P buffers (the 128 columns of the S buffers)
-            uint4 pa[8], pb[8];                                  // P of an even and of an odd tile, loaded two tiles ahead
-            float alpha_a = 1.f, alpha_b = 1.f;
-            auto load_p = [&](int i, uint4 (&dst)[8], float& alpha) {
-                const uint4* src = reinterpret_cast<const uint4*>(my_p + static_cast<size_t>(i) * kSaScratchTileBytes);
+            // Each thread stages its own 128-byte row of P (and its factor) four tiles ahead with cp.async, in the
+            // shared memory that held Q (unused in pass 2): the scratch area has usually left the L2 by now, and a
+            // round trip to HBM is longer than two tiles of work.
+            uint8_t* const p_ring = q_smem;                                            // [4][128 rows x 128 B], chunks swizzled by row
+            float* const a_ring = reinterpret_cast<float*>(q_smem + 4 * kSaQBlockBytes);   // [4][128]
+            auto stage_p = [&](int i) {
+                if (i < nt) {
+                    const uint8_t* src = my_p + static_cast<size_t>(i) * kSaScratchTileBytes;
+                    const uint32_t dst = smem_u32(p_ring) + (i & 3) * kSaQBlockBytes + row * 128;
 #pragma unroll
-                for (int v = 0; v < 8; ++v) dst[v] = __ldcg(src + v);
-                alpha = __ldcg(reinterpret_cast<const float*>(my_alpha + static_cast<size_t>(i) * kSaScratchTileBytes));
+                    for (int c = 0; c < 8; ++c) cp_async_16(dst + ((c ^ (row & 7)) << 4), src + c * 16);
+                    cp_async_4(smem_u32(a_ring + (i & 3) * 128 + row), my_alpha + static_cast<size_t>(i) * kSaScratchTileBytes);
+                }
+                cp_async_commit_group();                                               // one group per tile, empty past the end
             };
-            // the scratch area has usually left the L2 by now: pull this thread's lines back in well ahead of their use
-            auto prefetch_p = [&](int i) {
-                asm volatile("prefetch.global.L2 [%0];" ::"l"(my_p + static_cast<size_t>(i) * kSaScratchTileBytes));
+            auto fetch_p = [&](int i, uint4 (&dst)[8], float& alpha) {                 // after cp_async_wait_group: own data only
+                const uint8_t* src = p_ring + (i & 3) * kSaQBlockBytes + row * 128;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) dst[c] = *reinterpret_cast<const uint4*>(src + ((c ^ (row & 7)) << 4));
+                alpha = a_ring[(i & 3) * 128 + row];
             };
             // hands P(i) to the MMA warp: wait for its ring buffer, replay the rescale of pass 1, store, signal
             auto hand_over = [&](int i, const uint4 (&src)[8], float alpha) -> bool {
@@ -615,22 +624,17 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 ++pv_tiles;
                 return true;
             };
-            for (int i = 0; i < 8 && i < nt; ++i) prefetch_p(i);
-            load_p(0, pa, alpha_a);
-            if (nt > 1) load_p(1, pb, alpha_b);
+            for (int i = 0; i < 4; ++i) stage_p(i);
 #pragma unroll 1
-            for (int i = 0; i < nt && ok; i += 2) {
-                ok = hand_over(i, pa, alpha_a);
-                if (!ok) break;
-                if (i + 2 < nt) load_p(i + 2, pa, alpha_a);
-                if (i + 8 < nt) prefetch_p(i + 8);
-                if (i + 1 < nt) {
-                    ok = hand_over(i + 1, pb, alpha_b);
-                    if (!ok) break;
-                    if (i + 3 < nt) load_p(i + 3, pb, alpha_b);
-                    if (i + 9 < nt) prefetch_p(i + 9);
-                }
+            for (int i = 0; i < nt && ok; ++i) {
+                uint4 pv[8];
+                float alpha;
+                cp_async_wait_group<3>();                                               // tile i's group has landed
+                fetch_p(i, pv, alpha);
+                ok = hand_over(i, pv, alpha);
+                stage_p(i + 4);                                                         // its ring slot is free again
             }
+            cp_async_wait_all();
             if (!ok) break;
             ok = write_out(out_row + 256, inv);
         }
