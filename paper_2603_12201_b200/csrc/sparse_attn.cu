@@ -53,7 +53,7 @@ static_assert(kSaQT * kSaQBlockBytes <= 2 * kSaStageBytes, "the Q staging area l
 static_assert(kSaSmemBytes <= 232448, "shared memory budget of one CTA");
 constexpr uint32_t kColO = 0, kColS = 256, kColQ = 384;   // S buffer b at kColS + 64 b; P in its first 32 columns
 constexpr float kRescaleThreshold = 8.f;  // log2 units: P stays below 2^8
-constexpr uint32_t kSaScratchTileBytes = 128 * kSaBK * 2 + 128 * 4;   // P [128][64] bf16 + rescale factors [128] fp32
+constexpr uint32_t kSaScratchTileBytes = 128 * kSaBK * 2 + 128 * 4;   // P as [8 chunks][128 rows][16 B] + rescale factors [128] fp32
 
 struct SaParams {
     const uint8_t* kv;          // [n_kv, 576] bf16
@@ -407,7 +407,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         uint32_t pv_tiles = 0;                         // PV tiles before the current one, over the whole kernel
         int stage = 0;
         bool ok = true;
-        uint8_t* my_p = scratch + row * (kSaBK * 2);                  // + tile * kSaScratchTileBytes: this row's P, 128 bytes
+        // Saved P of a tile: [8 chunks of 16 bytes][128 rows]: a warp's store or copy of one chunk touches 512 contiguous bytes
+        uint8_t* my_p = scratch + row * 16;                           // + tile * kSaScratchTileBytes + chunk * 2048
         uint8_t* my_alpha = scratch + 128 * kSaBK * 2 + row * 4;      // + tile * kSaScratchTileBytes: this row's factor
         // multiplies this thread's row of O by alpha (the caller has made sure that every earlier PV product is complete)
         auto scale_o = [&](float alpha) {
@@ -544,8 +545,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                         pr[j] = pack_bf16x2(p0, p1);
                     }
                     tmem_st_32x32b_x8(s_tmem + 8 * c, pr);
-                    __stcg(dst + 2 * c, make_uint4(pr[0], pr[1], pr[2], pr[3]));
-                    __stcg(dst + 2 * c + 1, make_uint4(pr[4], pr[5], pr[6], pr[7]));
+                    __stcg(dst + (2 * c) * 128, make_uint4(pr[0], pr[1], pr[2], pr[3]));
+                    __stcg(dst + (2 * c + 1) * 128, make_uint4(pr[4], pr[5], pr[6], pr[7]));
                 };
                 {
                     uint32_t ra[16], rb[16];
@@ -588,7 +589,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     const uint8_t* src = my_p + static_cast<size_t>(i) * kSaScratchTileBytes;
                     const uint32_t dst = smem_u32(p_ring) + (i & 3) * kSaQBlockBytes + row * 128;
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) cp_async_16(dst + ((c ^ (row & 7)) << 4), src + c * 16);
+                    for (int c = 0; c < 8; ++c) cp_async_16(dst + ((c ^ (row & 7)) << 4), src + c * 2048);
                     cp_async_4(smem_u32(a_ring + (i & 3) * 128 + row), my_alpha + static_cast<size_t>(i) * kSaScratchTileBytes);
                 }
                 cp_async_commit_group();                                               // one group per tile, empty past the end
