@@ -10,25 +10,28 @@
 //   pass 1  gathers whole rows (576 columns), S = Q K^T, softmax, O[:, 0:256] += P V; the bf16 probabilities P
 //           and the rescale factors of the running maximum also go to a per-CTA scratch area in global memory
 //   pass 2  gathers only columns 256..511 of the same rows, reads P back and does O[:, 256:512] += P V with the
-//           same sequence of rescales: no second score product, half the gather bytes.
+//           same sequence of rescales: no second score product, half the gather bytes. Each softmax thread stages
+//           its own row of P four tiles ahead (cp.async into the shared memory that held Q): the scratch area does
+//           not stay in the L2 and a round trip to HBM is longer than two tiles of work.
 // Tensor memory (512 columns): O half [0,256) | S double-buffered [256,320), [320,384); P overwrites the first
-//   32 columns of its S buffer as bf16 pairs and is the A operand of the PV MMAs | Q blocks 0..3 (of 9 blocks of
-//   64 columns) as bf16 pairs [384,512), the A operand of their score MMAs; Q blocks 4..8 stay in shared memory.
+//   32 columns of its S buffer as bf16 pairs and is the A operand of the PV MMAs (pass 2: a ring of four P buffers
+//   in the same 128 columns) | Q blocks 0..3 (of 9 blocks of 64 columns) as bf16 pairs [384,512), the A operand of
+//   their score MMAs; Q blocks 4..8 stay in shared memory.
 // Shared memory: 2 stages x 9 blocks of [64 gathered rows x 128 B] (128-byte swizzle) | 5 blocks of Q
 //   [128 rows x 128 B]. A block of gathered rows is at once the K-major B operand of S (rows = keys) and the
 //   MN-major B operand of P V (64 contiguous value columns). A stage is two slots with their own barriers:
 //   "V" = blocks 0..3 (needed until the PV product) and "E" = blocks 4..8 (free again once the scores are
 //   done), so the next tile's E part is gathered while this tile is still in its softmax. Pass 2 uses the four
 //   slots as a ring of four value tiles.
-// Warps: 0 MMA issuer (tile i+1's scores are issued before tile i's PV product, so the tensor pipe works
-//   while the softmax warps turn S(i) into P(i)), 1 Q loader (TMA), 2-9 row gather (16-byte cp.async into the
-//   swizzled layout; two warps per slot, each slot its own acquire/copy/publish stream), 10-13 softmax: running reference maximum with a lazy rescale of O (only when the maximum
-//   grows by more than 2^8).
+// Warps: 0 MMA issuer (warp-uniform, one elected lane issues; order S(i+1) blocks 4..8 | P(i) V(i) | S(i+1)
+//   blocks 0..3), 1 Q loader (TMA), 2-9 row gather (16-byte cp.async into the swizzled layout; two warps per
+//   slot, each slot its own acquire/copy/publish stream), 10-13 softmax (running reference maximum with a lazy
+//   rescale of O, only when the maximum grows by more than 2^8).
+// The hot loops are rolled on purpose: with everything unrolled the kernel was 150 KB of code and every role
+// stalled on instruction fetch.
 // Entries < 0 or pointing outside the cache are skipped; a query's tiles end at its last usable entry
 // (counted by a small kernel first).
 #include <cuda_bf16.h>
-
-#include <type_traits>
 
 #include "kernels.h"
 #include "ptx_sm100.cuh"
