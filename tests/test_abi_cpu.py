@@ -80,6 +80,29 @@ def test_argument_validation_happens_before_any_device_work(idxc):
     assert L.idxc_topk_rows(one, 10, 2, 1, 1, None, 4, one, None) == idxc.ERR_INVALID_ARG
 
 
+def test_sparse_attention_validation_and_workspace(idxc):
+    L = idxc.lib()
+    one = ctypes.c_void_p(16)      # never dereferenced
+    f = ctypes.c_float(1.0)
+    args = lambda **kw: [kw.get("q", one), kw.get("kv", one), kw.get("topk", one), None, kw.get("n_q", 4), kw.get("n_kv", 100),
+                         kw.get("H", 128), kw.get("d_qk", 576), kw.get("d_v", 512), kw.get("k_top", 64), f, kw.get("out", one), None,
+                         kw.get("ws", one), kw.get("ws_bytes", 1 << 30), None]
+    assert L.idxc_sparse_attention(*args(k_top=0)) == idxc.ERR_INVALID_ARG
+    assert L.idxc_sparse_attention(*args(n_q=-1)) == idxc.ERR_INVALID_ARG
+    assert L.idxc_sparse_attention(*args(d_v=640)) == idxc.ERR_INVALID_ARG          # values wider than the row
+    assert L.idxc_sparse_attention(*args(d_qk=512, d_v=512)) == idxc.ERR_UNSUPPORTED
+    assert L.idxc_sparse_attention(*args(H=256)) == idxc.ERR_UNSUPPORTED
+    assert L.idxc_sparse_attention(*args(q=None)) == idxc.ERR_INVALID_ARG
+    assert L.idxc_sparse_attention(*args(out=ctypes.c_void_p(24))) == idxc.ERR_INVALID_ARG   # misaligned
+    assert L.idxc_sparse_attention(*args(ws_bytes=64)) == idxc.ERR_WORKSPACE
+    assert L.idxc_sparse_attention(*args(n_q=0)) == idxc.OK                          # nothing to do, nothing touched
+    # workspace: per-query counts plus the saved probabilities of the resident CTAs (16.5 KB per 64 selected rows)
+    assert L.idxc_sparse_attention_workspace_bytes(0, 2048) == 0
+    few, many = L.idxc_sparse_attention_workspace_bytes(4, 2048), L.idxc_sparse_attention_workspace_bytes(102400, 2048)
+    assert few == 256 + 4 * 32 * (16384 + 512)
+    assert many == 102400 * 4 + 160 * 32 * (16384 + 512)                            # capped at the largest grid
+
+
 def test_workspace_queries(idxc):
     assert idxc.prefill_workspace_bytes(0, 0, 16, 64, 8) == 0
     b = idxc.prefill_workspace_bytes(2048, 2048, 16, 64, 256)
