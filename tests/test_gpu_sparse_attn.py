@@ -150,3 +150,13 @@ def test_bench_size_chain_sampled_queries():
     rows = [0, 1, 147, 148, 2047, 4096, n_q - 149, n_q - 1]
     o_out, o_lse = osa.sparse_attention(codes(inp.q[rows]), codes(inp.kv), topk[rows].cpu().numpy(), D_V, scale)
     _check(out, lse, o_out, o_lse, np.asarray(rows), "bench size")
+
+
+@pytest.mark.parametrize("n_q,n_kv,h,k_top", [(1, 1, 1, 1), (3, 70, 7, 65), (2, 5000, 128, 4096), (149, 64, 33, 64)])
+def test_degenerate_shapes(n_q, n_kv, h, k_top):
+    # one head, one cache row, k_top below / just above / far above a tile, more selected slots than cache rows
+    # (entries repeat: duplicates count twice), one query more than there are SMs
+    inp = synth.attention_inputs(n_q, n_kv, h, D_QK, seed=21, device="cuda")
+    g = torch.Generator().manual_seed(n_q * 1000 + k_top)
+    topk = torch.randint(0, n_kv, (n_q, k_top), generator=g, dtype=torch.int32).cuda()
+    _run(inp, topk, 0.05, h=h, what=f"degenerate {n_q}x{n_kv}x{h}x{k_top}")
