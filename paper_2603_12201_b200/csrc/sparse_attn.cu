@@ -106,7 +106,9 @@ __global__ void sparse_attn_count_kernel(const int32_t* __restrict__ topk, const
 __global__ void __launch_bounds__(kSaThreads, 1)
 sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap kv_map, const SaParams p) {
     extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    // aligned by an offset into the array (not by an integer round trip), so that the compiler still knows that these
+    // pointers are shared memory and emits shared-space loads and stores for them
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     uint8_t* stage_smem = smem;                               // [2][9][64 x 128 B]; Q blocks 0..3 are staged here first
     uint8_t* q_smem = smem + 2 * kSaStageBytes;               // [5][128 x 128 B]: Q blocks 4..8
     uint64_t* bars = reinterpret_cast<uint64_t*>(q_smem + kSaQSmemBytes);
@@ -493,7 +495,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 ph_s_full[sbuf] ^= 1u;
                 tcgen05_fence_after_sync();
                 const uint32_t s_tmem = lane_base + kColS + sbuf * 64;
-                const uint32_t mlo = tile_mask[stage * 2], mhi = tile_mask[stage * 2 + 1];
+                uint32_t mlo, mhi;                                  // explicit shared-memory load: a generic one queues behind the global traffic
+                asm volatile("ld.volatile.shared.v2.u32 {%0, %1}, [%2];" : "=r"(mlo), "=r"(mhi) : "r"(smem_u32(const_cast<uint32_t*>(tile_mask) + stage * 2)) : "memory");
                 // Both sweeps over the 64 scores are rolled loops over 16-column chunks, read from tensor memory
                 // twice: the instruction footprint of the hot loop stays small.
                 // (the load of the next chunk is in flight while a chunk is processed: a tensor-memory load takes ~200 cycles)
