@@ -65,8 +65,11 @@ cudaError_t launch_quantize_e4m3(const void* x, int64_t n_tokens, int row_elems,
 constexpr int kSparseAttnMaxGrid = 160;
 bool sparse_attn_supported(int H, int d_qk, int d_v);
 size_t sparse_attn_scratch_bytes(int64_t n_q, int k_top);
+// With few queries (a decode step) a query's rows are split over several CTAs, whose fp32 partial results (sized for
+// 128 heads) are merged by a second kernel; 0 bytes when every query has its own CTA.
+size_t sparse_attn_partial_bytes(int64_t n_q);
 cudaError_t launch_sparse_attn(const void* kv, const int32_t* topk, const int64_t* kv_base, int64_t n_q, int64_t n_kv, int H,
-                               int k_top, float scale, void* out, float* lse, int32_t* n_eff, void* scratch,
+                               int k_top, float scale, void* out, float* lse, int32_t* n_eff, void* scratch, void* partial,
                                const CUtensorMap& q_map, const CUtensorMap& kv_map, unsigned int* status, int sm_count,
                                cudaStream_t stream);
 

@@ -69,6 +69,9 @@ struct SaParams {
     float scale_log2;           // scale * log2(e)
     __nv_bfloat16* out;         // [n_q, H, 512]
     float* lse;                 // [n_q, H] or nullptr
+    int splits;                 // CTAs that share a query's selected rows (few queries: decode); 1 = the CTA writes out itself
+    float* part_out;            // splits > 1: [n_q, splits, H, 512] fp32, each split's own normalised result
+    float* part_lse;            // splits > 1: [n_q, splits, H] natural-log sum of the split (-inf: nothing usable)
     unsigned int* status;
 };
 
@@ -160,6 +163,15 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     const uint32_t tmem_base = *tmem_base_slot;
 
     auto tiles_of = [&](int64_t t) -> int { return (__ldg(p.n_eff + t) + kSaBK - 1) / kSaBK; };
+    // work item = (query t, split s): split s of a query covers its tiles [nt * s / splits, nt * (s + 1) / splits)
+    const int64_t n_items = p.n_q * p.splits;
+    auto item_of = [&](int64_t item, int64_t& t, int& i0) -> int {
+        t = item / p.splits;
+        const int s = static_cast<int>(item - t * p.splits);
+        const int nt_all = tiles_of(t);
+        i0 = nt_all * s / p.splits;
+        return nt_all * (s + 1) / p.splits - i0;
+    };
     // first block of a slot's data inside the stage area
     auto slot_smem = [&](int slot) -> uint8_t* { return stage_smem + (slot >> 1) * kSaStageBytes + (slot & 1) * (kSaNVH * kSaKBlockBytes); };
     const int tiles_per_query = (p.k_top + kSaBK - 1) / kSaBK;
@@ -193,8 +205,10 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 umma_f16_ts_elect_acc(tmem_base + kColO, tmem_base + p_col + ks * 8, v_desc0 + (ks * 16 * 128) / 16, kIdescPV,
                                       (first_tile && ks == 0) ? 0u : 1u);
         };
-        for (int64_t t = blockIdx.x; t < p.n_q && ok; t += gridDim.x) {
-            const int nt = tiles_of(t);
+        for (int64_t item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+            int64_t t;
+            int i0;
+            const int nt = item_of(item, t, i0);
             if (nt == 0) continue;
             ok = wait_bar(bar_q_full, ph_q_full) && wait_bar(bar_q_ready, ph_q_ready);
             if (!ok) break;
@@ -289,8 +303,10 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             tma_prefetch_desc(&kv_map);
             uint32_t ph_q_empty = 0;
             bool ok = true;
-            for (int64_t t = blockIdx.x; t < p.n_q; t += gridDim.x) {
-                if (tiles_of(t) == 0) continue;
+            for (int64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+                int64_t t;
+                int i0;
+                if (item_of(item, t, i0) == 0) continue;
                 ok = mbar_wait(bar_q_empty, ph_q_empty ^ 1u, abort_flag, kWaitCycleBudget, 500);   // every MMA of the previous query is done
                 if (!ok) break;
                 ph_q_empty ^= 1u;
@@ -314,8 +330,10 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         uint32_t tile_seq = 0;                        // pass-1 tiles before the current query: tile i sits in stage (tile_seq + i) & 1
         bool ok = true;
         uint8_t* const slot_base = slot_smem(slot);
-        for (int64_t t = blockIdx.x; t < p.n_q && ok; t += gridDim.x) {
-            const int nt = tiles_of(t);
+        for (int64_t item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+            int64_t t;
+            int i0;
+            const int nt = item_of(item, t, i0);
             if (nt == 0) continue;
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_q_ready, ph_q_ready, abort_flag, kWaitCycleBudget, 200));   // the staging area is free again
             if (!ok) break;
@@ -324,7 +342,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             const int32_t* row_idx = p.topk + t * p.k_top;
             // lane l looks up row row0 + l of tile i; returns the mask of usable entries
             auto lookup = [&](int i, int& src_row) -> uint32_t {
-                const int j = i * kSaBK + row0 + lane;
+                const int j = (i0 + i) * kSaBK + row0 + lane;
                 src_row = -1;
                 if (j < p.k_top) {
                     const int64_t idx = __ldg(row_idx + j);
@@ -428,8 +446,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 tmem_st_32x32b_x32(lane_base + kColO + c * 32, o);
             }
         };
-        // normalises this thread's row of O and writes 256 output columns
-        auto write_out = [&](__nv_bfloat16* dst_row, float inv) -> bool {
+        // normalises this thread's row of O and writes 256 output columns: bf16 to the output, or fp32 to this split's
+        // partial result when several CTAs share the query (part_row != nullptr)
+        auto write_out = [&](__nv_bfloat16* dst_row, float* part_row, float inv) -> bool {
             if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar_o_full, ph_o_full, abort_flag))) return false;
             ph_o_full ^= 1u;
             tcgen05_fence_after_sync();
@@ -438,7 +457,13 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 uint32_t o[32];
                 tmem_ld_32x32b_x32(lane_base + kColO + c * 32, o);
                 tmem_ld_wait(o);
-                if (row < p.H) {
+                if (row < p.H && part_row != nullptr) {
+                    float4* dst = reinterpret_cast<float4*>(part_row + c * 32);
+#pragma unroll
+                    for (int v = 0; v < 8; ++v)
+                        dst[v] = make_float4(__uint_as_float(o[4 * v + 0]) * inv, __uint_as_float(o[4 * v + 1]) * inv,
+                                             __uint_as_float(o[4 * v + 2]) * inv, __uint_as_float(o[4 * v + 3]) * inv);
+                } else if (row < p.H) {
                     uint4* dst = reinterpret_cast<uint4*>(dst_row + c * 32);
 #pragma unroll
                     for (int v = 0; v < 4; ++v) {
@@ -456,13 +481,21 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             if (lane == 0) mbar_arrive(bar_o_free);
             return true;
         };
-        for (int64_t t = blockIdx.x; t < p.n_q && ok; t += gridDim.x) {
-            const int nt = tiles_of(t);
+        for (int64_t item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+            int64_t t;
+            int i0;
+            const int nt = item_of(item, t, i0);
             __nv_bfloat16* out_row = p.out + (t * p.H + row) * 512;
-            if (nt == 0) {                              // nothing selected: zeros
+            float* part_row = p.splits > 1 ? p.part_out + (item * p.H + row) * 512 : nullptr;
+            if (nt == 0) {                              // nothing (usable) in this item's range: zeros, weight 0 in the merge
                 if (row < p.H) {
-                    for (int c = 0; c < 512 / 8; ++c) reinterpret_cast<uint4*>(out_row)[c] = make_uint4(0u, 0u, 0u, 0u);
-                    if (p.lse) p.lse[t * p.H + row] = -INFINITY;
+                    if (part_row) {
+                        for (int c = 0; c < 512 / 4; ++c) reinterpret_cast<float4*>(part_row)[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        p.part_lse[item * p.H + row] = -INFINITY;
+                    } else {
+                        for (int c = 0; c < 512 / 8; ++c) reinterpret_cast<uint4*>(out_row)[c] = make_uint4(0u, 0u, 0u, 0u);
+                        if (p.lse) p.lse[t * p.H + row] = -INFINITY;
+                    }
                 }
                 continue;
             }
@@ -579,9 +612,13 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             }
             if (!ok) break;
             const float inv = l > 0.f ? 1.f / l : 0.f;
-            ok = write_out(out_row, inv);
+            ok = write_out(out_row, part_row, inv);
             if (!ok) break;
-            if (p.lse && row < p.H) p.lse[t * p.H + row] = l > 0.f ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
+            if (row < p.H) {
+                const float lse_val = l > 0.f ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
+                if (part_row) p.part_lse[item * p.H + row] = lse_val;
+                else if (p.lse) p.lse[t * p.H + row] = lse_val;
+            }
 
             // ---- pass 2: P and the factors come back from the scratch area, two tiles ahead, into a ring of four
             // P buffers (the 128 columns of the S buffers)
@@ -643,7 +680,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             }
             cp_async_wait_all();
             if (!ok) break;
-            ok = write_out(out_row + 256, inv);
+            ok = write_out(out_row + 256, part_row ? part_row + 256 : nullptr, inv);
         }
         if (!ok && lane == 0) sa_give_up(abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
     }
@@ -662,31 +699,78 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     }
 }
 
+// Merges the splits of a query: out = sum_s w_s out_s / sum_s w_s with w_s = exp(lse_s - max_s lse_s). One CTA per
+// (query, head), 128 threads x 4 columns.
+__global__ void sparse_attn_merge_kernel(const float* __restrict__ part_out, const float* __restrict__ part_lse, int H, int splits,
+                                         __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
+    const int64_t t = blockIdx.x / H;
+    const int h = static_cast<int>(blockIdx.x - t * H);
+    float m = -INFINITY;
+    for (int s = 0; s < splits; ++s) m = fmaxf(m, part_lse[(t * splits + s) * H + h]);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float denom = 0.f;
+    if (m > -INFINITY) {
+        for (int s = 0; s < splits; ++s) {
+            const float w = __expf(part_lse[(t * splits + s) * H + h] - m);
+            if (w == 0.f) continue;
+            const float4 v = reinterpret_cast<const float4*>(part_out + ((t * splits + s) * H + h) * 512)[threadIdx.x];
+            acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+            denom += w;
+        }
+    }
+    const float inv = denom > 0.f ? 1.f / denom : 0.f;
+    uint2 packed;
+    packed.x = pack_bf16x2(acc.x * inv, acc.y * inv);
+    packed.y = pack_bf16x2(acc.z * inv, acc.w * inv);
+    reinterpret_cast<uint2*>(out + (t * H + h) * 512)[threadIdx.x] = packed;
+    if (lse && threadIdx.x == 0) lse[t * H + h] = denom > 0.f ? m + logf(denom) : -INFINITY;
+}
+
 }  // namespace
 
 bool sparse_attn_supported(int H, int d_qk, int d_v) { return H >= 1 && H <= 128 && d_qk == 64 * kSaNB && d_v == 128 * kSaNVH; }
 
-int sparse_attn_grid(int64_t n_q, int sm_count) {
-    const int cap = sm_count < kSparseAttnMaxGrid ? sm_count : kSparseAttnMaxGrid;
-    return static_cast<int>(n_q < cap ? n_q : cap);
+// Few queries (a decode step) would leave most SMs idle: their selected rows are split over several CTAs.
+int sparse_attn_splits(int64_t n_q) {
+    if (n_q <= 0 || n_q >= 64) return 1;
+    const int64_t s = 128 / n_q;
+    return static_cast<int>(s > 8 ? 8 : s);
 }
 size_t sparse_attn_scratch_bytes(int64_t n_q, int k_top) {
-    const int64_t ctas = n_q < kSparseAttnMaxGrid ? n_q : kSparseAttnMaxGrid;
+    const int64_t items = n_q * sparse_attn_splits(n_q);
+    const int64_t ctas = items < kSparseAttnMaxGrid ? items : kSparseAttnMaxGrid;
     return static_cast<size_t>(ctas) * ((k_top + kSaBK - 1) / kSaBK) * kSaScratchTileBytes;
+}
+size_t sparse_attn_partial_bytes(int64_t n_q) {        // sized for 128 heads
+    const int splits = sparse_attn_splits(n_q);
+    return splits > 1 ? static_cast<size_t>(n_q) * splits * 128 * (512 + 1) * sizeof(float) : 0;
 }
 
 cudaError_t launch_sparse_attn(const void* kv, const int32_t* topk, const int64_t* kv_base, int64_t n_q, int64_t n_kv, int H,
-                               int k_top, float scale, void* out, float* lse, int32_t* n_eff, void* scratch,
-                               const CUtensorMap& q_map, const CUtensorMap& kv_map, unsigned int* status, int sm_count, cudaStream_t stream) {
+                               int k_top, float scale, void* out, float* lse, int32_t* n_eff, void* scratch, void* partial,
+                               const CUtensorMap& q_map, const CUtensorMap& kv_map, unsigned int* status, int sm_count,
+                               cudaStream_t stream) {
     if (n_q <= 0) return cudaSuccess;
     const int64_t count_blocks = (n_q * 32 + 255) / 256;
     sparse_attn_count_kernel<<<static_cast<unsigned>(count_blocks), 256, 0, stream>>>(topk, kv_base, n_q, n_kv, k_top, n_eff);
     if (cudaError_t e = cudaGetLastError(); e != cudaSuccess) return e;
     if (cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(sparse_attn_kernel), kSaSmemBytes); e != cudaSuccess) return e;
+    const int splits = sparse_attn_splits(n_q);
+    float* part_out = static_cast<float*>(partial);
+    float* part_lse = part_out ? part_out + static_cast<size_t>(n_q) * splits * 128 * 512 : nullptr;
     SaParams p{static_cast<const uint8_t*>(kv), topk, kv_base, n_eff, static_cast<uint8_t*>(scratch), n_q, n_kv, H, k_top,
-               scale * 1.4426950408889634f, static_cast<__nv_bfloat16*>(out), lse, status};
-    sparse_attn_kernel<<<sparse_attn_grid(n_q, sm_count), kSaThreads, kSaSmemBytes, stream>>>(q_map, kv_map, p);
-    return cudaGetLastError();
+               scale * 1.4426950408889634f, static_cast<__nv_bfloat16*>(out), lse, splits, part_out, part_lse, status};
+    const int64_t items = n_q * splits;
+    const int cap = sm_count < kSparseAttnMaxGrid ? sm_count : kSparseAttnMaxGrid;
+    const int grid = static_cast<int>(items < cap ? items : cap);
+    sparse_attn_kernel<<<grid, kSaThreads, kSaSmemBytes, stream>>>(q_map, kv_map, p);
+    if (cudaError_t e = cudaGetLastError(); e != cudaSuccess) return e;
+    if (splits > 1) {
+        sparse_attn_merge_kernel<<<static_cast<unsigned>(n_q * H), 128, 0, stream>>>(part_out, part_lse, H, splits,
+                                                                                      static_cast<__nv_bfloat16*>(out), lse);
+        return cudaGetLastError();
+    }
+    return cudaSuccess;
 }
 
 }  // namespace idxc
