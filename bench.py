@@ -198,7 +198,26 @@ def time_decode(idxc, synth, dev, peaks, steps, warmup):
     bytes_k = keys * c["d"] * 2
     us_score, us_total = statistics.median(t_score), statistics.median(t_total)
     gbs = bytes_k / (us_score * 1e-6) / 1e9
+    # the consumer of the step's indices: sparse attention of the B new tokens over their selected cache rows
+    # (128 heads, 576/512-column latent rows in a cache with the same row offsets; few queries: rows split over CTAs)
+    att = synth.attention_inputs(B, x.k_cache.shape[0], 128, 576, seed=c["seed"], device=dev)
+    a_out = torch.empty((B, 128, 512), dtype=torch.bfloat16, device=dev)
+    a_ws = idxc.alloc_workspace(idxc.lib().idxc_sparse_attention_workspace_bytes(B, k_top), dev)
+    for _ in range(3):
+        idxc.sparse_attention(att.q, att.kv, topk, 512, 1.0 / 24.0, kv_base=x.k_offsets, out=a_out, workspace=a_ws, want_lse=False)
+    ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ea.record()
+    for _ in range(10):
+        idxc.sparse_attention(att.q, att.kv, topk, 512, 1.0 / 24.0, kv_base=x.k_offsets, out=a_out, workspace=a_ws, want_lse=False)
+    eb.record()
+    torch.cuda.synchronize()
+    idxc.poll_device_status()
+    us_attn = ea.elapsed_time(eb) * 1e3 / 10
+    attn_tf = 2.0 * 128 * (576 + 512) * B * k_top / (us_attn * 1e-6) / 1e12
     return {
+        "sparse_attention_after": {"us": us_attn, "tflops_useful": attn_tf, "frac_of_bf16_peak": attn_tf / peaks["bf16_tflops"],
+                                   "gathered_bytes": B * k_top * (576 + 256) * 2,
+                                   "note": "B queries x k_top selected rows; with 32 queries four CTAs share a query and a second kernel merges their results"},
         "workload": f"cfg3: decode B={B} H_I={c['H']} d_I={c['d']} k_top={k_top}, sum(lens)={keys}",
         "us_per_step": us_total, "us_scorer": us_score, "us_topk": us_total - us_score,
         "k_cache_bytes": bytes_k,
