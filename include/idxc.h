@@ -280,7 +280,8 @@ idxc_status idxc_distill_kl(const float* scores, int64_t ld, int64_t rows, int64
  *   out      DEVICE bf16 [n_q, H, d_v], 16-byte aligned        lse  NULL or DEVICE fp32 [n_q, H]
  *   workspace DEVICE, idxc_sparse_attention_workspace_bytes(n_q, k_top) bytes, 16-byte aligned; caller-owned.
  *            It holds per-query entry counts and, per resident CTA, a query's probabilities between its two
- *            passes over the selected rows (about 0.5 MB per CTA at k_top = 2048)
+ *            passes over the selected rows (about 0.5 MB per CTA at k_top = 2048) and, with fewer than 64
+ *            queries, the fp32 partial results of the thread blocks that share a query
  * Supported shape: 1 <= H <= 128, d_qk = 576, d_v = 512 (tcgen05 path); anything else IDXC_ERR_UNSUPPORTED.
  * Arithmetic: bf16 products with fp32 accumulation, fp32 softmax with the probabilities rounded to bf16 for
  * the second product, bf16 output. Unselected rows are never read, except that row 0 of kv stands in for
