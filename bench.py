@@ -267,6 +267,43 @@ def time_schedule(idxc, synth, dev, L, H, d, k_top, n_layers, every, seed, reps)
             "gpairs_per_s_full_layers": pairs * calls_full / (t_full * 1e-3) / 1e9}
 
 
+def time_layer_loop(idxc, synth, dev, L, k_top, n_layers, every, seed):
+    """Fig. 2(b) with its attention step: per layer, a Full layer runs indexer + top-k, a Shared layer reuses the cached
+    indices, and every layer runs the sparse attention over them (128 heads, 576/512-column latent rows; the same
+    synthetic q and kv serve all layers). Compares the 1-in-`every` pattern with all-Full."""
+    H_i, d_i = 64, 128
+    pin = synth.prefill_inputs(L, H_i, d_i, seed=seed, device=dev, clustered=True)
+    att = synth.attention_inputs(L, L, 128, 576, seed=seed, device=dev)
+    topk = torch.empty((L, k_top), dtype=torch.int32, device=dev)
+    out = torch.empty((L, 128, 512), dtype=torch.bfloat16, device=dev)
+    ws_i = idxc.alloc_workspace(idxc.prefill_workspace_bytes(L, L, H_i, d_i, k_top), dev)
+    ws_a = idxc.alloc_workspace(idxc.lib().idxc_sparse_attention_workspace_bytes(L, k_top), dev)
+    scale = 1.0 / math.sqrt(576)
+
+    def run(pattern):
+        sch = idxc.Schedule(pattern)
+        sch.begin_pass()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for layer, c in enumerate(pattern):
+            if c == "F":
+                t = sch.prefill_layer(layer, pin.q, pin.k, pin.w, k_top, topk_buf=topk, workspace=ws_i)
+            else:
+                t = sch.prefill_layer(layer, k_top=k_top, q_len=L)
+            idxc.sparse_attention(att.q, att.kv, t, 512, scale, out=out, workspace=ws_a, want_lse=False)
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b)
+
+    sched, full = synth.uniform_pattern(n_layers, every), "F" * n_layers
+    run(sched)
+    t_sched, t_full = run(sched), run(full)
+    idxc.poll_device_status()
+    return {"workload": f"{n_layers} layers, L={L}, k_top={k_top}: indexer (F layers only) + sparse attention (every layer)",
+            "ms_scheduled": t_sched, "ms_all_full": t_full, "ratio": t_full / t_sched,
+            "note": "the paper's end-to-end figures (1.82x prefill at 200K) include an FP8 indexer and the rest of the model; context only"}
+
+
 def time_fp8_chunked(idxc, synth, dev, peaks, L, chunk, H, d, k_top, seed, decode_B):
     """Config-5 shape: one Full layer of FP8 (e4m3 + per-token scales) chunked prefill, query chunks of
     `chunk` rows against the full causal K, then one decode step at batch `decode_B` on caches of length L."""
@@ -469,6 +506,7 @@ def main():
     ap.add_argument("--L", type=int, default=0, help="override the workload's sequence length (small profiling cases)")
     ap.add_argument("--only-decode", action="store_true", help="run only the decode section (profiling)")
     ap.add_argument("--only-sparse-attention", action="store_true", help="run only the sparse-attention section (profiling)")
+    ap.add_argument("--only-layer-loop", action="store_true", help="run only the indexer + attention layer loop section")
     ap.add_argument("--sa-queries", type=int, default=8192, help="queries of the sparse-attention section")
     args = ap.parse_args()
     if args.warmup < 3:
@@ -501,6 +539,9 @@ def main():
     if args.only_decode:
         print(json.dumps({"decode": time_decode(idxc, synth, dev, peaks, steps=max(args.steps, 1), warmup=args.warmup)}),
               flush=True)
+        return
+    if args.only_layer_loop:
+        print(json.dumps({"layer_loop": time_layer_loop(idxc, synth, dev, args.L or 32768, 2048, 4, 4, seed=8)}), flush=True)
         return
     if args.only_sparse_attention:
         print(json.dumps({"sparse_attention": time_sparse_attention(idxc, synth, dev, peaks, args.L or 32768, args.sa_queries, 2048,
@@ -676,6 +717,8 @@ def main():
                                              seed=c4["seed"], reps=1 if args.full else 2)
             torch.cuda.empty_cache()
             line["sparse_attention"] = time_sparse_attention(idxc, synth, dev, peaks, 32768, args.sa_queries, c4["k_top"], seed=7)
+            torch.cuda.empty_cache()
+            line["layer_loop"] = time_layer_loop(idxc, synth, dev, 32768, c4["k_top"], 4, c4["every"], seed=8)
             torch.cuda.empty_cache()
             line["distill_kl"] = time_distill(idxc, dev, peaks, 16384, 2)
             torch.cuda.empty_cache()
