@@ -284,10 +284,9 @@ idxc_status idxc_distill_kl(const float* scores, int64_t ld, int64_t rows, int64
  *            queries, the fp32 partial results of the thread blocks that share a query
  * Supported shape: 1 <= H <= 128, d_qk = 576, d_v = 512 (tcgen05 path); anything else IDXC_ERR_UNSUPPORTED.
  * Arithmetic: bf16 products with fp32 accumulation, fp32 softmax with the probabilities rounded to bf16 for
- * the second product, bf16 output. Unselected rows are never read, except that row 0 of kv stands in for
- * skipped entries with weight 0 and must therefore hold finite numbers. Enqueues 2 kernels (3 with fewer than 64
- * queries, whose rows are split over several thread blocks and merged by the third); nothing is
- * allocated. Errors: IDXC_ERR_INVALID_ARG (null or misaligned pointer, sizes out of range),
+ * the second product, bf16 output. Rows that are not selected are never read (they may hold anything).
+ * Enqueues 2 kernels (3 with fewer than 64 queries, whose rows are split over several thread blocks and merged
+ * by the third); nothing is allocated. Errors: IDXC_ERR_INVALID_ARG (null or misaligned pointer, sizes out of range),
  * IDXC_ERR_WORKSPACE, IDXC_ERR_UNSUPPORTED, IDXC_ERR_CUDA.
  * ------------------------------------------------------------------------- */
 size_t idxc_sparse_attention_workspace_bytes(int64_t n_q, int k_top);

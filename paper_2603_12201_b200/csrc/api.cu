@@ -413,7 +413,7 @@ idxc_status idxc_quantize_e4m3(const void* x, int64_t n_tokens, int row_elems, v
 
 size_t idxc_sparse_attention_workspace_bytes(int64_t n_q, int k_top) {
     if (n_q <= 0 || k_top < 1) return 0;
-    return static_cast<size_t>(round_up(n_q * 4, 256)) + static_cast<size_t>(round_up(sparse_attn_scratch_bytes(n_q, k_top), 256)) +
+    return static_cast<size_t>(round_up(n_q * 8, 256)) + static_cast<size_t>(round_up(sparse_attn_scratch_bytes(n_q, k_top), 256)) +
            sparse_attn_partial_bytes(n_q);
 }
 
@@ -438,7 +438,7 @@ idxc_status idxc_sparse_attention(const void* q, const void* kv, const int32_t* 
     // an empty cache has no usable entry and is never read: any valid address serves as the base then
     if (!encode_operand_map(&kv_map, n_kv > 0 ? kv : q, n_kv > 0 ? n_kv : 1, d_qk, false, 1)) return IDXC_ERR_CUDA;
     g_launches += 2;
-    uint8_t* scratch = static_cast<uint8_t*>(workspace) + round_up(n_q * 4, 256);
+    uint8_t* scratch = static_cast<uint8_t*>(workspace) + round_up(n_q * 8, 256);
     void* partial = sparse_attn_partial_bytes(n_q) ? scratch + round_up(sparse_attn_scratch_bytes(n_q, k_top), 256) : nullptr;
     g_launches += partial ? 1 : 0;
     return launch_sparse_attn(kv, topk, kv_base, n_q, n_kv, H, k_top, scale, out, lse, static_cast<int32_t*>(workspace), scratch,

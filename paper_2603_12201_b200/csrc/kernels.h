@@ -60,7 +60,7 @@ cudaError_t launch_quantize_e4m3(const void* x, int64_t n_tokens, int row_elems,
                                  const int64_t* dst_rows, cudaStream_t stream);
 
 // sparse_attn.cu: attention over the selected rows. q_map: q as [n_q * H, 576] bf16, 128-byte swizzle, box
-// 64 columns x H rows; kv_map: kv as [n_kv, 576] bf16, 128-byte swizzle, box 64 columns x 1 row (gather form). n_eff: [n_q] int32 scratch; scratch: sparse_attn_scratch_bytes(n_q, k_top) bytes, 16-byte
+// 64 columns x H rows; kv_map: kv as [n_kv, 576] bf16, 128-byte swizzle, box 64 columns x 1 row (gather form). n_eff: [n_q][2] int32 scratch; scratch: sparse_attn_scratch_bytes(n_q, k_top) bytes, 16-byte
 // aligned (the probabilities of a query between its two passes, per CTA). At most kSparseAttnMaxGrid CTAs run.
 constexpr int kSparseAttnMaxGrid = 160;
 bool sparse_attn_supported(int H, int d_qk, int d_v);

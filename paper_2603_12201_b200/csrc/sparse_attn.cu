@@ -62,7 +62,7 @@ struct SaParams {
     const uint8_t* kv;          // [n_kv, 576] bf16
     const int32_t* topk;        // [n_q, k_top]
     const int64_t* kv_base;     // [n_q] or nullptr
-    const int32_t* n_eff;       // [n_q] entries to visit per query
+    const int32_t* n_eff;       // [n_q][2] entries to visit per query, cache row of its first usable entry
     uint8_t* scratch;           // [grid][tiles per query][kSaScratchTileBytes]
     int64_t n_q, n_kv;
     int H, k_top;
@@ -89,7 +89,9 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<const uint32_t*>(&v);
 }
 
-// n_eff[t] = 1 + position of the last entry of row t that is >= 0 and inside the cache (0 if none).
+// n_eff[2t] = 1 + position of the last entry of row t that is >= 0 and inside the cache (0 if none);
+// n_eff[2t+1] = the cache row of its first usable entry (stands in for skipped entries, with weight 0: rows that
+// are not selected are never read).
 __global__ void sparse_attn_count_kernel(const int32_t* __restrict__ topk, const int64_t* __restrict__ kv_base, int64_t n_q,
                                          int64_t n_kv, int k_top, int32_t* __restrict__ n_eff) {
     const int64_t t = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
@@ -97,13 +99,24 @@ __global__ void sparse_attn_count_kernel(const int32_t* __restrict__ topk, const
     if (t >= n_q) return;
     const int64_t base = kv_base ? kv_base[t] : 0;
     int last = 0;
+    unsigned long long first = ~0ull;          // (position << 32) | cache row of the first usable entry
     for (int j = lane; j < k_top; j += 32) {
         const int64_t idx = topk[t * k_top + j];
-        if (idx >= 0 && base + idx >= 0 && base + idx < n_kv) last = j + 1;
+        if (idx >= 0 && base + idx >= 0 && base + idx < n_kv) {
+            last = j + 1;
+            if (first == ~0ull) first = (static_cast<unsigned long long>(j) << 32) | static_cast<unsigned long long>(base + idx);
+        }
     }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) last = max(last, __shfl_xor_sync(0xFFFFFFFFu, last, o));
-    if (lane == 0) n_eff[t] = last;
+    for (int o = 16; o > 0; o >>= 1) {
+        last = max(last, __shfl_xor_sync(0xFFFFFFFFu, last, o));
+        const unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, first, o);
+        first = other < first ? other : first;
+    }
+    if (lane == 0) {
+        n_eff[2 * t] = last;
+        n_eff[2 * t + 1] = last ? static_cast<int32_t>(first & 0xFFFFFFFFull) : 0;
+    }
 }
 
 __global__ void __launch_bounds__(kSaThreads, 1)
@@ -162,7 +175,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     tcgen05_fence_after_sync();
     const uint32_t tmem_base = *tmem_base_slot;
 
-    auto tiles_of = [&](int64_t t) -> int { return (__ldg(p.n_eff + t) + kSaBK - 1) / kSaBK; };
+    auto tiles_of = [&](int64_t t) -> int { return (__ldg(p.n_eff + 2 * t) + kSaBK - 1) / kSaBK; };
     // work item = (query t, split s): split s of a query covers its tiles [nt * s / splits, nt * (s + 1) / splits)
     const int64_t n_items = p.n_q * p.splits;
     auto item_of = [&](int64_t item, int64_t& t, int& i0) -> int {
@@ -340,6 +353,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             ph_q_ready ^= 1u;
             const int64_t base = p.kv_base ? __ldg(p.kv_base + t) : 0;
             const int32_t* row_idx = p.topk + t * p.k_top;
+            const int stand_in = __ldg(p.n_eff + 2 * t + 1);     // a selected row: skipped entries load it and get weight 0
             // lane l looks up row row0 + l of tile i; returns the mask of usable entries
             auto lookup = [&](int i, int& src_row) -> uint32_t {
                 const int j = (i0 + i) * kSaBK + row0 + lane;
@@ -349,7 +363,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     if (idx >= 0 && base + idx >= 0 && base + idx < p.n_kv) src_row = static_cast<int>(base + idx);
                 }
                 const uint32_t valid = __ballot_sync(0xFFFFFFFFu, src_row >= 0);
-                if (src_row < 0) src_row = 0;                 // skipped entries load row 0 and get weight 0
+                if (src_row < 0) src_row = stand_in;
                 return valid;
             };
             // Copies column blocks [cb0, cb0 + n_blocks) of this warp's 32 rows into the slot's blocks 0..n_blocks-1 with

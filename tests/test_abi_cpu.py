@@ -100,8 +100,8 @@ def test_sparse_attention_validation_and_workspace(idxc):
     assert L.idxc_sparse_attention_workspace_bytes(0, 2048) == 0
     few, many = L.idxc_sparse_attention_workspace_bytes(4, 2048), L.idxc_sparse_attention_workspace_bytes(102400, 2048)
     # 4 queries are split over 8 CTAs each: 32 resident CTAs' scratch plus their fp32 partial results (sized for 128 heads)
-    assert few == 256 + 32 * 32 * (16384 + 512) + 4 * 8 * 128 * (512 + 1) * 4
-    assert many == 102400 * 4 + 160 * 32 * (16384 + 512)                            # capped at the largest grid
+    assert few == 256 + 32 * 32 * (16384 + 512) + 4 * 8 * 128 * (512 + 1) * 4    # 4 queries x 8 bytes round up to 256
+    assert many == 102400 * 8 + 160 * 32 * (16384 + 512)                            # capped at the largest grid
 
 
 def test_workspace_queries(idxc):

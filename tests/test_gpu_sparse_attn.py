@@ -92,6 +92,27 @@ def test_skipped_entries_anywhere_out_of_range_and_empty_rows():
     assert torch.equal(out[5], inp.kv[only, :D_V].expand(H, D_V))
 
 
+def test_rows_outside_the_selection_are_never_read():
+    # every cache row that no query selects is filled with NaN: the result must not change (skipped entries stand in
+    # with a selected row, never with an arbitrary one)
+    n_q, n_kv, k_top = 70, 2000, 200
+    inp = synth.attention_inputs(n_q, n_kv, H, D_QK, seed=16, device="cuda")
+    g = torch.Generator().manual_seed(3)
+    topk = torch.randint(1, n_kv, (n_q, k_top), generator=g, dtype=torch.int32).cuda()      # row 0 is never selected
+    topk[:, ::7] = -1
+    topk[5, :] = -1
+    used = torch.zeros(n_kv, dtype=torch.bool, device="cuda")
+    used[topk[topk >= 0].long()] = True
+    ref, ref_lse = binding.sparse_attention(inp.q, inp.kv, topk, D_V, 0.07)
+    poisoned = inp.kv.clone()
+    poisoned[~used] = float("nan")
+    out, lse = binding.sparse_attention(inp.q, poisoned, topk, D_V, 0.07)
+    binding.poll_device_status()
+    assert not bool(used[0]) and bool(torch.isnan(poisoned[0]).all())
+    assert torch.equal(out, ref) and torch.equal(lse, ref_lse)
+    assert bool(torch.isfinite(out.float()).all())
+
+
 def test_fewer_heads_and_decode_style_base_offsets():
     h, B = 16, 5
     lens = [700, 64, 2100, 1, 300]
