@@ -1,4 +1,4 @@
-// Thin inline-PTX wrappers for sm_100a: mbarrier, TMA tiled loads (no multicast),
+// Thin inline-PTX wrappers for sm_100a: mbarrier, TMA tiled loads (each CTA loads for itself),
 // tcgen05 (TMEM allocation, UMMA issue/commit, TMEM loads) and descriptor builders.
 // Every wait is bounded: it gives up after a cycle budget and reports failure so the
 // caller can record a status code and leave instead of spinning on a shared GPU.

@@ -10,7 +10,7 @@
 // Prefill kernel (persistent, one CTA per SM, warp-specialised):
 //   warp 0      TMA producer: a block of 2*256/H queries (two 256-column B tiles) is loaded
 //               once per work item and stays in shared memory; 128-key A tiles stream
-//               through a ring of stages. Per-CTA loads only (no multicast).
+//               through a ring of stages. Per-CTA loads only.
 //   warp 1      MMA issuer: per key tile, one 128 x 256 x d UMMA chain into each of the two
 //               256-column TMEM accumulators, so accumulator A is drained while B is filled.
 //   warps 2-9   epilogue: tcgen05.ld (16x256b), ReLU, FMA with w held in registers, two shuffles per
