@@ -55,3 +55,22 @@ def test_single_rank_needs_no_process_group():
     assert pdist.max_over_ranks(3.5, 1) == 3.5
     pdist.barrier(1)
     assert pdist.whole_job_rate(10.0, 2, 4.0, 1) == pytest.approx(5000.0)
+
+
+def test_attention_input_generators_on_cpu():
+    # the seeded generators of the attention step: shapes, dtype, determinism; selections are causal, distinct,
+    # ascending and padded with -1
+    import torch
+    from paper_2603_12201_b200 import synth
+    a = synth.attention_inputs(3, 50, 4, 64, seed=5)
+    b = synth.attention_inputs(3, 50, 4, 64, seed=5)
+    assert a.q.shape == (3, 4, 64) and a.kv.shape == (50, 64) and a.q.dtype == torch.bfloat16
+    assert torch.equal(a.q, b.q) and torch.equal(a.kv, b.kv)
+    pos = [0, 3, 10, 49]
+    sel = synth.random_selection(pos, 8, seed=5)
+    assert sel.shape == (4, 8) and sel.dtype == torch.int32
+    for t, row in zip(pos, sel.tolist()):
+        valid = [x for x in row if x >= 0]
+        assert len(valid) == min(8, t + 1) and row[len(valid):] == [-1] * (8 - len(valid))
+        assert valid == sorted(set(valid)) and all(0 <= x <= t for x in valid)
+    assert torch.equal(sel, synth.random_selection(pos, 8, seed=5))
