@@ -306,6 +306,19 @@ __device__ __forceinline__ uint64_t umma_smem_desc_sw128_mn(uint32_t smem_addr, 
 }
 constexpr uint32_t kUmmaBMajorMN = 1u << 16;
 
+// K-major operand without swizzle: 8-row x 16-byte core matrices of 128 contiguous bytes; `k_step_bytes`
+// separates the two core matrices of a row group along K (the leading byte offset), `row_group_bytes`
+// consecutive 8-row groups along M or N (the stride byte offset). With k_step_bytes = rows * 16 and
+// row_group_bytes = 128 the tile is stored as [16-byte chunk along K][row][16 bytes].
+__device__ __forceinline__ uint64_t umma_smem_desc_noswizzle(uint32_t smem_addr, uint32_t k_step_bytes, uint32_t row_group_bytes) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
+    d |= static_cast<uint64_t>(k_step_bytes >> 4) << 16;
+    d |= static_cast<uint64_t>(row_group_bytes >> 4) << 32;
+    d |= static_cast<uint64_t>(1) << 46;
+    return d;
+}
+
 // ---------------------------------------------------------------- cp.async (16-byte gathers) and proxy fence
 __device__ __forceinline__ void cp_async_16(uint32_t dst_smem, const void* src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
@@ -327,6 +340,17 @@ __device__ __forceinline__ void cp_async_wait_all() {
 // Makes this thread's completed generic-proxy writes to shared memory visible to the async proxy (UMMA, TMA).
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// Orders this thread's earlier generic-proxy writes to global memory before later async-proxy reads of them
+// (a bulk copy issued after a synchronisation with this thread).
+__device__ __forceinline__ void fence_proxy_async_global() {
+    asm volatile("fence.proxy.async.global;" ::: "memory");
+}
+// Bulk copy global -> shared (both 16-byte aligned, size a multiple of 16), completion counted in bytes on `bar`.
+__device__ __forceinline__ void bulk_load_1d(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
 // Instruction descriptor: fp32 accumulate, A and B K-major, dense.

@@ -9,14 +9,14 @@
 // 256-column half of d_v:
 //   pass 1  gathers whole rows (576 columns), S = Q K^T, softmax, O[:, 0:256] += P V; the bf16 probabilities P
 //           and the rescale factors of the running maximum also go to a per-CTA scratch area in global memory
-//   pass 2  gathers only columns 256..511 of the same rows, reads P back and does O[:, 256:512] += P V with the
-//           same sequence of rescales: no second score product, half the gather bytes. Each softmax thread stages
-//           its own row of P four tiles ahead (cp.async into the shared memory that held Q): the scratch area does
-//           not stay in the L2 and a round trip to HBM is longer than two tiles of work.
-// Tensor memory (512 columns): O half [0,256) | S double-buffered [256,320), [320,384); P overwrites the first
-//   32 columns of its S buffer as bf16 pairs and is the A operand of the PV MMAs (pass 2: a ring of four P buffers
-//   in the same 128 columns) | Q blocks 0..3 (of 9 blocks of 64 columns) as bf16 pairs [384,512), the A operand of
-//   their score MMAs; Q blocks 4..8 stay in shared memory.
+//   pass 2  gathers only columns 256..511 of the same rows and does O[:, 256:512] += P V with the saved P and the
+//           same sequence of rescales: no second score product, half the gather bytes. A saved tile of P is stored
+//           as [16-byte chunk][row][16 B], which is at once what a warp of softmax threads writes contiguously and
+//           the unswizzled K-major operand layout, so one bulk copy per tile brings it back (four tiles ahead, into
+//           the shared memory that held Q) and the PV MMAs read it there: no thread touches P in pass 2.
+// Tensor memory (512 columns): O half [0,256) | S double-buffered [256,320), [320,384); in pass 1 P overwrites the
+//   first 32 columns of its S buffer as bf16 pairs and is the A operand of the PV MMAs | Q blocks 0..3 (of 9 blocks
+//   of 64 columns) as bf16 pairs [384,512), the A operand of their score MMAs; Q blocks 4..8 stay in shared memory.
 // Shared memory: 2 stages x 9 blocks of [64 gathered rows x 128 B] (128-byte swizzle) | 5 blocks of Q
 //   [128 rows x 128 B]. A block of gathered rows is at once the K-major B operand of S (rows = keys) and the
 //   MN-major B operand of P V (64 contiguous value columns). A stage is two slots with their own barriers:
@@ -24,7 +24,7 @@
 //   done), so the next tile's E part is gathered while this tile is still in its softmax. Pass 2 uses the four
 //   slots as a ring of four value tiles.
 // Warps: 0 MMA issuer (warp-uniform, one elected lane issues; order S(i+1) blocks 4..8 | P(i) V(i) | S(i+1)
-//   blocks 0..3), 1 Q loader (TMA), 2-9 row gather (16-byte cp.async into the swizzled layout; two warps per
+//   blocks 0..3), 1 Q loader (TMA) and, in pass 2, loader of the saved P, 2-9 row gather (16-byte cp.async into the swizzled layout; two warps per
 //   slot, each slot its own acquire/copy/publish stream), 10-13 softmax (running reference maximum with a lazy
 //   rescale of O, only when the maximum grows by more than 2^8).
 // The hot loops are rolled on purpose: with everything unrolled the kernel was 150 KB of code and every role
@@ -54,9 +54,12 @@ constexpr uint32_t kSaQSmemBytes = kSaQS * kSaQBlockBytes;            // 81920
 constexpr uint32_t kSaSmemBytes = 2 * kSaStageBytes + kSaQSmemBytes + 256 + 1024;
 static_assert(kSaQT * kSaQBlockBytes <= 2 * kSaStageBytes, "the Q staging area lives in the tile stages");
 static_assert(kSaSmemBytes <= 232448, "shared memory budget of one CTA");
+constexpr int kSaPRing = 4;               // pass 2: saved P tiles in flight
 constexpr uint32_t kColO = 0, kColS = 256, kColQ = 384;   // S buffer b at kColS + 64 b; P in its first 32 columns
 constexpr float kRescaleThreshold = 8.f;  // log2 units: P stays below 2^8
-constexpr uint32_t kSaScratchTileBytes = 128 * kSaBK * 2 + 128 * 4;   // P as [8 chunks][128 rows][16 B] + rescale factors [128] fp32
+constexpr uint32_t kSaPTileBytes = 128 * kSaBK * 2;
+constexpr uint32_t kSaScratchTileBytes = kSaPTileBytes + 128 * 4;     // P as [8 chunks][128 rows][16 B] + rescale factors [128] fp32
+static_assert(kSaPRing * kSaScratchTileBytes <= kSaQSmemBytes && kSaScratchTileBytes % 16 == 0, "the P ring lives where Q blocks 4..8 were");
 
 struct SaParams {
     const uint8_t* kv;          // [n_kv, 576] bf16
@@ -135,14 +138,16 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     const uint32_t bar_slot_full = smem_u32(bars + 3);        // [4]
     const uint32_t bar_slot_empty = smem_u32(bars + 7);       // [4]
     const uint32_t bar_s_full = smem_u32(bars + 11);          // [2] S buffers
-    const uint32_t bar_p_ready = smem_u32(bars + 13);         // [4] pass 1 uses two (P in its S buffer), pass 2 a ring of four
-    const uint32_t bar_p_free = smem_u32(bars + 17);          // [4] pass 2: the PV product has read P buffer b
+    const uint32_t bar_p_ready = smem_u32(bars + 13);         // [4] pass 1 uses two (P in its S buffer); pass 2: rescales of tile i replayed, ring of four
+    const uint32_t bar_p_free = smem_u32(bars + 17);          // [4] pass 2: the PV product has read P ring buffer b
     const uint32_t bar_o_full = smem_u32(bars + 21);
     const uint32_t bar_o_free = smem_u32(bars + 22);
     const uint32_t bar_pv_done = smem_u32(bars + 23);         // one phase per PV tile
     uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(bars + 24);
     volatile uint32_t* abort_flag = tmem_base_slot + 1;
     volatile uint32_t* tile_mask = reinterpret_cast<volatile uint32_t*>(bars + 25);   // [2 stages][2]: usable entries of the tile, rows 0..31 and 32..63
+    const uint32_t bar_p_full = smem_u32(bars + 27);          // [4] pass 2: the saved P tile has landed in ring buffer b
+    const uint32_t bar_p2_go = smem_u32(bars + 31);           // pass 1 is over: P is in the scratch area and Q's shared memory is free
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -159,7 +164,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         for (int i = 0; i < 4; ++i) {
             mbar_init(bar_p_ready + 8 * i, 4);
             mbar_init(bar_p_free + 8 * i, 1);
+            mbar_init(bar_p_full + 8 * i, 1);
         }
+        mbar_init(bar_p2_go, 4);
         mbar_init(bar_o_full, 1);
         mbar_init(bar_o_free, 4);
         mbar_init(bar_pv_done, 1);
@@ -197,7 +204,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         constexpr uint32_t kIdescS = umma_idesc(1, 1, 128, kSaBK);
         constexpr uint32_t kIdescPV = umma_idesc(1, 1, 128, 64 * kSaNVH) | kUmmaBMajorMN;
         uint32_t ph_q_full = 0, ph_q_ready = 0, ph_o_free = 0;
-        uint32_t ph_slot_full[4] = {0u, 0u, 0u, 0u}, ph_p_ready[4] = {0u, 0u, 0u, 0u};
+        uint32_t ph_slot_full[4] = {0u, 0u, 0u, 0u}, ph_p_ready[4] = {0u, 0u, 0u, 0u}, ph_p_full[4] = {0u, 0u, 0u, 0u};
         int stage_s = 0, stage_pv = 0;      // pass 1: stage of the next tile to score / to multiply by V
         bool ok = true;
         const uint64_t q_desc0 = umma_smem_desc_sw128(smem_u32(q_smem));
@@ -296,11 +303,18 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             ph_o_free ^= 1u;
             for (int i = 0; i < nt; ++i) {
                 const int slot = i & 3;
-                ok = wait_slot(slot) && wait_bar(bar_p_ready + 8 * slot, ph_p_ready[slot]);
+                ok = wait_slot(slot) && wait_bar(bar_p_full + 8 * slot, ph_p_full[slot]) && wait_bar(bar_p_ready + 8 * slot, ph_p_ready[slot]);
                 if (!ok) break;
+                ph_p_full[slot] ^= 1u;
                 ph_p_ready[slot] ^= 1u;
                 tcgen05_fence_after_sync();
-                issue_pv(smem_u32(slot_smem(slot)), kColS + slot * 32, i == 0);
+                // P from the ring: chunks of a row are 2048 bytes apart, 8-row groups 128 bytes; 16 gathered rows per MMA
+                const uint64_t p_desc0 = umma_smem_desc_noswizzle(smem_u32(q_smem) + slot * kSaScratchTileBytes, 128 * 16, 128);
+                const uint64_t v_desc0 = umma_smem_desc_sw128_mn(smem_u32(slot_smem(slot)), kSaKBlockBytes);
+#pragma unroll
+                for (int ks = 0; ks < kSaBK / 16; ++ks)
+                    umma_f16_elect_acc(tmem_base + kColO, p_desc0 + (ks * 2 * 128 * 16) / 16, v_desc0 + (ks * 16 * 128) / 16, kIdescPV,
+                                       (i == 0 && ks == 0) ? 0u : 1u);
                 umma_commit_elect(bar_slot_empty + 8 * slot);
                 umma_commit_elect(bar_p_free + 8 * slot);
                 umma_commit_elect(bar_pv_done);
@@ -314,12 +328,14 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             // ------------------------------------------------------------ Q loader
             tma_prefetch_desc(&q_map);
             tma_prefetch_desc(&kv_map);
-            uint32_t ph_q_empty = 0;
+            uint32_t ph_q_empty = 0, ph_go = 0;
+            uint32_t ph_p_free[kSaPRing] = {0u, 0u, 0u, 0u};
             bool ok = true;
-            for (int64_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+            for (int64_t item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
                 int64_t t;
                 int i0;
-                if (item_of(item, t, i0) == 0) continue;
+                const int nt = item_of(item, t, i0);
+                if (nt == 0) continue;
                 ok = mbar_wait(bar_q_empty, ph_q_empty ^ 1u, abort_flag, kWaitCycleBudget, 500);   // every MMA of the previous query is done
                 if (!ok) break;
                 ph_q_empty ^= 1u;
@@ -328,6 +344,19 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 for (int b = 0; b < kSaNB; ++b) {
                     uint8_t* dst = b < kSaQT ? stage_smem + b * kSaQBlockBytes : q_smem + (b - kSaQT) * kSaQBlockBytes;
                     tma_load_2d(smem_u32(dst), &q_map, bar_q_full, b * 64, row0);
+                }
+                // ---- pass 2: the saved P tiles (and their rescale factors) come back, kSaPRing tiles ahead
+                ok = mbar_wait(bar_p2_go, ph_go, abort_flag, kWaitCycleBudget, 500);
+                if (!ok) break;
+                ph_go ^= 1u;
+                for (int i = 0; i < nt; ++i) {
+                    const int b = i & (kSaPRing - 1);
+                    ok = mbar_wait(bar_p_free + 8 * b, ph_p_free[b] ^ 1u, abort_flag, kWaitCycleBudget, 100);   // the PV product that read this buffer is done
+                    if (!ok) break;
+                    ph_p_free[b] ^= 1u;
+                    mbar_arrive_expect_tx(bar_p_full + 8 * b, kSaScratchTileBytes);
+                    bulk_load_1d(smem_u32(q_smem) + b * kSaScratchTileBytes, scratch + static_cast<size_t>(i) * kSaScratchTileBytes,
+                                 kSaScratchTileBytes, bar_p_full + 8 * b);
                 }
             }
             if (!ok) sa_give_up(abort_flag, p.status, DEV_TIMEOUT_PRODUCER);
@@ -440,7 +469,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         const int row = quarter * 32 + lane;           // head
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
         uint32_t ph_q_full = 0, ph_o_full = 0;
-        uint32_t ph_s_full[2] = {0u, 0u}, ph_p_free[4] = {0u, 0u, 0u, 0u};
+        uint32_t ph_s_full[2] = {0u, 0u}, ph_p_free[4] = {0u, 0u, 0u, 0u}, ph_p_full[4] = {0u, 0u, 0u, 0u};
         uint32_t pv_tiles = 0;                         // PV tiles before the current one, over the whole kernel
         int stage = 0;
         bool ok = true;
@@ -584,7 +613,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 }
                 const float m_sub = m_ref == -INFINITY ? 0.f : m_ref;   // no usable score yet: every P is exp2(-inf) = 0
                 // P(i) goes over the first half of S(i) chunk by chunk (columns 8c..8c+7 hold scores this thread has
-                // already read) and, with the factor, to the scratch area for pass 2 (read back by this same thread)
+                // already read) and, with the factor, to the scratch area for pass 2
                 uint4* dst = reinterpret_cast<uint4*>(my_p + static_cast<size_t>(i) * kSaScratchTileBytes);
                 float sum = 0.f;
                 auto exp16 = [&](const uint32_t (&r)[16], uint32_t m16, int c) {
@@ -625,6 +654,13 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 stage ^= 1;
             }
             if (!ok) break;
+            // P and the factors of every tile are written: order them before the bulk copies of pass 2 (async proxy),
+            // which the loader issues once all four warps have arrived. Every score product has completed by now, so
+            // the shared memory that held Q is free for the ring.
+            __threadfence();
+            fence_proxy_async_global();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_p2_go);
             const float inv = l > 0.f ? 1.f / l : 0.f;
             ok = write_out(out_row, part_row, inv);
             if (!ok) break;
@@ -634,65 +670,32 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 else if (p.lse) p.lse[t * p.H + row] = lse_val;
             }
 
-            // ---- pass 2: P and the factors come back from the scratch area, two tiles ahead, into a ring of four
-            // P buffers (the 128 columns of the S buffers)
-            // Each thread stages its own 128-byte row of P (and its factor) four tiles ahead with cp.async, in the
-            // shared memory that held Q (unused in pass 2): the scratch area has usually left the L2 by now, and a
-            // round trip to HBM is longer than two tiles of work.
-            uint8_t* const p_ring = q_smem;                                            // [4][128 rows x 128 B], chunks swizzled by row
-            float* const a_ring = reinterpret_cast<float*>(q_smem + 4 * kSaQBlockBytes);   // [4][128]
-            auto stage_p = [&](int i) {
-                if (i < nt) {
-                    const uint8_t* src = my_p + static_cast<size_t>(i) * kSaScratchTileBytes;
-                    const uint32_t dst = smem_u32(p_ring) + (i & 3) * kSaQBlockBytes + row * 128;
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) cp_async_16(dst + ((c ^ (row & 7)) << 4), src + c * 2048);
-                    cp_async_4(smem_u32(a_ring + (i & 3) * 128 + row), my_alpha + static_cast<size_t>(i) * kSaScratchTileBytes);
-                }
-                cp_async_commit_group();                                               // one group per tile, empty past the end
-            };
-            auto fetch_p = [&](int i, uint4 (&dst)[8], float& alpha) {                 // after cp_async_wait_group: own data only
-                const uint8_t* src = p_ring + (i & 3) * kSaQBlockBytes + row * 128;
-#pragma unroll
-                for (int c = 0; c < 8; ++c) dst[c] = *reinterpret_cast<const uint4*>(src + ((c ^ (row & 7)) << 4));
-                alpha = a_ring[(i & 3) * 128 + row];
-            };
-            // hands P(i) to the MMA warp: wait for its ring buffer, replay the rescale of pass 1, store, signal
-            auto hand_over = [&](int i, const uint4 (&src)[8], float alpha) -> bool {
-                const int pbuf = i & 3;
-                if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar_p_free + 8 * pbuf, ph_p_free[pbuf] ^ 1u, abort_flag))) return false;   // PV(i-4) has read this buffer
-                ph_p_free[pbuf] ^= 1u;
-                if (i > 0 && __any_sync(0xFFFFFFFFu, alpha != 1.f)) {
-                    // The factor applies to the sum over the tiles before i: PV(i-1) must be complete. It arrives on the
-                    // p_free barrier of its buffer; the parity is the one this thread's next wait on that buffer will use
-                    // (no PV product from tile i on can have been issued, so the barrier cannot be further ahead).
-                    const int prev = (i - 1) & 3;
-                    if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar_p_free + 8 * prev, ph_p_free[prev] ^ 1u, abort_flag))) return false;
-                    scale_o(alpha);
-                }
-                uint32_t pr[32];
-#pragma unroll
-                for (int v = 0; v < 8; ++v) { pr[4 * v] = src[v].x; pr[4 * v + 1] = src[v].y; pr[4 * v + 2] = src[v].z; pr[4 * v + 3] = src[v].w; }
-                tcgen05_fence_after_sync();
-                tmem_st_32x32b_x32(lane_base + kColS + pbuf * 32, pr);
-                tmem_st_wait();
-                tcgen05_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_p_ready + 8 * pbuf);
-                ++pv_tiles;
-                return true;
-            };
-            for (int i = 0; i < 4; ++i) stage_p(i);
+            // ---- pass 2: the MMA warp reads P from the ring itself; this thread only replays the rescales of its row
+            // (the factor of tile i applies to the sum over the tiles before i)
 #pragma unroll 1
             for (int i = 0; i < nt && ok; ++i) {
-                uint4 pv[8];
+                const int b = i & (kSaPRing - 1);
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_p_full + 8 * b, ph_p_full[b], abort_flag));
+                if (!ok) break;
+                ph_p_full[b] ^= 1u;
                 float alpha;
-                cp_async_wait_group<3>();                                               // tile i's group has landed
-                fetch_p(i, pv, alpha);
-                ok = hand_over(i, pv, alpha);
-                stage_p(i + 4);                                                         // its ring slot is free again
+                asm volatile("ld.shared.f32 %0, [%1];" : "=f"(alpha) : "r"(smem_u32(q_smem) + b * kSaScratchTileBytes + kSaPTileBytes + row * 4) : "memory");
+                if (i > 0 && __any_sync(0xFFFFFFFFu, alpha != 1.f)) {
+                    // PV(i-1) must be complete: it arrives on the p_free barrier of its buffer, in the phase this thread
+                    // noted when it passed tile i-1 (the loader refilled that buffer only after the phase before it, and
+                    // no PV product from tile i on can have been issued, so the barrier is in that phase or the next)
+                    const int prev = (i - 1) & (kSaPRing - 1);
+                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_p_free + 8 * prev, ph_p_free[prev] ^ 1u, abort_flag));
+                    if (!ok) break;
+                    scale_o(alpha);
+                    tmem_st_wait();
+                    tcgen05_fence_before_sync();
+                }
+                ph_p_free[b] ^= 1u;                      // the phase PV(i) will complete
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_p_ready + 8 * b);
+                ++pv_tiles;
             }
-            cp_async_wait_all();
             if (!ok) break;
             ok = write_out(out_row + 256, part_row ? part_row + 256 : nullptr, inv);
         }
