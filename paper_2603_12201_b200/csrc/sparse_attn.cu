@@ -13,7 +13,8 @@
 //           same sequence of rescales: no second score product, half the gather bytes. A saved tile of P is stored
 //           as [16-byte chunk][row][16 B], which is at once what a warp of softmax threads writes contiguously and
 //           the unswizzled K-major operand layout, so one bulk copy per tile brings it back (four tiles ahead, into
-//           the shared memory that held Q) and the PV MMAs read it there: no thread touches P in pass 2.
+//           the shared memory that held Q) and the PV MMAs read it there: no thread touches P in pass 2. The softmax
+//           warps note in pass 1 which tiles moved a reference maximum; only those tiles wait for them in pass 2.
 // Tensor memory (512 columns): O half [0,256) | S double-buffered [256,320), [320,384); in pass 1 P overwrites the
 //   first 32 columns of its S buffer as bf16 pairs and is the A operand of the PV MMAs | Q blocks 0..3 (of 9 blocks
 //   of 64 columns) as bf16 pairs [384,512), the A operand of their score MMAs; Q blocks 4..8 stay in shared memory.
@@ -23,9 +24,9 @@
 //   "V" = blocks 0..3 (needed until the PV product) and "E" = blocks 4..8 (free again once the scores are
 //   done), so the next tile's E part is gathered while this tile is still in its softmax. Pass 2 uses the four
 //   slots as a ring of four value tiles.
-// Warps: 0 MMA issuer (warp-uniform, one elected lane issues; order S(i+1) blocks 4..8 | P(i) V(i) | S(i+1)
-//   blocks 0..3), 1 Q loader (TMA) and, in pass 2, loader of the saved P, 2-9 row gather (16-byte cp.async into the swizzled layout; two warps per
-//   slot, each slot its own acquire/copy/publish stream), 10-13 softmax (running reference maximum with a lazy
+// Warps (16; three idle): 0 MMA issuer (warp-uniform, one elected lane issues; order S(i+1) blocks 4..8 | P(i) V(i) | S(i+1)
+//   blocks 0..3), 4 Q loader (TMA) and, in pass 2, loader of the saved P, eight row-gather warps (16-byte cp.async into the swizzled layout; two warps per
+//   slot, each slot its own acquire/copy/publish stream), 12-15 softmax (running reference maximum with a lazy
 //   rescale of O, only when the maximum grows by more than 2^8).
 // The hot loops are rolled on purpose: with everything unrolled the kernel was 150 KB of code and every role
 // stalled on instruction fetch.
@@ -40,7 +41,7 @@ namespace idxc {
 namespace {
 
 constexpr int kSaGatherWarps = 8;          // warps 2 .. 9
-constexpr int kSaThreads = 32 * (2 + kSaGatherWarps + 4);
+constexpr int kSaThreads = 32 * 16;
 static_assert(kSaGatherWarps == 8, "two gather warps per slot, four slots");
 constexpr int kSaBK = 64;                 // gathered rows per tile
 constexpr int kSaNB = 9;                  // 64-column blocks of d_qk = 576
@@ -51,7 +52,9 @@ constexpr uint32_t kSaQBlockBytes = 128 * 128;
 constexpr uint32_t kSaKBlockBytes = kSaBK * 128;
 constexpr uint32_t kSaStageBytes = kSaNB * kSaKBlockBytes;            // 73728
 constexpr uint32_t kSaQSmemBytes = kSaQS * kSaQBlockBytes;            // 81920
-constexpr uint32_t kSaSmemBytes = 2 * kSaStageBytes + kSaQSmemBytes + 256 + 1024;
+constexpr uint32_t kSaBarBytes = 512;     // mbarriers and a few words of per-query state
+constexpr uint32_t kSaSmemBytes = 2 * kSaStageBytes + kSaQSmemBytes + kSaBarBytes + 1024;
+constexpr int kSaFlagTiles = 256;         // tiles of a query whose "rescaled" flag is kept; later tiles count as flagged
 static_assert(kSaQT * kSaQBlockBytes <= 2 * kSaStageBytes, "the Q staging area lives in the tile stages");
 static_assert(kSaSmemBytes <= 232448, "shared memory budget of one CTA");
 constexpr int kSaPRing = 4;               // pass 2: saved P tiles in flight
@@ -59,7 +62,7 @@ constexpr uint32_t kColO = 0, kColS = 256, kColQ = 384;   // S buffer b at kColS
 constexpr float kRescaleThreshold = 8.f;  // log2 units: P stays below 2^8
 constexpr uint32_t kSaPTileBytes = 128 * kSaBK * 2;
 constexpr uint32_t kSaScratchTileBytes = kSaPTileBytes + 128 * 4;     // P as [8 chunks][128 rows][16 B] + rescale factors [128] fp32
-static_assert(kSaPRing * kSaScratchTileBytes <= kSaQSmemBytes && kSaScratchTileBytes % 16 == 0, "the P ring lives where Q blocks 4..8 were");
+static_assert(kSaPRing * kSaPTileBytes <= kSaQSmemBytes && kSaScratchTileBytes % 16 == 0, "the P ring lives where Q blocks 4..8 were");
 
 struct SaParams {
     const uint8_t* kv;          // [n_kv, 576] bf16
@@ -148,9 +151,19 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
     volatile uint32_t* tile_mask = reinterpret_cast<volatile uint32_t*>(bars + 25);   // [2 stages][2]: usable entries of the tile, rows 0..31 and 32..63
     const uint32_t bar_p_full = smem_u32(bars + 27);          // [4] pass 2: the saved P tile has landed in ring buffer b
     const uint32_t bar_p2_go = smem_u32(bars + 31);           // pass 1 is over: P is in the scratch area and Q's shared memory is free
+    // bit i: some row's reference maximum moved at tile i of the current query (O must be rescaled before PV(i))
+    volatile uint32_t* resc_mask = reinterpret_cast<volatile uint32_t*>(bars + 32);   // [kSaFlagTiles / 32]
+    const uint32_t bar_resc_go = smem_u32(bars + 36);         // pass 2: every PV product before a flagged tile is complete
+    static_assert(37 * 8 <= kSaBarBytes && kSaFlagTiles / 8 <= 32, "barrier area");
+    auto tile_rescales = [&](int i) -> bool { return i > 0 && (i >= kSaFlagTiles || ((resc_mask[i >> 5] >> (i & 31)) & 1u)); };
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    // Roles by warp. A warp's scheduler is warp % 4: the MMA warp shares its scheduler with the loader (mostly asleep),
+    // an idle warp and one softmax warp only, so that its issue slots are not taken by polling or copying warps.
+    //   0 MMA | 4 loader | 8, 11 idle | 1 2 3 5 6 7 9 10 gather | 12..15 softmax (TMEM lane quarter = warp % 4)
+    const int gather_index = warp < 4 ? warp - 1 : (warp < 8 ? warp - 2 : warp - 3);   // for warps 1 2 3 5 6 7 9 10
+    const bool is_gather = warp != 0 && warp != 4 && warp != 8 && warp < 11;
 
     if (threadIdx.x == 0) {
         mbar_init(bar_q_full, 1);
@@ -167,6 +180,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             mbar_init(bar_p_full + 8 * i, 1);
         }
         mbar_init(bar_p2_go, 4);
+        mbar_init(bar_resc_go, 1);
         mbar_init(bar_o_full, 1);
         mbar_init(bar_o_free, 4);
         mbar_init(bar_pv_done, 1);
@@ -303,13 +317,17 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             ph_o_free ^= 1u;
             for (int i = 0; i < nt; ++i) {
                 const int slot = i & 3;
-                ok = wait_slot(slot) && wait_bar(bar_p_full + 8 * slot, ph_p_full[slot]) && wait_bar(bar_p_ready + 8 * slot, ph_p_ready[slot]);
+                ok = wait_slot(slot) && wait_bar(bar_p_full + 8 * slot, ph_p_full[slot]);
                 if (!ok) break;
                 ph_p_full[slot] ^= 1u;
-                ph_p_ready[slot] ^= 1u;
+                if (tile_rescales(i)) {                          // the softmax warps rescale O first (rare after the first tiles)
+                    ok = wait_bar(bar_p_ready + 8 * slot, ph_p_ready[slot]);
+                    if (!ok) break;
+                    ph_p_ready[slot] ^= 1u;
+                }
                 tcgen05_fence_after_sync();
                 // P from the ring: chunks of a row are 2048 bytes apart, 8-row groups 128 bytes; 16 gathered rows per MMA
-                const uint64_t p_desc0 = umma_smem_desc_noswizzle(smem_u32(q_smem) + slot * kSaScratchTileBytes, 128 * 16, 128);
+                const uint64_t p_desc0 = umma_smem_desc_noswizzle(smem_u32(q_smem) + slot * kSaPTileBytes, 128 * 16, 128);
                 const uint64_t v_desc0 = umma_smem_desc_sw128_mn(smem_u32(slot_smem(slot)), kSaKBlockBytes);
 #pragma unroll
                 for (int ks = 0; ks < kSaBK / 16; ++ks)
@@ -319,11 +337,12 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 umma_commit_elect(bar_p_free + 8 * slot);
                 umma_commit_elect(bar_pv_done);
                 if (i == nt - 1) umma_commit_elect(bar_o_full);
+                else if (tile_rescales(i + 1)) umma_commit_elect(bar_resc_go);   // tells the softmax warps when O may be rescaled
             }
             if (ok) umma_commit_elect(bar_q_empty);
         }
         if (!ok && lane == 0) sa_give_up(abort_flag, p.status, DEV_TIMEOUT_MMA);
-    } else if (warp == 1) {
+    } else if (warp == 4) {
         if (lane == 0) {
             // ------------------------------------------------------------ Q loader
             tma_prefetch_desc(&q_map);
@@ -345,7 +364,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     uint8_t* dst = b < kSaQT ? stage_smem + b * kSaQBlockBytes : q_smem + (b - kSaQT) * kSaQBlockBytes;
                     tma_load_2d(smem_u32(dst), &q_map, bar_q_full, b * 64, row0);
                 }
-                // ---- pass 2: the saved P tiles (and their rescale factors) come back, kSaPRing tiles ahead
+                // ---- pass 2: the saved P tiles come back, kSaPRing tiles ahead
                 ok = mbar_wait(bar_p2_go, ph_go, abort_flag, kWaitCycleBudget, 500);
                 if (!ok) break;
                 ph_go ^= 1u;
@@ -354,18 +373,18 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     ok = mbar_wait(bar_p_free + 8 * b, ph_p_free[b] ^ 1u, abort_flag, kWaitCycleBudget, 100);   // the PV product that read this buffer is done
                     if (!ok) break;
                     ph_p_free[b] ^= 1u;
-                    mbar_arrive_expect_tx(bar_p_full + 8 * b, kSaScratchTileBytes);
-                    bulk_load_1d(smem_u32(q_smem) + b * kSaScratchTileBytes, scratch + static_cast<size_t>(i) * kSaScratchTileBytes,
-                                 kSaScratchTileBytes, bar_p_full + 8 * b);
+                    mbar_arrive_expect_tx(bar_p_full + 8 * b, kSaPTileBytes);
+                    bulk_load_1d(smem_u32(q_smem) + b * kSaPTileBytes, scratch + static_cast<size_t>(i) * kSaScratchTileBytes,
+                                 kSaPTileBytes, bar_p_full + 8 * b);
                 }
             }
             if (!ok) sa_give_up(abort_flag, p.status, DEV_TIMEOUT_PRODUCER);
         }
-    } else if (warp < 2 + kSaGatherWarps) {
+    } else if (is_gather) {
         // ---------------------------------------------------------------- row gather
         // Two warps per slot (32 rows each): a pair only ever fills its own slot, so the four slots are four
         // independent acquire -> copy -> publish streams and a tile's landing time overlaps other tiles' copies.
-        const int gw = warp - 2;
+        const int gw = gather_index;
         const int slot = gw >> 1;                     // 2 * stage + group
         const int row0 = (gw & 1) * 32;               // this warp's rows of every tile it handles
         uint32_t ph_q_ready = 0, ph_empty = 0;
@@ -463,13 +482,13 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             }
         }
         if (!ok && lane == 0) sa_give_up(abort_flag, p.status, DEV_TIMEOUT_GATHER);
-    } else {
+    } else if (warp >= 12) {
         // ---------------------------------------------------------------- softmax and output
         const int quarter = warp & 3;                  // TMEM lane quarter this warp may access
         const int row = quarter * 32 + lane;           // head
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
         uint32_t ph_q_full = 0, ph_o_full = 0;
-        uint32_t ph_s_full[2] = {0u, 0u}, ph_p_free[4] = {0u, 0u, 0u, 0u}, ph_p_full[4] = {0u, 0u, 0u, 0u};
+        uint32_t ph_s_full[2] = {0u, 0u}, ph_resc_go = 0;
         uint32_t pv_tiles = 0;                         // PV tiles before the current one, over the whole kernel
         int stage = 0;
         bool ok = true;
@@ -546,6 +565,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_q_full, ph_q_full, abort_flag));
             if (!ok) break;
             ph_q_full ^= 1u;
+            // every reader of the previous query's flags is done (its last PV product was issued before this thread
+            // wrote its output); the arrival on q_ready below orders the reset before this query's tiles
+            if (quarter == 0 && lane < kSaFlagTiles / 32) resc_mask[lane] = 0u;
 #pragma unroll 1
             for (int b = 0; b < kSaQT; ++b) {
                 uint32_t r[32];
@@ -605,6 +627,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     l *= alpha;
                 }
                 if (i > 0 && __any_sync(0xFFFFFFFFu, move)) {
+                    if (lane == 0 && i < kSaFlagTiles) atomicOr(const_cast<uint32_t*>(resc_mask) + (i >> 5), 1u << (i & 31));
                     // PV(i-1) was issued before the second part of S(i), whose completion this thread has seen; the wait
                     // below (one phase per PV tile: the barrier is in phase pv_tiles-1 or pv_tiles) then passes at once
                     ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_pv_done, (pv_tiles - 1u) & 1u, abort_flag));
@@ -671,31 +694,24 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             }
 
             // ---- pass 2: the MMA warp reads P from the ring itself; this thread only replays the rescales of its row
-            // (the factor of tile i applies to the sum over the tiles before i)
+            // (the factor of tile i applies to the sum over the tiles before i) at the tiles flagged in pass 1: the MMA
+            // warp signals when the products before such a tile are complete and waits for the arrival below
 #pragma unroll 1
-            for (int i = 0; i < nt && ok; ++i) {
-                const int b = i & (kSaPRing - 1);
-                ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_p_full + 8 * b, ph_p_full[b], abort_flag));
+            for (int i = 1; i < nt && ok; ++i) {
+                if (!tile_rescales(i)) continue;
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_resc_go, ph_resc_go, abort_flag));
                 if (!ok) break;
-                ph_p_full[b] ^= 1u;
-                float alpha;
-                asm volatile("ld.shared.f32 %0, [%1];" : "=f"(alpha) : "r"(smem_u32(q_smem) + b * kSaScratchTileBytes + kSaPTileBytes + row * 4) : "memory");
-                if (i > 0 && __any_sync(0xFFFFFFFFu, alpha != 1.f)) {
-                    // PV(i-1) must be complete: it arrives on the p_free barrier of its buffer, in the phase this thread
-                    // noted when it passed tile i-1 (the loader refilled that buffer only after the phase before it, and
-                    // no PV product from tile i on can have been issued, so the barrier is in that phase or the next)
-                    const int prev = (i - 1) & (kSaPRing - 1);
-                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_p_free + 8 * prev, ph_p_free[prev] ^ 1u, abort_flag));
-                    if (!ok) break;
+                ph_resc_go ^= 1u;
+                const float alpha = __ldcg(reinterpret_cast<const float*>(my_alpha + static_cast<size_t>(i) * kSaScratchTileBytes));
+                if (__any_sync(0xFFFFFFFFu, alpha != 1.f)) {
                     scale_o(alpha);
                     tmem_st_wait();
-                    tcgen05_fence_before_sync();
                 }
-                ph_p_free[b] ^= 1u;                      // the phase PV(i) will complete
+                tcgen05_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_p_ready + 8 * b);
-                ++pv_tiles;
+                if (lane == 0) mbar_arrive(bar_p_ready + 8 * (i & (kSaPRing - 1)));
             }
+            pv_tiles += static_cast<uint32_t>(nt);
             if (!ok) break;
             ok = write_out(out_row + 256, part_row ? part_row + 256 : nullptr, inv);
         }

@@ -181,3 +181,14 @@ def test_degenerate_shapes(n_q, n_kv, h, k_top):
     g = torch.Generator().manual_seed(n_q * 1000 + k_top)
     topk = torch.randint(0, n_kv, (n_q, k_top), generator=g, dtype=torch.int32).cuda()
     _run(inp, topk, 0.05, h=h, what=f"degenerate {n_q}x{n_kv}x{h}x{k_top}")
+
+
+def test_more_tiles_than_rescale_flags():
+    # k_top beyond 256 tiles of 64 entries: the per-tile "rescaled" flags of the second pass cover 256 tiles, later
+    # tiles always take the hand-over with the softmax warps; 64 queries so that no query is split over several CTAs
+    n_q, n_kv, h, k_top = 64, 900, 4, 16384 + 192
+    inp = synth.attention_inputs(n_q, n_kv, h, D_QK, seed=23, device="cuda")
+    g = torch.Generator().manual_seed(23)
+    topk = torch.randint(0, n_kv, (n_q, k_top), generator=g, dtype=torch.int32).cuda()
+    topk[1, 16400:] = -1                                    # ends inside the tiles beyond the flags
+    _run(inp, topk, 0.3, rows=[0, 1, 63], h=h, what="259 tiles")
