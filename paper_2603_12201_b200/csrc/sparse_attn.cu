@@ -15,7 +15,7 @@
 //           the unswizzled K-major operand layout, so one bulk copy per tile brings it back (four tiles ahead, into
 //           the shared memory that held Q) and the PV MMAs read it there: no thread touches P in pass 2. The softmax
 //           warps note in pass 1 which tiles moved a reference maximum; only those tiles wait for them in pass 2.
-// Tensor memory (512 columns): O half [0,256) | S double-buffered [256,320), [320,384); in pass 1 P overwrites the
+// Tensor memory (512 columns): O half of pass 1 [0,256), that of pass 2 [256,512) | S double-buffered [256,320), [320,384); in pass 1 P overwrites the
 //   first 32 columns of its S buffer as bf16 pairs and is the A operand of the PV MMAs | Q blocks 0..3 (of 9 blocks
 //   of 64 columns) as bf16 pairs [384,512), the A operand of their score MMAs; Q blocks 4..8 stay in shared memory.
 // Shared memory: 2 stages x 9 blocks of [64 gathered rows x 128 B] (128-byte swizzle) | 5 blocks of Q
@@ -59,6 +59,7 @@ static_assert(kSaQT * kSaQBlockBytes <= 2 * kSaStageBytes, "the Q staging area l
 static_assert(kSaSmemBytes <= 232448, "shared memory budget of one CTA");
 constexpr int kSaPRing = 4;               // pass 2: saved P tiles in flight
 constexpr uint32_t kColO = 0, kColS = 256, kColQ = 384;   // S buffer b at kColS + 64 b; P in its first 32 columns
+constexpr uint32_t kColO2 = 256;          // pass 2 accumulates over the S and Q columns (unused then), so it need not wait for pass 1's read-out
 constexpr float kRescaleThreshold = 8.f;  // log2 units: P stays below 2^8
 constexpr uint32_t kSaPTileBytes = 128 * kSaBK * 2;
 constexpr uint32_t kSaScratchTileBytes = kSaPTileBytes + 128 * 4;     // P as [8 chunks][128 rows][16 B] + rescale factors [128] fp32
@@ -249,7 +250,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             ph_q_full ^= 1u;
             ph_q_ready ^= 1u;
             // ---- pass 1: scores and the first half of the output
-            ok = wait_bar(bar_o_free, ph_o_free ^ 1u);        // the previous query's O has been read out
+            ok = wait_bar(bar_o_free, ph_o_free ^ 1u);        // the previous query's second half (and so all of its O) has been read out
             if (!ok) break;
             ph_o_free ^= 1u;
             // Issue order: S(i+1) blocks 4..8 | P(i) V(i) | S(i+1) blocks 0..3. The first part keeps the tensor pipe busy
@@ -312,9 +313,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             }
             if (!ok) break;
             // ---- pass 2: the second half of the output from the saved P; the four slots are a ring of value tiles
-            ok = wait_bar(bar_o_free, ph_o_free ^ 1u);
-            if (!ok) break;
-            ph_o_free ^= 1u;
+            // (accumulates in columns 256..511: no wait for the read-out of the first half)
             for (int i = 0; i < nt; ++i) {
                 const int slot = i & 3;
                 ok = wait_slot(slot) && wait_bar(bar_p_full + 8 * slot, ph_p_full[slot]);
@@ -331,7 +330,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 const uint64_t v_desc0 = umma_smem_desc_sw128_mn(smem_u32(slot_smem(slot)), kSaKBlockBytes);
 #pragma unroll
                 for (int ks = 0; ks < kSaBK / 16; ++ks)
-                    umma_f16_elect_acc(tmem_base + kColO, p_desc0 + (ks * 2 * 128 * 16) / 16, v_desc0 + (ks * 16 * 128) / 16, kIdescPV,
+                    umma_f16_elect_acc(tmem_base + kColO2, p_desc0 + (ks * 2 * 128 * 16) / 16, v_desc0 + (ks * 16 * 128) / 16, kIdescPV,
                                        (i == 0 && ks == 0) ? 0u : 1u);
                 umma_commit_elect(bar_slot_empty + 8 * slot);
                 umma_commit_elect(bar_p_free + 8 * slot);
@@ -496,37 +495,42 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         uint8_t* my_p = scratch + row * 16;                           // + tile * kSaScratchTileBytes + chunk * 2048
         uint8_t* my_alpha = scratch + 128 * kSaBK * 2 + row * 4;      // + tile * kSaScratchTileBytes: this row's factor
         // multiplies this thread's row of O by alpha (the caller has made sure that every earlier PV product is complete)
-        auto scale_o = [&](float alpha) {
+        auto scale_o = [&](float alpha, uint32_t col0) {
             tcgen05_fence_after_sync();
 #pragma unroll 1
             for (int c = 0; c < 8; ++c) {
                 uint32_t o[32];
-                tmem_ld_32x32b_x32(lane_base + kColO + c * 32, o);
+                tmem_ld_32x32b_x32(lane_base + col0 + c * 32, o);
                 tmem_ld_wait(o);
 #pragma unroll
                 for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
-                tmem_st_32x32b_x32(lane_base + kColO + c * 32, o);
+                tmem_st_32x32b_x32(lane_base + col0 + c * 32, o);
             }
         };
-        // normalises this thread's row of O and writes 256 output columns: bf16 to the output, or fp32 to this split's
-        // partial result when several CTAs share the query (part_row != nullptr)
-        auto write_out = [&](__nv_bfloat16* dst_row, float* part_row, float inv) -> bool {
+        // Normalises this thread's row of O and writes 256 output columns: fp32 to this split's partial result when
+        // several CTAs share the query (part_row != nullptr), else bf16 to the output. A thread holds 32 columns of one
+        // row at a time, and storing them directly makes every warp store touch 32 lines; so the warp transposes them
+        // through 2 KB of shared memory (the last block of a stage, which neither the value tiles of pass 2 nor the Q
+        // staging use) and stores 8 rows x 64 contiguous bytes per instruction.
+        uint8_t* const stg = stage_smem + 8 * kSaKBlockBytes + quarter * 2048;     // [32 rows][64 B], 16-byte chunks XORed by (row >> 1) & 3
+        auto write_out = [&](__nv_bfloat16* dst_query, float* part_row, float inv, uint32_t col0, bool last) -> bool {   // dst_query: row 0 of the query, first column of the half
             if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar_o_full, ph_o_full, abort_flag))) return false;
             ph_o_full ^= 1u;
             tcgen05_fence_after_sync();
 #pragma unroll 1
             for (int c = 0; c < 8; ++c) {
                 uint32_t o[32];
-                tmem_ld_32x32b_x32(lane_base + kColO + c * 32, o);
+                tmem_ld_32x32b_x32(lane_base + col0 + c * 32, o);
                 tmem_ld_wait(o);
-                if (row < p.H && part_row != nullptr) {
-                    float4* dst = reinterpret_cast<float4*>(part_row + c * 32);
+                if (part_row != nullptr) {
+                    if (row < p.H) {
+                        float4* dst = reinterpret_cast<float4*>(part_row + c * 32);
 #pragma unroll
-                    for (int v = 0; v < 8; ++v)
-                        dst[v] = make_float4(__uint_as_float(o[4 * v + 0]) * inv, __uint_as_float(o[4 * v + 1]) * inv,
-                                             __uint_as_float(o[4 * v + 2]) * inv, __uint_as_float(o[4 * v + 3]) * inv);
-                } else if (row < p.H) {
-                    uint4* dst = reinterpret_cast<uint4*>(dst_row + c * 32);
+                        for (int v = 0; v < 8; ++v)
+                            dst[v] = make_float4(__uint_as_float(o[4 * v + 0]) * inv, __uint_as_float(o[4 * v + 1]) * inv,
+                                                 __uint_as_float(o[4 * v + 2]) * inv, __uint_as_float(o[4 * v + 3]) * inv);
+                    }
+                } else {
 #pragma unroll
                     for (int v = 0; v < 4; ++v) {
                         uint4 w;
@@ -534,13 +538,22 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                         w.y = pack_bf16x2(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
                         w.z = pack_bf16x2(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
                         w.w = pack_bf16x2(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
-                        dst[v] = w;
+                        *reinterpret_cast<uint4*>(stg + lane * 64 + ((v ^ ((lane >> 1) & 3)) << 4)) = w;
                     }
+                    __syncwarp();
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int rr = (lane >> 2) + 8 * k, ch = lane & 3;     // 8 rows per instruction, 4 lanes per row
+                        const uint4 w = *reinterpret_cast<const uint4*>(stg + rr * 64 + ((ch ^ ((rr >> 1) & 3)) << 4));
+                        if (quarter * 32 + rr < p.H)
+                            *reinterpret_cast<uint4*>(dst_query + static_cast<int64_t>(quarter * 32 + rr) * 512 + c * 32 + ch * 8) = w;
+                    }
+                    __syncwarp();
                 }
             }
             tcgen05_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_o_free);
+            if (last && lane == 0) mbar_arrive(bar_o_free);    // both halves of O are read out: the next query may overwrite them
             return true;
         };
         for (int64_t item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
@@ -632,7 +645,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                     // below (one phase per PV tile: the barrier is in phase pv_tiles-1 or pv_tiles) then passes at once
                     ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_pv_done, (pv_tiles - 1u) & 1u, abort_flag));
                     if (!ok) break;
-                    scale_o(alpha);
+                    scale_o(alpha, kColO);
                 }
                 const float m_sub = m_ref == -INFINITY ? 0.f : m_ref;   // no usable score yet: every P is exp2(-inf) = 0
                 // P(i) goes over the first half of S(i) chunk by chunk (columns 8c..8c+7 hold scores this thread has
@@ -685,7 +698,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_p2_go);
             const float inv = l > 0.f ? 1.f / l : 0.f;
-            ok = write_out(out_row, part_row, inv);
+            ok = write_out(p.out + t * p.H * 512, part_row, inv, kColO, false);
             if (!ok) break;
             if (row < p.H) {
                 const float lse_val = l > 0.f ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
@@ -704,7 +717,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
                 ph_resc_go ^= 1u;
                 const float alpha = __ldcg(reinterpret_cast<const float*>(my_alpha + static_cast<size_t>(i) * kSaScratchTileBytes));
                 if (__any_sync(0xFFFFFFFFu, alpha != 1.f)) {
-                    scale_o(alpha);
+                    scale_o(alpha, kColO2);
                     tmem_st_wait();
                 }
                 tcgen05_fence_before_sync();
@@ -713,7 +726,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
             }
             pv_tiles += static_cast<uint32_t>(nt);
             if (!ok) break;
-            ok = write_out(out_row + 256, part_row ? part_row + 256 : nullptr, inv);
+            ok = write_out(p.out + t * p.H * 512 + 256, part_row ? part_row + 256 : nullptr, inv, kColO2, true);
         }
         if (!ok && lane == 0) sa_give_up(abort_flag, p.status, DEV_TIMEOUT_EPILOGUE);
     }
