@@ -99,16 +99,20 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // n_eff[2t] = 1 + position of the last entry of row t that is >= 0 and inside the cache (0 if none);
 // n_eff[2t+1] = the cache row of its first usable entry (stands in for skipped entries, with weight 0: rows that
 // are not selected are never read).
-__global__ void sparse_attn_count_kernel(const int32_t* __restrict__ topk, const int64_t* __restrict__ kv_base, int64_t n_q,
-                                         int64_t n_kv, int k_top, int32_t* __restrict__ n_eff) {
-    const int64_t t = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
-    const int lane = threadIdx.x & 31;
-    if (t >= n_q) return;
+constexpr int kSaCountThreads = 128;
+__global__ void __launch_bounds__(kSaCountThreads)
+sparse_attn_count_kernel(const int32_t* __restrict__ topk, const int64_t* __restrict__ kv_base, int64_t n_q, int64_t n_kv, int k_top,
+                         int32_t* __restrict__ n_eff) {
+    // one CTA per query: a decode step has few queries, and a single warp walking a row is one long chain of dependent loads
+    const int64_t t = blockIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t base = kv_base ? kv_base[t] : 0;
+    const int32_t* row = topk + t * k_top;
     int last = 0;
     unsigned long long first = ~0ull;          // (position << 32) | cache row of the first usable entry
-    for (int j = lane; j < k_top; j += 32) {
-        const int64_t idx = topk[t * k_top + j];
+#pragma unroll 4
+    for (int j = threadIdx.x; j < k_top; j += kSaCountThreads) {
+        const int64_t idx = __ldg(row + j);
         if (idx >= 0 && base + idx >= 0 && base + idx < n_kv) {
             last = j + 1;
             if (first == ~0ull) first = (static_cast<unsigned long long>(j) << 32) | static_cast<unsigned long long>(base + idx);
@@ -120,7 +124,16 @@ __global__ void sparse_attn_count_kernel(const int32_t* __restrict__ topk, const
         const unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, first, o);
         first = other < first ? other : first;
     }
-    if (lane == 0) {
+    __shared__ int s_last[kSaCountThreads / 32];
+    __shared__ unsigned long long s_first[kSaCountThreads / 32];
+    if (lane == 0) { s_last[warp] = last; s_first[warp] = first; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int w = 1; w < kSaCountThreads / 32; ++w) {
+            last = max(last, s_last[w]);
+            first = s_first[w] < first ? s_first[w] : first;
+        }
         n_eff[2 * t] = last;
         n_eff[2 * t + 1] = last ? static_cast<int32_t>(first & 0xFFFFFFFFull) : 0;
     }
@@ -747,20 +760,34 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
 
 // Merges the splits of a query: out = sum_s w_s out_s / sum_s w_s with w_s = exp(lse_s - max_s lse_s). One CTA per
 // (query, head), 128 threads x 4 columns.
-__global__ void sparse_attn_merge_kernel(const float* __restrict__ part_out, const float* __restrict__ part_lse, int H, int splits,
-                                         __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
+__global__ void __launch_bounds__(128)
+sparse_attn_merge_kernel(const float* __restrict__ part_out, const float* __restrict__ part_lse, int H, int splits,
+                         __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
+    constexpr int kMaxSplits = 8;              // sparse_attn_splits never returns more
     const int64_t t = blockIdx.x / H;
     const int h = static_cast<int>(blockIdx.x - t * H);
+    // all loads are issued before anything depends on them: one round trip to the L2 instead of one per split
+    float ls[kMaxSplits];
+    float4 v[kMaxSplits];
+#pragma unroll
+    for (int s = 0; s < kMaxSplits; ++s) {
+        ls[s] = -INFINITY;
+        v[s] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (s < splits) {
+            ls[s] = __ldg(part_lse + (t * splits + s) * H + h);
+            v[s] = __ldg(reinterpret_cast<const float4*>(part_out + ((t * splits + s) * H + h) * 512) + threadIdx.x);
+        }
+    }
     float m = -INFINITY;
-    for (int s = 0; s < splits; ++s) m = fmaxf(m, part_lse[(t * splits + s) * H + h]);
+#pragma unroll
+    for (int s = 0; s < kMaxSplits; ++s) m = fmaxf(m, ls[s]);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float denom = 0.f;
     if (m > -INFINITY) {
-        for (int s = 0; s < splits; ++s) {
-            const float w = __expf(part_lse[(t * splits + s) * H + h] - m);
-            if (w == 0.f) continue;
-            const float4 v = reinterpret_cast<const float4*>(part_out + ((t * splits + s) * H + h) * 512)[threadIdx.x];
-            acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+#pragma unroll
+        for (int s = 0; s < kMaxSplits; ++s) {
+            const float w = __expf(ls[s] - m);     // 0 for a split with nothing usable (its result is all zeros)
+            acc.x += w * v[s].x; acc.y += w * v[s].y; acc.z += w * v[s].z; acc.w += w * v[s].w;
             denom += w;
         }
     }
@@ -797,8 +824,7 @@ cudaError_t launch_sparse_attn(const void* kv, const int32_t* topk, const int64_
                                const CUtensorMap& q_map, const CUtensorMap& kv_map, unsigned int* status, int sm_count,
                                cudaStream_t stream) {
     if (n_q <= 0) return cudaSuccess;
-    const int64_t count_blocks = (n_q * 32 + 255) / 256;
-    sparse_attn_count_kernel<<<static_cast<unsigned>(count_blocks), 256, 0, stream>>>(topk, kv_base, n_q, n_kv, k_top, n_eff);
+    sparse_attn_count_kernel<<<static_cast<unsigned>(n_q), kSaCountThreads, 0, stream>>>(topk, kv_base, n_q, n_kv, k_top, n_eff);
     if (cudaError_t e = cudaGetLastError(); e != cudaSuccess) return e;
     if (cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(sparse_attn_kernel), kSaSmemBytes); e != cudaSuccess) return e;
     const int splits = sparse_attn_splits(n_q);
