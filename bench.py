@@ -486,7 +486,11 @@ def time_sparse_attention(idxc, synth, dev, peaks, L, n_q, k_top, seed, steps=3)
             "ms": ms, "queries_per_s": n_q / (ms * 1e-3), "selected_rows": selected,
             "gathered_bytes": gather_bytes,
             "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                         "frac": tf / peaks["bf16_tflops"], "of": peaks["source"] + " burst peak", "traffic": None}}
+                         "frac": tf / peaks["bf16_tflops"], "of": peaks["source"] + " burst peak",
+                         "frac_of_sustained": tf / peaks["bf16_tflops_sustained"], "traffic": None,
+                         "note": "the kernel draws the board's full power: after the sections before it in a default run the "
+                                 "clocks sit near 1.6 GHz (sw_power_cap) and the time is about 15-20 % above a cold run of this "
+                                 "section alone (--only-sparse-attention --steps 3)"}}
 
 
 def main():
@@ -507,6 +511,7 @@ def main():
     ap.add_argument("--only-decode", action="store_true", help="run only the decode section (profiling)")
     ap.add_argument("--only-sparse-attention", action="store_true", help="run only the sparse-attention section (profiling)")
     ap.add_argument("--only-layer-loop", action="store_true", help="run only the indexer + attention layer loop section")
+    ap.add_argument("--only-fp8", action="store_true", help="run only the FP8 chunked-prefill section (profiling; --L sets the length)")
     ap.add_argument("--sa-queries", type=int, default=8192, help="queries of the sparse-attention section")
     args = ap.parse_args()
     if args.warmup < 3:
@@ -542,6 +547,11 @@ def main():
         return
     if args.only_layer_loop:
         print(json.dumps({"layer_loop": time_layer_loop(idxc, synth, dev, args.L or 32768, 2048, 4, 4, seed=8)}), flush=True)
+        return
+    if args.only_fp8:
+        c5 = synth.CONFIGS["cfg5"]
+        print(json.dumps({"fp8_chunked": time_fp8_chunked(idxc, synth, dev, peaks, args.L or 32768, c5["chunk"], c5["H"], c5["d"],
+                                                          c5["k_top"], c5["seed"], c5["decode_B"])}), flush=True)
         return
     if args.only_sparse_attention:
         print(json.dumps({"sparse_attention": time_sparse_attention(idxc, synth, dev, peaks, args.L or 32768, args.sa_queries, 2048,
