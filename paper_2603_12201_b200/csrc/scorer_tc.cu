@@ -397,7 +397,7 @@ constexpr int kDecodeThreads = (2 + kDecodeEpiWarps) * 32;   // warp 0 producer,
 // Key tiles (of 128 keys) per work item. Measured on B200 (B = 32, 16K-128K keys per sequence): 16 tiles
 // stream at 6.1 TB/s; 6-8 tiles per item lose 20 % (all CTAs then walk HBM with the same 192-256 KB stride).
 constexpr int kDecodeChunkTiles = 16;
-constexpr int kDecodeAccSlots = 4;       // TMEM accumulators in flight (64 columns apart)
+constexpr int kDecodeAccSlots = 8;       // TMEM accumulators in flight (64 columns apart: all 512 columns)
 
 template <int NKH, int H>
 struct DecodeCfg {
@@ -405,7 +405,7 @@ struct DecodeCfg {
     static constexpr int kQRegion = H * kChunkBytes;                  // one 128-byte chunk of the query tile
     static constexpr int kQBytes = 2 * NKH * kQRegion;                // double buffered
     static constexpr int kKBytes = kStages * NKH * kKRegionBytes;
-    static constexpr int kWBytes = kDecodeEpiWarps * (64 + kDecodeChunkTiles * 32) * 4;   // per warp: w, and the key scales of one item
+    static constexpr int kWBytes = kDecodeEpiWarps * 64 * 4;          // per epilogue warp: w of the item's sequence
     static constexpr int kBarBytes = 512;
     static constexpr int kSmemBytes = kQBytes + kKBytes + kWBytes + kBarBytes + 1024;
 };
@@ -480,11 +480,12 @@ score_decode_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
     uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(w_smem) + Cfg::kWBytes);
     const uint32_t bar_q_full = smem_u32(bars + 0);          // [2]
     const uint32_t bar_q_empty = smem_u32(bars + 2);         // [2]
-    const uint32_t bar_acc_full = smem_u32(bars + 4);        // [4]
-    const uint32_t bar_acc_empty = smem_u32(bars + 8);       // [4]
-    const uint32_t bar_k_full = smem_u32(bars + 12);         // [kStages]
-    const uint32_t bar_k_empty = smem_u32(bars + 12 + kStages);
-    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(bars + 12 + 2 * kStages);
+    const uint32_t bar_acc_full = smem_u32(bars + 4);        // [kDecodeAccSlots]
+    const uint32_t bar_acc_empty = smem_u32(bars + 4 + kDecodeAccSlots);
+    const uint32_t bar_k_full = smem_u32(bars + 4 + 2 * kDecodeAccSlots);         // [kStages]
+    const uint32_t bar_k_empty = smem_u32(bars + 4 + 2 * kDecodeAccSlots + kStages);
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(bars + 4 + 2 * kDecodeAccSlots + 2 * kStages);
+    static_assert((5 + 2 * kDecodeAccSlots + 2 * kStages) * 8 <= Cfg::kBarBytes && kDecodeAccSlots * 64 <= 512, "barrier area, tensor memory");
     volatile uint32_t* abort_flag = tmem_base_slot + 1;
 
     const int warp = threadIdx.x >> 5;
@@ -506,7 +507,7 @@ score_decode_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
         fence_mbar_init();
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(tmem_base_slot), 256);
+        tmem_alloc(smem_u32(tmem_base_slot), kDecodeAccSlots * 64);
         tmem_relinquish_alloc_permit();
     }
     tcgen05_fence_before_sync();
@@ -547,52 +548,58 @@ score_decode_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
             if (!ok) give_up(abort_flag, p.status, DEV_TIMEOUT_PRODUCER);
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            int stage = 0, qbuf = 0, slot = 0;
-            uint32_t k_phase = 0, q_phase[2] = {0u, 0u}, acc_phase[kDecodeAccSlots] = {0u, 0u, 0u, 0u};
-            bool ok = true;
-            while (ok && walk.pop(seq, tile0, ntiles, len)) {
-                ok = mbar_wait(bar_q_full + 8 * qbuf, q_phase[qbuf], abort_flag);
+        // The whole warp runs this role with uniform control flow and one elected lane issues (a single diverged lane
+        // issues the same instruction stream about 1.5x slower); descriptors are a base plus 16-byte units.
+        int stage = 0, qbuf = 0, slot = 0;
+        uint32_t k_phase = 0, q_phase[2] = {0u, 0u}, acc_phase = 0;   // acc_phase: one bit per accumulator slot
+        bool ok = true;
+        const uint64_t a_desc0 = umma_smem_desc_sw128(smem_u32(k_smem));
+        const uint64_t b_desc0 = umma_smem_desc_sw128(smem_u32(q_smem));
+        auto wait_bar = [&](uint32_t bar, uint32_t parity) -> bool {
+            return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort_flag));
+        };
+        while (ok && walk.pop(seq, tile0, ntiles, len)) {
+            ok = wait_bar(bar_q_full + 8 * qbuf, q_phase[qbuf]);
+            if (!ok) break;
+            q_phase[qbuf] ^= 1u;
+            const uint64_t b_desc = b_desc0 + static_cast<uint64_t>(qbuf * NKH * Cfg::kQRegion / 16);
+            for (int kt = 0; kt < ntiles && ok; ++kt) {
+                ok = wait_bar(bar_k_full + 8 * stage, k_phase) && wait_bar(bar_acc_empty + 8 * slot, ((acc_phase >> slot) & 1u) ^ 1u);
                 if (!ok) break;
-                q_phase[qbuf] ^= 1u;
-                for (int kt = 0; kt < ntiles && ok; ++kt) {
-                    ok = mbar_wait(bar_k_full + 8 * stage, k_phase, abort_flag);
-                    if (!ok) break;
-                    ok = mbar_wait(bar_acc_empty + 8 * slot, acc_phase[slot] ^ 1u, abort_flag);
-                    if (!ok) break;
-                    acc_phase[slot] ^= 1u;
-                    tcgen05_fence_after_sync();
-                    const uint32_t d_tmem = tmem_base + slot * 64;
+                acc_phase ^= 1u << slot;
+                tcgen05_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + slot * 64;
+                const uint64_t a_desc = a_desc0 + static_cast<uint64_t>(stage * NKH * kKRegionBytes / 16);
 #pragma unroll
-                    for (int kh = 0; kh < NKH; ++kh) {
-                        const uint32_t a_base = smem_u32(k_smem + (stage * NKH + kh) * kKRegionBytes);
-                        const uint32_t b_base = smem_u32(q_smem + (qbuf * NKH + kh) * Cfg::kQRegion);
+                for (int kh = 0; kh < NKH; ++kh) {
 #pragma unroll
-                        for (int ks = 0; ks < 4; ++ks) {
-                            const uint64_t a_desc = umma_smem_desc_sw128(a_base + ks * 32);
-                            const uint64_t b_desc = umma_smem_desc_sw128(b_base + ks * 32);
-                            if constexpr (FP8) umma_f8(d_tmem, a_desc, b_desc, kIdesc, (kh | ks) != 0);
-                            else umma_f16(d_tmem, a_desc, b_desc, kIdesc, (kh | ks) != 0);
+                    for (int ks = 0; ks < 4; ++ks) {
+                        const uint64_t a = a_desc + (kh * kKRegionBytes + ks * 32) / 16, b = b_desc + (kh * Cfg::kQRegion + ks * 32) / 16;
+                        if constexpr (FP8) {
+                            if ((kh | ks) != 0) umma_f8_elect<true>(d_tmem, a, b, kIdesc);
+                            else umma_f8_elect<false>(d_tmem, a, b, kIdesc);
+                        } else {
+                            if ((kh | ks) != 0) umma_f16_elect<true>(d_tmem, a, b, kIdesc);
+                            else umma_f16_elect<false>(d_tmem, a, b, kIdesc);
                         }
                     }
-                    umma_commit(bar_acc_full + 8 * slot);
-                    umma_commit(bar_k_empty + 8 * stage);
-                    if (kt == ntiles - 1) umma_commit(bar_q_empty + 8 * qbuf);
-                    if (++stage == kStages) { stage = 0; k_phase ^= 1u; }
-                    slot = (slot + 1) & (kDecodeAccSlots - 1);
                 }
-                qbuf ^= 1;
+                umma_commit_elect(bar_acc_full + 8 * slot);
+                umma_commit_elect(bar_k_empty + 8 * stage);
+                if (kt == ntiles - 1) umma_commit_elect(bar_q_empty + 8 * qbuf);
+                if (++stage == kStages) { stage = 0; k_phase ^= 1u; }
+                slot = (slot + 1) & (kDecodeAccSlots - 1);
             }
-            if (!ok) give_up(abort_flag, p.status, DEV_TIMEOUT_MMA);
+            qbuf ^= 1;
         }
+        if (!ok && lane == 0) give_up(abort_flag, p.status, DEV_TIMEOUT_MMA);
     } else {
         const int quarter = warp & 3;
         const int grp = (warp - 2) >> 2;                 // which accumulator slots this warp drains
         const int key_in_tile = quarter * 32 + lane;
-        float* my_w = w_smem + (warp - 2) * (64 + kDecodeChunkTiles * 32);
-        float* my_ksc = my_w + 64;                       // FP8: k_scale of my key in every tile of the item
+        float* my_w = w_smem + (warp - 2) * 64;
         int slot = 0;
-        uint32_t acc_phase[kDecodeAccSlots] = {0u, 0u, 0u, 0u};
+        uint32_t acc_phase = 0;                          // one bit per accumulator slot
         bool ok = true;
         while (ok && walk.pop(seq, tile0, ntiles, len)) {
             __syncwarp();
@@ -602,30 +609,33 @@ score_decode_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                 my_w[h] = v;
             }
             const int64_t krow0 = p.k_offsets[seq];
-            if constexpr (FP8) {
-                // all key scales of the item at once: independent loads in flight instead of one exposed
-                // memory latency per tile
-#pragma unroll 4
-                for (int kt = 0; kt < ntiles; ++kt) {
-                    const int s2 = (tile0 + kt) * kTileKeys + key_in_tile;
-                    my_ksc[kt * 32 + lane] = s2 < len ? __ldg(p.k_scale + krow0 + s2) : 0.f;
-                }
-            }
             __syncwarp();
             const float4* w4 = reinterpret_cast<const float4*>(my_w);
             for (int kt = 0; kt < ntiles && ok; ++kt, slot = (slot + 1) & (kDecodeAccSlots - 1)) {
                 if ((slot & 1) != grp) continue;         // the other group's tile
                 const int s = (tile0 + kt) * kTileKeys + key_in_tile;
-                ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_acc_full + 8 * slot, acc_phase[slot], abort_flag));   // warp-uniform
+                // FP8: the key's scale is asked for before the wait and used after the head sums: its latency is hidden
+                // behind the accumulator's
+                float ksc = 1.f;
+                if constexpr (FP8) ksc = s < len ? __ldg(p.k_scale + krow0 + s) : 0.f;
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_acc_full + 8 * slot, (acc_phase >> slot) & 1u, abort_flag));   // warp-uniform
                 if (!ok) break;
-                acc_phase[slot] ^= 1u;
+                acc_phase ^= 1u << slot;
                 tcgen05_fence_after_sync();
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(slot * 64);
                 float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;    // four independent partial sums over the heads
+                // the accumulator is in registers once its loads have completed: the slot goes back to the MMA warp
+                // before the head sums, not after
+                auto release_slot = [&]() {
+                    tcgen05_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_acc_empty + 8 * slot);
+                };
                 if constexpr (H == 16) {
                     uint32_t r[16];
                     tmem_ld_32x32b_x16(taddr, r);
                     tmem_ld_wait(r);
+                    release_slot();
 #pragma unroll
                     for (int j4 = 0; j4 < 4; ++j4) {
                         const float4 wv = w4[j4];
@@ -640,6 +650,7 @@ score_decode_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                     if constexpr (H == 64) tmem_ld_32x32b_x32(taddr + 32, rb);
                     tmem_ld_wait(ra);                    // waits for every load issued so far
                     if constexpr (H == 64) tmem_ld_wait(rb);
+                    release_slot();
 #pragma unroll
                     for (int j4 = 0; j4 < 8; ++j4) {
                         const float4 wv = w4[j4];
@@ -659,12 +670,9 @@ score_decode_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                         }
                     }
                 }
-                tcgen05_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_acc_empty + 8 * slot);
                 if (s < len) {
                     float acc = (a0 + a1) + (a2 + a3);
-                    if constexpr (FP8) acc *= my_ksc[kt * 32 + lane];
+                    if constexpr (FP8) acc *= ksc;
                     p.scores[static_cast<int64_t>(seq) * p.ld + s] = acc;
                 }
             }
@@ -681,7 +689,7 @@ score_decode_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
     __syncthreads();
     if (warp == 1) {
         tcgen05_fence_after_sync();
-        tmem_dealloc(tmem_base, 256);
+        tmem_dealloc(tmem_base, kDecodeAccSlots * 64);
     }
 }
 
