@@ -510,7 +510,7 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2"])
     ap.add_argument("--ref-rows", type=int, default=128, help="rows per step of the reference (oracle) arm")
     ap.add_argument("--cpu-rows", type=int, default=1024, help="rows of the cpu_baseline sample")
-    ap.add_argument("--e2e-steps", type=int, default=8)
+    ap.add_argument("--e2e-steps", type=int, default=32, help="steps of the end-to-end loop (its first copy-in and last copy-out are not overlapped: few steps overstate them)")
     ap.add_argument("--no-extras", action="store_true", help="skip the decode and schedule sections")
     ap.add_argument("--schedule-layers", type=int, default=8)
     ap.add_argument("--schedule-L", type=int, default=32768)
