@@ -433,16 +433,13 @@ idxc_status idxc_sparse_attention(const void* q, const void* kv, const int32_t* 
     if (!di.ok) return IDXC_ERR_CUDA;
     CUtensorMap q_map;
     if (!encode_operand_map(&q_map, q, n_q * H, d_qk, false, H)) return IDXC_ERR_CUDA;
-    CUtensorMap kv_map;
     if (n_kv >= (int64_t(1) << 31)) return IDXC_ERR_INVALID_ARG;
-    // an empty cache has no usable entry and is never read: any valid address serves as the base then
-    if (!encode_operand_map(&kv_map, n_kv > 0 ? kv : q, n_kv > 0 ? n_kv : 1, d_qk, false, 1)) return IDXC_ERR_CUDA;
     g_launches += 2;
     uint8_t* scratch = static_cast<uint8_t*>(workspace) + round_up(n_q * 8, 256);
     void* partial = sparse_attn_partial_bytes(n_q) ? scratch + round_up(sparse_attn_scratch_bytes(n_q, k_top), 256) : nullptr;
     g_launches += partial ? 1 : 0;
     return launch_sparse_attn(kv, topk, kv_base, n_q, n_kv, H, k_top, scale, out, lse, static_cast<int32_t*>(workspace), scratch,
-                              partial, q_map, kv_map, di.status_ptr, di.sm_count, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+                              partial, q_map, di.status_ptr, di.sm_count, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
                ? IDXC_OK : IDXC_ERR_CUDA;
 }
 

@@ -70,7 +70,7 @@ size_t sparse_attn_scratch_bytes(int64_t n_q, int k_top);
 size_t sparse_attn_partial_bytes(int64_t n_q);
 cudaError_t launch_sparse_attn(const void* kv, const int32_t* topk, const int64_t* kv_base, int64_t n_q, int64_t n_kv, int H,
                                int k_top, float scale, void* out, float* lse, int32_t* n_eff, void* scratch, void* partial,
-                               const CUtensorMap& q_map, const CUtensorMap& kv_map, unsigned int* status, int sm_count,
+                               const CUtensorMap& q_map, unsigned int* status, int sm_count,
                                cudaStream_t stream);
 
 // selftest.cu: one tiny kernel whose only wait can never be satisfied; it must record a time-out in

@@ -40,7 +40,7 @@
 namespace idxc {
 namespace {
 
-constexpr int kSaGatherWarps = 8;          // warps 2 .. 9
+constexpr int kSaGatherWarps = 8;          // warps 1 2 3 5 6 7 9 10
 constexpr int kSaThreads = 32 * 16;
 static_assert(kSaGatherWarps == 8, "two gather warps per slot, four slots");
 constexpr int kSaBK = 64;                 // gathered rows per tile
@@ -140,7 +140,7 @@ sparse_attn_count_kernel(const int32_t* __restrict__ topk, const int64_t* __rest
 }
 
 __global__ void __launch_bounds__(kSaThreads, 1)
-sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap kv_map, const SaParams p) {
+sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) {
     extern __shared__ uint8_t smem_raw[];
     // aligned by an offset into the array (not by an integer round trip), so that the compiler still knows that these
     // pointers are shared memory and emits shared-space loads and stores for them
@@ -358,7 +358,6 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_const
         if (lane == 0) {
             // ------------------------------------------------------------ Q loader
             tma_prefetch_desc(&q_map);
-            tma_prefetch_desc(&kv_map);
             uint32_t ph_q_empty = 0, ph_go = 0;
             uint32_t ph_p_free[kSaPRing] = {0u, 0u, 0u, 0u};
             bool ok = true;
@@ -821,7 +820,7 @@ size_t sparse_attn_partial_bytes(int64_t n_q) {        // sized for 128 heads
 
 cudaError_t launch_sparse_attn(const void* kv, const int32_t* topk, const int64_t* kv_base, int64_t n_q, int64_t n_kv, int H,
                                int k_top, float scale, void* out, float* lse, int32_t* n_eff, void* scratch, void* partial,
-                               const CUtensorMap& q_map, const CUtensorMap& kv_map, unsigned int* status, int sm_count,
+                               const CUtensorMap& q_map, unsigned int* status, int sm_count,
                                cudaStream_t stream) {
     if (n_q <= 0) return cudaSuccess;
     sparse_attn_count_kernel<<<static_cast<unsigned>(n_q), kSaCountThreads, 0, stream>>>(topk, kv_base, n_q, n_kv, k_top, n_eff);
@@ -835,7 +834,7 @@ cudaError_t launch_sparse_attn(const void* kv, const int32_t* topk, const int64_
     const int64_t items = n_q * splits;
     const int cap = sm_count < kSparseAttnMaxGrid ? sm_count : kSparseAttnMaxGrid;
     const int grid = static_cast<int>(items < cap ? items : cap);
-    sparse_attn_kernel<<<grid, kSaThreads, kSaSmemBytes, stream>>>(q_map, kv_map, p);
+    sparse_attn_kernel<<<grid, kSaThreads, kSaSmemBytes, stream>>>(q_map, p);
     if (cudaError_t e = cudaGetLastError(); e != cudaSuccess) return e;
     if (splits > 1) {
         sparse_attn_merge_kernel<<<static_cast<unsigned>(n_q * H), 128, 0, stream>>>(part_out, part_lse, H, splits,
