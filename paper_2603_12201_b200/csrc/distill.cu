@@ -1,9 +1,9 @@
 // Forward value of the multi-layer distillation loss of training-aware IndexCache (Eq. 1):
 //     L_multi = sum_{j=0..m} 1/(m+1) sum_t KL( p_t^(l+j) || Softmax(I_t) )
 // over the causal positions s <= t of every row, or (sparse-training form) over the row's selected top-k
-// positions with p renormalised over them. One 256-thread CTA per row: an online max / sum-of-exponentials
-// sweep over the scores, then one sweep per target. HBM-bound: 4 * (1 + n_targets) bytes per (t, s) pair
-// (the second read of the scores comes from L2). exp / log in fp32, accumulation in fp64.
+// positions with p renormalised over them. One 256-thread CTA per row; the dense form reads the scores and every
+// target exactly once, in one sweep. HBM-bound: 4 * (1 + n_targets) bytes per (t, s) pair. exp / log and the
+// per-thread sums in fp32, block sums in fp64.
 #include "../../include/idxc.h"
 #include "kernels.h"
 
@@ -29,6 +29,9 @@ __device__ __forceinline__ double block_sum_f64(double v, double* sh) {
     return t;
 }
 
+// NT: targets handled by one dense sweep (1, 2 or 4: their sums live in registers); more targets take one sweep per
+// group of NT, the scores of the later sweeps coming from the L2.
+template <int NT>
 __global__ void __launch_bounds__(DK_THREADS)
 distill_kl_kernel(const float* __restrict__ scores, int64_t ld, int64_t rows, int64_t first_len, int64_t len_step,
                   DistillTargets tg, int n_targets, const int32_t* __restrict__ topk, int k_top, double* __restrict__ loss_out,
@@ -43,19 +46,65 @@ distill_kl_kernel(const float* __restrict__ scores, int64_t ld, int64_t rows, in
         const int count = T ? k_top : static_cast<int>(n);
         double row_loss = 0.0;
         if (!T) {
-            // ---- dense causal row: 128-bit loads; online max / sum-of-exponentials in one sweep
+            // ---- dense causal row, ONE sweep over the scores and all targets (128-bit loads). With lse = log sum exp(x):
+            //   KL(p || softmax(x)) = sum p log p - sum p x + lse * sum p,
+            // so a thread keeps the online (m, l) pair of the soft-max plus, per target, C = sum p log p,
+            // D = sum p (x - m) against its own running maximum m (when m moves to m', D += (m - m') * S) and S = sum p;
+            // the block then brings every thread to the row maximum and adds up. No second pass over the scores.
             const int nvec = static_cast<int>(n >> 2);
             const float4* I4 = reinterpret_cast<const float4*>(I);
+            for (int j0 = 0; j0 < n_targets; j0 += NT) {
+            const int nt = n_targets - j0 < NT ? n_targets - j0 : NT;     // targets of this sweep
             float m = -INFINITY, l = 0.f;
-            auto push = [&](float x) {
-                if (x > m) { l = l * __expf(m - x) + 1.f; m = x; } else { l += __expf(x - m); }
+            float C[NT], D[NT], S[NT];
+#pragma unroll
+            for (int j = 0; j < NT; ++j) C[j] = D[j] = S[j] = 0.f;
+            auto raise = [&](float x) {                    // the running maximum moves up to x
+                l *= __expf(m - x);                        // exp(-inf) = 0 for the first element
+                if (m > -INFINITY) {
+#pragma unroll
+                    for (int j = 0; j < NT; ++j)
+                        if (j < nt) D[j] += (m - x) * S[j];
+                }
+                m = x;
+            };
+            auto push4 = [&](const float4& x, const float4* pv) {
+                const float xm = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
+                if (xm > m) raise(xm);
+                const float d0 = x.x - m, d1 = x.y - m, d2 = x.z - m, d3 = x.w - m;
+                l += (__expf(d0) + __expf(d1)) + (__expf(d2) + __expf(d3));
+#pragma unroll
+                for (int j = 0; j < NT; ++j) {
+                    if (j < nt) {
+                        const float4 q = pv[j];
+                        if (q.x > 0.f) { C[j] += q.x * __logf(q.x); D[j] += q.x * d0; S[j] += q.x; }
+                        if (q.y > 0.f) { C[j] += q.y * __logf(q.y); D[j] += q.y * d1; S[j] += q.y; }
+                        if (q.z > 0.f) { C[j] += q.z * __logf(q.z); D[j] += q.z * d2; S[j] += q.z; }
+                        if (q.w > 0.f) { C[j] += q.w * __logf(q.w); D[j] += q.w * d3; S[j] += q.w; }
+                    }
+                }
             };
             for (int v = threadIdx.x; v < nvec; v += DK_THREADS) {
-                const float4 x = __ldg(I4 + v);
-                push(x.x); push(x.y); push(x.z); push(x.w);
+                float4 pv[NT];
+#pragma unroll
+                for (int j = 0; j < NT; ++j)
+                    if (j < nt) pv[j] = __ldg(reinterpret_cast<const float4*>(tg.p[j0 + j] + r * ld) + v);
+                push4(__ldg(I4 + v), pv);
             }
-            for (int i = 4 * nvec + threadIdx.x; i < n; i += DK_THREADS) push(__ldg(I + i));
-            // merge (m, l) pairs across the block
+            for (int i = 4 * nvec + threadIdx.x; i < n; i += DK_THREADS) {       // at most 3 elements of the row
+                const float x = __ldg(I + i);
+                if (x > m) raise(x);
+                const float d = x - m;
+                l += __expf(d);
+#pragma unroll
+                for (int j = 0; j < NT; ++j) {
+                    if (j < nt) {
+                        const float q = __ldg(tg.p[j0 + j] + r * ld + i);
+                        if (q > 0.f) { C[j] += q * __logf(q); D[j] += q * d; S[j] += q; }
+                    }
+                }
+            }
+            // row maximum, then every thread's sums relative to it
             float bm = m;
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) bm = fmaxf(bm, __shfl_xor_sync(0xFFFFFFFFu, bm, o));
@@ -65,18 +114,15 @@ distill_kl_kernel(const float* __restrict__ scores, int64_t ld, int64_t rows, in
 #pragma unroll
             for (int w = 0; w < DK_THREADS / 32; ++w) bm = fmaxf(bm, sh_m[w]);
             const double se = block_sum_f64(l > 0.f ? static_cast<double>(l * __expf(m - bm)) : 0.0, sh);
-            const float lse = bm + logf(static_cast<float>(se));
-            for (int j = 0; j < n_targets; ++j) {
-                const float4* P4 = reinterpret_cast<const float4*>(tg.p[j] + r * ld);
-                float acc = 0.f;
-                auto term = [&](float p, float x) { if (p > 0.f) acc += p * (__logf(p) - (x - lse)); };
-                for (int v = threadIdx.x; v < nvec; v += DK_THREADS) {
-                    const float4 pv = __ldg(P4 + v);
-                    const float4 x = __ldg(I4 + v);
-                    term(pv.x, x.x); term(pv.y, x.y); term(pv.z, x.z); term(pv.w, x.w);
-                }
-                for (int i = 4 * nvec + threadIdx.x; i < n; i += DK_THREADS) term(__ldg(tg.p[j] + r * ld + i), __ldg(I + i));
-                row_loss += block_sum_f64(static_cast<double>(acc), sh);
+            const double lse_rel = log(se);                                       // lse - bm
+#pragma unroll
+            for (int j = 0; j < NT; ++j) {
+                if (j >= nt) break;                        // block-uniform
+                // sum p log p - sum p (x - bm) + (lse - bm) * sum p
+                const double dj = m > -INFINITY ? static_cast<double>(D[j]) + static_cast<double>(m - bm) * static_cast<double>(S[j]) : 0.0;
+                const double part = static_cast<double>(C[j]) - dj + lse_rel * static_cast<double>(S[j]);
+                row_loss += block_sum_f64(part, sh);
+            }
             }
         } else {
             // ---- sparse-training form: the row's selected positions only
@@ -147,7 +193,11 @@ extern "C" idxc_status idxc_distill_kl(const float* scores, int64_t ld, int64_t 
         tg.p[j] = targets[j];
     }
     const unsigned grid = static_cast<unsigned>(rows < (1 << 20) ? rows : (1 << 20));
-    distill_kl_kernel<<<grid, DK_THREADS, 0, stream>>>(scores, ld, rows, first_len, len_step, tg, n_targets, topk, k_top, loss_out,
-                                                       row_loss_out);
+    auto launch = [&](auto kernel) {
+        kernel<<<grid, DK_THREADS, 0, stream>>>(scores, ld, rows, first_len, len_step, tg, n_targets, topk, k_top, loss_out, row_loss_out);
+    };
+    if (n_targets <= 1) launch(distill_kl_kernel<1>);
+    else if (n_targets <= 2) launch(distill_kl_kernel<2>);
+    else launch(distill_kl_kernel<4>);
     return cudaGetLastError() == cudaSuccess ? IDXC_OK : IDXC_ERR_CUDA;
 }

@@ -438,6 +438,13 @@ def test_distill_kl_matches_oracle():
     want, want_rows = odist.multi_layer_loss(scores.cpu().numpy(), [t.cpu().numpy() for t in targets])
     assert loss.item() == pytest.approx(want, rel=2e-5)
     assert np.allclose(rows.cpu().numpy(), want_rows, rtol=1e-4, atol=1e-6)
+    # more targets than one sweep holds in registers (groups of four), and a single one
+    more = targets + [targets[0].flip(0).contiguous() * 0 + targets[1], targets[2], targets[0]]
+    for tl in (more, targets[:1]):
+        loss_m, rows_m = idxc.distill_kl(scores, tl, want_rows=True)
+        want_m, want_rows_m = odist.multi_layer_loss(scores.cpu().numpy(), [t.cpu().numpy() for t in tl])
+        assert loss_m.item() == pytest.approx(want_m, rel=2e-5)
+        assert np.allclose(rows_m.cpu().numpy(), want_rows_m, rtol=1e-4, atol=1e-6)
     # sparse-training form on the indices the top-k kernel selected
     tk = torch.from_numpy(g_topk).to(DEV)
     loss_k, rows_k = idxc.distill_kl(scores, targets, topk=tk, want_rows=True)
