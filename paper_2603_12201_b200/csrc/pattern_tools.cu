@@ -1,7 +1,7 @@
 // Pattern tooling on index tensors (the paper's Appendix A, Appendix C and Algorithm 1).
 //   * overlap kernel: per query row |T_a n T_b| / (valid entries of T_a), for one pair of index tensors or
-//     for every pair of N layers in one launch. Both rows are ascending, so each element of one row is
-//     looked up in the other by binary search in shared memory. HBM-bound: 2 * 4 * k bytes per row pair.
+//     for every pair of N layers in one launch. Both rows are ascending: runs of one row are merged against the
+//     other in shared memory. 2 * 4 * k bytes per row pair (the pairs of a row run together: repeats hit the L2).
 //   * similarity DP (host): the exact pattern with M Full layers that maximises the summed similarity of
 //     the Shared layers to their source layers.
 //   * greedy layer selection (host): Algorithm 1 with the caller's loss function.
@@ -15,55 +15,67 @@ namespace {
 
 constexpr int OV_THREADS = 256;
 
-// grid.x: row blocks (grid-stride), grid.y: pair index. pairs[2p], pairs[2p+1]: layer indices of pair p.
+// grid.x: pair index (fastest, so that the pairs of one row run together and the row's index lists are read from HBM
+// once and from the L2 afterwards), grid.y: row blocks (grid-stride). pairs[2p], pairs[2p+1]: layer indices of pair p.
 // sums[p] accumulates the row ratios (double, atomicAdd); row_out (optional, single pair) gets each ratio.
+// Both rows are ascending: a thread takes a run of consecutive entries of T_a, finds where the run starts in T_b with
+// one binary search and then walks both lists together.
 __global__ void __launch_bounds__(OV_THREADS)
 overlap_kernel(const int32_t* const* __restrict__ layers, const int* __restrict__ pairs, int64_t rows, int k_top,
                double* __restrict__ sums, float* __restrict__ row_out) {
-    extern __shared__ int32_t sh[];                 // row of T_b, k_top entries
+    extern __shared__ int32_t sh[];                 // row of T_b, then row of T_a: k_top entries each
+    int32_t* sb = sh;
+    int32_t* sa = sh + k_top;
     __shared__ int warp_cnt[OV_THREADS / 32];
-    __shared__ int valid_b_s;
-    const int p = blockIdx.y;
+    __shared__ int valid_s[2];
+    const int p = blockIdx.x;
     const int32_t* Ta = layers[pairs[2 * p]];
     const int32_t* Tb = layers[pairs[2 * p + 1]];
+    const int run = (k_top + OV_THREADS - 1) / OV_THREADS;      // entries of T_a per thread
     double local_sum = 0.0;
-    for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
+    for (int64_t r = blockIdx.y; r < rows; r += gridDim.y) {
         const int32_t* a = Ta + r * k_top;
         const int32_t* b = Tb + r * k_top;
         __syncthreads();
-        if (threadIdx.x == 0) valid_b_s = 0;
+        if (threadIdx.x < 2) valid_s[threadIdx.x] = 0;
         __syncthreads();
-        int nb_local = 0;
+        int na_local = 0, nb_local = 0;
         for (int i = threadIdx.x; i < k_top; i += OV_THREADS) {
-            const int32_t v = __ldg(b + i);
-            sh[i] = v;
-            nb_local += v >= 0;
+            const int32_t vb = __ldg(b + i), va = __ldg(a + i);
+            sb[i] = vb;
+            sa[i] = va;
+            nb_local += vb >= 0;
+            na_local += va >= 0;
         }
-        if (nb_local) atomicAdd(&valid_b_s, nb_local);
+        if (na_local) atomicAdd(&valid_s[0], na_local);
+        if (nb_local) atomicAdd(&valid_s[1], nb_local);
         __syncthreads();
-        const int nb = valid_b_s;                   // valid entries come first (padding is at the end)
-        int hits = 0, valid_a = 0;
-        for (int i = threadIdx.x; i < k_top; i += OV_THREADS) {
-            const int32_t v = __ldg(a + i);
-            if (v < 0) continue;
-            ++valid_a;
-            int lo = 0, hi = nb;                    // first position with sh[pos] >= v
+        const int na = valid_s[0], nb = valid_s[1];  // valid entries come first (padding is at the end)
+        int hits = 0;
+        const int i0 = threadIdx.x * run;
+        const int i1 = i0 + run < na ? i0 + run : na;
+        if (i0 < i1) {
+            const int32_t first = sa[i0];
+            int lo = 0, hi = nb;                      // first position with sb[pos] >= first
             while (lo < hi) {
                 const int mid = (lo + hi) >> 1;
-                if (sh[mid] < v) lo = mid + 1; else hi = mid;
+                if (sb[mid] < first) lo = mid + 1; else hi = mid;
             }
-            hits += (lo < nb && sh[lo] == v);
+            int j = lo;
+            for (int i = i0; i < i1 && j < nb; ++i) {
+                const int32_t v = sa[i];
+                while (j < nb && sb[j] < v) ++j;
+                hits += (j < nb && sb[j] == v);
+            }
         }
-        int packed = hits | (valid_a << 16);        // both <= 2048
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) packed += __shfl_xor_sync(0xFFFFFFFFu, packed, o);
-        if ((threadIdx.x & 31) == 0) warp_cnt[threadIdx.x >> 5] = packed;
+        for (int o = 16; o > 0; o >>= 1) hits += __shfl_xor_sync(0xFFFFFFFFu, hits, o);
+        if ((threadIdx.x & 31) == 0) warp_cnt[threadIdx.x >> 5] = hits;
         __syncthreads();
         if (threadIdx.x == 0) {
-            int tot = 0;
-            for (int w = 0; w < OV_THREADS / 32; ++w) tot += warp_cnt[w];
-            const int h = tot & 0xFFFF, va = tot >> 16;
-            const double ratio = va ? static_cast<double>(h) / va : 0.0;
+            int h = 0;
+            for (int w = 0; w < OV_THREADS / 32; ++w) h += warp_cnt[w];
+            const double ratio = na ? static_cast<double>(h) / na : 0.0;
             local_sum += ratio;
             if (row_out) row_out[r] = static_cast<float>(ratio);
         }
@@ -76,9 +88,9 @@ overlap_kernel(const int32_t* const* __restrict__ layers, const int* __restrict_
 cudaError_t launch_overlap(const int32_t* const* layers_dev, const int* pairs_dev, int n_pairs, int64_t rows, int k_top,
                            double* sums_dev, float* row_out, cudaStream_t stream) {
     if (n_pairs <= 0 || rows <= 0) return cudaSuccess;
-    const unsigned gx = static_cast<unsigned>(rows < 4096 ? rows : 4096);
-    dim3 grid(gx, static_cast<unsigned>(n_pairs));
-    overlap_kernel<<<grid, OV_THREADS, k_top * sizeof(int32_t), stream>>>(layers_dev, pairs_dev, rows, k_top, sums_dev, row_out);
+    const unsigned gy = static_cast<unsigned>(rows < 4096 ? rows : 4096);
+    dim3 grid(static_cast<unsigned>(n_pairs), gy);
+    overlap_kernel<<<grid, OV_THREADS, 2 * k_top * sizeof(int32_t), stream>>>(layers_dev, pairs_dev, rows, k_top, sums_dev, row_out);
     return cudaGetLastError();
 }
 
