@@ -15,19 +15,20 @@
 //           the unswizzled K-major operand layout, so one bulk copy per tile brings it back (four tiles ahead, into
 //           the shared memory that held Q) and the PV MMAs read it there: no thread touches P in pass 2. The softmax
 //           warps note in pass 1 which tiles moved a reference maximum; only those tiles wait for them in pass 2.
-// Tensor memory (512 columns): O half of pass 1 [0,256), that of pass 2 [256,512) | S double-buffered [256,320), [320,384); in pass 1 P overwrites the
-//   first 32 columns of its S buffer as bf16 pairs and is the A operand of the PV MMAs | Q blocks 0..3 (of 9 blocks
+// Tensor memory (512 columns): O half of pass 1 [0,256) | S double-buffered [256,320), [320,384); in pass 1 P overwrites
+//   the first 32 columns of its S buffer as bf16 pairs and is the A operand of the PV MMAs | Q blocks 0..3 (of 9 blocks
 //   of 64 columns) as bf16 pairs [384,512), the A operand of their score MMAs; Q blocks 4..8 stay in shared memory.
+//   Pass 2 accumulates its half of O in [256,512): S and Q are not needed then, and pass 1's half can still be read out.
 // Shared memory: 2 stages x 9 blocks of [64 gathered rows x 128 B] (128-byte swizzle) | 5 blocks of Q
 //   [128 rows x 128 B]. A block of gathered rows is at once the K-major B operand of S (rows = keys) and the
 //   MN-major B operand of P V (64 contiguous value columns). A stage is two slots with their own barriers:
 //   "V" = blocks 0..3 (needed until the PV product) and "E" = blocks 4..8 (free again once the scores are
 //   done), so the next tile's E part is gathered while this tile is still in its softmax. Pass 2 uses the four
 //   slots as a ring of four value tiles.
-// Warps (16; three idle): 0 MMA issuer (warp-uniform, one elected lane issues; order S(i+1) blocks 4..8 | P(i) V(i) | S(i+1)
-//   blocks 0..3), 4 Q loader (TMA) and, in pass 2, loader of the saved P, eight row-gather warps (16-byte cp.async into the swizzled layout; two warps per
-//   slot, each slot its own acquire/copy/publish stream), 12-15 softmax (running reference maximum with a lazy
-//   rescale of O, only when the maximum grows by more than 2^8).
+// Warps (16; three idle): 0 MMA issuer (warp-uniform, one elected lane issues; order S(i+1) blocks 4..8 | P(i) V(i) |
+//   S(i+1) blocks 0..3), 4 Q loader (TMA) and, in pass 2, loader of the saved P, eight row-gather warps (16-byte
+//   cp.async into the swizzled layout; two warps per slot, each slot its own acquire/copy/publish stream), 12-15
+//   softmax (running reference maximum with a lazy rescale of O, only when the maximum grows by more than 2^8).
 // The hot loops are rolled on purpose: with everything unrolled the kernel was 150 KB of code and every role
 // stalled on instruction fetch.
 // Entries < 0 or pointing outside the cache are skipped; a query's tiles end at its last usable entry
