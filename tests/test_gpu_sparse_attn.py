@@ -192,3 +192,19 @@ def test_more_tiles_than_rescale_flags():
     topk = torch.randint(0, n_kv, (n_q, k_top), generator=g, dtype=torch.int32).cuda()
     topk[1, 16400:] = -1                                    # ends inside the tiles beyond the flags
     _run(inp, topk, 0.3, rows=[0, 1, 63], h=h, what="259 tiles")
+
+
+def test_repeated_calls_give_identical_bits():
+    # the result does not depend on timing between the roles of the kernel (gather, MMA, softmax, loaders): twenty calls
+    # on the same inputs, prefill-style and split (decode-style), agree bit for bit
+    for n_q, k_top in ((300, 1024), (24, 2048)):
+        n_kv = 6000
+        inp = synth.attention_inputs(n_q, n_kv, H, D_QK, seed=31, device="cuda")
+        g = torch.Generator().manual_seed(31 + n_q)
+        topk = torch.randint(0, n_kv, (n_q, k_top), generator=g, dtype=torch.int32).cuda()
+        topk[::5, k_top // 2:] = -1
+        ref, ref_lse = binding.sparse_attention(inp.q, inp.kv, topk, D_V, 0.2)
+        for _ in range(20):
+            out, lse = binding.sparse_attention(inp.q, inp.kv, topk, D_V, 0.2)
+            assert torch.equal(out, ref) and torch.equal(lse, ref_lse)
+        binding.poll_device_status()
