@@ -41,6 +41,8 @@ typedef enum { IDXC_BF16 = 0, IDXC_FP8_E4M3 = 1 } idxc_dtype;
 /* flags (bitwise or) */
 #define IDXC_FLAG_COPY_SHARED 0x1u  /* schedule: S layers copy the cached indices into topk_buf instead of aliasing */
 #define IDXC_FLAG_SIMT_SCORER 0x2u  /* debugging aid: score with the plain CUDA-core kernel instead of tcgen05     */
+#define IDXC_FLAG_FILL_MASKED 0x4u  /* prefill with scores_out: entries s > t of every row, up to column L_k - 1, are set
+                                       to -infinity (the causal mask as a soft-max expects it) instead of left untouched */
 
 /* Limits checked before any launch. */
 #define IDXC_MAX_K_TOP 2048
@@ -65,7 +67,8 @@ const char* idxc_status_string(idxc_status s);
  *   w        [q_len, H_I] fp32
  *   q_scale  [q_len] fp32, k_scale [L_k] fp32: IDXC_FP8_E4M3 only, else NULL
  *   scores_out  NULL, or [q_len, ld_scores] fp32 (ld_scores >= L_k, a multiple of 4;
- *               base 16-byte aligned). Only entries s <= t are written.
+ *               base 16-byte aligned). Only entries s <= t are written (IDXC_FLAG_FILL_MASKED: the other entries of the
+ *               row up to column L_k - 1 are set to -infinity).
  *   topk_out    NULL, or [q_len, k_top] int32
  *   workspace   at least idxc_prefill_workspace_bytes(...) bytes, 256-byte aligned;
  *               contents are scratch. With scores_out == NULL the scores go through it

@@ -78,7 +78,7 @@ idxc_status check_common(int H, int d, int k_top, idxc_dtype dt, uint32_t flags)
     if (dt != IDXC_BF16 && dt != IDXC_FP8_E4M3) return IDXC_ERR_INVALID_ARG;
     if (k_top < 1 || k_top > IDXC_MAX_K_TOP) return IDXC_ERR_INVALID_ARG;
     if (H < 1 || H > IDXC_MAX_HEADS || d < 1) return IDXC_ERR_INVALID_ARG;
-    if (flags & ~(IDXC_FLAG_COPY_SHARED | IDXC_FLAG_SIMT_SCORER)) return IDXC_ERR_INVALID_ARG;
+    if (flags & ~(IDXC_FLAG_COPY_SHARED | IDXC_FLAG_SIMT_SCORER | IDXC_FLAG_FILL_MASKED)) return IDXC_ERR_INVALID_ARG;
     if (!(flags & IDXC_FLAG_SIMT_SCORER) && !score_tc_supported(H, d, dt == IDXC_FP8_E4M3)) return IDXC_ERR_UNSUPPORTED;
     return IDXC_OK;
 }
@@ -202,7 +202,13 @@ idxc_status idxc_indexer_prefill(const void* q, const void* k, const float* w, c
         return IDXC_OK;
     };
 
-    if (scores_out) return run_rows(0, q_len, scores_out, ld_scores);
+    if (scores_out) {
+        if (flags & IDXC_FLAG_FILL_MASKED) {                   // disjoint from what the scorer writes: any order
+            g_launches += 1;
+            if (launch_fill_masked(scores_out, ld_scores, q_begin, q_len, L_k, stream) != cudaSuccess) return IDXC_ERR_CUDA;
+        }
+        return run_rows(0, q_len, scores_out, ld_scores);
+    }
 
     // scores go through the workspace in query chunks
     const int64_t ld = round_up(q_begin + q_len, 32);

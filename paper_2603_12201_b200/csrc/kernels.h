@@ -45,6 +45,8 @@ struct ScoreArgs {
 
 // Plain CUDA-core scorer (scorer_simt.cu): debugging aid and cross-check.
 cudaError_t launch_score_simt(const ScoreArgs& a, cudaStream_t stream);
+// -inf into columns q_begin + r + 1 .. n_cols - 1 of every row r (the causal mask, IDXC_FLAG_FILL_MASKED).
+cudaError_t launch_fill_masked(float* scores, int64_t ld, int64_t q_begin, int64_t n_rows, int64_t n_cols, cudaStream_t stream);
 
 // tcgen05 scorers (scorer_tc.cu). `status` is the device status word. The tensor maps are
 // encoded by the caller: q as [n_rows*H, d] and k as [k_rows, d], 128-byte swizzle, inner

@@ -47,7 +47,38 @@ score_simt_kernel(ScoreArgs a) {
     a.scores[r * a.ld + s] = I;
 }
 
+// Causal mask for callers that read whole rows (IDXC_FLAG_FILL_MASKED): row r of `scores` gets -inf in columns
+// q_begin + r + 1 .. n_cols - 1. One CTA per row, 4-byte stores up to the next 16-byte boundary, then 16-byte stores.
+__global__ void __launch_bounds__(256)
+fill_masked_kernel(float* __restrict__ scores, int64_t ld, int64_t q_begin, int64_t n_cols) {
+    const int64_t r = blockIdx.x;
+    float* row = scores + r * ld;
+    const int64_t c0 = q_begin + r + 1;
+    if (c0 >= n_cols) return;
+    const int64_t a0 = (c0 + 3) & ~int64_t(3);                 // rows start 16-byte aligned and ld is a multiple of 4
+    const int64_t a1 = n_cols & ~int64_t(3);
+    const float ninf = -INFINITY;
+    if (a0 >= a1) {
+        for (int64_t c = c0 + threadIdx.x; c < n_cols; c += blockDim.x) row[c] = ninf;
+        return;
+    }
+    for (int64_t c = c0 + threadIdx.x; c < a0; c += blockDim.x) row[c] = ninf;
+    const float4 v = make_float4(ninf, ninf, ninf, ninf);
+    for (int64_t c = a0 + 4 * static_cast<int64_t>(threadIdx.x); c < a1; c += 4 * static_cast<int64_t>(blockDim.x))
+        *reinterpret_cast<float4*>(row + c) = v;
+    for (int64_t c = a1 + threadIdx.x; c < n_cols; c += blockDim.x) row[c] = ninf;
+}
+
 }  // namespace
+
+cudaError_t launch_fill_masked(float* scores, int64_t ld, int64_t q_begin, int64_t n_rows, int64_t n_cols, cudaStream_t stream) {
+    for (int64_t r0 = 0; r0 < n_rows; r0 += (int64_t(1) << 30)) {
+        const int64_t nr = n_rows - r0 < (int64_t(1) << 30) ? n_rows - r0 : (int64_t(1) << 30);
+        fill_masked_kernel<<<static_cast<unsigned>(nr), 256, 0, stream>>>(scores + r0 * ld, ld, q_begin + r0, n_cols);
+        if (cudaError_t e = cudaGetLastError(); e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
 
 cudaError_t launch_score_simt(const ScoreArgs& a, cudaStream_t stream) {
     if (a.n_rows <= 0) return cudaSuccess;

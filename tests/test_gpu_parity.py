@@ -179,6 +179,30 @@ def test_prefill_duplicate_keys_pick_lowest_index_and_gate():
         assert t2[t, :kk].tolist() == list(range(kk))
 
 
+def test_prefill_fill_masked_writes_the_causal_mask():
+    # IDXC_FLAG_FILL_MASKED: s > t becomes -inf up to column L_k - 1, the scores s <= t and the columns beyond L_k stay
+    # as they are; chunked calls (q_begin > 0) mask relative to the absolute position
+    L, H, d, k_top = 333, 16, 64, 16
+    inp = _to_dev(synth.prefill_inputs(L, H, d, seed=12))
+    ld = 352
+    plain = torch.full((L, ld), 7.0, device=DEV)
+    idxc.indexer_prefill(inp.q, inp.k, inp.w, k_top, scores_out=plain)
+    filled = torch.full((L, ld), 7.0, device=DEV)
+    idxc.indexer_prefill(inp.q, inp.k, inp.w, k_top, scores_out=filled, flags=idxc.FLAG_FILL_MASKED)
+    t = torch.arange(L, device=DEV)[:, None]
+    s_ = torch.arange(ld, device=DEV)[None, :]
+    causal, masked, beyond = s_ <= t, (s_ > t) & (s_ < L), s_ >= L
+    assert torch.equal(filled[causal.expand(L, ld)], plain[causal.expand(L, ld)])
+    assert bool(torch.isneginf(filled[masked.expand(L, ld)]).all())
+    assert bool((filled[beyond.expand(L, ld)] == 7.0).all()) and bool((plain[masked.expand(L, ld)] == 7.0).all())
+    q0, q1 = 100, 230
+    part = torch.full((q1 - q0, ld), 7.0, device=DEV)
+    idxc.indexer_prefill(inp.q[q0:q1], inp.k, inp.w[q0:q1], k_top, q_begin=q0, scores_out=part, flags=idxc.FLAG_FILL_MASKED)
+    assert torch.equal(part, filled[q0:q1])
+    # the masked rows feed a soft-max directly
+    assert bool(torch.isfinite(torch.softmax(filled[:, :L], dim=1)).all())
+
+
 def test_prefill_rejects_bad_arguments():
     inp = _to_dev(synth.prefill_inputs(64, 16, 64, seed=1))
     topk = torch.empty((64, 8), dtype=torch.int32, device=DEV)
