@@ -312,6 +312,29 @@ def time_layer_loop(idxc, synth, dev, L, k_top, n_layers, every, seed):
             "note": "the paper's end-to-end figures (1.82x prefill at 200K) include an FP8 indexer and the rest of the model; context only"}
 
 
+def measure_fp8_gemm_peak(dev):
+    """A denominator for the FP8 lines only (MEASURED_PEAKS.json holds no FP8 figure): the library's e4m3 GEMM,
+    8192^3, best of 10 by CUDA events. None if this torch build has no such GEMM. Not on any timed path."""
+    try:
+        n = 8192
+        a = torch.randn(n, n, device=dev).to(torch.float8_e4m3fn)
+        b = torch.randn(n, n, device=dev).to(torch.float8_e4m3fn).t()
+        one = torch.tensor(1.0, device=dev)
+        for _ in range(3):
+            torch._scaled_mm(a, b, scale_a=one, scale_b=one, out_dtype=torch.bfloat16)
+        best = float("inf")
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            torch._scaled_mm(a, b, scale_a=one, scale_b=one, out_dtype=torch.bfloat16)
+            e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        return 2.0 * n ** 3 / (best * 1e-3) / 1e12
+    except Exception:
+        return None
+
+
 def time_fp8_chunked(idxc, synth, dev, peaks, L, chunk, H, d, k_top, seed, decode_B):
     """Config-5 shape: one Full layer of FP8 (e4m3 + per-token scales) chunked prefill, query chunks of
     `chunk` rows against the full causal K, then one decode step at batch `decode_B` on caches of length L."""
@@ -361,6 +384,10 @@ def time_fp8_chunked(idxc, synth, dev, peaks, L, chunk, H, d, k_top, seed, decod
            "ms_scorer": t_sc, "ms_topk": t_tk, "scorer_tflops": flops / (t_sc * 1e-3) / 1e12,
            "scorer_frac_of_2x_bf16_peak": flops / (t_sc * 1e-3) / 1e12 / (2 * peaks["bf16_tflops"]),
            "fp8_peak_note": "no measured FP8 peak on this pool: 2 x measured bf16 burst peak (nominal ratio)"}
+    fp8_peak = measure_fp8_gemm_peak(dev)
+    if fp8_peak:
+        out["fp8_gemm_peak_measured_here_tflops"] = fp8_peak
+        out["scorer_frac_of_fp8_gemm_peak_measured_here"] = out["scorer_tflops"] / fp8_peak
     # decode step on caches of length L
     x = synth.decode_inputs(decode_B, H, d, L, L, seed=seed, device=dev, layer=1, fp8=True, lens=[L] * decode_B)
     x.k_cache[:L] = inp.k
