@@ -173,52 +173,62 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
             if (!ok) give_up(abort_flag, p.status, DEV_TIMEOUT_PRODUCER);
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            // ------------------------------------------------------------ MMA issuer
-            int stage = 0;
-            uint32_t k_phase = 0, q_phase = 0;
-            uint32_t acc_phase[2] = {0u, 0u};
-            bool ok = true;
-            for (int64_t rho = 0; ok; ++rho) {
-                const int64_t item = item_of_round(rho);
-                if (item < 0) break;
-                const int nkt = key_tiles_of_item(item);
-                for (int kt = 0; kt < nkt && ok; ++kt) {
-                    ok = mbar_wait(bar_k_full + 8 * stage, k_phase, abort_flag);
-                    if (!ok) break;
-                    for (int half = 0; half < 2; ++half) {
-                        if (kt == 0) {
-                            ok = mbar_wait(bar_q_full + 8 * half, q_phase, abort_flag);
-                            if (!ok) break;
-                        }
-                        ok = mbar_wait(bar_acc_empty + 8 * half, acc_phase[half] ^ 1u, abort_flag);
+        // ---------------------------------------------------------------- MMA issuer
+        // The whole warp runs this role with uniform control flow and one elected lane issues; descriptors are a base
+        // plus 16-byte units.
+        int stage = 0;
+        uint32_t k_phase = 0, q_phase = 0;
+        uint32_t acc_phase[2] = {0u, 0u};
+        bool ok = true;
+        const uint64_t a_desc0 = umma_smem_desc_sw128(smem_u32(k_smem));
+        const uint64_t b_desc0 = umma_smem_desc_sw128(smem_u32(q_smem));
+        auto wait_bar = [&](uint32_t bar, uint32_t parity) -> bool {
+            return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort_flag));
+        };
+        for (int64_t rho = 0; ok; ++rho) {
+            const int64_t item = item_of_round(rho);
+            if (item < 0) break;
+            const int nkt = key_tiles_of_item(item);
+            for (int kt = 0; kt < nkt && ok; ++kt) {
+                ok = wait_bar(bar_k_full + 8 * stage, k_phase);
+                if (!ok) break;
+                const uint64_t a_stage = a_desc0 + static_cast<uint64_t>(stage * NKH * kKRegionBytes / 16);
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    if (kt == 0) {
+                        ok = wait_bar(bar_q_full + 8 * half, q_phase);
                         if (!ok) break;
-                        acc_phase[half] ^= 1u;
-                        tcgen05_fence_after_sync();
-                        const uint32_t d_tmem = tmem_base + half * kTileCols;
+                    }
+                    ok = wait_bar(bar_acc_empty + 8 * half, acc_phase[half] ^ 1u);
+                    if (!ok) break;
+                    acc_phase[half] ^= 1u;
+                    tcgen05_fence_after_sync();
+                    const uint32_t d_tmem = tmem_base + half * kTileCols;
+                    const uint64_t b_half = b_desc0 + static_cast<uint64_t>(half * NKH * kQRegionBytes / 16);
 #pragma unroll
-                        for (int kh = 0; kh < NKH; ++kh) {
-                            const uint32_t a_base = smem_u32(k_smem + (stage * NKH + kh) * kKRegionBytes);
-                            const uint32_t b_base = smem_u32(q_smem + (half * NKH + kh) * kQRegionBytes);
+                    for (int kh = 0; kh < NKH; ++kh) {
 #pragma unroll
-                            for (int ks = 0; ks < 4; ++ks) {   // 32 bytes of K per MMA: 16 bf16 or 32 fp8
-                                const uint64_t a_desc = umma_smem_desc_sw128(a_base + ks * 32);
-                                const uint64_t b_desc = umma_smem_desc_sw128(b_base + ks * 32);
-                                if constexpr (FP8) umma_f8(d_tmem, a_desc, b_desc, kIdesc, (kh | ks) != 0);
-                                else umma_f16(d_tmem, a_desc, b_desc, kIdesc, (kh | ks) != 0);
+                        for (int ks = 0; ks < 4; ++ks) {   // 32 bytes of K per MMA: 16 bf16 or 32 fp8
+                            const uint64_t a = a_stage + (kh * kKRegionBytes + ks * 32) / 16, b = b_half + (kh * kQRegionBytes + ks * 32) / 16;
+                            if constexpr (FP8) {
+                                if ((kh | ks) != 0) umma_f8_elect<true>(d_tmem, a, b, kIdesc);
+                                else umma_f8_elect<false>(d_tmem, a, b, kIdesc);
+                            } else {
+                                if ((kh | ks) != 0) umma_f16_elect<true>(d_tmem, a, b, kIdesc);
+                                else umma_f16_elect<false>(d_tmem, a, b, kIdesc);
                             }
                         }
-                        umma_commit(bar_acc_full + 8 * half);
-                        if (kt == nkt - 1) umma_commit(bar_q_empty + 8 * half);
                     }
-                    if (!ok) break;
-                    umma_commit(bar_k_empty + 8 * stage);
-                    if (++stage == kStages) { stage = 0; k_phase ^= 1u; }
+                    umma_commit_elect(bar_acc_full + 8 * half);
+                    if (kt == nkt - 1) umma_commit_elect(bar_q_empty + 8 * half);
                 }
-                q_phase ^= 1u;
+                if (!ok) break;
+                umma_commit_elect(bar_k_empty + 8 * stage);
+                if (++stage == kStages) { stage = 0; k_phase ^= 1u; }
             }
-            if (!ok) give_up(abort_flag, p.status, DEV_TIMEOUT_MMA);
+            q_phase ^= 1u;
         }
+        if (!ok && lane == 0) give_up(abort_flag, p.status, DEV_TIMEOUT_MMA);
     } else if (warp >= kEpilogueWarp0) {
         // ---------------------------------------------------------------- epilogue
         // TMEM is read with the 16x256b shape: a thread owns 4 keys (TMEM lanes g, g+8, g+16, g+24 of
