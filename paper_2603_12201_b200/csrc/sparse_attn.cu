@@ -158,7 +158,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
     const uint32_t bar_s_full = smem_u32(bars + 11);          // [2] S buffers
     const uint32_t bar_p_ready = smem_u32(bars + 13);         // [4] pass 1 uses two (P in its S buffer); pass 2: rescales of tile i replayed, ring of four
     const uint32_t bar_p_free = smem_u32(bars + 17);          // [4] pass 2: the PV product has read P ring buffer b
-    const uint32_t bar_o_full = smem_u32(bars + 21);
+    const uint32_t bar_o_full = smem_u32(bars + 21);          // pass 1's half of O is complete
     const uint32_t bar_o_free = smem_u32(bars + 22);
     const uint32_t bar_pv_done = smem_u32(bars + 23);         // one phase per PV tile
     uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(bars + 24);
@@ -169,7 +169,11 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
     // bit i: some row's reference maximum moved at tile i of the current query (O must be rescaled before PV(i))
     volatile uint32_t* resc_mask = reinterpret_cast<volatile uint32_t*>(bars + 32);   // [kSaFlagTiles / 32]
     const uint32_t bar_resc_go = smem_u32(bars + 36);         // pass 2: every PV product before a flagged tile is complete
-    static_assert(37 * 8 <= kSaBarBytes && kSaFlagTiles / 8 <= 32, "barrier area");
+    // Pass 2's half of O is complete. A barrier of its own: pass 2 does not wait for the softmax warps (unless a tile is
+    // flagged), so with few tiles it can end before a warp has even looked at pass 1's completion; on one barrier that
+    // warp would find the phase it waits for two completions back, which a parity wait cannot tell from "not yet".
+    const uint32_t bar_o2_full = smem_u32(bars + 37);
+    static_assert(38 * 8 <= kSaBarBytes && kSaFlagTiles / 8 <= 32, "barrier area");
     auto tile_rescales = [&](int i) -> bool { return i > 0 && (i >= kSaFlagTiles || ((resc_mask[i >> 5] >> (i & 31)) & 1u)); };
 
     const int warp = threadIdx.x >> 5;
@@ -197,6 +201,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
         mbar_init(bar_p2_go, 4);
         mbar_init(bar_resc_go, 1);
         mbar_init(bar_o_full, 1);
+        mbar_init(bar_o2_full, 1);
         mbar_init(bar_o_free, 4);
         mbar_init(bar_pv_done, 1);
         *abort_flag = 0u;
@@ -349,7 +354,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
                 umma_commit_elect(bar_slot_empty + 8 * slot);
                 umma_commit_elect(bar_p_free + 8 * slot);
                 umma_commit_elect(bar_pv_done);
-                if (i == nt - 1) umma_commit_elect(bar_o_full);
+                if (i == nt - 1) umma_commit_elect(bar_o2_full);
                 else if (tile_rescales(i + 1)) umma_commit_elect(bar_resc_go);   // tells the softmax warps when O may be rescaled
             }
             if (ok) umma_commit_elect(bar_q_empty);
@@ -527,8 +532,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
         // staging use) and stores 8 rows x 64 contiguous bytes per instruction.
         uint8_t* const stg = stage_smem + 8 * kSaKBlockBytes + quarter * 2048;     // [32 rows][64 B], 16-byte chunks XORed by (row >> 1) & 3
         auto write_out = [&](__nv_bfloat16* dst_query, float* part_row, float inv, uint32_t col0, bool last) -> bool {   // dst_query: row 0 of the query, first column of the half
-            if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar_o_full, ph_o_full, abort_flag))) return false;
-            ph_o_full ^= 1u;
+            // each of the two barriers completes once per query: the phase flips after the second half
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait(last ? bar_o2_full : bar_o_full, ph_o_full, abort_flag))) return false;
+            if (last) ph_o_full ^= 1u;
             tcgen05_fence_after_sync();
 #pragma unroll 1
             for (int c = 0; c < 8; ++c) {

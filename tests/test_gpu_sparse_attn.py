@@ -208,3 +208,25 @@ def test_repeated_calls_give_identical_bits():
             out, lse = binding.sparse_attention(inp.q, inp.kv, topk, D_V, 0.2)
             assert torch.equal(out, ref) and torch.equal(lse, ref_lse)
         binding.poll_device_status()
+
+
+def test_few_tiles_per_cta_after_unrelated_calls():
+    # Split mode with one to four tiles per CTA: the second pass can finish before a softmax warp has looked at the first
+    # pass's completion (regression: both completions once shared a barrier and the late warp waited for ever). Calls
+    # with full-head queries in between leave different leftovers in shared memory for the 112 head rows this call does
+    # not load, which varies the timing of its warps.
+    h, B = 16, 5
+    lens = [700, 64, 2100, 1, 300]
+    offs = np.concatenate([[0], np.cumsum([((n + 127) // 128) * 128 for n in lens])[:-1]])
+    n_kv = int(offs[-1] + lens[-1])
+    inp = synth.attention_inputs(B, n_kv, h, D_QK, seed=14, device="cuda")
+    topk = synth.random_selection([n - 1 for n in lens], 2048, seed=14, device="cuda")
+    base = torch.as_tensor(offs, dtype=torch.int64, device="cuda")
+    other = synth.attention_inputs(148, 4096, H, D_QK, seed=15, device="cuda")
+    other_topk = torch.randint(0, 4096, (148, 256), generator=torch.Generator().manual_seed(15), dtype=torch.int32).cuda()
+    ref, ref_lse = binding.sparse_attention(inp.q, inp.kv, topk, D_V, 0.06, kv_base=base)
+    for _ in range(150):
+        binding.sparse_attention(other.q, other.kv, other_topk, D_V, 0.05)
+        out, lse = binding.sparse_attention(inp.q, inp.kv, topk, D_V, 0.06, kv_base=base)
+        assert torch.equal(out, ref) and torch.equal(lse, ref_lse)
+    binding.poll_device_status()
