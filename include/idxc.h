@@ -75,7 +75,7 @@ const char* idxc_status_string(idxc_status s);
  *               in query chunks, so its size does not grow with q_len beyond a cap.
  * A full prefill is q_begin = 0, q_len = L_k = L; chunked prefill calls this once
  * per chunk with the full K and gives the same rows.
- * Supported: d_I in {64, 128}; H_I in {16, 32, 64}; 1 <= k_top <= 2048;
+ * Supported: d_I in {64, 128}; H_I in {16, 32, 64}; 1 <= k_top <= 2048; q_len * H_I < 2^31;
  * q, k, w 16-byte aligned. Other sizes return IDXC_ERR_UNSUPPORTED / INVALID_ARG
  * before anything is launched.
  * ------------------------------------------------------------------------- */
@@ -125,13 +125,18 @@ idxc_status idxc_indexer_decode(const void* q_step, const void* k_cache, int64_t
  * afford the device-wide stall of cudaMalloc / cudaFree.)
  * Same operation, arguments and rules as idxc_indexer_decode with scores_out == NULL, but the
  * fp32 score scratch lives in an array built into the library (IDXC_NOALLOC_SCRATCH_BYTES on
- * every GPU that loads the library, until the process exits) instead of a workspace. The call
- * allocates nothing on host or device. Limits and behaviour:
+ * every GPU this entry point is used on, until the process exits) instead of a workspace.
+ * Limits and behaviour:
+ *   - FIRST CALL ON A DEVICE: CUDA creates a library's device data lazily, so the array comes into
+ *     being when the first call on a device looks its address up. That call makes the driver set
+ *     aside the IDXC_NOALLOC_SCRATCH_BYTES (it fails with IDXC_ERR_CUDA if the device has no room
+ *     left) and sets up per-kernel attributes. Make it once per device at start-up -- a warm-up
+ *     step on small inputs is enough -- BEFORE the host gives the remaining HBM to its cache pool
+ *     and before any stream capture, with that device current. Every later call on the device,
+ *     whatever its shape or dtype, allocates nothing on the device or on the host.
  *   - B * round_up(max_len, 32) * 4 bytes must not exceed IDXC_NOALLOC_SCRATCH_BYTES (e.g.
  *     B = 32 sequences of up to 131072 keys); larger requests return IDXC_ERR_WORKSPACE and
  *     launch nothing. topk_out is required.
- *   - The first call on each device looks up the array's device address (that device must be
- *     current); make that first call before starting any stream capture.
  *   - Every call shares the one array. Calls whose kernels can overlap on the GPU (different
  *     streams without an ordering between them) race and return unspecified indices; calls on
  *     one stream, or ordered by events, are safe. The array keeps the previous call's scores

@@ -6,12 +6,15 @@ SparseAttn_l(X, T^(l)). The paper instantiates it under Multi-head Latent Attent
 reading taken here is the textbook definition restricted to the selected set, in the multi-query form MLA
 serves in: every head h of query t attends the same latent rows,
 
-    s[t,h,j] = scale * < q[t,h,:], kv[base_t + T_t[j], 0:d_qk] >            for the valid entries T_t[j] >= 0
+    s[t,h,j] = scale * < q[t,h,:], kv[base_t + T_t[j], 0:d_qk] >            for the usable entries of T_t
     p[t,h,:] = Softmax_j(s[t,h,:])
     out[t,h,:] = sum_j p[t,h,j] * kv[base_t + T_t[j], 0:d_v]                 (values = leading d_v columns of the row)
     lse[t,h]   = log sum_j exp(s[t,h,j])
 
-computed in float64 from the bf16 bit patterns. A query without any valid entry gets out = 0, lse = -inf.
+computed in float64 from the bf16 bit patterns. An entry is usable when T_t[j] >= 0 and the cache row it names,
+base_t + T_t[j], exists (lies in [0, n_kv)); the other entries are padding and take no part (reading taken: the paper
+only ever forms T_t from cached positions, so an entry that names no row selects nothing). A query without any usable
+entry gets out = 0, lse = -inf.
 Nothing here is blocked, fused or reordered: gather, one matrix product, a softmax, one matrix product.
 """
 from __future__ import annotations
@@ -39,10 +42,11 @@ def sparse_attention(q_bits, kv_bits, topk, d_v: int, scale: float, kv_base=None
     for i, t in enumerate(rows):
         sel = np.asarray(topk[t], dtype=np.int64)
         sel = sel[sel >= 0]
-        if sel.size == 0:
-            continue
         if kv_base is not None:
             sel = sel + int(kv_base[t])
+        sel = sel[(sel >= 0) & (sel < kv.shape[0])]           # entries that name no cache row select nothing
+        if sel.size == 0:
+            continue
         rows_kv = kv[sel]                                   # [n_sel, d_qk]
         s = scale * (bf16_bits_to_f64(q_bits[t]) @ rows_kv.T)   # [H, n_sel]
         m = s.max(axis=1, keepdims=True)

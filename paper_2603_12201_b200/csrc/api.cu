@@ -101,18 +101,27 @@ idxc_status launch_scorer(const ScoreArgs& a, bool decode, uint32_t flags, cudaS
 
 }  // namespace
 
-// Function attributes are per device: remember which (kernel, device) pairs have been raised.
+// Function attributes are per device: remember which (kernel, device) pairs have been raised. The table is a
+// fixed array in static storage (this function never allocates); once it is full the attribute is simply set again
+// on every call, which is harmless.
 cudaError_t ensure_max_dynamic_smem(const void* kernel, int bytes) {
+    constexpr int kSlots = 1024;
     static std::mutex mu;
-    static std::vector<std::pair<const void*, int>> done;
+    static const void* done_kernel[kSlots];
+    static int done_dev[kSlots];
+    static int n_done = 0;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     std::lock_guard<std::mutex> lock(mu);
-    for (const auto& p : done)
-        if (p.first == kernel && p.second == dev) return cudaSuccess;
+    for (int i = 0; i < n_done; ++i)
+        if (done_kernel[i] == kernel && done_dev[i] == dev) return cudaSuccess;
     e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    if (e == cudaSuccess) done.emplace_back(kernel, dev);
+    if (e == cudaSuccess && n_done < kSlots) {
+        done_kernel[n_done] = kernel;
+        done_dev[n_done] = dev;
+        ++n_done;
+    }
     return e;
 }
 
@@ -169,6 +178,8 @@ idxc_status idxc_indexer_prefill(const void* q, const void* k, const float* w, c
     idxc_status st = check_common(H_I, d_I, k_top, dt, flags);
     if (st != IDXC_OK) return st;
     if (q_begin < 0 || q_len < 0 || L_k < q_begin + q_len || L_k > (int64_t(1) << 30)) return IDXC_ERR_INVALID_ARG;
+    // the kernels address q through a tensor map whose row coordinate (query * H_I + head) is a 32-bit int
+    if (q_len * H_I >= (int64_t(1) << 31)) return IDXC_ERR_INVALID_ARG;
     if (q_len == 0) return IDXC_OK;
     if (!scores_out && !topk_out) return IDXC_ERR_INVALID_ARG;
     if (!q || !k || !w || !aligned(q, 16) || !aligned(k, 16) || !aligned(w, 16)) return IDXC_ERR_INVALID_ARG;
@@ -236,7 +247,9 @@ idxc_status idxc_indexer_decode(const void* q_step, const void* k_cache, int64_t
                                 void* workspace, size_t workspace_bytes, uint32_t flags, void* cuda_stream) {
     idxc_status st = check_common(H_I, d_I, k_top, dt, flags);
     if (st != IDXC_OK) return st;
-    if (B < 0 || max_len < 0 || max_len > (int64_t(1) << 30) || cache_rows < 0 || cache_rows > (int64_t(1) << 31) - 256)
+    // cache rows and (sequence, head) rows are 32-bit tensor-map coordinates in the kernels
+    if (B < 0 || max_len < 0 || max_len > (int64_t(1) << 30) || cache_rows < 0 || cache_rows > (int64_t(1) << 31) - 256 ||
+        static_cast<int64_t>(B) * H_I >= (int64_t(1) << 31))
         return IDXC_ERR_INVALID_ARG;
     if (B == 0) return IDXC_OK;
     if (!scores_out && !topk_out) return IDXC_ERR_INVALID_ARG;

@@ -56,6 +56,12 @@ cudaError_t launch_score_prefill_tc(const ScoreArgs& a, const CUtensorMap& q_map
 cudaError_t launch_score_decode_tc(const ScoreArgs& a, const CUtensorMap& q_map, const CUtensorMap& k_map,
                                    unsigned int* status, int sm_count, cudaStream_t stream);
 bool score_tc_supported(int H, int d, int fp8);
+// Load every kernel a decode step can launch on the current device and set its attributes (scorer_tc.cu, topk.cu,
+// topk_cluster.cu, scorer_simt.cu), so that later launches find them resident.
+cudaError_t preload_score_decode_tc();
+cudaError_t preload_topk_rows();
+cudaError_t preload_topk_rows_cluster();
+cudaError_t preload_score_simt();
 
 // quantize.cu: per-token e4m3 quantiser (row_elems a multiple of 8, at most 8192), optional row scatter.
 cudaError_t launch_quantize_e4m3(const void* x, int64_t n_tokens, int row_elems, void* codes, float* scale,

@@ -8,8 +8,12 @@
 // fixed-size array that is part of the library image, so the caller passes inputs and the
 // output only.
 //
-// The array costs IDXC_NOALLOC_SCRATCH_BYTES on every GPU that loads the library, for the life
-// of the process. All calls share it: two calls whose kernels may overlap on the GPU (different
+// The array costs IDXC_NOALLOC_SCRATCH_BYTES on every GPU this entry point is used on, for the
+// life of the process. CUDA loads a library's device code and data lazily, so the array comes into
+// being when the FIRST call on a device looks its address up: that one call makes the driver set
+// aside the 16 MiB and must therefore be made while the device still has them free, i.e. before
+// the host hands the rest of HBM to its cache pool (a warm-up step at start-up does it). Every
+// later call on that device allocates nothing, on the device or on the host. All calls share it: two calls whose kernels may overlap on the GPU (different
 // streams, no dependency between them) race on it and give unspecified indices. It keeps the
 // previous call's scores; nothing in it has to start at zero, because the scoring kernel writes
 // every score the top-k kernel reads before that kernel runs.
@@ -18,6 +22,7 @@
 #include <mutex>
 
 #include "../../include/idxc.h"
+#include "kernels.h"
 
 namespace {
 
@@ -29,7 +34,8 @@ constexpr int kMaxDevices = 64;
 std::mutex g_setup_mutex;
 void* g_scratch_addr[kMaxDevices] = {};   // device address of the array, per device ordinal
 
-// First call on a device: resolve the array's device address with that device current.
+// First call on a device: resolve the array's device address with that device current. With lazy module
+// loading this lookup is also what makes the driver create the array on that device.
 idxc_status scratch_for_current_device(void** out) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return IDXC_ERR_CUDA;
@@ -37,6 +43,11 @@ idxc_status scratch_for_current_device(void** out) {
     if (!g_scratch_addr[dev]) {
         void* p = nullptr;
         if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return IDXC_ERR_CUDA;
+        // The driver also loads a kernel's code when it is first used on a device. Load every kernel a decode step can
+        // launch now, so that a later call with another head count, dtype or batch shape finds it resident.
+        if (idxc::preload_score_decode_tc() != cudaSuccess || idxc::preload_topk_rows() != cudaSuccess ||
+            idxc::preload_topk_rows_cluster() != cudaSuccess || idxc::preload_score_simt() != cudaSuccess)
+            return IDXC_ERR_CUDA;
         g_scratch_addr[dev] = p;
     }
     *out = g_scratch_addr[dev];

@@ -80,6 +80,12 @@ cudaError_t launch_fill_masked(float* scores, int64_t ld, int64_t q_begin, int64
     return cudaSuccess;
 }
 
+cudaError_t preload_score_simt() {
+    cudaFuncAttributes fa;
+    if (cudaError_t e = cudaFuncGetAttributes(&fa, reinterpret_cast<const void*>(score_simt_kernel<false>)); e != cudaSuccess) return e;
+    return cudaFuncGetAttributes(&fa, reinterpret_cast<const void*>(score_simt_kernel<true>));
+}
+
 cudaError_t launch_score_simt(const ScoreArgs& a, cudaStream_t stream) {
     if (a.n_rows <= 0) return cudaSuccess;
     const int64_t max_keys = a.lens ? a.max_len : a.q_begin + a.n_rows;

@@ -731,6 +731,23 @@ cudaError_t launch_decode_instance(const ScoreArgs& a, const CUtensorMap& q_map,
 
 }  // namespace
 
+// Loads every decode scorer instance on the current device and raises its shared-memory limit, so that no later
+// launch has to (a kernel's first use on a device makes the driver load its code).
+cudaError_t preload_score_decode_tc() {
+    cudaError_t e = cudaSuccess;
+    auto one = [&](const void* kern, int smem) {
+        cudaFuncAttributes fa;
+        if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, kern);
+        if (e == cudaSuccess) e = ensure_max_dynamic_smem(kern, smem);
+    };
+#define IDXC_PRELOAD(NKH, H, FP8) one(reinterpret_cast<const void*>(score_decode_tc_kernel<NKH, H, FP8>), DecodeCfg<NKH, H>::kSmemBytes);
+    IDXC_PRELOAD(1, 16, false) IDXC_PRELOAD(1, 32, false) IDXC_PRELOAD(1, 64, false)
+    IDXC_PRELOAD(2, 16, false) IDXC_PRELOAD(2, 32, false) IDXC_PRELOAD(2, 64, false)
+    IDXC_PRELOAD(1, 16, true) IDXC_PRELOAD(1, 32, true) IDXC_PRELOAD(1, 64, true)
+#undef IDXC_PRELOAD
+    return e;
+}
+
 cudaError_t launch_score_decode_tc(const ScoreArgs& a, const CUtensorMap& q_map, const CUtensorMap& k_map,
                                    unsigned int* status, int sm_count, cudaStream_t stream) {
     if (a.n_rows <= 0 || a.max_len <= 0) return cudaSuccess;

@@ -1,28 +1,29 @@
 // Row-wise top-k select (Sec. 3 "Notation": T_t = Top-k(I_t)).
 //
-// One CTA per row, many rows in flight per SM (256 threads and <= 42 registers per thread when
-// there are many rows; 1024 threads for a handful of rows). A few LONG rows (decode) go to the
-// cluster kernel of topk_cluster.cu instead. Each warp
-// owns one contiguous segment of the row. Scores are compared through order-preserving 32-bit
-// keys (larger score <=> larger key, -0 == +0); the k-th largest is found exactly by a radix
-// select, 12 + 10 + 10 key bits, most significant first:
-//   sweep 1 (the HBM read)  4096-bin shared-memory histogram of the top 12 key bits; a suffix
-//                           scan finds the threshold bucket b1 holding the k-th largest score.
-//   sweep 2 (L2)            scores above bucket b1 are certainly selected, scores inside it
-//                           (typically < 2 % of the row) are candidates: both are flagged in a
-//                           shared-memory map (one byte per 128-bit load: low nibble "selected",
-//                           high nibble "candidate").
-//   candidates              gathered with key and position by walking the high nibbles (slots by
-//                           prefix popcount, no atomics); digits 2 and 3 on those only give the
-//                           exact threshold T; candidates above T, and the lowest-position ones
-//                           equal to T until k are reached, are flagged as selected.
-//   emission                a block-wide prefix popcount over the low nibbles ranks every selected
-//                           position: ascending indices, deterministic tie-break, no atomics on
-//                           the output.
-// Sweep 2 compares floats against the bucket bounds, which orders exactly like the keys. If the
-// threshold bucket holds more scores than the candidate buffer (many near-equal scores, e.g. a
-// constant row), or the row is longer than the map, digits 2 and 3 are histogrammed over the whole
-// row and the emission uses block-wide prefix sums over the row instead; same result, slower.
+// One CTA per row, many rows in flight per SM (128 threads when there are many rows; 1024 threads for a
+// handful of rows). A few LONG rows (decode) go to the cluster kernel of topk_cluster.cu instead. Each warp
+// owns one contiguous segment of the row. The exact top-k comes out of ONE sweep over the row:
+//   sample      a sixteenth of the row or more (128-score blocks spread over every warp's segment; the whole row
+//               when it is short) gives a mean and a spread, which fix a monotone map score -> bin
+//               floor(x * scale + offset), clamped to [0, 1023], with the bins laid around where the k-th largest
+//               score should lie. A histogram of the sample in these bins gives two pivot scores that bracket the
+//               k-th largest score of the whole row: bin edges next to the sample's scores of rank
+//               r -+ (3.5 standard deviations of that rank under sampling), r = k * sample / n.
+//   sweep       (the HBM read) every score at or above the upper pivot is certainly selected, the scores between
+//               the pivots (a few per cent of the row) are candidates: both are flagged in a shared-memory map (one
+//               byte per 128-bit load: low nibble "selected", high nibble "candidate") and counted.
+//   check       with A scores above and C candidates the bracket held iff A < k <= A + C. It then remains to take
+//               the k - A largest candidates.
+//   candidates  gathered into a list by walking the map; one histogram of the list in 1024 finer bins across the band
+//               leaves a handful of scores in the bin of the wanted rank; those are ranked by direct comparison of
+//               their order-preserving 32-bit keys (larger key first, lower position first among equal keys).
+//               Selected candidates are flagged in the map.
+//   emission    warp-wide prefix popcounts over the map rank every selected position: ascending indices,
+//               deterministic tie-break, no atomics on the output.
+// The result never depends on the sample: the pivots only decide how many scores become candidates, the counts are
+// exact, and when the bracket does not hold (a few rows in ten thousand for independent scores; constant rows,
+// heavy ties, infinities, or scores that drift along the row) or a list overflows, the row is selected on keys
+// alone by three histogram passes over the row; same result, slower. Rows longer than the map take that path too.
 #include "kernels.h"
 #include "topk_common.cuh"
 
@@ -30,25 +31,67 @@ namespace idxc {
 using namespace topk;
 namespace {
 
-// The candidate buffers live in the upper three quarters of the 4096-bin histogram, which is
-// only needed as a whole until the threshold bucket is known: 1536 keys + 1536 positions.
-constexpr int TK_CAP = (TK_BINS1 - TK_BINS23) / 2;
+constexpr int TK_BINS = 1024;
 constexpr int TK_MAP_MAX_BYTES = 128 * 1024;      // rows up to 524288 scores use the map
+constexpr int TK_SMALL = 128;                     // scores ranked by direct comparison at most
+constexpr float TK_MARGIN_SIGMAS = 3.5f;          // half-width of the bracket in standard deviations of the sampled rank
 
-// CAP_DYN = 0: the candidate buffers alias the histogram (TK_CAP entries). CAP_DYN > 0: they hold
-// CAP_DYN entries and live in dynamic shared memory behind the map (for launches with few, long rows,
-// whose threshold bucket holds more scores).
-template <int THREADS, int MIN_BLOCKS, int CAP_DYN>
+struct alignas(16) TopkRowSmem {
+    float part_sum[32], part_sq[32];
+    uint32_t part_cnt[32];
+    uint32_t part_a[32], part_c[32];
+    uint32_t cand_count;
+    uint32_t small_count;
+    uint32_t small_key[TK_SMALL];
+    uint32_t small_idx[TK_SMALL];
+};
+
+__device__ __forceinline__ void flag_selected(uint32_t* sel_map, uint32_t idx) {
+    atomicOr(&sel_map[idx >> 4], 1u << (8u * ((idx >> 2) & 3u) + (idx & 3u)));
+}
+// 0xFFFFFFFF if a >= b else 0 (false for NaN)
+__device__ __forceinline__ uint32_t ge_mask(float a, float b) {
+    uint32_t r;
+    asm("set.ge.u32.f32 %0, %1, %2;" : "=r"(r) : "f"(a), "f"(b));
+    return r;
+}
+// z with P(N(0,1) > z) = p, to about 1e-3 (Abramowitz & Stegun 26.2.23), clamped to [-2.5, 2.5]
+__device__ __forceinline__ float upper_quantile_z(float p) {
+    const bool upper = p <= 0.5f;
+    const float q = fminf(fmaxf(upper ? p : 1.f - p, 1e-6f), 0.5f);
+    const float t2 = -2.f * __logf(q);
+    const float t = t2 * rsqrtf(t2);
+    const float zz = t - __fdividef(2.515517f + t * (0.802853f + t * 0.010328f), 1.f + t * (1.432788f + t * (0.189269f + t * 0.001308f)));
+    return fminf(fmaxf(upper ? zz : -zz, -2.5f), 2.5f);
+}
+// bits 0-3, 8-11, 16-19, 24-27 of m (a map word's nibbles of one kind) as one 16-bit mask: bit j <-> position 16 w + j
+__device__ __forceinline__ uint32_t squeeze_nibbles(uint32_t m) {
+    return (m & 0xFu) | ((m >> 4) & 0xF0u) | ((m >> 8) & 0xF00u) | ((m >> 12) & 0xF000u);
+}
+// exclusive prefix sum of v over the lanes of a warp; total = the warp's sum
+__device__ __forceinline__ uint32_t warp_excl_scan(uint32_t v, int lane, uint32_t& total) {
+    uint32_t inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+        if (lane >= o) inc += y;
+    }
+    total = __shfl_sync(0xFFFFFFFFu, inc, 31);
+    return inc - v;
+}
+// CAP candidates (fine bin, position) in dynamic shared memory behind the map.
+template <int THREADS, int MIN_BLOCKS, int CAP>
 __global__ void __launch_bounds__(THREADS, MIN_BLOCKS)
 topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int64_t n_rows, int64_t first_len, int64_t len_step,
                  const int32_t* __restrict__ lens, int k_top, int32_t* __restrict__ out, int map_scores) {
     constexpr int WARPS = THREADS / 32;
-    __shared__ __align__(16) TopkSmem<WARPS> sm;
-    extern __shared__ uint32_t sel_map[];                        // map_scores / 16 words
+    constexpr int U = TK_UNROLL;
+    __shared__ __align__(16) TopkSmem<WARPS, 2048> sm;           // 2048 bins: the keys-only path needs them
+    __shared__ TopkRowSmem rs;
+    extern __shared__ uint32_t sel_map[];                        // map_scores / 16 words, then the candidates
     uint8_t* sel_bytes = reinterpret_cast<uint8_t*>(sel_map);
-    constexpr int CAP = CAP_DYN > 0 ? CAP_DYN : TK_CAP;
-    uint32_t* cand_key = CAP_DYN > 0 ? sel_map + map_scores / 16 : sm.hist + TK_BINS23;   // aliased: valid once b1 is known
-    uint32_t* cand_idx = cand_key + CAP;
+    uint32_t* cand_fb = sel_map + map_scores / 16;               // a candidate's fine bin ...
+    uint32_t* cand_idx = cand_fb + CAP;                          // ... and position
     int slot = 0;
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const uint32_t k = static_cast<uint32_t>(k_top);
@@ -64,123 +107,294 @@ topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int64_t n_rows, i
             continue;
         }
         const float* src = scores + row * ld;
+        if (n > map_scores) {                                    // longer than the map: keys alone
+            slow_path_full<THREADS>(sm, src, n, k, out_row, slot);
+            continue;
+        }
         // this warp's segment: a multiple of 128 scores, so every lane loads aligned float4s
         const int seg = (((n + WARPS - 1) / WARPS) + 127) & ~127;
         const int seg_begin = wid * seg < n ? wid * seg : n;
         const int seg_end = seg_begin + seg < n ? seg_begin + seg : n;
+        // this warp's sample: S blocks of 128 scores, `stride` apart, from the start of its segment; over the block
+        // 2048 scores per 32768 of the row, at least 2048
+        const int seg_blocks = seg >> 7;
+        int S = (16 * ((n + 32767) >> 15) + WARPS - 1) / WARPS;
+        S = S < U ? U : S;
+        S = S > seg_blocks ? seg_blocks : S;
+        const int stride = (seg_blocks / S) << 7;
+        // calls f(float4, index of its first score) for the lane's part of every sample block
+        auto for_sample = [&](auto f) {
+            for (int j0 = 0; j0 < S; j0 += U) {
+                float4 x[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int base = seg_begin + (j0 + u) * stride + 4 * lane;
+                    x[u] = (j0 + u < S && base < seg_end) ? __ldg(reinterpret_cast<const float4*>(src + base))
+                                                         : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int base = seg_begin + (j0 + u) * stride + 4 * lane;
+                    if (j0 + u < S && base < seg_end) f(x[u], base);
+                }
+            }
+        };
 
-        // ---- sweep 1: histogram of the top 12 key bits over the whole row
-        __syncthreads();   // earlier readers of sm are done
-        zero_hist<THREADS>(sm, TK_BINS1);
+        // ---- the sample: mean and spread
+        __syncthreads();   // earlier readers of sm, rs and the map are done
+        zero_hist<THREADS>(sm, TK_BINS);
+        {
+            float s1 = 0.f, s2 = 0.f;
+            uint32_t m = 0;
+            for_sample([&](const float4& x, int base) {
+                const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (base + e < n) { s1 += xs[e]; s2 = fmaf(xs[e], xs[e], s2); ++m; }
+            });
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                s1 += __shfl_xor_sync(0xFFFFFFFFu, s1, o);
+                s2 += __shfl_xor_sync(0xFFFFFFFFu, s2, o);
+                m += __shfl_xor_sync(0xFFFFFFFFu, m, o);
+            }
+            if (lane == 0) { rs.part_sum[wid] = s1; rs.part_sq[wid] = s2; rs.part_cnt[wid] = m; }
+            if (threadIdx.x == 0) { rs.cand_count = 0u; rs.small_count = 0u; }
+        }
         __syncthreads();
-        sweep_segment<TK_UNROLL>(src, n, seg_begin, seg_end, lane, [&](const float4& x, int base) {
+        float scale, offset;
+        uint32_t m_sample = 0;
+        {
+            float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+            for (int w = 0; w < WARPS; ++w) { s1 += rs.part_sum[w]; s2 += rs.part_sq[w]; m_sample += rs.part_cnt[w]; }
+            const float inv_m = __fdividef(1.f, static_cast<float>(m_sample));
+            const float mean = s1 * inv_m;
+            const float var = fmaxf(s2 * inv_m - mean * mean, 0.f);
+            const float sd = var * rsqrtf(fmaxf(var, 1e-37f));
+            // where the k-th largest of n draws of such a distribution is expected, in standard deviations from the mean
+            // (a rough inverse normal distribution is enough: it only centres the bins)
+            const float z = upper_quantile_z(__fdividef(static_cast<float>(k_top), static_cast<float>(n)));
+            const float half = 1.5f * sd;                         // the bins span [centre - half, centre + half)
+            scale = __fdividef(0.5f * TK_BINS, half);
+            offset = -(mean + z * sd - half) * scale;
+            // a constant sample, or one with infinities, gives no usable map: the row takes the keys-only path
+            if (!(sd > 0.f) || !(fabsf(scale) < 3.0e38f) || !(fabsf(offset) < 3.0e38f)) scale = 0.f;
+        }
+        if (scale == 0.f) {                                      // the same for every thread
+            slow_path_full<THREADS>(sm, src, n, k, out_row, slot);
+            continue;
+        }
+        // ---- histogram of the sample, pivots
+        for_sample([&](const float4& x, int base) {
             const float xs[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
-            for (int e = 0; e < 4; ++e)
-                if (base + e < n) atomicAdd(&sm.hist[score_digit1(xs[e])], 1u);
+            for (int e = 0; e < 4; ++e) {
+                if (base + e < n) {
+                    const int b = __float2int_rd(__fmaf_rn(xs[e], scale, offset));     // NaN -> 0; saturates
+                    atomicAdd(&sm.hist[min(max(b, 0), TK_BINS - 1)], 1u);
+                }
+            }
         });
         __syncthreads();
-        uint32_t b1, above1;
-        select_bucket<TK_BINS1, THREADS>(sm, k, slot, b1, above1);
-        const uint32_t c1 = sm.hist[b1];
-        uint32_t need = k - above1;          // rank inside bucket b1, 1-based
-        __syncthreads();                     // everyone has read hist[b1]: the candidate buffers may now overwrite the bins
+        // rank of the k-th largest of the row inside the sample, and its standard deviation under sampling without replacement
+        const float mf = static_cast<float>(m_sample), nf = static_cast<float>(n);
+        const float p = __fdividef(static_cast<float>(k_top), nf);
+        const float r = mf * p;
+        const float var_r = fmaxf(mf * p * (1.f - p) * __fdividef(nf - mf, fmaxf(nf - 1.f, 1.f)), 0.f);
+        const float sd_r = var_r * rsqrtf(fmaxf(var_r, 1e-37f));
+        const bool whole = m_sample == static_cast<uint32_t>(n);          // the sample is the row: ranks are exact
+        const float margin = whole ? 0.f : TK_MARGIN_SIGMAS * sd_r + 2.f;
+        const int r_hi = whole ? k_top : static_cast<int>(floorf(r - margin));  // sample ranks below r_hi: certainly selected
+        const int r_lo = whole ? k_top : static_cast<int>(ceilf(r + margin));   // sample ranks above r_lo: certainly not
+        const bool has_hi = r_hi >= 1;
+        const bool has_lo = r_lo <= static_cast<int>(m_sample);
+        uint32_t hi_bin, lo_bin, ab_hi, ab_lo;
+        select_two_buckets<TK_BINS, THREADS>(sm, has_hi ? r_hi : 1, has_lo ? r_lo : m_sample, slot, hi_bin, ab_hi, lo_bin, ab_lo);
+        // the pivots as scores: the upper edge of bin hi_bin and the lower edge of bin lo_bin (any bracket will do, so the
+        // rounding of these two divisions does not matter); an end bin has no edge on its outer side
+        const float inv_scale = __fdividef(1.f, scale);
+        const float lo_x = (!has_lo || lo_bin == 0u) ? -INFINITY : (static_cast<float>(lo_bin) - offset) * inv_scale;
+        const float hi_x = (!has_hi || hi_bin == TK_BINS - 1) ? INFINITY : (static_cast<float>(hi_bin + 1u) - offset) * inv_scale;
 
-        if (c1 <= static_cast<uint32_t>(CAP) && n <= map_scores) {
-            // ---- sweep 2: flag the scores above bucket b1 (selected) and inside it (candidates)
-            const float lo = key_to_score(b1 << 20);                       // smallest score of bucket b1
-            const bool has_above = b1 < TK_BINS1 - 1;
-            const float hi = key_to_score(has_above ? ((b1 + 1) << 20) : 0xFFFFFFFFu);   // smallest score above it
-            sweep_segment<TK_UNROLL>(src, n, seg_begin, seg_end, lane, [&](const float4& x4, int base) {
-                const float x[4] = {x4.x, x4.y, x4.z, x4.w};
-                uint32_t flags = 0;
+        // ---- the sweep: flag the scores at or above the upper pivot and those between the pivots
+        auto flag4 = [&](const float4& v) -> uint32_t {
+            const float x[4] = {v.x, v.y, v.z, v.w};
+            uint32_t sel = 0, ge_lo = 0;
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    if (base + e >= n || !(x[e] >= lo)) continue;
-                    flags |= (has_above && x[e] >= hi) ? (1u << e) : (16u << e);
-                }
-                sel_bytes[base >> 2] = static_cast<uint8_t>(flags);        // lanes past the end of the row write 0
-            });
-            __syncthreads();
-            // ---- gather the candidates (high nibbles) with their keys; slots by prefix popcount
-            const int words = (n + 15) >> 4;
-            const int wpt = (words + THREADS - 1) / THREADS;
-            const int w0 = static_cast<int>(threadIdx.x) * wpt < words ? static_cast<int>(threadIdx.x) * wpt : words;
-            const int w1 = w0 + wpt < words ? w0 + wpt : words;
-            {
-                uint32_t cnt = 0;
-                for (int w = w0; w < w1; ++w) cnt += __popc(sel_map[w] & 0xF0F0F0F0u);
-                uint32_t total;
-                uint32_t pos = block_excl_scan(cnt, sm, slot, total);
-                for (int w = w0; w < w1; ++w) {
-                    uint32_t m = sel_map[w] & 0xF0F0F0F0u;
-                    while (m) {
-                        const int b = __ffs(m) - 1;
-                        m &= m - 1;
-                        const int idx = 16 * w + 4 * (b >> 3) + (b & 7) - 4;
-                        if (pos < static_cast<uint32_t>(CAP)) {
-                            cand_key[pos] = score_key(__ldg(src + idx)) & 0xFFFFFu;
-                            cand_idx[pos] = static_cast<uint32_t>(idx);
-                        }
-                        ++pos;
-                    }
-                }
+            for (int e = 0; e < 4; ++e) {
+                sel |= ge_mask(x[e], hi_x) & (1u << e);
+                ge_lo |= ge_mask(x[e], lo_x) & (16u << e);
             }
-            // ---- digits 2 and 3 on the candidates
-            uint32_t t_low, need_eq, m_eq;
-            candidate_select<THREADS>(sm, cand_key, c1, need, slot, t_low, need_eq, m_eq);
-            // ---- flag the selected candidates
-            for (uint32_t i = threadIdx.x; i < c1; i += THREADS) {
-                const uint32_t c = cand_key[i];
-                bool take = c > t_low;
-                if (c == t_low) {
-                    take = true;
-                    if (m_eq != need_eq) {                       // ties compete: the lowest positions win
-                        uint32_t before = 0;
-                        for (uint32_t i2 = 0; i2 < c1; ++i2) before += (cand_key[i2] == t_low) & (cand_idx[i2] < cand_idx[i]);
-                        take = before < need_eq;
-                    }
-                }
-                if (take) {
-                    const uint32_t idx = cand_idx[i];
-                    atomicOr(&sel_map[idx >> 4], 1u << (8u * ((idx >> 2) & 3u) + (idx & 3u)));
-                }
+            return sel | (ge_lo & ~(sel << 4));                         // high nibble: between the pivots
+        };
+        {
+            // whole steps of U blocks that lie inside the segment and the row need no bounds checks
+            const int full_end = seg_begin + ((seg_end & ~3) - seg_begin) / (128 * U) * (128 * U);
+            const float* p = src + seg_begin + 4 * lane;
+            uint8_t* mb = sel_bytes + (seg_begin >> 2) + lane;
+            int cb = seg_begin;
+            for (; cb < full_end; cb += 128 * U, p += 128 * U, mb += 32 * U) {
+                float4 x4[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) x4[u] = __ldg(reinterpret_cast<const float4*>(p + 128 * u));
+#pragma unroll
+                for (int u = 0; u < U; ++u) mb[32 * u] = static_cast<uint8_t>(flag4(x4[u]));
             }
-            __syncthreads();
-            // ---- emission: rank the selected positions by a prefix popcount over the low nibbles
-            uint32_t cnt = 0;
-            for (int w = w0; w < w1; ++w) cnt += __popc(sel_map[w] & 0x0F0F0F0Fu);
+            for (; cb < seg_end; cb += 128) {                           // the ragged rest, one block at a time
+                const int base = cb + 4 * lane;
+                uint32_t flags = 0;
+                if (base < n) {
+                    flags = flag4(__ldg(reinterpret_cast<const float4*>(src + base)));
+                    const int left = n - base;                          // scores of this 128-bit load inside the row
+                    if (left < 4) flags &= (0x11u << left) - 0x11u;
+                }
+                sel_bytes[base >> 2] = static_cast<uint8_t>(flags);    // lanes past the end of the row write 0
+            }
+        }
+        __syncwarp();
+        // A = scores above the band, C = scores inside it: counted from this warp's part of the map, summed over the block
+        const int w_begin = seg_begin >> 4, w_end = seg_begin < seg_end ? (seg_end + 15) >> 4 : w_begin;
+        {
+            uint32_t n_sel = 0, n_cand = 0;
+            for (int w = w_begin + lane; w < w_end; w += 32) {
+                const uint32_t m = sel_map[w];
+                n_sel += __popc(m & 0x0F0F0F0Fu);
+                n_cand += __popc(m & 0xF0F0F0F0u);
+            }
+            n_sel = __reduce_add_sync(0xFFFFFFFFu, n_sel);
+            n_cand = __reduce_add_sync(0xFFFFFFFFu, n_cand);
+            if (lane == 0) { rs.part_a[wid] = n_sel; rs.part_c[wid] = n_cand; }
+        }
+        __syncthreads();
+        uint32_t A = 0, C = 0;
+#pragma unroll
+        for (int w = 0; w < WARPS; ++w) { A += rs.part_a[w]; C += rs.part_c[w]; }
+        if (!(A < k && k - A <= C && C <= static_cast<uint32_t>(CAP))) { // the bracket did not hold, or the list would overflow
+            slow_path_full<THREADS>(sm, src, n, k, out_row, slot);
+            continue;
+        }
+        const uint32_t need = k - A;                                    // candidates to take, 1..C
+        // ---- gather the candidates: each warp walks the map words of its segment, 32 words at a time
+        zero_hist<THREADS>(sm, TK_BINS);
+        // every lane owns a run of consecutive map words of its warp's segment
+        const int wpl = (w_end - w_begin + 31) >> 5;
+        const int lw0 = w_begin + lane * wpl < w_end ? w_begin + lane * wpl : w_end;
+        const int lw1 = lw0 + wpl < w_end ? lw0 + wpl : w_end;
+        {
+            uint32_t c = 0;
+            for (int w = lw0; w < lw1; ++w) c += __popc(sel_map[w] & 0xF0F0F0F0u);
             uint32_t total;
-            uint32_t rank = block_excl_scan(cnt, sm, slot, total);
-            for (int w = w0; w < w1; ++w) {
-                uint32_t m = sel_map[w] & 0x0F0F0F0Fu;
+            uint32_t pos = warp_excl_scan(c, lane, total);
+            uint32_t basepos = 0;
+            if (lane == 0 && total != 0u) basepos = atomicAdd(&rs.cand_count, total);
+            pos += __shfl_sync(0xFFFFFFFFu, basepos, 0);
+            for (int w = lw0; w < lw1; ++w) {
+                uint32_t m = squeeze_nibbles(sel_map[w] >> 4);
+                const uint32_t idx0 = 16u * static_cast<uint32_t>(w);
+                while (m) {
+                    const uint32_t b = __ffs(m) - 1;
+                    m &= m - 1;
+                    if (pos < static_cast<uint32_t>(CAP)) cand_idx[pos] = idx0 + b;
+                    ++pos;
+                }
+            }
+        }
+        __syncthreads();
+        // ---- candidates: finer bins across the band
+        const float y_lo = (has_lo && lo_bin != 0u) ? static_cast<float>(lo_bin) : 0.f;
+        const float y_hi = (has_hi && hi_bin != TK_BINS - 1) ? static_cast<float>(hi_bin + 1u) : static_cast<float>(TK_BINS);
+        const float fscale = __fdividef(static_cast<float>(TK_BINS), y_hi - y_lo);
+        auto fine_bin = [&](float x) -> uint32_t {
+            const float y = __fmaf_rn(x, scale, offset);
+            const int b = __float2int_rd((y - y_lo) * fscale);
+            return static_cast<uint32_t>(min(max(b, 0), TK_BINS - 1));
+        };
+        for (uint32_t i = threadIdx.x; i < C; i += THREADS) {             // independent loads (L2), all in flight together
+            const uint32_t fb = fine_bin(__ldg(src + cand_idx[i]));
+            cand_fb[i] = fb;
+            atomicAdd(&sm.hist[fb], 1u);
+        }
+        __syncthreads();
+        uint32_t fb1, above_f;
+        select_bucket<TK_BINS, THREADS>(sm, need, slot, fb1, above_f);
+        const uint32_t m1 = sm.hist[fb1];
+        if (m1 > static_cast<uint32_t>(TK_SMALL)) {                     // many near-equal scores at the threshold
+            slow_path_full<THREADS>(sm, src, n, k, out_row, slot);
+            continue;
+        }
+        const uint32_t need1 = need - above_f;                          // scores to take from fine bin fb1, 1..m1
+        for (uint32_t i = threadIdx.x; i < C; i += THREADS) {
+            const uint32_t fb = cand_fb[i];
+            if (fb > fb1) {
+                flag_selected(sel_map, cand_idx[i]);
+            } else if (fb == fb1) {
+                const uint32_t pos = atomicAdd(&rs.small_count, 1u);
+                const uint32_t idx = cand_idx[i];
+                if (pos < static_cast<uint32_t>(TK_SMALL)) { rs.small_key[pos] = score_key(__ldg(src + idx)); rs.small_idx[pos] = idx; }
+            }
+        }
+        __syncthreads();
+        for (uint32_t i = threadIdx.x; i < m1; i += THREADS) {          // larger key first, lower position first among equal keys
+            const uint32_t ki = rs.small_key[i], ii = rs.small_idx[i];
+            uint32_t beaten_by = 0;
+            for (uint32_t j = 0; j < m1; ++j) {
+                const uint32_t kj = rs.small_key[j], ij = rs.small_idx[j];
+                beaten_by += (kj > ki) | ((kj == ki) & (ij < ii));
+            }
+            if (beaten_by < need1) flag_selected(sel_map, ii);
+        }
+        __syncthreads();
+        // ---- emission: a lane ranks the selected positions of its run of map words; lanes and warps are offset by
+        // prefix sums of their counts
+        {
+            uint32_t c = 0;
+            for (int w = lw0; w < lw1; ++w) c += __popc(sel_map[w] & 0x0F0F0F0Fu);
+            uint32_t total;
+            uint32_t pos = warp_excl_scan(c, lane, total);
+            if (lane == 0) rs.part_a[wid] = total;
+            __syncthreads();
+#pragma unroll
+            for (int w = 0; w < WARPS; ++w) pos += w < wid ? rs.part_a[w] : 0u;
+            for (int w = lw0; w < lw1; ++w) {
+                uint32_t m = squeeze_nibbles(sel_map[w]);
+                const int idx0 = 16 * w;
                 while (m) {
                     const int b = __ffs(m) - 1;
                     m &= m - 1;
-                    if (rank < k) out_row[rank] = 16 * w + 4 * (b >> 3) + (b & 7);
-                    ++rank;
+                    if (pos < k) out_row[pos] = idx0 + b;
+                    ++pos;
                 }
             }
-            continue;
         }
-
-        // ---- slow path: digits 2 and 3 over the whole row, then block-scan emission
-        slow_path<THREADS>(sm, src, n, b1, need, k, out_row, slot);
     }
 }
 
-template <int THREADS, int MIN_BLOCKS, int CAP_DYN>
+template <int THREADS, int MIN_BLOCKS, int CAP>
 cudaError_t launch_instance(const float* scores, int64_t ld, int64_t n_rows, int64_t first_len, int64_t len_step,
                             const int32_t* lens, int k_top, int32_t* out, int map_bytes, cudaStream_t stream) {
-    auto kern = topk_rows_kernel<THREADS, MIN_BLOCKS, CAP_DYN>;
-    if (cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(kern), TK_MAP_MAX_BYTES + 8 * CAP_DYN); e != cudaSuccess) return e;
+    auto kern = topk_rows_kernel<THREADS, MIN_BLOCKS, CAP>;
+    if (cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(kern), TK_MAP_MAX_BYTES + 8 * CAP); e != cudaSuccess) return e;
     const int64_t max_grid = 1 << 20;
     const unsigned grid = static_cast<unsigned>(n_rows < max_grid ? n_rows : max_grid);
-    kern<<<grid, THREADS, map_bytes + 8 * CAP_DYN, stream>>>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, map_bytes * 4);
+    kern<<<grid, THREADS, map_bytes + 8 * CAP, stream>>>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, map_bytes * 4);
     return cudaGetLastError();
 }
 
+constexpr int kCapMany = 1536, kCapFew = 8192;    // candidate slots of the two instances
+
 }  // namespace
+
+
+cudaError_t preload_topk_rows() {
+    cudaFuncAttributes fa;
+    const void* many = reinterpret_cast<const void*>(topk_rows_kernel<128, 8, kCapMany>);
+    const void* few = reinterpret_cast<const void*>(topk_rows_kernel<1024, 1, kCapFew>);
+    if (cudaError_t e = cudaFuncGetAttributes(&fa, many); e != cudaSuccess) return e;
+    if (cudaError_t e = cudaFuncGetAttributes(&fa, few); e != cudaSuccess) return e;
+    if (cudaError_t e = ensure_max_dynamic_smem(many, TK_MAP_MAX_BYTES + 8 * kCapMany); e != cudaSuccess) return e;
+    return ensure_max_dynamic_smem(few, TK_MAP_MAX_BYTES + 8 * kCapFew);
+}
 
 cudaError_t launch_topk_rows(const float* scores, int64_t ld, int64_t n_rows, int64_t first_len, int64_t len_step,
                              const int32_t* lens, int k_top, int32_t* out, cudaStream_t stream) {
@@ -195,8 +409,8 @@ cudaError_t launch_topk_rows(const float* scores, int64_t ld, int64_t n_rows, in
     if (map_bytes > TK_MAP_MAX_BYTES) map_bytes = TK_MAP_MAX_BYTES;
     // many rows: small CTAs, many per SM; few rows: more threads per row
     if (n_rows >= 1024)
-        return launch_instance<256, 6, 0>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, static_cast<int>(map_bytes), stream);
-    return launch_instance<1024, 1, 8192>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, static_cast<int>(map_bytes), stream);
+        return launch_instance<128, 8, kCapMany>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, static_cast<int>(map_bytes), stream);
+    return launch_instance<1024, 1, kCapFew>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, static_cast<int>(map_bytes), stream);
 }
 
 }  // namespace idxc

@@ -27,6 +27,8 @@ namespace idxc {
 using namespace topk;
 namespace {
 
+constexpr int CL_D1 = 12;             // first digit: top 12 key bits
+constexpr int TK_BINS1 = 1 << CL_D1;
 constexpr int CL_SIZE = 8;            // CTAs per row
 constexpr int CL_THREADS = 512;
 constexpr int CL_WARPS = CL_THREADS / 32;
@@ -49,7 +51,7 @@ __global__ void __launch_bounds__(CL_THREADS, 2)
 topk_rows_cluster_kernel(const float* __restrict__ scores, int64_t ld, int64_t n_rows, int64_t first_len, int64_t len_step,
                          const int32_t* __restrict__ lens, int k_top, int32_t* __restrict__ out, int map_bytes) {
     cg::cluster_group cluster = cg::this_cluster();
-    __shared__ __align__(16) TopkSmem<CL_WARPS> sm;
+    __shared__ __align__(16) TopkSmem<CL_WARPS, TK_BINS1> sm;
     __shared__ ClusterExchange ex;
     extern __shared__ uint32_t dyn[];
     uint32_t* sel_map = dyn;                                   // map_bytes: one byte per 4 scores of my part
@@ -92,7 +94,7 @@ topk_rows_cluster_kernel(const float* __restrict__ scores, int64_t ld, int64_t n
             const float xs[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e)
-                if (base + e < n) atomicAdd(&sm.hist[score_digit1(xs[e])], 1u);
+                if (base + e < n) atomicAdd(&sm.hist[score_digit1<CL_D1>(xs[e])], 1u);
         });
         cluster.sync();                                                                        // (1)
         // ---- 2. sum my 512 bins over the cluster
@@ -101,7 +103,7 @@ topk_rows_cluster_kernel(const float* __restrict__ scores, int64_t ld, int64_t n
         for (int r = 0; r < CL_SIZE; ++r) v += cluster.map_shared_rank(sm.hist, r)[rank * CL_BINS_PER_RANK + tid];
         ex.red[tid] = v;
         uint32_t my_total;
-        (void)block_excl_scan(v, sm, slot, my_total);
+        (void)block_excl_scan<CL_WARPS>(v, sm, slot, my_total);
         if (tid < CL_SIZE) cluster.map_shared_rank(ex.part_tot, tid)[rank] = my_total;
         cluster.sync();                                                                        // (2)
         // ---- 3. the CTA whose bins hold the k-th largest score selects the bucket
@@ -123,8 +125,8 @@ topk_rows_cluster_kernel(const float* __restrict__ scores, int64_t ld, int64_t n
         const uint32_t b1 = ex.bcast[0];
         const uint32_t c1 = ex.bcast[2];
         const uint32_t need = k - ex.bcast[1];                 // rank inside bucket b1, 1-based
-        if (c1 > static_cast<uint32_t>(CL_CAP) || part > map_bytes * 4) {                      // cluster-uniform
-            if (rank == 0) slow_path<CL_THREADS>(sm, src, n, b1, need, k, out_row, slot);
+        if (c1 > static_cast<uint32_t>(CL_CAP) || part > map_bytes * 4 || !bucket_is_finite<CL_D1>(b1)) {   // cluster-uniform
+            if (rank == 0) slow_path<CL_THREADS, CL_D1>(sm, src, n, b1, need, k, out_row, slot);
             continue;
         }
         // ---- 4. flag my scores above bucket b1 (selected) and inside it (candidates)
@@ -150,7 +152,7 @@ topk_rows_cluster_kernel(const float* __restrict__ scores, int64_t ld, int64_t n
             uint32_t cnt = 0;
             for (int w = w0; w < w1; ++w) cnt += __popc(sel_map[w] & 0xF0F0F0F0u);
             uint32_t mine;
-            uint32_t pos = block_excl_scan(cnt, sm, slot, mine);
+            uint32_t pos = block_excl_scan<CL_WARPS>(cnt, sm, slot, mine);
             if (tid == 0) ex.cand_base = atomicAdd(cluster.map_shared_rank(&ex.cand_total, 0), mine);
             __syncthreads();
             pos += ex.cand_base;
@@ -174,7 +176,7 @@ topk_rows_cluster_kernel(const float* __restrict__ scores, int64_t ld, int64_t n
         // ---- 5. the leader finds the exact threshold among the candidates
         if (rank == 0) {
             uint32_t t_low, need_eq, m_eq;
-            candidate_select<CL_THREADS>(sm, cand_key, c1, need, slot, t_low, need_eq, m_eq);
+            candidate_select<CL_THREADS, 32 - CL_D1>(sm, cand_key, c1, need, slot, t_low, need_eq, m_eq);
             if (tid == 0) ex.cand_base = 0xFFFFFFFFu;          // reused: position limit for ties (none: take all)
             __syncthreads();
             if (m_eq != need_eq) {                             // ties compete: the need_eq lowest positions win
@@ -211,7 +213,7 @@ topk_rows_cluster_kernel(const float* __restrict__ scores, int64_t ld, int64_t n
             cnt += __popc(word);
         }
         uint32_t mine;
-        uint32_t rnk = block_excl_scan(cnt, sm, slot, mine);
+        uint32_t rnk = block_excl_scan<CL_WARPS>(cnt, sm, slot, mine);
         if (tid < CL_SIZE) cluster.map_shared_rank(ex.sel_cnt, tid)[rank] = mine;
         cluster.sync();                                                                        // (6)
         // ---- 7. emission
@@ -230,6 +232,12 @@ topk_rows_cluster_kernel(const float* __restrict__ scores, int64_t ld, int64_t n
 }
 
 }  // namespace
+
+cudaError_t preload_topk_rows_cluster() {
+    cudaFuncAttributes fa;
+    if (cudaError_t e = cudaFuncGetAttributes(&fa, reinterpret_cast<const void*>(topk_rows_cluster_kernel)); e != cudaSuccess) return e;
+    return ensure_max_dynamic_smem(reinterpret_cast<const void*>(topk_rows_cluster_kernel), CL_MAX_PART / 4 + 2 * CL_CAP * 4);
+}
 
 bool topk_cluster_applicable(int64_t n_rows, int64_t longest) {
     return n_rows >= 1 && n_rows <= 128 && longest >= 16384 && longest <= static_cast<int64_t>(CL_MAX_PART) * CL_SIZE;

@@ -78,6 +78,10 @@ def test_argument_validation_happens_before_any_device_work(idxc):
     assert L.idxc_indexer_decode(one, one, 100, one, None, None, one, None, 2, 10, 16, 64, 8, idxc.BF16, None, 0, one, one, 1 << 20, 0, None) == idxc.ERR_INVALID_ARG
     # top-k: ld not a multiple of 4
     assert L.idxc_topk_rows(one, 10, 2, 1, 1, None, 4, one, None) == idxc.ERR_INVALID_ARG
+    # tensor-map row coordinates are 32-bit: (query, head) rows and (sequence, head) rows must stay below 2^31
+    assert L.idxc_indexer_prefill(one, one, one, None, None, 0, 1 << 25, 1 << 25, 64, 128, 8, idxc.BF16, None, 0, one, one, 1 << 20, 0, None) == idxc.ERR_INVALID_ARG
+    assert L.idxc_indexer_decode(one, one, 100, one, None, None, one, one, 1 << 25, 10, 64, 128, 8, idxc.BF16, None, 0, one, one, 1 << 20, 0, None) == idxc.ERR_INVALID_ARG
+
 
 
 def test_sparse_attention_validation_and_workspace(idxc):

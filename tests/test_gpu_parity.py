@@ -94,6 +94,89 @@ def test_topk_rows_matches_oracle(n, k_top):
         assert np.array_equal(out[r], want), f"row {r}"
 
 
+def test_topk_rows_many_rows_constant_tied_and_crowded():
+    """More than 1024 rows (the many-rows kernel instance) with the rows that defeat the fast path: constant rows,
+    heavy ties, and rows whose scores all share their leading key bits, so that the threshold bucket holds the whole
+    row and the select has to finish over the row itself. Bit-exact against the oracle, every row."""
+    g = torch.Generator().manual_seed(99)
+    n_rows, ld, k_top = 1100, 3000, 512
+    s = torch.randn(n_rows, ld, generator=g)
+    s[::7] = 0.0                                                        # constant rows
+    s[1::7] = torch.round(s[1::7] * 2) / 2                              # a handful of distinct values
+    s[2::7] = 1.0 + torch.rand(s[2::7].shape, generator=g) * 2.0 ** -6  # one crowded bucket: all in [1, 1.016)
+    s[3::7] = -(1.0 + torch.randint(0, 3, s[3::7].shape, generator=g).float() * 2.0 ** -20)   # crowded and tied
+    s[4::7, ::2] = -0.0
+    s[4::7, 1::2] = 0.0                                                 # -0 == +0
+    lens = torch.randint(0, ld + 1, (n_rows,), generator=g, dtype=torch.int32)
+    lens[:40] = ld
+    out = torch.full((n_rows, k_top), -7, dtype=torch.int32, device=DEV)
+    idxc.topk_rows(s.to(DEV), k_top, out, lens=lens.to(DEV))
+    out = out.cpu().numpy()
+    s64 = s.to(torch.float64).numpy()
+    for r in range(n_rows):
+        assert np.array_equal(out[r], oracle.topk(s64[r, : int(lens[r])], k_top)), f"row {r}"
+
+
+def _selected_dominate(scores: torch.Tensor, topk: torch.Tensor, lens: torch.Tensor, k_top: int):
+    """Property that holds for any correct selection: per row min(k, len) distinct ascending in-range indices, and no
+    unselected score of the row exceeds a selected one (checked on the device over the whole output)."""
+    n_rows, ld = scores.shape
+    kk = torch.clamp(lens.long(), max=k_top)
+    col = torch.arange(k_top, device=scores.device)
+    valid = col[None, :] < kk[:, None]
+    assert bool(((topk >= 0) == valid).all())
+    assert bool((topk[:, 1:] > topk[:, :-1])[valid[:, 1:]].all())
+    assert bool((torch.where(valid, topk.long(), torch.zeros_like(topk, dtype=torch.long)) < torch.clamp(lens.long(), min=1)[:, None]).all())
+    for r0 in range(0, n_rows, 64):                                     # slabs bound the transient memory
+        sl = slice(r0, min(n_rows, r0 + 64))
+        sc = scores[sl]
+        chosen = torch.zeros_like(sc, dtype=torch.bool)
+        idx = torch.where(valid[sl], topk[sl].long(), torch.zeros_like(topk[sl], dtype=torch.long))
+        chosen.scatter_(1, idx, valid[sl])
+        inside = torch.arange(ld, device=sc.device)[None, :] < lens[sl].long()[:, None]
+        lo_sel = torch.where(chosen, sc, torch.full_like(sc, float("inf"))).amin(dim=1)
+        hi_rest = torch.where(inside & ~chosen, sc, torch.full_like(sc, float("-inf"))).amax(dim=1)
+        assert bool((hi_rest <= lo_sel).all())
+
+
+@pytest.mark.parametrize("n_rows", [5, 1024])
+def test_topk_rows_longer_than_the_selection_map(n_rows):
+    """Rows of more than 524288 scores exceed the shared-memory selection map of both one-CTA kernel instances
+    (few rows: 1024 threads; 1024 rows and more: 256 threads) and are finished over the row itself."""
+    n, k_top = 524288 + 517, 2048
+    ld = (n + 3) // 4 * 4
+    g = torch.Generator(device=DEV).manual_seed(n_rows)
+    s = torch.randn(n_rows, ld, generator=g, device=DEV)
+    s[1] = torch.round(s[1] * 4) / 4                                     # ties across the threshold
+    s[2] = 0.0
+    lens = torch.full((n_rows,), n, dtype=torch.int32, device=DEV)
+    lens[3] = n - 5
+    out = torch.full((n_rows, k_top), -7, dtype=torch.int32, device=DEV)
+    idxc.topk_rows(s, k_top, out, lens=lens)
+    _selected_dominate(s, out, lens, k_top)
+    for r in sorted({0, 1, 2, 3, n_rows - 1}):
+        want = oracle.topk(s[r, : int(lens[r])].to(torch.float64).cpu().numpy(), k_top)
+        assert np.array_equal(out[r].cpu().numpy(), want), f"row {r}"
+
+
+def test_topk_rows_with_masked_entries_read_at_full_length():
+    """Rows filled under IDXC_FLAG_FILL_MASKED hold -inf beyond the causal part. Read at full length with fewer than k
+    finite scores, the k-th largest is -inf itself: every finite position is selected first, then the lowest masked
+    positions; every output slot is written."""
+    L, H, d, k_top = 300, 16, 64, 64
+    inp = _to_dev(synth.prefill_inputs(L, H, d, seed=14))
+    ld = 304
+    sc = torch.zeros((L, ld), device=DEV)
+    idxc.indexer_prefill(inp.q, inp.k, inp.w, k_top, scores_out=sc, flags=idxc.FLAG_FILL_MASKED)
+    out = torch.full((L, k_top), -7, dtype=torch.int32, device=DEV)
+    idxc.topk_rows(sc, k_top, out, first_len=L, len_step=0)
+    out = out.cpu().numpy()
+    host = sc.cpu().to(torch.float64).numpy()
+    for r in range(L):
+        assert np.array_equal(out[r], oracle.topk(host[r, :L], k_top)), f"row {r}"
+    assert out[10].tolist() == list(range(k_top))                        # 11 finite scores, then masked ones in order
+
+
 def test_topk_rows_causal_lengths_and_empty():
     g = torch.Generator().manual_seed(5)
     n_rows, ld, k_top = 70, 72, 16
@@ -117,6 +200,15 @@ def test_topk_rows_causal_lengths_and_empty():
     (700, 32, 128, 64, False, 0),
     (900, 64, 128, 100, True, 0),
     (333, 16, 128, 40, True, 0),
+    # the remaining (d_I, H_I, dtype) kernels the library accepts
+    (640, 64, 64, 50, False, 0),
+    (450, 16, 128, 33, False, 0),
+    (520, 32, 128, 77, True, 0),
+    # odd sizes around a key tile and a work item
+    (1, 64, 128, 4, False, 0),
+    (127, 64, 128, 16, False, 0),
+    (129, 64, 128, 16, True, 0),
+    (2049, 64, 128, 256, False, 0),
 ])
 def test_prefill_matches_oracle(L, H, d, k_top, fp8, flags):
     inp = _to_dev(synth.prefill_inputs(L, H, d, seed=10 + L, fp8=fp8))
@@ -229,6 +321,12 @@ def test_prefill_rejects_bad_arguments():
     (5, 16, 64, 32, False, [129, 2048, 31, 1025, 4000], 0),
     (3, 32, 128, 48, True, [999, 2500, 50], 0),
     (2, 64, 128, 2048, False, [2047, 5000], 0),
+    # the remaining (d_I, H_I, dtype) kernels the library accepts
+    (3, 32, 64, 16, False, [640, 129, 3000], 0),
+    (2, 64, 64, 40, False, [2500, 77], 0),
+    (3, 16, 128, 24, False, [128, 1000, 2305], 0),
+    (4, 32, 128, 64, False, [1, 2049, 300, 4097], 0),
+    (3, 16, 128, 20, True, [700, 2100, 33], 0),
 ])
 def test_decode_matches_oracle(B, H, d, k_top, fp8, lens, flags):
     inp = _to_dev(synth.decode_inputs(B, H, d, 0, 0, seed=20 + B, fp8=fp8, lens=lens, row_align=8))

@@ -139,3 +139,25 @@ def test_empty_selection():
     out, lse = sparse_attn.sparse_attention(qb, kb, topk, 2, 1.0)
     assert np.all(out[0] == 0) and np.all(np.isneginf(lse[0]))
     assert np.all(lse[1] == 0.0)
+
+
+def test_entries_that_name_no_cache_row_select_nothing():
+    # an entry past the end of the cache (or, with a sequence base, before its start) is padding: the result equals the
+    # one with those entries removed, and a query whose entries all fall outside gets out = 0, lse = -inf
+    rng = np.random.default_rng(17)
+    n_kv, H, d_qk, d_v = 12, 2, 8, 4
+    qb, _ = _rand_bf16(rng, (3, H, d_qk))
+    kb, _ = _rand_bf16(rng, (n_kv, d_qk))
+    dirty = np.array([[3, 12, 7, 500, -1, 0], [12, 13, 99, -1, -1, -1], [11, 2 ** 30, 5, -1, 12, 1]], dtype=np.int32)
+    clean = np.array([[3, 7, 0, -1, -1, -1], [-1, -1, -1, -1, -1, -1], [11, 5, 1, -1, -1, -1]], dtype=np.int32)
+    out_d, lse_d = sparse_attn.sparse_attention(qb, kb, dirty, d_v, 0.3)
+    out_c, lse_c = sparse_attn.sparse_attention(qb, kb, clean, d_v, 0.3)
+    assert np.array_equal(out_d, out_c) and np.array_equal(lse_d, lse_c)
+    assert np.all(out_d[1] == 0) and np.all(np.isneginf(lse_d[1]))
+    # with a base offset the test is on the row actually named: base + entry
+    base = np.array([4, 10, 0], dtype=np.int64)
+    rel = np.array([[0, 7, 8, -1, -1, -1], [1, 2, 5, -1, -1, -1], [0, 11, 12, -1, -1, -1]], dtype=np.int32)
+    rel_clean = np.array([[0, 7, -1, -1, -1, -1], [1, -1, -1, -1, -1, -1], [0, 11, -1, -1, -1, -1]], dtype=np.int32)
+    a = sparse_attn.sparse_attention(qb, kb, rel, d_v, 0.3, kv_base=base)
+    b = sparse_attn.sparse_attention(qb, kb, rel_clean, d_v, 0.3, kv_base=base)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
