@@ -315,6 +315,14 @@ idxc_status idxc_poll_device_status(void* cuda_stream);
  * once, and IDXC_OK afterwards. Nothing traps or faults. */
 idxc_status idxc_selftest_bounded_wait(uint32_t wait_cycles, void* cuda_stream);
 
+/* Measurement aid (no counterpart in the paper): the rate at which the prefill scorer's epilogue can read fp32
+ * accumulators out of tensor memory, which bounds the FP8 scorer (its tensor work per accumulator is half the bf16
+ * scorer's, its read-out the same). Enqueues one kernel with the scorer's CTA shape (one CTA per SM, 8 reading warps)
+ * in which every reading warp reads its share (32 lanes x 128 columns) of accumulators_per_warp accumulators with the
+ * epilogue's own loads and nothing else runs. *bytes_read_out (HOST, may be NULL) = accumulator bytes the launch reads
+ * over all SMs; time the launch with events around the call to get bytes per second. 1 <= accumulators_per_warp <= 2^24. */
+idxc_status idxc_selftest_tmem_readout(uint32_t accumulators_per_warp, int64_t* bytes_read_out, void* cuda_stream);
+
 /* Number of kernel launches this library has made in this process (all streams). */
 int64_t idxc_launch_count(void);
 

@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = [
     "idxc_indexer_decode", "idxc_topk_rows", "idxc_schedule_create", "idxc_schedule_destroy",
     "idxc_schedule_begin_pass", "idxc_schedule_source", "idxc_schedule_stats", "idxc_schedule_prefill_layer",
     "idxc_schedule_decode_layer", "idxc_poll_device_status", "idxc_launch_count", "idxc_indexer_decode_noalloc",
-    "idxc_selftest_bounded_wait", "idxc_quantize_e4m3", "idxc_topk_overlap", "idxc_pattern_search_dp",
+    "idxc_selftest_bounded_wait", "idxc_selftest_tmem_readout", "idxc_quantize_e4m3", "idxc_topk_overlap", "idxc_pattern_search_dp",
     "idxc_pattern_search_greedy", "idxc_distill_kl", "idxc_sparse_attention_workspace_bytes", "idxc_sparse_attention",
 ]
 NOALLOC_SCRATCH_BYTES = 16 << 20
@@ -101,6 +101,8 @@ def lib() -> ctypes.CDLL:
         L.idxc_quantize_e4m3.argtypes = [vp, i64, i32, vp, vp, vp, vp]
         L.idxc_selftest_bounded_wait.restype = i32
         L.idxc_selftest_bounded_wait.argtypes = [u32, vp]
+        L.idxc_selftest_tmem_readout.restype = i32
+        L.idxc_selftest_tmem_readout.argtypes = [u32, ctypes.POINTER(i64), vp]
         L.idxc_poll_device_status.restype = i32
         L.idxc_poll_device_status.argtypes = [vp]
         _lib = L
@@ -352,6 +354,15 @@ def selftest_bounded_wait(wait_cycles: int = 1_000_000, stream=None):
     """idxc_selftest_bounded_wait: enqueue a kernel whose wait can never be satisfied; the next
     poll_device_status() must raise IdxcError(ERR_DEVICE_TIMEOUT)."""
     _check(lib().idxc_selftest_bounded_wait(int(wait_cycles), _stream(stream)), "idxc_selftest_bounded_wait")
+
+
+def selftest_tmem_readout(accumulators_per_warp: int, stream=None) -> int:
+    """idxc_selftest_tmem_readout: enqueue the tensor-memory read-out measurement kernel; returns the accumulator bytes
+    the launch reads over all SMs (time the call with CUDA events)."""
+    nbytes = ctypes.c_int64()
+    _check(lib().idxc_selftest_tmem_readout(int(accumulators_per_warp), ctypes.byref(nbytes), _stream(stream)),
+           "idxc_selftest_tmem_readout")
+    return int(nbytes.value)
 
 
 def poll_device_status(stream=None):

@@ -470,6 +470,18 @@ idxc_status idxc_selftest_bounded_wait(uint32_t wait_cycles, void* cuda_stream) 
                ? IDXC_OK : IDXC_ERR_CUDA;
 }
 
+idxc_status idxc_selftest_tmem_readout(uint32_t accumulators_per_warp, int64_t* bytes_read_out, void* cuda_stream) {
+    DeviceInfo& di = device_info();
+    if (!di.ok) return IDXC_ERR_CUDA;
+    if (accumulators_per_warp == 0 || accumulators_per_warp > (1u << 24)) return IDXC_ERR_INVALID_ARG;
+    // each of the 8 reading warps of an SM reads its 32 lanes x 128 columns share of `accumulators_per_warp` accumulators
+    if (bytes_read_out) *bytes_read_out = static_cast<int64_t>(di.sm_count) * 8 * accumulators_per_warp * (32 * 128 * 4);
+    g_launches += 1;
+    // the status word doubles as the sink: the kernel never writes it in practice (see selftest.cu)
+    return launch_selftest_tmem_readout(accumulators_per_warp, di.status_ptr, di.sm_count, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+               ? IDXC_OK : IDXC_ERR_CUDA;
+}
+
 idxc_status idxc_poll_device_status(void* cuda_stream) {
     if (!device_info().ok) return IDXC_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);

@@ -84,5 +84,8 @@ cudaError_t launch_sparse_attn(const void* kv, const int32_t* topk, const int64_
 // selftest.cu: one tiny kernel whose only wait can never be satisfied; it must record a time-out in
 // `status` after `budget_cycles` and return.
 cudaError_t launch_selftest_bounded_wait(unsigned int* status, long long budget_cycles, cudaStream_t stream);
+// selftest.cu: every SM reads `iters` 128 x 256 fp32 accumulators per reading warp out of tensor memory with the
+// prefill epilogue's load pattern (8 warps per SM); `sink` is a device word that is never written in practice.
+cudaError_t launch_selftest_tmem_readout(uint32_t iters, uint32_t* sink, int sm_count, cudaStream_t stream);
 
 }  // namespace idxc
