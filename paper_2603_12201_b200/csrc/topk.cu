@@ -34,11 +34,8 @@ namespace {
 constexpr int TK_BINS = 1024;
 constexpr int TK_MAP_MAX_BYTES = 128 * 1024;      // rows up to 524288 scores use the map
 constexpr int TK_SMALL = 128;                     // scores ranked by direct comparison at most
-constexpr float TK_MARGIN_SIGMAS = 3.5f;          // half-width of the bracket in standard deviations of the sampled rank
 
-struct alignas(16) TopkRowSmem {
-    float part_sum[32], part_sq[32];
-    uint32_t part_cnt[32];
+struct alignas(16) TopkRowSmem : SampleSmem {
     uint32_t part_a[32], part_c[32];
     uint32_t cand_count;
     uint32_t small_count;
@@ -46,39 +43,6 @@ struct alignas(16) TopkRowSmem {
     uint32_t small_idx[TK_SMALL];
 };
 
-__device__ __forceinline__ void flag_selected(uint32_t* sel_map, uint32_t idx) {
-    atomicOr(&sel_map[idx >> 4], 1u << (8u * ((idx >> 2) & 3u) + (idx & 3u)));
-}
-// 0xFFFFFFFF if a >= b else 0 (false for NaN)
-__device__ __forceinline__ uint32_t ge_mask(float a, float b) {
-    uint32_t r;
-    asm("set.ge.u32.f32 %0, %1, %2;" : "=r"(r) : "f"(a), "f"(b));
-    return r;
-}
-// z with P(N(0,1) > z) = p, to about 1e-3 (Abramowitz & Stegun 26.2.23), clamped to [-2.5, 2.5]
-__device__ __forceinline__ float upper_quantile_z(float p) {
-    const bool upper = p <= 0.5f;
-    const float q = fminf(fmaxf(upper ? p : 1.f - p, 1e-6f), 0.5f);
-    const float t2 = -2.f * __logf(q);
-    const float t = t2 * rsqrtf(t2);
-    const float zz = t - __fdividef(2.515517f + t * (0.802853f + t * 0.010328f), 1.f + t * (1.432788f + t * (0.189269f + t * 0.001308f)));
-    return fminf(fmaxf(upper ? zz : -zz, -2.5f), 2.5f);
-}
-// bits 0-3, 8-11, 16-19, 24-27 of m (a map word's nibbles of one kind) as one 16-bit mask: bit j <-> position 16 w + j
-__device__ __forceinline__ uint32_t squeeze_nibbles(uint32_t m) {
-    return (m & 0xFu) | ((m >> 4) & 0xF0u) | ((m >> 8) & 0xF00u) | ((m >> 12) & 0xF000u);
-}
-// exclusive prefix sum of v over the lanes of a warp; total = the warp's sum
-__device__ __forceinline__ uint32_t warp_excl_scan(uint32_t v, int lane, uint32_t& total) {
-    uint32_t inc = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-        if (lane >= o) inc += y;
-    }
-    total = __shfl_sync(0xFFFFFFFFu, inc, 31);
-    return inc - v;
-}
 // CAP candidates (fine bin, position) in dynamic shared memory behind the map.
 template <int THREADS, int MIN_BLOCKS, int CAP>
 __global__ void __launch_bounds__(THREADS, MIN_BLOCKS)
@@ -115,119 +79,17 @@ topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int64_t n_rows, i
         const int seg = (((n + WARPS - 1) / WARPS) + 127) & ~127;
         const int seg_begin = wid * seg < n ? wid * seg : n;
         const int seg_end = seg_begin + seg < n ? seg_begin + seg : n;
-        // this warp's sample: S blocks of 128 scores, `stride` apart, from the start of its segment; over the block
-        // 2048 scores per 32768 of the row, at least 2048
-        const int seg_blocks = seg >> 7;
-        int S = (16 * ((n + 32767) >> 15) + WARPS - 1) / WARPS;
-        S = S < U ? U : S;
-        S = S > seg_blocks ? seg_blocks : S;
-        const int stride = (seg_blocks / S) << 7;
-        // calls f(float4, index of its first score) for the lane's part of every sample block
-        auto for_sample = [&](auto f) {
-            for (int j0 = 0; j0 < S; j0 += U) {
-                float4 x[U];
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    const int base = seg_begin + (j0 + u) * stride + 4 * lane;
-                    x[u] = (j0 + u < S && base < seg_end) ? __ldg(reinterpret_cast<const float4*>(src + base))
-                                                         : make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    const int base = seg_begin + (j0 + u) * stride + 4 * lane;
-                    if (j0 + u < S && base < seg_end) f(x[u], base);
-                }
-            }
-        };
-
-        // ---- the sample: mean and spread
+        // ---- the sample and the two pivot scores around the k-th largest (the same code serves the cluster kernel)
         __syncthreads();   // earlier readers of sm, rs and the map are done
-        zero_hist<THREADS>(sm, TK_BINS);
-        {
-            float s1 = 0.f, s2 = 0.f;
-            uint32_t m = 0;
-            for_sample([&](const float4& x, int base) {
-                const float xs[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (base + e < n) { s1 += xs[e]; s2 = fmaf(xs[e], xs[e], s2); ++m; }
-            });
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                s1 += __shfl_xor_sync(0xFFFFFFFFu, s1, o);
-                s2 += __shfl_xor_sync(0xFFFFFFFFu, s2, o);
-                m += __shfl_xor_sync(0xFFFFFFFFu, m, o);
-            }
-            if (lane == 0) { rs.part_sum[wid] = s1; rs.part_sq[wid] = s2; rs.part_cnt[wid] = m; }
-            if (threadIdx.x == 0) { rs.cand_count = 0u; rs.small_count = 0u; }
-        }
-        __syncthreads();
-        float scale, offset;
-        uint32_t m_sample = 0;
-        {
-            float s1 = 0.f, s2 = 0.f;
-#pragma unroll
-            for (int w = 0; w < WARPS; ++w) { s1 += rs.part_sum[w]; s2 += rs.part_sq[w]; m_sample += rs.part_cnt[w]; }
-            const float inv_m = __fdividef(1.f, static_cast<float>(m_sample));
-            const float mean = s1 * inv_m;
-            const float var = fmaxf(s2 * inv_m - mean * mean, 0.f);
-            const float sd = var * rsqrtf(fmaxf(var, 1e-37f));
-            // where the k-th largest of n draws of such a distribution is expected, in standard deviations from the mean
-            // (a rough inverse normal distribution is enough: it only centres the bins)
-            const float z = upper_quantile_z(__fdividef(static_cast<float>(k_top), static_cast<float>(n)));
-            const float half = 1.5f * sd;                         // the bins span [centre - half, centre + half)
-            scale = __fdividef(0.5f * TK_BINS, half);
-            offset = -(mean + z * sd - half) * scale;
-            // a constant sample, or one with infinities, gives no usable map: the row takes the keys-only path
-            if (!(sd > 0.f) || !(fabsf(scale) < 3.0e38f) || !(fabsf(offset) < 3.0e38f)) scale = 0.f;
-        }
-        if (scale == 0.f) {                                      // the same for every thread
+        if (threadIdx.x == 0) { rs.cand_count = 0u; rs.small_count = 0u; }
+        const Pivots pv = sample_pivots<THREADS, TK_BINS>(sm, rs, src, n, k_top, slot);
+        if (!pv.usable) {                                        // the same for every thread
             slow_path_full<THREADS>(sm, src, n, k, out_row, slot);
             continue;
         }
-        // ---- histogram of the sample, pivots
-        for_sample([&](const float4& x, int base) {
-            const float xs[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                if (base + e < n) {
-                    const int b = __float2int_rd(__fmaf_rn(xs[e], scale, offset));     // NaN -> 0; saturates
-                    atomicAdd(&sm.hist[min(max(b, 0), TK_BINS - 1)], 1u);
-                }
-            }
-        });
-        __syncthreads();
-        // rank of the k-th largest of the row inside the sample, and its standard deviation under sampling without replacement
-        const float mf = static_cast<float>(m_sample), nf = static_cast<float>(n);
-        const float p = __fdividef(static_cast<float>(k_top), nf);
-        const float r = mf * p;
-        const float var_r = fmaxf(mf * p * (1.f - p) * __fdividef(nf - mf, fmaxf(nf - 1.f, 1.f)), 0.f);
-        const float sd_r = var_r * rsqrtf(fmaxf(var_r, 1e-37f));
-        const bool whole = m_sample == static_cast<uint32_t>(n);          // the sample is the row: ranks are exact
-        const float margin = whole ? 0.f : TK_MARGIN_SIGMAS * sd_r + 2.f;
-        const int r_hi = whole ? k_top : static_cast<int>(floorf(r - margin));  // sample ranks below r_hi: certainly selected
-        const int r_lo = whole ? k_top : static_cast<int>(ceilf(r + margin));   // sample ranks above r_lo: certainly not
-        const bool has_hi = r_hi >= 1;
-        const bool has_lo = r_lo <= static_cast<int>(m_sample);
-        uint32_t hi_bin, lo_bin, ab_hi, ab_lo;
-        select_two_buckets<TK_BINS, THREADS>(sm, has_hi ? r_hi : 1, has_lo ? r_lo : m_sample, slot, hi_bin, ab_hi, lo_bin, ab_lo);
-        // the pivots as scores: the upper edge of bin hi_bin and the lower edge of bin lo_bin (any bracket will do, so the
-        // rounding of these two divisions does not matter); an end bin has no edge on its outer side
-        const float inv_scale = __fdividef(1.f, scale);
-        const float lo_x = (!has_lo || lo_bin == 0u) ? -INFINITY : (static_cast<float>(lo_bin) - offset) * inv_scale;
-        const float hi_x = (!has_hi || hi_bin == TK_BINS - 1) ? INFINITY : (static_cast<float>(hi_bin + 1u) - offset) * inv_scale;
+        const float lo_x = pv.lo_x, hi_x = pv.hi_x;
 
         // ---- the sweep: flag the scores at or above the upper pivot and those between the pivots
-        auto flag4 = [&](const float4& v) -> uint32_t {
-            const float x[4] = {v.x, v.y, v.z, v.w};
-            uint32_t sel = 0, ge_lo = 0;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                sel |= ge_mask(x[e], hi_x) & (1u << e);
-                ge_lo |= ge_mask(x[e], lo_x) & (16u << e);
-            }
-            return sel | (ge_lo & ~(sel << 4));                         // high nibble: between the pivots
-        };
         {
             // whole steps of U blocks that lie inside the segment and the row need no bounds checks
             const int full_end = seg_begin + ((seg_end & ~3) - seg_begin) / (128 * U) * (128 * U);
@@ -239,13 +101,13 @@ topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int64_t n_rows, i
 #pragma unroll
                 for (int u = 0; u < U; ++u) x4[u] = __ldg(reinterpret_cast<const float4*>(p + 128 * u));
 #pragma unroll
-                for (int u = 0; u < U; ++u) mb[32 * u] = static_cast<uint8_t>(flag4(x4[u]));
+                for (int u = 0; u < U; ++u) mb[32 * u] = static_cast<uint8_t>(flag4(x4[u], lo_x, hi_x));
             }
             for (; cb < seg_end; cb += 128) {                           // the ragged rest, one block at a time
                 const int base = cb + 4 * lane;
                 uint32_t flags = 0;
                 if (base < n) {
-                    flags = flag4(__ldg(reinterpret_cast<const float4*>(src + base)));
+                    flags = flag4(__ldg(reinterpret_cast<const float4*>(src + base)), lo_x, hi_x);
                     const int left = n - base;                          // scores of this 128-bit load inside the row
                     if (left < 4) flags &= (0x11u << left) - 0x11u;
                 }
@@ -302,14 +164,7 @@ topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int64_t n_rows, i
         }
         __syncthreads();
         // ---- candidates: finer bins across the band
-        const float y_lo = (has_lo && lo_bin != 0u) ? static_cast<float>(lo_bin) : 0.f;
-        const float y_hi = (has_hi && hi_bin != TK_BINS - 1) ? static_cast<float>(hi_bin + 1u) : static_cast<float>(TK_BINS);
-        const float fscale = __fdividef(static_cast<float>(TK_BINS), y_hi - y_lo);
-        auto fine_bin = [&](float x) -> uint32_t {
-            const float y = __fmaf_rn(x, scale, offset);
-            const int b = __float2int_rd((y - y_lo) * fscale);
-            return static_cast<uint32_t>(min(max(b, 0), TK_BINS - 1));
-        };
+        auto fine_bin = [&](float x) -> uint32_t { return pv.fine_bin<TK_BINS>(x); };
         for (uint32_t i = threadIdx.x; i < C; i += THREADS) {             // independent loads (L2), all in flight together
             const uint32_t fb = fine_bin(__ldg(src + cand_idx[i]));
             cand_fb[i] = fb;

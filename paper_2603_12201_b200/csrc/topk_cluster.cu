@@ -1,21 +1,20 @@
 // Top-k select for a FEW LONG rows (decode: one row of up to 128K scores per sequence), Sec. 3
 // "Notation" T_t = Top-k(I_t) as in topk.cu, but with one thread-block CLUSTER of 8 CTAs per row so
-// that a batch of 8-32 rows fills the GPU. Each CTA owns one eighth of the row; the CTAs exchange
-// their results through distributed shared memory:
-//   1. every CTA histograms the top 12 key bits of its part                           (cluster sync)
-//   2. CTA r sums bins [512r, 512r+512) over the 8 histograms and publishes the total (cluster sync)
-//   3. the CTA whose bins hold the k-th largest score finds the threshold bucket b1 and
-//      broadcasts it                                                                   (cluster sync)
-//   4. every CTA flags its scores above b1 (selected) and inside it (candidates) in a local map
-//      and copies its candidates (low key bits, position) into the leader's buffer     (cluster sync)
-//   5. the leader finds the exact threshold among the candidates (digits 2 and 3) and the
-//      position limit for ties, and broadcasts them                                    (cluster sync)
-//   6. every CTA flags its selected candidates, counts its selected positions and
-//      publishes the count                                                             (cluster sync)
-//   7. every CTA emits its positions at rank (selected in lower parts) + local prefix.
-// Same result as the one-CTA kernel: ascending positions, ties to the lowest position.
-// Rows whose threshold bucket holds more candidates than the leader's buffer are finished by the
-// leader alone with the slow path of topk_common.cuh.
+// that a batch of 8-32 rows fills the GPU. Same one-sweep algorithm as the row kernel; each CTA owns one
+// eighth of the row and the CTAs exchange their counts through distributed shared memory:
+//   1. every CTA samples the WHOLE row and derives the same two pivot scores (identical arithmetic on identical
+//      data: no exchange needed), then sweeps its own part once: scores at or above the upper pivot are flagged
+//      in a local map, scores between the pivots are candidates; it publishes its two counts   (cluster sync)
+//   2. with A scores above and C candidates over the cluster the bracket held iff A < k <= A + C. Every CTA sorts
+//      its candidates into 1024 finer bins across the band                                    (cluster sync)
+//   3. every CTA adds the eight histograms up, finds the bin of the wanted rank, flags its candidates in higher
+//      bins and appends those inside that bin (a handful) to a list in the leader              (cluster sync)
+//   4. every CTA ranks that list by direct comparison of the 32-bit keys (larger key first, lower position first
+//      among equal keys), flags its own winners, counts its selected positions and publishes   (cluster sync)
+//   5. every CTA emits its positions at rank (selected in lower parts) + local prefix.
+// Same result as the one-CTA kernel: ascending positions, ties to the lowest position. Rows the fast path cannot
+// separate (bracket missed, crowded threshold bin, a list overflow, constant or non-finite sample, parts longer
+// than the map) are selected by the leader alone on keys (slow_path_full of topk_common.cuh).
 #include <cooperative_groups.h>
 
 #include "kernels.h"
@@ -27,37 +26,45 @@ namespace idxc {
 using namespace topk;
 namespace {
 
-constexpr int CL_D1 = 12;             // first digit: top 12 key bits
-constexpr int TK_BINS1 = 1 << CL_D1;
 constexpr int CL_SIZE = 8;            // CTAs per row
 constexpr int CL_THREADS = 512;
 constexpr int CL_WARPS = CL_THREADS / 32;
-constexpr int CL_BINS_PER_RANK = TK_BINS1 / CL_SIZE;      // 512: one bin per thread in the reduction
-constexpr int CL_CAP = 4096;          // candidates the leader can hold
+constexpr int CL_BINS = 1024;         // bins of the sample histogram and of the finer candidate histogram
+constexpr int CL_CAP = 1024;          // candidates one CTA can list
+constexpr int CL_SMALL = 128;         // scores ranked by direct comparison at most
 constexpr int CL_MAX_PART = 65536;    // scores per CTA the local map can flag (rows up to 524288)
-static_assert(CL_BINS_PER_RANK == CL_THREADS, "the bin reduction assigns one bin per thread");
+constexpr int U = TK_UNROLL;
 
+// The per-rank counts are written by the other CTAs of the cluster. They exist twice and successive rows alternate
+// between the copies: a CTA that has run ahead into the next row then never writes into counts a slower CTA is still
+// reading (it cannot get two rows ahead: every row has a cluster barrier).
 struct ClusterExchange {
-    uint32_t red[CL_BINS_PER_RANK];   // my 512 bins summed over the cluster
-    uint32_t part_tot[CL_SIZE];       // total of each rank's 512 bins
-    uint32_t bcast[4];                // b1, scores above b1, scores inside b1
-    uint32_t cand_total;              // leader: candidate slots handed out
-    uint32_t cand_base;               // first slot of this CTA's candidates
-    uint32_t tsel[2];                 // low 20 key bits of the threshold, position limit for ties
-    uint32_t sel_cnt[CL_SIZE];        // selected positions per part
+    uint32_t part_a[2][CL_SIZE];      // scores above the band, per rank (every CTA holds all eight)
+    uint32_t part_c[2][CL_SIZE];      // candidates, per rank
+    uint32_t sel_cnt[2][CL_SIZE];     // selected positions, per rank
+    uint32_t small_count;             // leader: entries of the list below
+    uint32_t small_key[CL_SMALL];     // leader: keys and positions of the candidates inside the threshold bin
+    uint32_t small_idx[CL_SMALL];
+};
+
+struct ClusterRowSmem : SampleSmem {
+    uint32_t warp_cnt[2][CL_WARPS];
+    uint32_t cand_count;
 };
 
 __global__ void __launch_bounds__(CL_THREADS, 2)
 topk_rows_cluster_kernel(const float* __restrict__ scores, int64_t ld, int64_t n_rows, int64_t first_len, int64_t len_step,
                          const int32_t* __restrict__ lens, int k_top, int32_t* __restrict__ out, int map_bytes) {
     cg::cluster_group cluster = cg::this_cluster();
-    __shared__ __align__(16) TopkSmem<CL_WARPS, TK_BINS1> sm;
+    __shared__ __align__(16) TopkSmem<CL_WARPS, 2048> sm;      // [0, 1024): sample histogram, then the summed fine histogram;
+                                                               // [1024, 2048): this CTA's fine histogram; all 2048: keys-only path
+    __shared__ ClusterRowSmem rs;
     __shared__ ClusterExchange ex;
     extern __shared__ uint32_t dyn[];
     uint32_t* sel_map = dyn;                                   // map_bytes: one byte per 4 scores of my part
     uint8_t* sel_bytes = reinterpret_cast<uint8_t*>(sel_map);
-    uint32_t* cand_key = dyn + map_bytes / 4;                  // leader only: CL_CAP keys, CL_CAP positions
-    uint32_t* cand_idx = cand_key + CL_CAP;
+    uint32_t* cand_fb = dyn + map_bytes / 4;                   // my candidates: fine bin ...
+    uint32_t* cand_idx = cand_fb + CL_CAP;                     // ... and position in the row
     const unsigned rank = cluster.block_rank();
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const int tid = threadIdx.x;
@@ -65,7 +72,9 @@ topk_rows_cluster_kernel(const float* __restrict__ scores, int64_t ld, int64_t n
     const int64_t n_clusters = gridDim.x / CL_SIZE;
     int slot = 0;
 
+    int par = 1;
     for (int64_t row = blockIdx.x / CL_SIZE; row < n_rows; row += n_clusters) {
+        par ^= 1;                                              // which copy of the exchanged counts this row uses
         int64_t len = lens ? static_cast<int64_t>(lens[row]) : first_len + row * len_step;
         len = len < 0 ? 0 : (len > ld ? ld : len);
         const int n = static_cast<int>(len);
@@ -84,147 +93,181 @@ topk_rows_cluster_kernel(const float* __restrict__ scores, int64_t ld, int64_t n
         const int seg = (((pn + CL_WARPS - 1) / CL_WARPS) + 127) & ~127;
         const int seg_begin = pb + (wid * seg < pn ? wid * seg : pn);
         const int seg_end = seg_begin + seg < pe ? seg_begin + seg : pe;
-
-        // ---- 1. local histogram of the top 12 key bits
-        __syncthreads();
-        zero_hist<CL_THREADS>(sm, TK_BINS1);
-        if (tid == 0) ex.cand_total = 0u;
-        __syncthreads();
-        sweep_segment<TK_UNROLL>(src, n, seg_begin, seg_end, lane, [&](const float4& x, int base) {
-            const float xs[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e)
-                if (base + e < n) atomicAdd(&sm.hist[score_digit1<CL_D1>(xs[e])], 1u);
-        });
-        cluster.sync();                                                                        // (1)
-        // ---- 2. sum my 512 bins over the cluster
-        uint32_t v = 0;
-#pragma unroll
-        for (int r = 0; r < CL_SIZE; ++r) v += cluster.map_shared_rank(sm.hist, r)[rank * CL_BINS_PER_RANK + tid];
-        ex.red[tid] = v;
-        uint32_t my_total;
-        (void)block_excl_scan<CL_WARPS>(v, sm, slot, my_total);
-        if (tid < CL_SIZE) cluster.map_shared_rank(ex.part_tot, tid)[rank] = my_total;
-        cluster.sync();                                                                        // (2)
-        // ---- 3. the CTA whose bins hold the k-th largest score selects the bucket
-        uint32_t above_mine = 0;
-        for (unsigned r = rank + 1; r < CL_SIZE; ++r) above_mine += ex.part_tot[r];            // higher ranks hold higher bins
-        if (above_mine < k && k <= above_mine + my_total) {                                    // block-uniform
-            sm.hist[tid] = ex.red[tid];                                                        // remote readers of hist are done
-            __syncthreads();
-            uint32_t bl, al;
-            select_bucket<CL_BINS_PER_RANK, CL_THREADS>(sm, k - above_mine, slot, bl, al);
-            if (tid < CL_SIZE) {
-                uint32_t* dst = cluster.map_shared_rank(ex.bcast, tid);
-                dst[0] = rank * CL_BINS_PER_RANK + bl;
-                dst[1] = above_mine + al;
-                dst[2] = ex.red[bl];
-            }
-        }
-        cluster.sync();                                                                        // (3)
-        const uint32_t b1 = ex.bcast[0];
-        const uint32_t c1 = ex.bcast[2];
-        const uint32_t need = k - ex.bcast[1];                 // rank inside bucket b1, 1-based
-        if (c1 > static_cast<uint32_t>(CL_CAP) || part > map_bytes * 4 || !bucket_is_finite<CL_D1>(b1)) {   // cluster-uniform
-            if (rank == 0) slow_path<CL_THREADS, CL_D1>(sm, src, n, b1, need, k, out_row, slot);
+        if (part > map_bytes * 4) {                            // cluster-uniform: parts longer than the map
+            if (rank == 0) slow_path_full<CL_THREADS>(sm, src, n, k, out_row, slot);
             continue;
         }
-        // ---- 4. flag my scores above bucket b1 (selected) and inside it (candidates)
-        const float lo = key_to_score(b1 << 20);
-        const bool has_above = b1 < TK_BINS1 - 1;
-        const float hi = key_to_score(has_above ? ((b1 + 1) << 20) : 0xFFFFFFFFu);
-        sweep_segment<TK_UNROLL>(src, n, seg_begin, seg_end, lane, [&](const float4& x4, int base) {
-            const float x[4] = {x4.x, x4.y, x4.z, x4.w};
-            uint32_t flags = 0;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                if (base + e >= n || !(x[e] >= lo)) continue;
-                flags |= (has_above && x[e] >= hi) ? (1u << e) : (16u << e);
-            }
-            sel_bytes[(base - pb) >> 2] = static_cast<uint8_t>(flags);
-        });
-        __syncthreads();
-        const int words = (pn + 15) >> 4;
-        const int wpt = (words + CL_THREADS - 1) / CL_THREADS;
-        const int w0 = tid * wpt < words ? tid * wpt : words;
-        const int w1 = w0 + wpt < words ? w0 + wpt : words;
+        // ---- 1. pivots from a sample of the whole row (the same in every CTA), then one sweep over my part
+        __syncthreads();                                       // earlier readers of sm, rs and the map are done
+        if (tid == 0) { rs.cand_count = 0u; if (rank == 0) ex.small_count = 0u; }
+        const Pivots pv = sample_pivots<CL_THREADS, CL_BINS>(sm, rs, src, n, k_top, slot);
+        if (!pv.usable) {                                      // cluster-uniform
+            if (rank == 0) slow_path_full<CL_THREADS>(sm, src, n, k, out_row, slot);
+            continue;
+        }
         {
-            uint32_t cnt = 0;
-            for (int w = w0; w < w1; ++w) cnt += __popc(sel_map[w] & 0xF0F0F0F0u);
-            uint32_t mine;
-            uint32_t pos = block_excl_scan<CL_WARPS>(cnt, sm, slot, mine);
-            if (tid == 0) ex.cand_base = atomicAdd(cluster.map_shared_rank(&ex.cand_total, 0), mine);
-            __syncthreads();
-            pos += ex.cand_base;
-            uint32_t* lk = cluster.map_shared_rank(cand_key, 0);
-            uint32_t* li = cluster.map_shared_rank(cand_idx, 0);
-            for (int w = w0; w < w1; ++w) {
-                uint32_t m = sel_map[w] & 0xF0F0F0F0u;
+            const float lo_x = pv.lo_x, hi_x = pv.hi_x;
+            const int full_end = seg_begin + (seg_end - seg_begin) / (128 * U) * (128 * U);
+            const float* p = src + seg_begin + 4 * lane;
+            uint8_t* mb = sel_bytes + ((seg_begin - pb) >> 2) + lane;
+            int cb = seg_begin;
+            for (; cb < full_end; cb += 128 * U, p += 128 * U, mb += 32 * U) {
+                float4 x4[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) x4[u] = __ldg(reinterpret_cast<const float4*>(p + 128 * u));
+#pragma unroll
+                for (int u = 0; u < U; ++u) mb[32 * u] = static_cast<uint8_t>(flag4(x4[u], lo_x, hi_x));
+            }
+            for (; cb < seg_end; cb += 128) {                  // the ragged rest, one block at a time
+                const int base = cb + 4 * lane;
+                uint32_t flags = 0;
+                if (base < n) {
+                    flags = flag4(__ldg(reinterpret_cast<const float4*>(src + base)), lo_x, hi_x);
+                    const int left = n - base;                 // scores of this 128-bit load inside the row
+                    if (left < 4) flags &= (0x11u << left) - 0x11u;
+                }
+                sel_bytes[(base - pb) >> 2] = static_cast<uint8_t>(flags);
+            }
+        }
+        __syncwarp();
+        // my warp's map words, and every lane's run of them
+        const int w_begin = (seg_begin - pb) >> 4, w_end = seg_begin < seg_end ? (seg_end - pb + 15) >> 4 : w_begin;
+        const int wpl = (w_end - w_begin + 31) >> 5;
+        const int lw0 = w_begin + lane * wpl < w_end ? w_begin + lane * wpl : w_end;
+        const int lw1 = lw0 + wpl < w_end ? lw0 + wpl : w_end;
+        uint32_t my_cand = 0;                                  // candidates in this lane's run
+        {
+            uint32_t n_sel = 0;
+            for (int w = lw0; w < lw1; ++w) {
+                const uint32_t m = sel_map[w];
+                n_sel += __popc(m & 0x0F0F0F0Fu);
+                my_cand += __popc(m & 0xF0F0F0F0u);
+            }
+            n_sel = __reduce_add_sync(0xFFFFFFFFu, n_sel);
+            const uint32_t n_cand = __reduce_add_sync(0xFFFFFFFFu, my_cand);
+            if (lane == 0) { rs.warp_cnt[0][wid] = n_sel; rs.warp_cnt[1][wid] = n_cand; }
+        }
+        __syncthreads();
+        if (tid < CL_SIZE) {                                   // publish my two counts in every CTA of the cluster
+            uint32_t a = 0, c = 0;
+#pragma unroll
+            for (int w = 0; w < CL_WARPS; ++w) { a += rs.warp_cnt[0][w]; c += rs.warp_cnt[1][w]; }
+            cluster.map_shared_rank(ex.part_a[par], tid)[rank] = a;
+            cluster.map_shared_rank(ex.part_c[par], tid)[rank] = c;
+        }
+        cluster.sync();                                                                        // (1)
+        uint32_t A = 0, C = 0, c_max = 0;
+#pragma unroll
+        for (int r = 0; r < CL_SIZE; ++r) {
+            A += ex.part_a[par][r];
+            C += ex.part_c[par][r];
+            c_max = ex.part_c[par][r] > c_max ? ex.part_c[par][r] : c_max;
+        }
+        if (!(A < k && k - A <= C && c_max <= static_cast<uint32_t>(CL_CAP))) {                // cluster-uniform
+            if (rank == 0) slow_path_full<CL_THREADS>(sm, src, n, k, out_row, slot);
+            continue;
+        }
+        const uint32_t need = k - A;                           // candidates to take, 1..C
+        // ---- 2. list my candidates, sort them into the finer bins
+        for (int i = tid; i < CL_BINS; i += CL_THREADS) sm.hist[CL_BINS + i] = 0u;
+        const uint32_t my_c = ex.part_c[par][rank];
+        {
+            uint32_t total;
+            uint32_t pos = warp_excl_scan(my_cand, lane, total);
+            uint32_t basepos = 0;
+            if (lane == 0 && total != 0u) basepos = atomicAdd(&rs.cand_count, total);
+            pos += __shfl_sync(0xFFFFFFFFu, basepos, 0);
+            for (int w = lw0; w < lw1; ++w) {
+                uint32_t m = squeeze_nibbles(sel_map[w] >> 4);
+                const uint32_t idx0 = static_cast<uint32_t>(pb) + 16u * static_cast<uint32_t>(w);
                 while (m) {
-                    const int b = __ffs(m) - 1;
+                    const uint32_t b = __ffs(m) - 1;
                     m &= m - 1;
-                    const int idx = pb + 16 * w + 4 * (b >> 3) + (b & 7) - 4;
-                    if (pos < static_cast<uint32_t>(CL_CAP)) {
-                        lk[pos] = score_key(__ldg(src + idx)) & 0xFFFFFu;
-                        li[pos] = static_cast<uint32_t>(idx);
-                    }
+                    if (pos < static_cast<uint32_t>(CL_CAP)) cand_idx[pos] = idx0 + b;
                     ++pos;
                 }
             }
         }
-        cluster.sync();                                                                        // (4)
-        // ---- 5. the leader finds the exact threshold among the candidates
-        if (rank == 0) {
-            uint32_t t_low, need_eq, m_eq;
-            candidate_select<CL_THREADS, 32 - CL_D1>(sm, cand_key, c1, need, slot, t_low, need_eq, m_eq);
-            if (tid == 0) ex.cand_base = 0xFFFFFFFFu;          // reused: position limit for ties (none: take all)
-            __syncthreads();
-            if (m_eq != need_eq) {                             // ties compete: the need_eq lowest positions win
-                for (uint32_t i = tid; i < c1; i += CL_THREADS) {
-                    if (cand_key[i] != t_low) continue;
-                    uint32_t before = 0;
-                    for (uint32_t i2 = 0; i2 < c1; ++i2) before += (cand_key[i2] == t_low) & (cand_idx[i2] < cand_idx[i]);
-                    if (before == need_eq - 1) ex.cand_base = cand_idx[i];
+        __syncthreads();
+        for (uint32_t i = tid; i < my_c; i += CL_THREADS) {    // independent loads (L2), all in flight together
+            const uint32_t fb = pv.fine_bin<CL_BINS>(__ldg(src + cand_idx[i]));
+            cand_fb[i] = fb;
+            atomicAdd(&sm.hist[CL_BINS + fb], 1u);
+        }
+        cluster.sync();                                                                        // (2)
+        // ---- 3. the summed histogram, the bin of the wanted rank
+        for (int i = tid; i < CL_BINS; i += CL_THREADS) {
+            uint32_t v = 0;
+#pragma unroll
+            for (int r = 0; r < CL_SIZE; ++r) v += cluster.map_shared_rank(sm.hist, r)[CL_BINS + i];
+            sm.hist[i] = v;
+        }
+        __syncthreads();
+        uint32_t fb1, above_f;
+        select_bucket<CL_BINS, CL_THREADS>(sm, need, slot, fb1, above_f);
+        const uint32_t m1 = sm.hist[fb1];
+        const uint32_t need1 = need - above_f;                 // scores to take from fine bin fb1, 1..m1
+        if (m1 <= static_cast<uint32_t>(CL_SMALL)) {
+            uint32_t* l_count = cluster.map_shared_rank(&ex.small_count, 0);
+            uint32_t* l_key = cluster.map_shared_rank(ex.small_key, 0);
+            uint32_t* l_idx = cluster.map_shared_rank(ex.small_idx, 0);
+            for (uint32_t i = tid; i < my_c; i += CL_THREADS) {
+                const uint32_t fb = cand_fb[i];
+                const uint32_t idx = cand_idx[i];
+                if (fb > fb1) {
+                    flag_selected(sel_map, idx - static_cast<uint32_t>(pb));
+                } else if (fb == fb1) {
+                    const uint32_t pos = atomicAdd(l_count, 1u);
+                    if (pos < static_cast<uint32_t>(CL_SMALL)) { l_key[pos] = score_key(__ldg(src + idx)); l_idx[pos] = idx; }
                 }
             }
-            __syncthreads();
-            if (tid < CL_SIZE) {
-                uint32_t* dst = cluster.map_shared_rank(ex.tsel, tid);
-                dst[0] = t_low;
-                dst[1] = ex.cand_base;
+        }
+        cluster.sync();                                                                        // (3)
+        if (m1 > static_cast<uint32_t>(CL_SMALL)) {            // cluster-uniform: many near-equal scores at the threshold
+            if (rank == 0) slow_path_full<CL_THREADS>(sm, src, n, k, out_row, slot);
+            continue;
+        }
+        // ---- 4. rank the listed scores; flag my winners; count my selected positions
+        {
+            const uint32_t* l_key = cluster.map_shared_rank(ex.small_key, 0);
+            const uint32_t* l_idx = cluster.map_shared_rank(ex.small_idx, 0);
+            for (uint32_t i = tid; i < m1; i += CL_THREADS) {
+                const uint32_t ki = l_key[i], ii = l_idx[i];
+                if (ii < static_cast<uint32_t>(pb) || ii >= static_cast<uint32_t>(pe)) continue;      // not mine
+                uint32_t beaten_by = 0;
+                for (uint32_t j = 0; j < m1; ++j) {
+                    const uint32_t kj = l_key[j], ij = l_idx[j];
+                    beaten_by += (kj > ki) | ((kj == ki) & (ij < ii));
+                }
+                if (beaten_by < need1) flag_selected(sel_map, ii - static_cast<uint32_t>(pb));
             }
         }
-        cluster.sync();                                                                        // (5)
-        const uint32_t t_low = ex.tsel[0], idx_limit = ex.tsel[1];
-        // ---- 6. flag my selected candidates; count my selected positions
-        uint32_t cnt = 0;
-        for (int w = w0; w < w1; ++w) {
-            uint32_t word = sel_map[w];
-            uint32_t m = word & 0xF0F0F0F0u;
+        __syncthreads();
+        uint32_t c_sel = 0;
+        for (int w = lw0; w < lw1; ++w) c_sel += __popc(sel_map[w] & 0x0F0F0F0Fu);
+        uint32_t w_total;
+        uint32_t pos = warp_excl_scan(c_sel, lane, w_total);
+        if (lane == 0) rs.warp_cnt[0][wid] = w_total;
+        __syncthreads();
+        if (tid < CL_SIZE) {
+            uint32_t s = 0;
+#pragma unroll
+            for (int w = 0; w < CL_WARPS; ++w) s += rs.warp_cnt[0][w];
+            cluster.map_shared_rank(ex.sel_cnt[par], tid)[rank] = s;
+        }
+        cluster.sync();                                                                        // (4)
+        // ---- 5. emission
+        for (unsigned r = 0; r < rank; ++r) pos += ex.sel_cnt[par][r];
+#pragma unroll
+        for (int w = 0; w < CL_WARPS; ++w) pos += w < wid ? rs.warp_cnt[0][w] : 0u;
+        for (int w = lw0; w < lw1; ++w) {
+            uint32_t m = squeeze_nibbles(sel_map[w]);
+            const int idx0 = pb + 16 * w;
             while (m) {
                 const int b = __ffs(m) - 1;
                 m &= m - 1;
-                const uint32_t idx = static_cast<uint32_t>(pb + 16 * w + 4 * (b >> 3) + (b & 7) - 4);
-                const uint32_t low = score_key(__ldg(src + idx)) & 0xFFFFFu;
-                if (low > t_low || (low == t_low && idx <= idx_limit)) word |= 1u << (b - 4);
-            }
-            word &= 0x0F0F0F0Fu;
-            sel_map[w] = word;                                 // only this thread touches its words
-            cnt += __popc(word);
-        }
-        uint32_t mine;
-        uint32_t rnk = block_excl_scan<CL_WARPS>(cnt, sm, slot, mine);
-        if (tid < CL_SIZE) cluster.map_shared_rank(ex.sel_cnt, tid)[rank] = mine;
-        cluster.sync();                                                                        // (6)
-        // ---- 7. emission
-        for (unsigned r = 0; r < rank; ++r) rnk += ex.sel_cnt[r];
-        for (int w = w0; w < w1; ++w) {
-            uint32_t m = sel_map[w];
-            while (m) {
-                const int b = __ffs(m) - 1;
-                m &= m - 1;
-                if (rnk < k) out_row[rnk] = pb + 16 * w + 4 * (b >> 3) + (b & 7);
-                ++rnk;
+                if (pos < k) out_row[pos] = idx0 + b;
+                ++pos;
             }
         }
     }

@@ -303,6 +303,191 @@ __device__ __forceinline__ void slow_path(SM& sm, const float* __restrict__ src,
     }
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// Building blocks of the one-sweep select: a sample of the row fixes two pivot scores that bracket the k-th largest.
+
+__device__ __forceinline__ void flag_selected(uint32_t* sel_map, uint32_t idx) {
+    atomicOr(&sel_map[idx >> 4], 1u << (8u * ((idx >> 2) & 3u) + (idx & 3u)));
+}
+// 0xFFFFFFFF if a >= b else 0 (false for NaN)
+__device__ __forceinline__ uint32_t ge_mask(float a, float b) {
+    uint32_t r;
+    asm("set.ge.u32.f32 %0, %1, %2;" : "=r"(r) : "f"(a), "f"(b));
+    return r;
+}
+// z with P(N(0,1) > z) = p, to about 1e-3 (Abramowitz & Stegun 26.2.23), clamped to [-2.5, 2.5]
+__device__ __forceinline__ float upper_quantile_z(float p) {
+    const bool upper = p <= 0.5f;
+    const float q = fminf(fmaxf(upper ? p : 1.f - p, 1e-6f), 0.5f);
+    const float t2 = -2.f * __logf(q);
+    const float t = t2 * rsqrtf(t2);
+    const float zz = t - __fdividef(2.515517f + t * (0.802853f + t * 0.010328f), 1.f + t * (1.432788f + t * (0.189269f + t * 0.001308f)));
+    return fminf(fmaxf(upper ? zz : -zz, -2.5f), 2.5f);
+}
+// bits 0-3, 8-11, 16-19, 24-27 of m (a map word's nibbles of one kind) as one 16-bit mask: bit j <-> position 16 w + j
+__device__ __forceinline__ uint32_t squeeze_nibbles(uint32_t m) {
+    return (m & 0xFu) | ((m >> 4) & 0xF0u) | ((m >> 8) & 0xF00u) | ((m >> 12) & 0xF000u);
+}
+// exclusive prefix sum of v over the lanes of a warp; total = the warp's sum
+__device__ __forceinline__ uint32_t warp_excl_scan(uint32_t v, int lane, uint32_t& total) {
+    uint32_t inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+        if (lane >= o) inc += y;
+    }
+    total = __shfl_sync(0xFFFFFFFFu, inc, 31);
+    return inc - v;
+}
+
+constexpr float TK_MARGIN_SIGMAS = 3.5f;          // half-width of the bracket in standard deviations of the sampled rank
+
+struct SampleSmem {
+    float part_sum[32], part_sq[32];
+    uint32_t part_cnt[32];
+};
+
+// What the sample yields. Scores map monotonically to bins floor(x * scale + offset); lo_x and hi_x are the pivot scores
+// (x >= hi_x: certainly among the k largest; lo_x <= x < hi_x: candidate; below lo_x: certainly not), either may be
+// infinite. [y_lo, y_hi) is the band in bin units, for the finer bins the candidates are sorted into.
+struct Pivots {
+    float scale, offset, lo_x, hi_x, y_lo, fscale;
+    bool usable;
+    template <int BINS>
+    __device__ __forceinline__ uint32_t fine_bin(float x) const {
+        const int b = __float2int_rd((__fmaf_rn(x, scale, offset) - y_lo) * fscale);
+        return static_cast<uint32_t>(min(max(b, 0), BINS - 1));
+    }
+};
+
+// Samples the row (n scores at src, n > k_top): every warp of the block reads S blocks of 128 scores spread evenly over
+// its share n / WARPS of the row (2048 scores per 32768 of the row over the whole block, at least U blocks per warp; the
+// whole row when it is short), the block computes their mean and spread, histograms them in BINS monotone bins laid
+// around where the k-th largest score should lie, and takes as pivots the bin edges next to the sample's scores of rank
+// r -+ (TK_MARGIN_SIGMAS standard deviations of that rank under sampling without replacement), r = k * sample / n.
+// Every thread of the block must call it; it uses sm.hist[0..BINS) and ends after a barrier. A block that calls it
+// with the same row gets the same pivots whatever its place in a cluster. usable = false: the sample is constant or not
+// finite (the caller selects on keys alone).
+template <int THREADS, int BINS, typename SM, typename RS>
+__device__ __forceinline__ Pivots sample_pivots(SM& sm, RS& rs, const float* __restrict__ src, int n, int k_top, int& slot) {
+    constexpr int WARPS = THREADS / 32;
+    constexpr int U = TK_UNROLL;
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const int seg = (((n + WARPS - 1) / WARPS) + 127) & ~127;
+    const int seg_begin = wid * seg < n ? wid * seg : n;
+    const int seg_end = seg_begin + seg < n ? seg_begin + seg : n;
+    const int seg_blocks = seg >> 7;
+    int S = (16 * ((n + 32767) >> 15) + WARPS - 1) / WARPS;
+    S = S < U ? U : S;
+    S = S > seg_blocks ? seg_blocks : S;
+    const int stride = (seg_blocks / S) << 7;
+    // calls f(float4, index of its first score) for the lane's part of every sample block
+    auto for_sample = [&](auto f) {
+        for (int j0 = 0; j0 < S; j0 += U) {
+            float4 x[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int base = seg_begin + (j0 + u) * stride + 4 * lane;
+                x[u] = (j0 + u < S && base < seg_end) ? __ldg(reinterpret_cast<const float4*>(src + base))
+                                                     : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int base = seg_begin + (j0 + u) * stride + 4 * lane;
+                if (j0 + u < S && base < seg_end) f(x[u], base);
+            }
+        }
+    };
+    Pivots pv;
+    // ---- mean and spread
+    zero_hist<THREADS>(sm, BINS);
+    {
+        float s1 = 0.f, s2 = 0.f;
+        uint32_t m = 0;
+        for_sample([&](const float4& x, int base) {
+            const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (base + e < n) { s1 += xs[e]; s2 = fmaf(xs[e], xs[e], s2); ++m; }
+        });
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            s1 += __shfl_xor_sync(0xFFFFFFFFu, s1, o);
+            s2 += __shfl_xor_sync(0xFFFFFFFFu, s2, o);
+            m += __shfl_xor_sync(0xFFFFFFFFu, m, o);
+        }
+        if (lane == 0) { rs.part_sum[wid] = s1; rs.part_sq[wid] = s2; rs.part_cnt[wid] = m; }
+    }
+    __syncthreads();
+    uint32_t m_sample = 0;
+    {
+        float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+        for (int w = 0; w < WARPS; ++w) { s1 += rs.part_sum[w]; s2 += rs.part_sq[w]; m_sample += rs.part_cnt[w]; }
+        const float inv_m = __fdividef(1.f, static_cast<float>(m_sample));
+        const float mean = s1 * inv_m;
+        const float var = fmaxf(s2 * inv_m - mean * mean, 0.f);
+        const float sd = var * rsqrtf(fmaxf(var, 1e-37f));
+        // where the k-th largest of n draws of such a distribution is expected, in standard deviations from the mean
+        // (a rough inverse normal distribution is enough: it only centres the bins)
+        const float z = upper_quantile_z(__fdividef(static_cast<float>(k_top), static_cast<float>(n)));
+        const float half = 1.5f * sd;                         // the bins span [centre - half, centre + half)
+        pv.scale = __fdividef(0.5f * BINS, half);
+        pv.offset = -(mean + z * sd - half) * pv.scale;
+        // a constant sample, or one with infinities, gives no usable map
+        pv.usable = sd > 0.f && fabsf(pv.scale) < 3.0e38f && fabsf(pv.offset) < 3.0e38f;
+    }
+    if (!pv.usable) return pv;                                // the same for every thread
+    // ---- histogram of the sample
+    for_sample([&](const float4& x, int base) {
+        const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (base + e < n) {
+                const int b = __float2int_rd(__fmaf_rn(xs[e], pv.scale, pv.offset));     // NaN -> 0; saturates
+                atomicAdd(&sm.hist[min(max(b, 0), BINS - 1)], 1u);
+            }
+        }
+    });
+    __syncthreads();
+    // ---- rank of the k-th largest of the row inside the sample, and its standard deviation under sampling without replacement
+    const float mf = static_cast<float>(m_sample), nf = static_cast<float>(n);
+    const float p = __fdividef(static_cast<float>(k_top), nf);
+    const float r = mf * p;
+    const float var_r = fmaxf(mf * p * (1.f - p) * __fdividef(nf - mf, fmaxf(nf - 1.f, 1.f)), 0.f);
+    const float sd_r = var_r * rsqrtf(fmaxf(var_r, 1e-37f));
+    const bool whole = m_sample == static_cast<uint32_t>(n);          // the sample is the row: ranks are exact
+    const float margin = whole ? 0.f : TK_MARGIN_SIGMAS * sd_r + 2.f;
+    const int r_hi = whole ? k_top : static_cast<int>(floorf(r - margin));  // sample ranks below r_hi: certainly selected
+    const int r_lo = whole ? k_top : static_cast<int>(ceilf(r + margin));   // sample ranks above r_lo: certainly not
+    const bool has_hi = r_hi >= 1;
+    const bool has_lo = r_lo <= static_cast<int>(m_sample);
+    uint32_t hi_bin, lo_bin, ab_hi, ab_lo;
+    select_two_buckets<BINS, THREADS>(sm, has_hi ? r_hi : 1, has_lo ? r_lo : m_sample, slot, hi_bin, ab_hi, lo_bin, ab_lo);
+    // the pivots as scores: the upper edge of bin hi_bin and the lower edge of bin lo_bin (any bracket will do, so the
+    // rounding of these divisions does not matter); an end bin has no edge on its outer side
+    const float inv_scale = __fdividef(1.f, pv.scale);
+    const bool open_lo = !has_lo || lo_bin == 0u, open_hi = !has_hi || hi_bin == BINS - 1;
+    pv.lo_x = open_lo ? -INFINITY : (static_cast<float>(lo_bin) - pv.offset) * inv_scale;
+    pv.hi_x = open_hi ? INFINITY : (static_cast<float>(hi_bin + 1u) - pv.offset) * inv_scale;
+    pv.y_lo = open_lo ? 0.f : static_cast<float>(lo_bin);
+    const float y_hi = open_hi ? static_cast<float>(BINS) : static_cast<float>(hi_bin + 1u);
+    pv.fscale = __fdividef(static_cast<float>(BINS), y_hi - pv.y_lo);
+    return pv;
+}
+
+// Flags of four consecutive scores: bit e (low nibble) = at or above the upper pivot, bit 4 + e = between the pivots.
+__device__ __forceinline__ uint32_t flag4(const float4& v, float lo_x, float hi_x) {
+    const float x[4] = {v.x, v.y, v.z, v.w};
+    uint32_t sel = 0, ge_lo = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        sel |= ge_mask(x[e], hi_x) & (1u << e);
+        ge_lo |= ge_mask(x[e], lo_x) & (16u << e);
+    }
+    return sel | (ge_lo & ~(sel << 4));
+}
+
 // Radix select over a LIST of c full 32-bit keys (11 + 11 + 10 bits): finds the key T of the need-th largest entry
 // (1-based), how many entries equal to T are to be taken (need_eq >= 1) and how many there are (m_eq).
 // Uses hist[0..2047]; every thread of the block must call it.

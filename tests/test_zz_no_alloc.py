@@ -56,6 +56,36 @@ def test_noalloc_decode_matches_regular_entry_point_twice_in_a_row():
     assert torch.equal(_noalloc(third, 128), _regular(third, 128))
 
 
+def test_noalloc_decode_allocates_nothing_after_its_first_call_on_a_device():
+    """The first call on a device makes the driver create the built-in array and load the decode kernels; from then on
+    a call must leave the device's free memory untouched, whatever head count, dtype or batch shape it brings (a
+    serving host makes the first call at start-up, then hands the rest of HBM to its cache pool). Outputs and inputs
+    are allocated before the free memory is read, so only the library's own behaviour is measured."""
+    warm = _case(51, [300, 40])
+    out_w = torch.full((2, 8), -7, dtype=torch.int32, device=DEV)
+    idxc.indexer_decode_noalloc(warm.q_step, warm.k_cache, warm.w, warm.k_offsets, warm.lens, warm.max_len, 8, out_w,
+                                warm.q_scale, warm.k_scale)                      # first call (unless an earlier test made it)
+    idxc.poll_device_status()
+    cases = []
+    for seed, (H, d, fp8, lens, k_top) in enumerate([(16, 64, False, [5000, 129], 32), (32, 128, True, [700], 64),
+                                                       (64, 128, False, [20000, 17000, 300], 2048), (64, 64, False, [9, 2000], 16)]):
+        x = synth.decode_inputs(len(lens), H, d, 0, 0, seed=60 + seed, fp8=fp8, lens=lens)
+        for name in ("q_step", "k_cache", "w", "q_scale", "k_scale", "k_offsets", "lens"):
+            v = getattr(x, name)
+            if v is not None:
+                setattr(x, name, v.to(DEV))
+        cases.append((x, k_top, torch.full((len(lens), k_top), -7, dtype=torch.int32, device=DEV)))
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    for x, k_top, out in cases:
+        idxc.indexer_decode_noalloc(x.q_step, x.k_cache, x.w, x.k_offsets, x.lens, x.max_len, k_top, out, x.q_scale, x.k_scale)
+    idxc.poll_device_status()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, f"free device memory moved by {free_before - free_after} bytes"
+    for x, k_top, out in cases:
+        assert torch.equal(out, _regular(x, k_top))
+
+
 def test_noalloc_decode_rejects_steps_larger_than_its_array():
     x = _case(44, [100, 200])
     out = torch.empty((2, 16), dtype=torch.int32, device=DEV)
