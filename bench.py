@@ -114,6 +114,11 @@ class ClockSampler:
             self._thread.start()
         return self
 
+    def reset(self):
+        """Forgets what was sampled so far (the sampler keeps running): call at the start of the timed region."""
+        self.samples.clear()
+        self.reasons.clear()
+
     def __exit__(self, *exc):
         self._stop.set()
         if self._thread is not None:
@@ -631,13 +636,13 @@ def time_overlap(idxc, dev, peaks, rows, k_top, n_layers):
     pairs = [(a, b) for a in range(n_layers) for b in range(a + 1, n_layers)]
     ptrs = torch.tensor([t.data_ptr() for t in tops], dtype=torch.int64, device=dev)
     pr = torch.tensor(pairs, dtype=torch.int32, device=dev).reshape(-1)
-    sums = torch.empty((len(pairs),), dtype=torch.float64, device=dev)
+    means = torch.empty((len(pairs),), dtype=torch.float64, device=dev)
     L_ = idxc.lib()
     stream = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
 
     def call():
         st = L_.idxc_topk_overlap(ctypes.c_void_p(ptrs.data_ptr()), ctypes.c_void_p(pr.data_ptr()), len(pairs), rows, k_top,
-                                  ctypes.c_void_p(sums.data_ptr()), None, stream)
+                                  ctypes.c_void_p(means.data_ptr()), None, stream)
         assert st == 0
     call()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -649,7 +654,7 @@ def time_overlap(idxc, dev, peaks, rows, k_top, n_layers):
     ms = a.elapsed_time(b) / 5
     nbytes = len(pairs) * 2 * rows * k_top * 4
     gbs = nbytes / (ms * 1e-3) / 1e9
-    return {"layers": n_layers, "pairs": len(pairs), "rows": rows, "k_top": k_top, "ms": ms, "mean_overlap": float((sums / rows).mean()),
+    return {"layers": n_layers, "pairs": len(pairs), "rows": rows, "k_top": k_top, "ms": ms, "mean_overlap": float(means.mean()),
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
                          "of": peaks["source"], "note": "every tensor is read n_layers-1 times; the index tensors (403 MB) exceed L2"}}
 
@@ -819,13 +824,14 @@ def main():
         if evs:
             evs[2].record()
 
-    for _ in range(W):
-        step()
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
-    torch.cuda.synchronize()
-    barrier(world)
-    launches0 = idxc.launch_count()
-    with ClockSampler(local) as clk:
+    with ClockSampler(local) as clk:                 # started before the warm-up: its first queries are slow and hold the interpreter
+        for _ in range(W):
+            step()
+        torch.cuda.synchronize()
+        barrier(world)
+        launches0 = idxc.launch_count()
+        clk.reset()
         t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t_start.record()
         for i in range(K):

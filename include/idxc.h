@@ -228,10 +228,10 @@ idxc_status idxc_schedule_decode_layer(idxc_schedule* s, int layer,
  *
  * idxc_topk_overlap -- the cross-layer top-k index overlap of Appendix A: for a pair of index tensors
  * T_a, T_b ([rows, k_top] int32, ascending, -1 padded, as produced above) the per-row ratio
- * |T_a[r] n T_b[r]| / (valid entries of T_a[r]) and its sum over the rows.
+ * |T_a[r] n T_b[r]| / (valid entries of T_a[r]) and its mean over the rows (the figure Appendix A plots).
  *   layers   DEVICE array of device pointers to the index tensors
  *   pairs    DEVICE int32 [2 * n_pairs]: pair p compares layers[pairs[2p]] with layers[pairs[2p+1]]
- *   sums_out DEVICE double [n_pairs]: sum over rows of the ratio (divide by rows for the mean); zeroed by the call
+ *   means_out DEVICE double [n_pairs]: mean over the rows of the ratio; zeroed by the call
  *   row_out  NULL, or DEVICE float [rows] (only with n_pairs == 1): the per-row ratios
  * One launch covers all pairs (n_pairs <= 65535).
  *
@@ -249,7 +249,7 @@ idxc_status idxc_schedule_decode_layer(idxc_schedule* s, int layer,
 typedef double (*idxc_eval_loss_fn)(const char* pattern, int N, void* user);
 
 idxc_status idxc_topk_overlap(const int32_t* const* layers, const int32_t* pairs, int n_pairs, int64_t rows, int k_top,
-                              double* sums_out, float* row_out, void* cuda_stream);
+                              double* means_out, float* row_out, void* cuda_stream);
 idxc_status idxc_pattern_search_dp(const double* S, int N, int M, char* pattern_out, double* value_out);
 idxc_status idxc_pattern_search_greedy(int N, int K, idxc_eval_loss_fn eval_loss, void* user, char* pattern_out,
                                        int* order_out, int64_t* evaluations_out);

@@ -278,11 +278,10 @@ def topk_overlap(layers, pairs=None, want_rows=False, stream=None):
     dev = layers[0].device
     ptrs = torch.tensor([t.data_ptr() for t in layers], dtype=torch.int64, device=dev)
     pr = torch.tensor(pairs, dtype=torch.int32, device=dev).reshape(-1)
-    sums = torch.empty((len(pairs),), dtype=torch.float64, device=dev)
+    mean = torch.empty((len(pairs),), dtype=torch.float64, device=dev)
     row_out = torch.empty((rows,), dtype=torch.float32, device=dev) if want_rows else None
-    _check(lib().idxc_topk_overlap(_ptr(ptrs), _ptr(pr), len(pairs), rows, k_top, _ptr(sums), _ptr(row_out), _stream(stream)),
+    _check(lib().idxc_topk_overlap(_ptr(ptrs), _ptr(pr), len(pairs), rows, k_top, _ptr(mean), _ptr(row_out), _stream(stream)),
            "idxc_topk_overlap")
-    mean = sums / max(rows, 1)
     return (mean, row_out) if want_rows else mean
 
 

@@ -17,12 +17,13 @@ constexpr int OV_THREADS = 256;
 
 // grid.x: pair index (fastest, so that the pairs of one row run together and the row's index lists are read from HBM
 // once and from the L2 afterwards), grid.y: row blocks (grid-stride). pairs[2p], pairs[2p+1]: layer indices of pair p.
-// sums[p] accumulates the row ratios (double, atomicAdd); row_out (optional, single pair) gets each ratio.
+// means[p] accumulates the row ratios divided by the number of rows (double, atomicAdd): the average of Appendix A;
+// row_out (optional, single pair) gets each ratio.
 // Both rows are ascending: a thread takes a run of consecutive entries of T_a, finds where the run starts in T_b with
 // one binary search and then walks both lists together.
 __global__ void __launch_bounds__(OV_THREADS)
 overlap_kernel(const int32_t* const* __restrict__ layers, const int* __restrict__ pairs, int64_t rows, int k_top,
-               double* __restrict__ sums, float* __restrict__ row_out) {
+               double* __restrict__ means, float* __restrict__ row_out) {
     extern __shared__ int32_t sh[];                 // row of T_b, then row of T_a: k_top entries each
     int32_t* sb = sh;
     int32_t* sa = sh + k_top;
@@ -80,7 +81,7 @@ overlap_kernel(const int32_t* const* __restrict__ layers, const int* __restrict_
             if (row_out) row_out[r] = static_cast<float>(ratio);
         }
     }
-    if (threadIdx.x == 0) atomicAdd(&sums[p], local_sum);
+    if (threadIdx.x == 0) atomicAdd(&means[p], local_sum / static_cast<double>(rows));
 }
 
 }  // namespace
