@@ -243,8 +243,8 @@ idxc_status idxc_schedule_decode_layer(idxc_schedule* s, int layer,
  * idxc_pattern_search_greedy -- Algorithm 1 (HOST driver): starting from all-Full, K times flip to Shared the
  * remaining layer (never layer 0) whose flip gives the lowest eval_loss(pattern, N, user); ties go to the
  * lowest layer. eval_loss receives a NUL-terminated pattern. order_out (HOST, K ints, may be NULL) gets the
- * flipped layers in order, evaluations_out (HOST, may be NULL) the number of loss evaluations
- * (N(N-1)/2 for K = N-1).
+ * flipped layers in order, step_loss_out (HOST, K doubles, may be NULL) the loss of the pattern after each step,
+ * evaluations_out (HOST, may be NULL) the number of loss evaluations (N(N-1)/2 for K = N-1).
  * ------------------------------------------------------------------------- */
 typedef double (*idxc_eval_loss_fn)(const char* pattern, int N, void* user);
 
@@ -252,7 +252,7 @@ idxc_status idxc_topk_overlap(const int32_t* const* layers, const int32_t* pairs
                               double* means_out, float* row_out, void* cuda_stream);
 idxc_status idxc_pattern_search_dp(const double* S, int N, int M, char* pattern_out, double* value_out);
 idxc_status idxc_pattern_search_greedy(int N, int K, idxc_eval_loss_fn eval_loss, void* user, char* pattern_out,
-                                       int* order_out, int64_t* evaluations_out);
+                                       int* order_out, double* step_loss_out, int64_t* evaluations_out);
 
 /* ---------------------------------------------------------------------------
  * Multi-layer distillation loss of training-aware IndexCache, forward value (Eq. 1):

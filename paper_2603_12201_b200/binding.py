@@ -90,7 +90,7 @@ def lib() -> ctypes.CDLL:
         L.idxc_pattern_search_dp.argtypes = [vp, i32, i32, ctypes.c_char_p, ctypes.POINTER(ctypes.c_double)]
         L.idxc_pattern_search_greedy.restype = i32
         L.idxc_pattern_search_greedy.argtypes = [i32, i32, EVAL_LOSS_FN, vp, ctypes.c_char_p, ctypes.POINTER(i32),
-                                                 ctypes.POINTER(i64)]
+                                                 ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
         L.idxc_distill_kl.restype = i32
         L.idxc_distill_kl.argtypes = [vp, i64, i64, i64, i64, ctypes.POINTER(vp), i32, vp, i32, vp, vp, vp]
         L.idxc_sparse_attention_workspace_bytes.restype = sz
@@ -297,15 +297,17 @@ def pattern_search_dp(S, M: int):
     return buf.raw[:N].decode(), val.value
 
 
-def pattern_search_greedy(N: int, K: int, eval_loss):
+def pattern_search_greedy(N: int, K: int, eval_loss, want_losses: bool = False):
     """idxc_pattern_search_greedy (Algorithm 1). eval_loss(pattern: str) -> float.
-    Returns (pattern, order of flipped layers, number of evaluations)."""
+    Returns (pattern, order of flipped layers, number of evaluations[, loss after each step])."""
     cb = EVAL_LOSS_FN(lambda p, n, user: float(eval_loss(p[:n].decode())))
     buf = ctypes.create_string_buffer(N)
     order = (ctypes.c_int * max(K, 1))()
+    losses = (ctypes.c_double * max(K, 1))()
     evals = ctypes.c_int64()
-    _check(lib().idxc_pattern_search_greedy(N, K, cb, None, buf, order, ctypes.byref(evals)), "idxc_pattern_search_greedy")
-    return buf.raw[:N].decode(), list(order)[:K], evals.value
+    _check(lib().idxc_pattern_search_greedy(N, K, cb, None, buf, order, losses, ctypes.byref(evals)), "idxc_pattern_search_greedy")
+    out = (buf.raw[:N].decode(), list(order)[:K], evals.value)
+    return out + (list(losses)[:K],) if want_losses else out
 
 
 def distill_kl(scores, targets, first_len=1, len_step=1, topk=None, want_rows=False, stream=None):

@@ -5,6 +5,7 @@
 //   * similarity DP (host): the exact pattern with M Full layers that maximises the summed similarity of
 //     the Shared layers to their source layers.
 //   * greedy layer selection (host): Algorithm 1 with the caller's loss function.
+#include <string>
 #include <vector>
 
 #include "../../include/idxc.h"
@@ -17,8 +18,8 @@ constexpr int OV_THREADS = 256;
 
 // grid.x: pair index (fastest, so that the pairs of one row run together and the row's index lists are read from HBM
 // once and from the L2 afterwards), grid.y: row blocks (grid-stride). pairs[2p], pairs[2p+1]: layer indices of pair p.
-// means[p] accumulates the row ratios divided by the number of rows (double, atomicAdd): the average of Appendix A;
-// row_out (optional, single pair) gets each ratio.
+// means[p] accumulates the row ratios (double, atomicAdd); a second, tiny kernel divides by the number of rows: the
+// average of Appendix A. row_out (optional, single pair) gets each ratio.
 // Both rows are ascending: a thread takes a run of consecutive entries of T_a, finds where the run starts in T_b with
 // one binary search and then walks both lists together.
 __global__ void __launch_bounds__(OV_THREADS)
@@ -81,7 +82,12 @@ overlap_kernel(const int32_t* const* __restrict__ layers, const int* __restrict_
             if (row_out) row_out[r] = static_cast<float>(ratio);
         }
     }
-    if (threadIdx.x == 0) atomicAdd(&means[p], local_sum / static_cast<double>(rows));
+    if (threadIdx.x == 0) atomicAdd(&means[p], local_sum);
+}
+
+__global__ void overlap_mean_kernel(double* __restrict__ means, int n_pairs, double rows) {
+    const int p = blockIdx.x * blockDim.x + threadIdx.x;
+    if (p < n_pairs) means[p] /= rows;
 }
 
 }  // namespace
@@ -92,6 +98,8 @@ cudaError_t launch_overlap(const int32_t* const* layers_dev, const int* pairs_de
     const unsigned gy = static_cast<unsigned>(rows < 4096 ? rows : 4096);
     dim3 grid(static_cast<unsigned>(n_pairs), gy);
     overlap_kernel<<<grid, OV_THREADS, 2 * k_top * sizeof(int32_t), stream>>>(layers_dev, pairs_dev, rows, k_top, sums_dev, row_out);
+    if (cudaError_t e = cudaGetLastError(); e != cudaSuccess) return e;
+    overlap_mean_kernel<<<(n_pairs + 255) / 256, 256, 0, stream>>>(sums_dev, n_pairs, static_cast<double>(rows));
     return cudaGetLastError();
 }
 
@@ -154,32 +162,30 @@ idxc_status idxc_pattern_search_dp(const double* S, int N, int M, char* pattern_
     return IDXC_OK;
 }
 
-// Algorithm 1. Ties go to the lowest layer.
+// Greedy layer selection (Algorithm 1): from the all-Full pattern, K times turn into a Shared layer the still-Full
+// layer (never layer 0) whose conversion leaves the lowest loss. State is one pattern buffer in which a trial is a
+// single character flipped and restored; the lowest trial of a step wins, the lowest layer among equal losses.
 idxc_status idxc_pattern_search_greedy(int N, int K, idxc_eval_loss_fn eval_loss, void* user, char* pattern_out,
-                                       int* order_out, int64_t* evaluations_out) {
+                                       int* order_out, double* step_loss_out, int64_t* evaluations_out) {
     if (N < 1 || K < 0 || K > N - 1 || !eval_loss || !pattern_out) return IDXC_ERR_INVALID_ARG;
-    std::vector<char> c(N + 1, 'F');
-    c[N] = '\0';
-    std::vector<int> remaining;
-    for (int l = 1; l < N; ++l) remaining.push_back(l);
+    std::string pattern(static_cast<size_t>(N), 'F');            // NUL-terminated through c_str()
     int64_t evals = 0;
     for (int step = 0; step < K; ++step) {
-        int best_pos = -1;
-        double best_loss = 0.0;
-        for (size_t pos = 0; pos < remaining.size(); ++pos) {
-            const int l = remaining[pos];
-            c[l] = 'S';
-            const double loss = eval_loss(c.data(), N, user);
-            c[l] = 'F';
+        int winner = -1;
+        double winner_loss = 0.0;
+        for (int l = 1; l < N; ++l) {
+            if (pattern[l] != 'F') continue;                     // already Shared
+            pattern[l] = 'S';
+            const double loss = eval_loss(pattern.c_str(), N, user);
+            pattern[l] = 'F';
             ++evals;
-            if (best_pos < 0 || loss < best_loss) { best_pos = static_cast<int>(pos); best_loss = loss; }
+            if (winner < 0 || loss < winner_loss) { winner = l; winner_loss = loss; }
         }
-        const int l = remaining[best_pos];
-        c[l] = 'S';
-        remaining.erase(remaining.begin() + best_pos);
-        if (order_out) order_out[step] = l;
+        pattern[winner] = 'S';                                   // K <= N - 1: a Full layer other than 0 is always left
+        if (order_out) order_out[step] = winner;
+        if (step_loss_out) step_loss_out[step] = winner_loss;
     }
-    for (int l = 0; l < N; ++l) pattern_out[l] = c[l];
+    pattern.copy(pattern_out, static_cast<size_t>(N));
     if (evaluations_out) *evaluations_out = evals;
     return IDXC_OK;
 }

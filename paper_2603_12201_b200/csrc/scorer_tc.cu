@@ -150,6 +150,19 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
                 const int64_t item = item_of_round(rho);
                 if (item < 0) break;
                 const int nkt = key_tiles_of_item(item);
+                auto load_k = [&](int kt) -> bool {
+                    if (!mbar_wait(bar_k_empty + 8 * stage, k_phase ^ 1u, abort_flag)) return false;
+                    mbar_arrive_expect_tx(bar_k_full + 8 * stage, NKH * kKRegionBytes);
+                    for (int kh = 0; kh < NKH; ++kh)
+                        tma_load_2d(smem_u32(k_smem + (stage * NKH + kh) * kKRegionBytes), &k_map, bar_k_full + 8 * stage,
+                                    kh * kElemsPerChunk, kt * kTileKeys);
+                    if (++stage == kStages) { stage = 0; k_phase ^= 1u; }
+                    return true;
+                };
+                // The first key tiles of this item go out before the wait for the query buffers: their ring stages come
+                // free while the previous item's last tiles are still being multiplied, the query buffers only after them.
+                const int pre = nkt < kStages ? nkt : kStages;
+                for (int kt = 0; kt < pre && ok; ++kt) ok = load_k(kt);
                 for (int half = 0; half < 2 && ok; ++half) {
                     ok = mbar_wait(bar_q_empty + 8 * half, q_phase ^ 1u, abort_flag);
                     if (!ok) break;
@@ -159,15 +172,7 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
                         tma_load_2d(smem_u32(q_smem + (half * NKH + kh) * kQRegionBytes), &q_map, bar_q_full + 8 * half,
                                     kh * kElemsPerChunk, row0);
                 }
-                for (int kt = 0; kt < nkt && ok; ++kt) {
-                    ok = mbar_wait(bar_k_empty + 8 * stage, k_phase ^ 1u, abort_flag);
-                    if (!ok) break;
-                    mbar_arrive_expect_tx(bar_k_full + 8 * stage, NKH * kKRegionBytes);
-                    for (int kh = 0; kh < NKH; ++kh)
-                        tma_load_2d(smem_u32(k_smem + (stage * NKH + kh) * kKRegionBytes), &k_map, bar_k_full + 8 * stage,
-                                    kh * kElemsPerChunk, kt * kTileKeys);
-                    if (++stage == kStages) { stage = 0; k_phase ^= 1u; }
-                }
+                for (int kt = pre; kt < nkt && ok; ++kt) ok = load_k(kt);
                 q_phase ^= 1u;
             }
             if (!ok) give_up(abort_flag, p.status, DEV_TIMEOUT_PRODUCER);

@@ -650,6 +650,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
                         max16(rb, m32 >> 16);
                     }
                 }
+                // rows beyond the query's heads hold whatever the staging area held before (only H rows are loaded): they
+                // must never ask for a rescale of O, which would cost every tile of the query an extra pass
+                if (row >= p.H) mt = -INFINITY;
                 // lazy reference maximum: move it only when the row maximum outgrew it by 2^8
                 const bool move = mt > m_ref + kRescaleThreshold;      // also true for the first usable score (m_ref = -inf)
                 float alpha = 1.f;

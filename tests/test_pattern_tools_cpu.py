@@ -70,5 +70,11 @@ def test_greedy_matches_oracle_loop(idxc):
             want = opat.greedy_select(9, K, loss)
             assert got == want
     assert idxc.pattern_search_greedy(9, 8, additive)[2] == 9 * 8 // 2       # N(N-1)/2 evaluations for a full search
+    # the loss after each step is the loss of the pattern with exactly the layers flipped so far
+    pat, order, _, losses = idxc.pattern_search_greedy(9, 5, runs, want_losses=True)
+    for step in range(5):
+        p = "".join("S" if l in order[: step + 1] else "F" for l in range(9))
+        assert losses[step] == pytest.approx(runs(p), rel=1e-15)
+    assert pat == "".join("S" if l in order else "F" for l in range(9))
     with pytest.raises(idxc.IdxcError):
         idxc.pattern_search_greedy(9, 9, additive)                            # layer 0 can never be Shared
