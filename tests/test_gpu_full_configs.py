@@ -167,8 +167,8 @@ def test_config5_fp8_chunked_prefill_and_decode():
     o_sc, _ = oracle.indexer_prefill(codes(inp.q[t:t + 1]), codes_cached(inp), f32(inp.w[t:t + 1]), k_top, dt,
                                      f32(inp.q_scale[t:t + 1]), f32(inp.k_scale), q_begin=t)
     assert_scores_close(score_rows[t][: t + 1], o_sc[0, : t + 1], RTOL_BF16, what="fp8 row, tight bound")
-    # one decode step on the resulting cache (sequence 0) and two fresh caches of the same length
-    B = 3
+    # one decode step at the workload's batch: the resulting cache (sequence 0) and fresh caches of the same length
+    B = c["decode_B"]
     fresh = synth.decode_inputs(B, H, d, L, L, seed=c["seed"], device=DEV, layer=1, fp8=True, lens=[L] * B)
     fresh.k_cache[:L] = inp.k
     fresh.k_scale[:L] = inp.k_scale
