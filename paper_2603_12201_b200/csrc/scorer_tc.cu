@@ -408,9 +408,11 @@ cudaError_t launch_score_prefill_tc(const ScoreArgs& a, const CUtensorMap& q_map
 namespace {
 
 constexpr int kDecodeEpiWarps = 8;       // two groups of 4 (one warp per TMEM lane quarter); group g drains slots g, g+2
-constexpr int kDecodeThreads = (2 + kDecodeEpiWarps) * 32;   // warp 0 producer, warp 1 MMA, warps 2-9 epilogue
-// Key tiles (of 128 keys) per work item. Measured on B200 (B = 32, 16K-128K keys per sequence): 16 tiles
-// stream at 6.1 TB/s; 6-8 tiles per item lose 20 % (all CTAs then walk HBM with the same 192-256 KB stride).
+constexpr int kDecodeMmaWarps = 2;      // warp 1 and (if 2) the last warp: key tiles alternate between them
+constexpr int kDecodeThreads = (1 + kDecodeMmaWarps + kDecodeEpiWarps) * 32;   // warp 0 producer, warp 1 MMA, warps 2-9 epilogue, warp 10 MMA
+// Key tiles (of 128 keys, 256-byte rows) per work item; twice as many when a row is 128 bytes, so that an item is
+// the same stretch of HBM. Measured on B200 (bf16, d = 128, B = 32, 16K-128K keys per sequence): 16 tiles stream
+// at 6.1 TB/s; 6-8 tiles per item lose 20 % (all CTAs then walk HBM with the same 192-256 KB stride).
 constexpr int kDecodeChunkTiles = 16;
 constexpr int kDecodeAccSlots = 8;       // TMEM accumulators in flight (64 columns apart: all 512 columns)
 
@@ -421,8 +423,11 @@ struct DecodeCfg {
     static constexpr int kQBytes = 2 * NKH * kQRegion;                // double buffered
     static constexpr int kKBytes = kStages * NKH * kKRegionBytes;
     static constexpr int kWBytes = kDecodeEpiWarps * 64 * 4;          // per epilogue warp: w of the item's sequence
+    static constexpr int kMaxChunk = kDecodeChunkTiles * 2 / NKH;     // key tiles per work item, at most
+    static constexpr int kMaxOwn = (kMaxChunk + 1) / 2;               // ... of which one group of epilogue warps drains
+    static constexpr int kScaleBytes = kDecodeEpiWarps * 2 * kMaxOwn * 32 * 4;   // FP8 key scales: [warp][2 items][own tile][lane]
     static constexpr int kBarBytes = 512;
-    static constexpr int kSmemBytes = kQBytes + kKBytes + kWBytes + kBarBytes + 1024;
+    static constexpr int kSmemBytes = kQBytes + kKBytes + kWBytes + kScaleBytes + kBarBytes + 1024;
 };
 
 struct DecodeParams {
@@ -486,13 +491,18 @@ score_decode_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
     constexpr int kStages = Cfg::kStages;
     constexpr int kElemsPerChunk = FP8 ? 128 : 64;
     constexpr uint32_t kIdesc = FP8 ? umma_idesc(0, 0, kTileKeys, H) : umma_idesc(1, 1, kTileKeys, H);
+    // Two MMA warps only when the key ring has an even number of stages: a stage then always belongs to the same warp.
+    // With an odd ring a warp would wait for every other phase of a stage's barrier, and a parity wait cannot tell the
+    // phase it wants from the one two before it.
+    constexpr int kMmaWarps = (kStages % 2 == 0 && kDecodeAccSlots % 2 == 0) ? kDecodeMmaWarps : 1;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint8_t* k_smem = smem;                                  // [kStages][NKH][128 x 128 B]
     uint8_t* q_smem = k_smem + Cfg::kKBytes;                 // [2][NKH][H x 128 B]
     float* w_smem = reinterpret_cast<float*>(q_smem + Cfg::kQBytes);   // [4 warps][64]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(w_smem) + Cfg::kWBytes);
+    float* scale_smem = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(w_smem) + Cfg::kWBytes);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(scale_smem) + Cfg::kScaleBytes);
     const uint32_t bar_q_full = smem_u32(bars + 0);          // [2]
     const uint32_t bar_q_empty = smem_u32(bars + 2);         // [2]
     const uint32_t bar_acc_full = smem_u32(bars + 4);        // [kDecodeAccSlots]
@@ -508,7 +518,7 @@ score_decode_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
     if (threadIdx.x == 0) {
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar_q_full + 8 * i, 1);
-            mbar_init(bar_q_empty + 8 * i, 1);
+            mbar_init(bar_q_empty + 8 * i, kMmaWarps);
         }
         for (int i = 0; i < kDecodeAccSlots; ++i) {
             mbar_init(bar_acc_full + 8 * i, 1);
@@ -562,9 +572,14 @@ score_decode_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
             }
             if (!ok) give_up(abort_flag, p.status, DEV_TIMEOUT_PRODUCER);
         }
-    } else if (warp == 1) {
+    } else if (warp == 1 || (kMmaWarps == 2 && warp == 2 + kDecodeEpiWarps)) {
         // The whole warp runs this role with uniform control flow and one elected lane issues (a single diverged lane
         // issues the same instruction stream about 1.5x slower); descriptors are a base plus 16-byte units.
+        // With two such warps the key tiles alternate between them (a tile is four to eight small MMAs, two commits and
+        // two barrier waits, and one warp gets through that more slowly than 16 KB tiles arrive): warp m takes the tiles
+        // whose running number has parity m, which are also the accumulator slots of parity m; both walk all tiles to
+        // keep the ring position and the phases.
+        const int mma_id = warp == 1 ? 0 : 1;
         int stage = 0, qbuf = 0, slot = 0;
         uint32_t k_phase = 0, q_phase[2] = {0u, 0u}, acc_phase = 0;   // acc_phase: one bit per accumulator slot
         bool ok = true;
@@ -579,28 +594,32 @@ score_decode_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
             q_phase[qbuf] ^= 1u;
             const uint64_t b_desc = b_desc0 + static_cast<uint64_t>(qbuf * NKH * Cfg::kQRegion / 16);
             for (int kt = 0; kt < ntiles && ok; ++kt) {
-                ok = wait_bar(bar_k_full + 8 * stage, k_phase) && wait_bar(bar_acc_empty + 8 * slot, ((acc_phase >> slot) & 1u) ^ 1u);
-                if (!ok) break;
-                acc_phase ^= 1u << slot;
-                tcgen05_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + slot * 64;
-                const uint64_t a_desc = a_desc0 + static_cast<uint64_t>(stage * NKH * kKRegionBytes / 16);
+                if (kMmaWarps == 1 || (slot & 1) == mma_id) {
+                    ok = wait_bar(bar_k_full + 8 * stage, k_phase) && wait_bar(bar_acc_empty + 8 * slot, ((acc_phase >> slot) & 1u) ^ 1u);
+                    if (!ok) break;
+                    acc_phase ^= 1u << slot;
+                    tcgen05_fence_after_sync();
+                    const uint32_t d_tmem = tmem_base + slot * 64;
+                    const uint64_t a_desc = a_desc0 + static_cast<uint64_t>(stage * NKH * kKRegionBytes / 16);
 #pragma unroll
-                for (int kh = 0; kh < NKH; ++kh) {
+                    for (int kh = 0; kh < NKH; ++kh) {
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {
-                        const uint64_t a = a_desc + (kh * kKRegionBytes + ks * 32) / 16, b = b_desc + (kh * Cfg::kQRegion + ks * 32) / 16;
-                        if constexpr (FP8) {
-                            if ((kh | ks) != 0) umma_f8_elect<true>(d_tmem, a, b, kIdesc);
-                            else umma_f8_elect<false>(d_tmem, a, b, kIdesc);
-                        } else {
-                            if ((kh | ks) != 0) umma_f16_elect<true>(d_tmem, a, b, kIdesc);
-                            else umma_f16_elect<false>(d_tmem, a, b, kIdesc);
+                        for (int ks = 0; ks < 4; ++ks) {
+                            const uint64_t a = a_desc + (kh * kKRegionBytes + ks * 32) / 16, b = b_desc + (kh * Cfg::kQRegion + ks * 32) / 16;
+                            if constexpr (FP8) {
+                                if ((kh | ks) != 0) umma_f8_elect<true>(d_tmem, a, b, kIdesc);
+                                else umma_f8_elect<false>(d_tmem, a, b, kIdesc);
+                            } else {
+                                if ((kh | ks) != 0) umma_f16_elect<true>(d_tmem, a, b, kIdesc);
+                                else umma_f16_elect<false>(d_tmem, a, b, kIdesc);
+                            }
                         }
                     }
+                    umma_commit_elect(bar_acc_full + 8 * slot);
+                    umma_commit_elect(bar_k_empty + 8 * stage);
                 }
-                umma_commit_elect(bar_acc_full + 8 * slot);
-                umma_commit_elect(bar_k_empty + 8 * stage);
+                // the query buffer is free once the item's MMAs of BOTH warps are complete: each commits after its last
+                // tile of the item (a commit with nothing outstanding arrives at once)
                 if (kt == ntiles - 1) umma_commit_elect(bar_q_empty + 8 * qbuf);
                 if (++stage == kStages) { stage = 0; k_phase ^= 1u; }
                 slot = (slot + 1) & (kDecodeAccSlots - 1);
@@ -608,7 +627,7 @@ score_decode_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
             qbuf ^= 1;
         }
         if (!ok && lane == 0) give_up(abort_flag, p.status, DEV_TIMEOUT_MMA);
-    } else {
+    } else if (warp < 2 + kDecodeEpiWarps) {
         const int quarter = warp & 3;
         const int grp = (warp - 2) >> 2;                 // which accumulator slots this warp drains
         const int key_in_tile = quarter * 32 + lane;
@@ -616,23 +635,61 @@ score_decode_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
         int slot = 0;
         uint32_t acc_phase = 0;                          // one bit per accumulator slot
         bool ok = true;
+        // What a work item needs besides its accumulators is fetched one item ahead, by a second walker: w of the item's
+        // sequence (times its query scale) into registers and, FP8, the scales of this thread's keys in the tiles this
+        // warp will drain, by 4-byte cp.async into a staging area of its own (two items deep, a slot per lane and tile).
+        // Asked for tile by tile they cost the warp a memory latency each, and any per-tile bookkeeping is dear in a warp
+        // that has its scheduler almost to itself (a dependent instruction every 4-6 cycles).
+        constexpr int kWPerLane = (H + 31) / 32;
+        constexpr int kMaxOwn = Cfg::kMaxOwn;
+        float* my_scales = scale_smem + (warp - 2) * (2 * kMaxOwn * 32) + lane;
+        DecodeItemWalker walk_next(p, blockIdx.x, gridDim.x);
+        float w_next[kWPerLane];
+        int next_slot0 = 0;                              // accumulator slot of the next item's first tile
+        int stage_buf = 0;                               // staging buffer the next fetch goes to
+        auto fetch_next = [&]() {                        // always commits one cp.async group
+            int s2, t2, n2, l2;
+            if (walk_next.pop(s2, t2, n2, l2)) {
+                float qs = 1.f;
+                if constexpr (FP8) qs = __ldg(p.q_scale + s2);
+#pragma unroll
+                for (int i = 0; i < kWPerLane; ++i) {
+                    const int h = lane + 32 * i;
+                    w_next[i] = h < H ? __ldg(p.w + static_cast<int64_t>(s2) * H + h) * qs : 0.f;
+                }
+                if constexpr (FP8) {
+                    const int kt0 = ((next_slot0 & 1) != grp) ? 1 : 0;          // this group's first tile of the item
+                    const int s_first = (t2 + kt0) * kTileKeys + key_in_tile;
+                    const float* src = p.k_scale + p.k_offsets[s2] + s_first;
+                    const uint32_t dst = smem_u32(my_scales + stage_buf * (kMaxOwn * 32));
+#pragma unroll
+                    for (int j = 0; j < kMaxOwn; ++j)
+                        if (kt0 + 2 * j < n2 && s_first + 2 * kTileKeys * j < l2) cp_async_4(dst + j * 128, src + 2 * kTileKeys * j);
+                }
+                next_slot0 = (next_slot0 + n2) & (kDecodeAccSlots - 1);
+            }
+            if constexpr (FP8) cp_async_commit();
+            stage_buf ^= 1;
+        };
+        fetch_next();
         while (ok && walk.pop(seq, tile0, ntiles, len)) {
             __syncwarp();
-            for (int h = lane; h < H; h += 32) {
-                float v = __ldg(p.w + static_cast<int64_t>(seq) * H + h);
-                if constexpr (FP8) v *= __ldg(p.q_scale + seq);
-                my_w[h] = v;
-            }
-            const int64_t krow0 = p.k_offsets[seq];
+#pragma unroll
+            for (int i = 0; i < kWPerLane; ++i)
+                if (lane + 32 * i < H) my_w[lane + 32 * i] = w_next[i];
+            const float* item_scales = my_scales + (stage_buf ^ 1) * (kMaxOwn * 32);   // where the last fetch went
+            fetch_next();
+            if constexpr (FP8) cp_async_wait_group<1>();   // this item's scales (the group before the one just committed) are in
             __syncwarp();
             const float4* w4 = reinterpret_cast<const float4*>(my_w);
             for (int kt = 0; kt < ntiles && ok; ++kt, slot = (slot + 1) & (kDecodeAccSlots - 1)) {
                 if ((slot & 1) != grp) continue;         // the other group's tile
                 const int s = (tile0 + kt) * kTileKeys + key_in_tile;
-                // FP8: the key's scale is asked for before the wait and used after the head sums: its latency is hidden
-                // behind the accumulator's
                 float ksc = 1.f;
-                if constexpr (FP8) ksc = s < len ? __ldg(p.k_scale + krow0 + s) : 0.f;
+                if constexpr (FP8) {
+                    if (s < len) ksc = *item_scales;       // (slots of keys past the end were not written)
+                    item_scales += 32;
+                }
                 ok = __all_sync(0xFFFFFFFFu, mbar_wait(bar_acc_full + 8 * slot, (acc_phase >> slot) & 1u, abort_flag));   // warp-uniform
                 if (!ok) break;
                 acc_phase ^= 1u << slot;
@@ -715,13 +772,14 @@ cudaError_t launch_decode_instance(const ScoreArgs& a, const CUtensorMap& q_map,
     auto kern = score_decode_tc_kernel<NKH, H, FP8>;
     if (cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(kern), Cfg::kSmemBytes); e != cudaSuccess) return e;
     const int64_t tiles = (a.max_len + kTileKeys - 1) / kTileKeys;
-    // Tiles per work item: 16 streams best (shorter items cost about 5 % at a large batch), but a small batch leaves the
-    // last round of the static schedule half empty. Estimated with every sequence at max_len (the lengths live on the
-    // device): the item size in 10..16 with the fewest rounds x size, the larger one on a tie (items of 6 to 8 tiles
-    // make the CTAs walk HBM in lock-step at a stride that costs a fifth of the bandwidth).
-    int chunk = kDecodeChunkTiles;
+    // Tiles per work item: 512 KB of keys streams best (shorter items cost about 5 % at a large batch), but a small batch
+    // leaves the last round of the static schedule half empty. Estimated with every sequence at max_len (the lengths live
+    // on the device): the item size in 320..512 KB with the fewest rounds x size, the larger one on a tie (items of 192 to
+    // 256 KB make the CTAs walk HBM in lock-step at a stride that costs a fifth of the bandwidth).
+    const int cmax = Cfg::kMaxChunk, cmin = 10 * 2 / NKH;
+    int chunk = cmax;
     int64_t best = -1;
-    for (int c = kDecodeChunkTiles; c >= 10; --c) {
+    for (int c = cmax; c >= cmin; --c) {
         const int64_t n_items = a.n_rows * ((tiles + c - 1) / c);
         const int64_t cost = ((n_items + sm_count - 1) / sm_count) * c;
         if (best < 0 || cost < best) { best = cost; chunk = c; }
