@@ -183,6 +183,10 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
     //   0 MMA | 4 loader | 8, 11 idle | 1 2 3 5 6 7 9 10 gather | 12..15 softmax (TMEM lane quarter = warp % 4)
     const int gather_index = warp < 4 ? warp - 1 : (warp < 8 ? warp - 2 : warp - 3);   // for warps 1 2 3 5 6 7 9 10
     const bool is_gather = warp != 0 && warp != 4 && warp != 8 && warp < 11;
+    // L2 residency: the cache rows (read again by later queries) and the saved probabilities (read back within the
+    // query) are kept in preference to q and the output, which stream through once
+    const uint64_t pol_keep = l2_policy_evict_last();
+    const uint64_t pol_stream = l2_policy_evict_first();
 
     if (threadIdx.x == 0) {
         mbar_init(bar_q_full, 1);
@@ -379,7 +383,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
                 const int row0 = static_cast<int>(t * p.H);
                 for (int b = 0; b < kSaNB; ++b) {
                     uint8_t* dst = b < kSaQT ? stage_smem + b * kSaQBlockBytes : q_smem + (b - kSaQT) * kSaQBlockBytes;
-                    tma_load_2d(smem_u32(dst), &q_map, bar_q_full, b * 64, row0);
+                    tma_load_2d_hint(smem_u32(dst), &q_map, bar_q_full, b * 64, row0, pol_stream);
                 }
                 // ---- pass 2: the saved P tiles come back, kSaPRing tiles ahead
                 ok = mbar_wait(bar_p2_go, ph_go, abort_flag, kWaitCycleBudget, 500);
@@ -390,9 +394,16 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
                     ok = mbar_wait(bar_p_free + 8 * b, ph_p_free[b] ^ 1u, abort_flag, kWaitCycleBudget, 100);   // the PV product that read this buffer is done
                     if (!ok) break;
                     ph_p_free[b] ^= 1u;
+                    // the tile that was in this buffer has been multiplied: its saved copy is dead, and L2 need not write it
+                    // back (the last kSaPRing tiles of a query are left alone: the next query's pass 1 overwrites them)
+                    if (i >= kSaPRing) {
+                        const uint8_t* dead = scratch + static_cast<size_t>(i - kSaPRing) * kSaScratchTileBytes;
+#pragma unroll 4
+                        for (uint32_t o = 0; o < kSaPTileBytes; o += 128) l2_discard_128(dead + o);
+                    }
                     mbar_arrive_expect_tx(bar_p_full + 8 * b, kSaPTileBytes);
-                    bulk_load_1d(smem_u32(q_smem) + b * kSaPTileBytes, scratch + static_cast<size_t>(i) * kSaScratchTileBytes,
-                                 kSaPTileBytes, bar_p_full + 8 * b);
+                    bulk_load_1d_hint(smem_u32(q_smem) + b * kSaPTileBytes, scratch + static_cast<size_t>(i) * kSaScratchTileBytes,
+                                      kSaPTileBytes, bar_p_full + 8 * b, pol_keep);
                 }
             }
             if (!ok) sa_give_up(abort_flag, p.status, DEV_TIMEOUT_PRODUCER);
@@ -450,8 +461,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
 #pragma unroll
                     for (int rr = 0; rr < 8; ++rr) {
                         const uint32_t off = (bt * 8 + rr) * 128;
-                        cp_async_16((dst0 ^ (rr << 4)) + off, src[rr]);
-                        if (second) cp_async_16((dst1 ^ (rr << 4)) + off, src[rr] + 512);
+                        cp_async_16_hint((dst0 ^ (rr << 4)) + off, src[rr], pol_keep);
+                        if (second) cp_async_16_hint((dst1 ^ (rr << 4)) + off, src[rr] + 512, pol_keep);
                     }
                 }
                 cp_async_wait_all();
@@ -565,7 +576,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
                         const int rr = (lane >> 2) + 8 * k, ch = lane & 3;     // 8 rows per instruction, 4 lanes per row
                         const uint4 w = *reinterpret_cast<const uint4*>(stg + rr * 64 + ((ch ^ ((rr >> 1) & 3)) << 4));
                         if (quarter * 32 + rr < p.H)
-                            *reinterpret_cast<uint4*>(dst_query + static_cast<int64_t>(quarter * 32 + rr) * 512 + c * 32 + ch * 8) = w;
+                            st_global_v4_hint(dst_query + static_cast<int64_t>(quarter * 32 + rr) * 512 + c * 32 + ch * 8, w, pol_stream);
                     }
                     __syncwarp();
                 }
@@ -685,8 +696,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap q_map, const SaParams p) 
                         pr[j] = pack_bf16x2(p0, p1);
                     }
                     tmem_st_32x32b_x8(s_tmem + 8 * c, pr);
-                    __stcg(dst + (2 * c) * 128, make_uint4(pr[0], pr[1], pr[2], pr[3]));
-                    __stcg(dst + (2 * c + 1) * 128, make_uint4(pr[4], pr[5], pr[6], pr[7]));
+                    st_global_v4_hint(dst + (2 * c) * 128, make_uint4(pr[0], pr[1], pr[2], pr[3]), pol_keep);
+                    st_global_v4_hint(dst + (2 * c + 1) * 128, make_uint4(pr[4], pr[5], pr[6], pr[7]), pol_keep);
                 };
                 {
                     uint32_t ra[16], rb[16];

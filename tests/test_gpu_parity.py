@@ -327,9 +327,13 @@ def test_prefill_rejects_bad_arguments():
     (3, 16, 128, 24, False, [128, 1000, 2305], 0),
     (4, 32, 128, 64, False, [1, 2049, 300, 4097], 0),
     (3, 16, 128, 20, True, [700, 2100, 33], 0),
+    # FP8 at the paper's head count: several work items per sequence (the key scales are staged one item ahead and the
+    # key tiles alternate between two MMA warps), an empty sequence, one of a single key, ragged ends
+    (6, 64, 128, 64, True, [0, 9000, 4097, 129, 1, 6500], 0),
+    (2, 64, 64, 32, False, [7000, 3333], 0),          # 128-byte rows in bf16: two MMA warps, no scales
 ])
 def test_decode_matches_oracle(B, H, d, k_top, fp8, lens, flags):
-    inp = _to_dev(synth.decode_inputs(B, H, d, 0, 0, seed=20 + B, fp8=fp8, lens=lens, row_align=8))
+    inp = _to_dev(synth.decode_inputs(B, H, d, 0, 0, seed=20 + B, fp8=fp8, lens=lens, row_align=8 if B != 6 else 1))
     ld = (inp.max_len + 3) // 4 * 4
     scores = torch.full((B, ld), float("nan"), device=DEV)
     topk = torch.full((B, k_top), -7, dtype=torch.int32, device=DEV)
