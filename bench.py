@@ -462,6 +462,47 @@ def time_tmem_readout(idxc, dev, accumulators_per_warp=4096):
             "what": "fp32 accumulator bytes read out of tensor memory per second over all SMs, the scorer's load pattern alone"}
 
 
+def time_decode_fp8(idxc, synth, dev, peaks, L, H, d, k_top, seed, decode_B, first_k=None, first_k_scale=None):
+    """Decode step (one idxc_indexer_decode call: scorer + select) at batch decode_B on e4m3 caches of length L, timed on
+    two cache sets used in turn so that no step finds its keys in L2. first_k / first_k_scale: keys of a prefill that
+    become sequence 0 of set 0."""
+    sets = []
+    for si in range(2):
+        x = synth.decode_inputs(decode_B, H, d, L, L, seed=seed, device=dev, layer=1 + si, fp8=True, lens=[L] * decode_B)
+        if si == 0 and first_k is not None:
+            x.k_cache[:L] = first_k
+            x.k_scale[:L] = first_k_scale
+        sets.append(x)
+    dtop = torch.empty((decode_B, k_top), dtype=torch.int32, device=dev)
+    dws = idxc.alloc_workspace(idxc.decode_workspace_bytes(decode_B, L, H, d, k_top, idxc.FP8_E4M3), dev)
+    dld = (L + 31) // 32 * 32
+    dscores = dws[: decode_B * dld * 4].view(torch.float32).view(decode_B, dld)
+    ev_step, ev_score = [], []
+    for i in range(26):                                 # enqueued back to back: no host round trip inside a timed interval
+        x = sets[i & 1]
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        idxc.indexer_decode(x.q_step, x.k_cache, x.w, x.k_offsets, x.lens, L, k_top, x.q_scale, x.k_scale, topk_out=dtop, workspace=dws)
+        b.record()
+        ev_step.append((a, b))
+    for i in range(26):
+        x = sets[i & 1]
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        idxc.indexer_decode(x.q_step, x.k_cache, x.w, x.k_offsets, x.lens, L, k_top, x.q_scale, x.k_scale, scores_out=dscores)
+        b.record()
+        ev_score.append((a, b))
+    torch.cuda.synchronize()
+    idxc.poll_device_status()
+    us = median_event_ms(ev_step[6:]) * 1e3
+    us_sc = median_event_ms(ev_score[6:]) * 1e3
+    nbytes = decode_B * L * (d + 4)
+    return {"B": decode_B, "us_per_step": us, "us_scorer": us_sc, "us_topk": us - us_sc, "bytes": nbytes,
+            "frac_of_hbm": nbytes / (us * 1e-6) / 1e9 / peaks["hbm_gbs"],
+            "scorer_frac_of_hbm": nbytes / (us_sc * 1e-6) / 1e9 / peaks["hbm_gbs"],
+            "l2": f"two cache sets of {nbytes >> 20} MiB alternate between steps ({2 * nbytes >> 20} MiB > 126 MB L2): every step streams its keys from HBM"}
+
+
 def time_fp8_chunked(idxc, synth, dev, peaks, L, chunk, H, d, k_top, seed, decode_B, n_layers, every, readout):
     """Config 5: FP8 (e4m3 + per-token scales) chunked prefill, query chunks of `chunk` rows against the full causal K:
     one Full layer (with the two kernels timed apart), the N-layer 1-in-`every` schedule against all-Full, then one
@@ -559,41 +600,7 @@ def time_fp8_chunked(idxc, synth, dev, peaks, L, chunk, H, d, k_top, seed, decod
     del layers[1:]
     torch.cuda.empty_cache()
     # ---- decode step on caches of length L: sequence 0 of set 0 holds the prefill's keys; two cache sets alternate
-    sets = []
-    for si in range(2):
-        x = synth.decode_inputs(decode_B, H, d, L, L, seed=seed, device=dev, layer=1 + si, fp8=True, lens=[L] * decode_B)
-        if si == 0:
-            x.k_cache[:L] = inp.k
-            x.k_scale[:L] = inp.k_scale
-        sets.append(x)
-    dtop = torch.empty((decode_B, k_top), dtype=torch.int32, device=dev)
-    dws = idxc.alloc_workspace(idxc.decode_workspace_bytes(decode_B, L, H, d, k_top, idxc.FP8_E4M3), dev)
-    dld = (L + 31) // 32 * 32
-    dscores = dws[: decode_B * dld * 4].view(torch.float32).view(decode_B, dld)
-    ev_step, ev_score = [], []
-    for i in range(26):                                 # enqueued back to back: no host round trip inside a timed interval
-        x = sets[i & 1]
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        idxc.indexer_decode(x.q_step, x.k_cache, x.w, x.k_offsets, x.lens, L, k_top, x.q_scale, x.k_scale, topk_out=dtop, workspace=dws)
-        b.record()
-        ev_step.append((a, b))
-    for i in range(26):
-        x = sets[i & 1]
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        idxc.indexer_decode(x.q_step, x.k_cache, x.w, x.k_offsets, x.lens, L, k_top, x.q_scale, x.k_scale, scores_out=dscores)
-        b.record()
-        ev_score.append((a, b))
-    torch.cuda.synchronize()
-    idxc.poll_device_status()
-    us = median_event_ms(ev_step[6:]) * 1e3
-    us_sc = median_event_ms(ev_score[6:]) * 1e3
-    nbytes = decode_B * L * (d + 4)
-    out["decode"] = {"B": decode_B, "us_per_step": us, "us_scorer": us_sc, "us_topk": us - us_sc, "bytes": nbytes,
-                     "frac_of_hbm": nbytes / (us * 1e-6) / 1e9 / peaks["hbm_gbs"],
-                     "scorer_frac_of_hbm": nbytes / (us_sc * 1e-6) / 1e9 / peaks["hbm_gbs"],
-                     "l2": f"two cache sets of {nbytes >> 20} MiB alternate between steps ({2 * nbytes >> 20} MiB > 126 MB L2): every step streams its keys from HBM"}
+    out["decode"] = time_decode_fp8(idxc, synth, dev, peaks, L, H, d, k_top, seed, decode_B, inp.k, inp.k_scale)
     return out
 
 
@@ -741,6 +748,7 @@ def main():
     ap.add_argument("--full", action="store_true", help="accepted for compatibility: full sizes are the default")
     ap.add_argument("--L", type=int, default=0, help="override the workload's sequence length (small profiling cases)")
     ap.add_argument("--only-decode", action="store_true", help="run only the decode section (profiling)")
+    ap.add_argument("--only-decode-fp8", action="store_true", help="run only the batch-8 e4m3 decode step of config 5 (profiling)")
     ap.add_argument("--only-sparse-attention", action="store_true", help="run only the sparse-attention section (profiling)")
     ap.add_argument("--only-layer-loop", action="store_true", help="run only the indexer + attention layer loop section")
     ap.add_argument("--only-fp8", action="store_true", help="run only the FP8 chunked-prefill section (profiling; --L sets the length)")
@@ -786,6 +794,10 @@ def main():
     if args.only_decode:
         print(json.dumps({"decode": section(time_decode, idxc, synth, dev, peaks, steps=max(args.steps, 1), warmup=args.warmup)}),
               flush=True)
+        return
+    if args.only_decode_fp8:
+        print(json.dumps({"decode_fp8": section(time_decode_fp8, idxc, synth, dev, peaks, args.L or c5["L"], c5["H"], c5["d"], c5["k_top"],
+                                                c5["seed"], c5["decode_B"])}), flush=True)
         return
     if args.only_layer_loop:
         print(json.dumps({"layer_loop": section(time_layer_loop, idxc, synth, dev, args.L or 32768, 2048, 4, 4, seed=8)}), flush=True)
