@@ -44,6 +44,9 @@ typedef enum { IDXC_BF16 = 0, IDXC_FP8_E4M3 = 1 } idxc_dtype;
 #define IDXC_FLAG_FILL_MASKED 0x4u  /* prefill with scores_out: entries s > t of every row, up to column L_k - 1, are set
                                        to -infinity (the causal mask as a soft-max expects it) instead of left untouched */
 
+#define IDXC_FLAG_STREAM_TOPK 0x8u  /* prefill with topk_out only: the scorer keeps, per query row, only the scores that can
+                                       still be among the k_top largest (see idxc_indexer_prefill) instead of writing all */
+
 /* Limits checked before any launch. */
 #define IDXC_MAX_K_TOP 2048
 #define IDXC_MAX_HEADS 64
@@ -73,6 +76,13 @@ const char* idxc_status_string(idxc_status s);
  *   workspace   at least idxc_prefill_workspace_bytes(...) bytes, 256-byte aligned;
  *               contents are scratch. With scores_out == NULL the scores go through it
  *               in query chunks, so its size does not grow with q_len beyond a cap.
+ * IDXC_FLAG_STREAM_TOPK (north star: "the score write or streaming top-k in the epilogue"; needs topk_out, scores_out
+ * == NULL, L_k <= 262144 and a workspace sized with the same flag): the scorer visits a strided sample of a row's
+ * keys first, takes from it a threshold that almost surely lies below the row's k_top-th largest score, and from then
+ * on writes only (score, position) pairs at or above it to a per-row list; a second kernel selects exactly from the
+ * list after checking, with its own count, that at least k_top listed scores reach the threshold. Rows that fail the
+ * check (or whose list overflowed: many equal scores) are computed again by the ordinary score + select kernels,
+ * which run after it and skip every other row. T is the same as without the flag, entry for entry.
  * A full prefill is q_begin = 0, q_len = L_k = L; chunked prefill calls this once
  * per chunk with the full K and gives the same rows.
  * Supported: d_I in {64, 128}; H_I in {16, 32, 64}; 1 <= k_top <= 2048; q_len * H_I < 2^31;

@@ -20,6 +20,7 @@ BF16, FP8_E4M3 = 0, 1
 FLAG_COPY_SHARED = 0x1
 FLAG_SIMT_SCORER = 0x2
 FLAG_FILL_MASKED = 0x4
+FLAG_STREAM_TOPK = 0x8
 
 EXPORTED_SYMBOLS = [
     "idxc_status_string", "idxc_prefill_workspace_bytes", "idxc_indexer_prefill", "idxc_decode_workspace_bytes",

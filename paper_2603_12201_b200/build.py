@@ -10,7 +10,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libidxc.so"
-SOURCES = ["api.cu", "topk.cu", "topk_cluster.cu", "scorer_simt.cu", "scorer_tc.cu", "noalloc.cu", "selftest.cu", "quantize.cu", "pattern_tools.cu", "distill.cu", "sparse_attn.cu"]
+SOURCES = ["api.cu", "topk.cu", "topk_cluster.cu", "topk_stream.cu", "scorer_simt.cu", "scorer_tc.cu", "noalloc.cu", "selftest.cu", "quantize.cu", "pattern_tools.cu", "distill.cu", "sparse_attn.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr",

@@ -78,10 +78,16 @@ idxc_status check_common(int H, int d, int k_top, idxc_dtype dt, uint32_t flags)
     if (dt != IDXC_BF16 && dt != IDXC_FP8_E4M3) return IDXC_ERR_INVALID_ARG;
     if (k_top < 1 || k_top > IDXC_MAX_K_TOP) return IDXC_ERR_INVALID_ARG;
     if (H < 1 || H > IDXC_MAX_HEADS || d < 1) return IDXC_ERR_INVALID_ARG;
-    if (flags & ~(IDXC_FLAG_COPY_SHARED | IDXC_FLAG_SIMT_SCORER | IDXC_FLAG_FILL_MASKED)) return IDXC_ERR_INVALID_ARG;
+    if (flags & ~(IDXC_FLAG_COPY_SHARED | IDXC_FLAG_SIMT_SCORER | IDXC_FLAG_FILL_MASKED | IDXC_FLAG_STREAM_TOPK)) return IDXC_ERR_INVALID_ARG;
+    if ((flags & IDXC_FLAG_STREAM_TOPK) && (flags & IDXC_FLAG_SIMT_SCORER)) return IDXC_ERR_INVALID_ARG;
     if (!(flags & IDXC_FLAG_SIMT_SCORER) && !score_tc_supported(H, d, dt == IDXC_FP8_E4M3)) return IDXC_ERR_UNSUPPORTED;
     return IDXC_OK;
 }
+
+// Streaming top-k: bytes of workspace per query row of a chunk (full scores for the rows that are computed again, the
+// candidate lists, their lengths, the threshold, two flag bytes) and the slack for aligning the seven regions.
+int64_t stream_bytes_per_row(int64_t ld) { return ld * 4 + static_cast<int64_t>(kStreamRowSlots) * 8 + kStreamLanes + 4 + 4 + 2; }
+constexpr int64_t kStreamSlack = 7 * 256;
 
 idxc_status launch_scorer(const ScoreArgs& a, bool decode, uint32_t flags, cudaStream_t stream) {
     if (flags & IDXC_FLAG_SIMT_SCORER) {
@@ -160,14 +166,15 @@ int64_t idxc_launch_count(void) { return g_launches.load(); }
 
 size_t idxc_prefill_workspace_bytes(int64_t q_len, int64_t L_k, int H_I, int d_I, int k_top, idxc_dtype dt,
                                     uint32_t flags) {
-    (void)L_k; (void)H_I; (void)d_I; (void)k_top; (void)dt; (void)flags;
+    (void)L_k; (void)H_I; (void)d_I; (void)k_top; (void)dt;
     if (q_len <= 0) return 0;
     // scratch rows of round_up(L_k, 32) floats; L_k bounds q_begin + q_len
     const int64_t ld = round_up(L_k > q_len ? L_k : q_len, 32);
+    const int64_t per_row = (flags & IDXC_FLAG_STREAM_TOPK) ? stream_bytes_per_row(ld) : ld * 4;
     int64_t rows = round_up(q_len, kMinChunkRows);
-    const int64_t cap = (kPreferredScratchBytes / (ld * 4)) / kMinChunkRows * kMinChunkRows;
+    const int64_t cap = (kPreferredScratchBytes / per_row) / kMinChunkRows * kMinChunkRows;
     if (rows > cap) rows = cap < kMinChunkRows ? kMinChunkRows : cap;
-    return static_cast<size_t>(rows * ld * 4);
+    return static_cast<size_t>(rows * per_row + ((flags & IDXC_FLAG_STREAM_TOPK) ? kStreamSlack : 0));
 }
 
 idxc_status idxc_indexer_prefill(const void* q, const void* k, const float* w, const float* q_scale,
@@ -187,6 +194,11 @@ idxc_status idxc_indexer_prefill(const void* q, const void* k, const float* w, c
     if (fp8 && (!q_scale || !k_scale)) return IDXC_ERR_INVALID_ARG;
     if (scores_out && (ld_scores < L_k || (ld_scores & 3) || !aligned(scores_out, 16))) return IDXC_ERR_INVALID_ARG;
     if (topk_out && !aligned(topk_out, 4)) return IDXC_ERR_INVALID_ARG;
+    const bool streaming = (flags & IDXC_FLAG_STREAM_TOPK) != 0;
+    if (streaming) {
+        if (scores_out || !topk_out) return IDXC_ERR_INVALID_ARG;
+        if (L_k > kStreamMaxKeys || !score_prefill_stream_supported(H_I, d_I, fp8 ? 1 : 0)) return IDXC_ERR_UNSUPPORTED;
+    }
     if (!device_info().ok) return IDXC_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int64_t elem = fp8 ? 1 : 2;
@@ -224,6 +236,48 @@ idxc_status idxc_indexer_prefill(const void* q, const void* k, const float* w, c
     // scores go through the workspace in query chunks
     const int64_t ld = round_up(q_begin + q_len, 32);
     if (!workspace || !aligned(workspace, 256)) return IDXC_ERR_WORKSPACE;
+    if (streaming) {
+        if (workspace_bytes < static_cast<size_t>(kStreamSlack)) return IDXC_ERR_WORKSPACE;
+        const int64_t per_row = stream_bytes_per_row(ld);
+        const int64_t chunk = static_cast<int64_t>((workspace_bytes - kStreamSlack) / static_cast<size_t>(per_row)) / kMinChunkRows * kMinChunkRows;
+        if (chunk < kMinChunkRows) return IDXC_ERR_WORKSPACE;
+        // regions of the workspace, each 256-byte aligned (chunk is a multiple of 32 rows)
+        char* base = static_cast<char*>(workspace);
+        auto take = [&](int64_t bytes) { char* r = base; base += round_up(bytes, 256); return r; };
+        float* sc = reinterpret_cast<float*>(take(chunk * ld * 4));
+        StreamTopk stt{};
+        stt.cand = reinterpret_cast<uint2*>(take(chunk * kStreamRowSlots * 8));
+        stt.sample_count = reinterpret_cast<uint32_t*>(take(chunk * 4));
+        stt.lane_count = reinterpret_cast<uint8_t*>(take(chunk * kStreamLanes));
+        stt.tau = reinterpret_cast<float*>(take(chunk * 4));
+        stt.k_top = k_top;
+        uint8_t* row_fail = reinterpret_cast<uint8_t*>(take(chunk));
+        uint8_t* item_fail = reinterpret_cast<uint8_t*>(take(chunk));
+        const int rows_per_item = score_prefill_rows_per_item(H_I);
+        for (int64_t r0 = 0; r0 < q_len; r0 += chunk) {
+            const int64_t nr = q_len - r0 < chunk ? q_len - r0 : chunk;
+            a.q = static_cast<const char*>(q) + r0 * H_I * d_I * elem;
+            a.w = w + r0 * H_I;
+            a.q_scale = fp8 ? q_scale + r0 : nullptr;
+            a.q_begin = q_begin + r0;
+            a.n_rows = nr;
+            // 1. scorer with the filtered lists instead of the score write; 2. exact selection from the lists
+            a.scores = nullptr; a.ld = 0; a.stream = stt; a.item_mask = nullptr;
+            st = launch_scorer(a, false, flags, stream);
+            if (st != IDXC_OK) return st;
+            g_launches += 1;
+            if (launch_finish_topk_stream(stt, nr, q_begin + r0, rows_per_item, topk_out + r0 * k_top, row_fail, item_fail, stream) != cudaSuccess)
+                return IDXC_ERR_CUDA;
+            // 3. the blocks of rows with a flagged row, scored in full; 4. the flagged rows, selected the ordinary way
+            a.scores = sc; a.ld = ld; a.stream = StreamTopk{}; a.item_mask = item_fail;
+            st = launch_scorer(a, false, flags, stream);
+            if (st != IDXC_OK) return st;
+            g_launches += 1;
+            if (launch_topk_rows(sc, ld, nr, q_begin + r0 + 1, 1, nullptr, k_top, topk_out + r0 * k_top, stream, row_fail) != cudaSuccess)
+                return IDXC_ERR_CUDA;
+        }
+        return IDXC_OK;
+    }
     int64_t chunk = static_cast<int64_t>(workspace_bytes / static_cast<size_t>(ld * 4)) / kMinChunkRows * kMinChunkRows;
     if (chunk < kMinChunkRows) return IDXC_ERR_WORKSPACE;
     for (int64_t r0 = 0; r0 < q_len; r0 += chunk) {

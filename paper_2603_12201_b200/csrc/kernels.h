@@ -12,17 +12,45 @@ namespace idxc {
 cudaError_t ensure_max_dynamic_smem(const void* kernel, int bytes);
 
 // Row-wise top-k select (topk.cu). Row r has length lens[r] (device) if lens != nullptr,
-// else first_len + r * len_step, clamped to [0, ld].
+// else first_len + r * len_step, clamped to [0, ld]. row_mask: nullptr, or one byte per row: rows whose byte is 0 are
+// left alone (neither read nor written).
 cudaError_t launch_topk_rows(const float* scores, int64_t ld, int64_t n_rows, int64_t first_len,
                              int64_t len_step, const int32_t* lens, int k_top, int32_t* out,
-                             cudaStream_t stream);
+                             cudaStream_t stream, const uint8_t* row_mask = nullptr);
 
 // Cluster variant for a few long rows (topk_cluster.cu): 8 CTAs per row exchanging through
 // distributed shared memory. `longest` = longest row of the launch.
 bool topk_cluster_applicable(int64_t n_rows, int64_t longest);
 cudaError_t launch_topk_rows_cluster(const float* scores, int64_t ld, int64_t n_rows, int64_t first_len,
                                      int64_t len_step, const int32_t* lens, int k_top, int32_t* out,
-                                     int64_t longest, cudaStream_t stream);
+                                     int64_t longest, cudaStream_t stream, const uint8_t* row_mask = nullptr);
+
+// Streaming top-k of the prefill scorer (the score write replaced by a filtered candidate list per query row):
+// the scorer visits a strided sample of a work item's key tiles first, takes from each row's sample a threshold that
+// with high probability lies below the row's k_top-th largest score, and from then on appends only the (score, key
+// index) pairs at or above the threshold. finish_topk_stream (topk_stream.cu) takes the exact top-k of each list,
+// or flags the row (threshold too high after all, or a list overflow) for the ordinary score + select path.
+// A row's list is kStreamRowSlots pairs (x = score bits, y = key index): first the sample's own scores at or above the
+// threshold (up to kStreamSampleCap), then 128 lists of kStreamLaneCap slots, one per scorer thread that sees keys of the
+// row (TMEM lane quarter * 32 + lane): a thread appends at a position it keeps in a register, with no vote or atomic.
+constexpr int kStreamSampleCap = 1024;
+constexpr int kStreamLaneCap = 64;
+constexpr int kStreamLanes = 128;
+constexpr int kStreamRowSlots = kStreamSampleCap + kStreamLanes * kStreamLaneCap;   // 9216 pairs = 72 KB per row
+constexpr int kStreamMaxKeys = 262144;      // longest row the second half's position bitmap covers
+struct StreamTopk {
+    uint2* cand;            // [n_rows, kStreamRowSlots]; nullptr: ordinary score write
+    uint32_t* sample_count; // [n_rows] pairs in the sample part
+    uint8_t* lane_count;    // [n_rows, kStreamLanes] pairs appended by each thread, saturating at 255 (> kStreamLaneCap: overflow)
+    float* tau;             // [n_rows] the row's threshold (-inf: none)
+    int k_top;
+};
+
+// topk_stream.cu: exact top-k of every row's candidate list into out [n_rows, k_top] (ascending key indices, -1
+// padding), or row_fail[row] = 1 where the list cannot give it; item_fail[b] = 1 where block b of rows_per_item rows
+// holds a flagged row (both arrays are written in full).
+cudaError_t launch_finish_topk_stream(const StreamTopk& st, int64_t n_rows, int64_t q_begin, int rows_per_item, int32_t* out,
+                                      uint8_t* row_fail, uint8_t* item_fail, cudaStream_t stream);
 
 // Arguments shared by the scorers. A "row" is one query vector set [H, d].
 struct ScoreArgs {
@@ -41,6 +69,8 @@ struct ScoreArgs {
     int fp8;                // 0: bf16, 1: e4m3 codes with scales
     float* scores;          // [n_rows, ld]
     int64_t ld;
+    StreamTopk stream;      // prefill only; cand == nullptr: scores are written
+    const uint8_t* item_mask;   // prefill only: nullptr, or one byte per block of rows_per_item rows: 0 = skip the block
 };
 
 // Plain CUDA-core scorer (scorer_simt.cu): debugging aid and cross-check.
@@ -56,6 +86,10 @@ cudaError_t launch_score_prefill_tc(const ScoreArgs& a, const CUtensorMap& q_map
 cudaError_t launch_score_decode_tc(const ScoreArgs& a, const CUtensorMap& q_map, const CUtensorMap& k_map,
                                    unsigned int* status, int sm_count, cudaStream_t stream);
 bool score_tc_supported(int H, int d, int fp8);
+// Streaming top-k is built for the shapes whose work item leaves room for the sample (scorer_tc.cu).
+bool score_prefill_stream_supported(int H, int d, int fp8);
+// Query rows per work item of the prefill scorer (the granularity of item_mask).
+int score_prefill_rows_per_item(int H);
 // Load every kernel a decode step can launch on the current device and set its attributes (scorer_tc.cu, topk.cu,
 // topk_cluster.cu, scorer_simt.cu), so that later launches find them resident.
 cudaError_t preload_score_decode_tc();

@@ -23,6 +23,7 @@
 // epilogue warps drain alternate TMEM accumulator slots.
 #include "kernels.h"
 #include "ptx_sm100.cuh"
+#include "topk_common.cuh"
 
 namespace idxc {
 namespace {
@@ -45,13 +46,21 @@ constexpr int kColsPerEpiWarp = kTileCols / (kNumEpilogueWarps / 4);   // 128 or
 constexpr int kGroupsPerEpiWarp = kColsPerEpiWarp / 8;               // 8-column groups per warp
 constexpr int kChunksPerEpiWarp = kColsPerEpiWarp / 32;              // 32-column TMEM loads per 16 lanes
 
-template <int NKH>
+// STREAM: streaming top-k (kernels.h, StreamTopk). The sample of a work item's rows lives in shared memory
+// (kStreamSampleBytes over all rows of the item); with 256-byte operand rows the key ring gives up a stage for it.
+constexpr int kStreamSampleBytes = 32 * 1024;
+template <int NKH, int H, bool STREAM>
 struct PrefillCfg {
-    static constexpr int kStages = NKH == 2 ? 3 : 4;
+    static constexpr int QB = 2 * (kTileCols / H);
+    static constexpr int kStages = NKH == 2 ? (STREAM ? 2 : 3) : 4;
     static constexpr int kQBytes = 2 * NKH * kQRegionBytes;
     static constexpr int kKBytes = kStages * NKH * kKRegionBytes;
-    static constexpr int kBarBytes = 256;
-    static constexpr int kSmemBytes = kQBytes + kKBytes + kBarBytes + 1024;   // + alignment slack
+    static constexpr int kSampleBytes = STREAM ? kStreamSampleBytes : 0;
+    static constexpr int kSampleMax = kStreamSampleBytes / 4 / QB;          // sample scores per row: 1024, 512, 256
+    static constexpr int kSampleTiles = kSampleMax / kTileKeys;             // key tiles visited before the threshold exists
+    static constexpr int kBarBytes = 256 + (STREAM ? 16 * QB + 1024 : 0);   // + per-row counter, threshold; 32 bins per epilogue warp
+    static constexpr int kSmemBytes = kQBytes + kKBytes + kSampleBytes + kBarBytes + 1024;   // + alignment slack
+    static constexpr bool kFits = kSmemBytes <= 227 * 1024 && kSampleTiles >= 2;
 };
 
 struct PrefillParams {
@@ -64,6 +73,24 @@ struct PrefillParams {
     int64_t n_rows;
     int64_t k_rows;
     unsigned int* status;
+    StreamTopk st;
+    const uint8_t* item_mask;
+};
+
+// Order in which a work item of nkt key tiles is visited when the top-k streams: `ns` sample tiles 0, stride,
+// 2 stride, ... first, then the others in ascending order. Without a sample (ns == nkt) the order is plain.
+struct TileOrder {
+    int nkt, stride, ns;
+    __device__ TileOrder(int nkt_, int max_sample_tiles) : nkt(nkt_) {
+        stride = (nkt + max_sample_tiles - 1) / max_sample_tiles;
+        if (stride < 2) { stride = 1; ns = nkt; }
+        else ns = (nkt + stride - 1) / stride;
+    }
+    __device__ int tile(int j) const {
+        if (j < ns) return j * stride;
+        const int r = j - ns;                       // r-th tile that is not a multiple of stride
+        return r + r / (stride - 1) + 1;
+    }
 };
 
 __device__ __forceinline__ void give_up(volatile uint32_t* abort_flag, unsigned int* status, unsigned int code) {
@@ -72,11 +99,11 @@ __device__ __forceinline__ void give_up(volatile uint32_t* abort_flag, unsigned 
 }
 
 // NKH: 128-byte chunks per operand row (d * element size / 128). H: indexer heads.
-template <int NKH, int H, bool FP8>
+template <int NKH, int H, bool FP8, bool STREAM>
 __global__ void __launch_bounds__(kPrefillThreads, 1)
 score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                         const PrefillParams p) {
-    using Cfg = PrefillCfg<NKH>;
+    using Cfg = PrefillCfg<NKH, H, STREAM>;
     constexpr int kStages = Cfg::kStages;
     constexpr int QPA = kTileCols / H;       // queries per accumulator
     constexpr int QB = 2 * QPA;              // queries per work item
@@ -87,7 +114,8 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint8_t* q_smem = smem;                                   // [2][NKH][256 x 128 B]
     uint8_t* k_smem = q_smem + Cfg::kQBytes;                  // [kStages][NKH][128 x 128 B]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(k_smem + Cfg::kKBytes);
+    float* sample = reinterpret_cast<float*>(k_smem + Cfg::kKBytes);          // STREAM: [QB][kSampleMax] scores of the sample tiles
+    uint64_t* bars = reinterpret_cast<uint64_t*>(k_smem + Cfg::kKBytes + Cfg::kSampleBytes);
     // barrier map
     const uint32_t bar_q_full = smem_u32(bars + 0);           // [2]
     const uint32_t bar_q_empty = smem_u32(bars + 2);          // [2]
@@ -95,8 +123,12 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
     const uint32_t bar_acc_empty = smem_u32(bars + 6);        // [2]
     const uint32_t bar_k_full = smem_u32(bars + 8);           // [kStages]
     const uint32_t bar_k_empty = smem_u32(bars + 8 + kStages);
-    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(bars + 8 + 2 * kStages);
+    const uint32_t bar_group = smem_u32(bars + 8 + 2 * kStages);   // STREAM: [2] the four warps that share a set of query rows
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(bars + 10 + 2 * kStages);
     volatile uint32_t* abort_flag = tmem_base_slot + 1;
+    float* row_tau = reinterpret_cast<float*>(tmem_base_slot + 4);   // STREAM: [QB] the row's threshold
+    uint32_t* warp_hist = reinterpret_cast<uint32_t*>(row_tau + QB);   // STREAM: [epilogue warps][32]
+    static_assert((10 + 2 * kStages) * 8 + 16 + (STREAM ? 4 * QB + 128 * kNumEpilogueWarps : 0) <= Cfg::kBarBytes, "barrier area");
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -112,6 +144,8 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
             mbar_init(bar_k_full + 8 * i, 1);
             mbar_init(bar_k_empty + 8 * i, 1);
         }
+        mbar_init(bar_group, kNumEpilogueWarps / 2);
+        mbar_init(bar_group + 8, kNumEpilogueWarps / 2);
         *abort_flag = 0u;
         fence_mbar_init();
     }
@@ -128,9 +162,13 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
     const int G = gridDim.x;
     const int cta = blockIdx.x;
     // work item of this CTA in round `rho` (longest first, boustrophedon), or -1
+    // (-2: the item is masked out and every role passes over it)
     auto item_of_round = [&](int64_t rho) -> int64_t {
         const int64_t seq = rho * G + ((rho & 1) ? (G - 1 - cta) : cta);
-        return seq < n_items ? n_items - 1 - seq : -1;
+        if (seq >= n_items) return -1;
+        const int64_t item = n_items - 1 - seq;
+        if (p.item_mask != nullptr && p.item_mask[item] == 0) return -2;
+        return item;
     };
     auto key_tiles_of_item = [&](int64_t item) -> int {
         int64_t last = item * QB + QB;
@@ -148,9 +186,12 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
             bool ok = true;
             for (int64_t rho = 0; ok; ++rho) {
                 const int64_t item = item_of_round(rho);
+                if (item == -2) continue;
                 if (item < 0) break;
                 const int nkt = key_tiles_of_item(item);
-                auto load_k = [&](int kt) -> bool {
+                const TileOrder ord(nkt, STREAM ? Cfg::kSampleTiles : nkt);
+                auto load_k = [&](int j) -> bool {
+                    const int kt = STREAM ? ord.tile(j) : j;
                     if (!mbar_wait(bar_k_empty + 8 * stage, k_phase ^ 1u, abort_flag)) return false;
                     mbar_arrive_expect_tx(bar_k_full + 8 * stage, NKH * kKRegionBytes);
                     for (int kh = 0; kh < NKH; ++kh)
@@ -192,6 +233,7 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
         };
         for (int64_t rho = 0; ok; ++rho) {
             const int64_t item = item_of_round(rho);
+            if (item == -2) continue;
             if (item < 0) break;
             const int nkt = key_tiles_of_item(item);
             for (int kt = 0; kt < nkt && ok; ++kt) {
@@ -249,12 +291,33 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
         const int j = lane & 3, g = lane >> 2;
         const int key_written = quarter * 32 + g + 8 * j;    // the key (of the thread's four) this thread stores
         uint32_t acc_phase[2] = {0u, 0u};
+        uint32_t grp_phase = 0;                      // STREAM: phase of this warp group's barrier
         bool ok = true;
+        // STREAM: the four warps that hold the same columns (one per TMEM lane quarter) share 2 QPW query rows; they meet
+        // at a barrier of their own (bounded like every other wait)
+        auto group_sync = [&]() -> bool {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_group + 8 * colhalf);
+            const bool good = __all_sync(0xFFFFFFFFu, mbar_wait(bar_group + 8 * colhalf, grp_phase, abort_flag));
+            grp_phase ^= 1u;
+            return good;
+        };
         for (int64_t rho = 0; ok; ++rho) {
             const int64_t item = item_of_round(rho);
+            if (item == -2) continue;
             if (item < 0) break;
             const int nkt = key_tiles_of_item(item);
+            const TileOrder ord(nkt, STREAM ? Cfg::kSampleTiles : nkt);
             const int64_t row_base = item * QB;
+            // STREAM: every thread has a list of its own per row (it sees one key of each tile), so it appends at a position
+            // it keeps in a register: no vote, no atomic, nothing to wait for
+            uint32_t my_count[STREAM ? 2 * QPW : 1];
+#pragma unroll
+            for (int c = 0; c < (STREAM ? 2 * QPW : 1); ++c) my_count[c] = 0u;
+            // this thread's list of the group's first row; row c of the group is c / QPW * QPA + c % QPW rows further
+            uint2* const my_list = STREAM ? p.st.cand + (row_base + colhalf * QPW) * kStreamRowSlots + kStreamSampleCap +
+                                                (quarter * 32 + lane) * kStreamLaneCap
+                                          : nullptr;
             uint64_t wreg[2][kGroupsPerEpiWarp];       // (w of column 8g+2j, w of column 8g+2j+1), packed
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
@@ -273,7 +336,8 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
                     wreg[half][grp] = pack_f32x2(v.x, v.y);
                 }
             }
-            for (int kt = 0; kt < nkt && ok; ++kt) {
+            for (int jt = 0; jt < nkt && ok; ++jt) {
+                const int kt = STREAM ? ord.tile(jt) : jt;
                 const int64_t s = static_cast<int64_t>(kt) * kTileKeys + key_written;
                 float ksc = 1.f;
                 if constexpr (FP8) ksc = s < p.k_rows ? __ldg(p.k_scale + s) : 0.f;
@@ -333,12 +397,129 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
                             v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
                             if (r == j) mine = v;                      // thread j of the group stores key g + 8j
                         }
-                        const int64_t row = row_base + half * QPA + colhalf * QPW + i;
+                        const int r_item = half * QPA + colhalf * QPW + i;
+                        const int64_t row = row_base + r_item;
                         const int64_t t = p.q_begin + row;
-                        if (row < p.n_rows && s <= t) {
-                            if constexpr (FP8) mine *= ksc;
-                            p.scores[row * p.ld + s] = mine;
+                        if constexpr (FP8) mine *= ksc;
+                        if constexpr (!STREAM) {
+                            if (row < p.n_rows && s <= t) p.scores[row * p.ld + s] = mine;
+                        } else if (jt < ord.ns) {
+                            // a sample tile: every score goes to the row's sample (which of them are real is worked out
+                            // from their place when the sample is read)
+                            sample[r_item * Cfg::kSampleMax + jt * kTileKeys + key_written] = mine;
+                        } else {
+                            // past the sample: only scores that are not below the row's threshold (a NaN stays in)
+                            if (row < p.n_rows && s <= t && !(mine < row_tau[r_item])) {
+                                const uint32_t pos = my_count[half * QPW + i]++;
+                                if (pos < static_cast<uint32_t>(kStreamLaneCap))
+                                    my_list[(half * QPA + i) * kStreamRowSlots + pos] = make_uint2(__float_as_uint(mine), static_cast<uint32_t>(s));
+                            }
                         }
+                    }
+                }
+                if constexpr (STREAM) {
+                    if (ok && jt == ord.ns - 1) {
+                        // ---- the sample is complete: each warp of the group takes the thresholds of its share of the rows
+                        ok = group_sync();
+                        if (!ok) break;
+                        for (int idx = quarter; idx < 2 * QPW; idx += 4) {
+                            const int r_item = (idx / QPW) * QPA + colhalf * QPW + idx % QPW;
+                            const int64_t row = row_base + r_item;
+                            if (row >= p.n_rows) continue;                          // warp-uniform
+                            const int64_t t = p.q_begin + row;
+                            const float* smp = sample + r_item * Cfg::kSampleMax;
+                            // place p of the sample is key (p / 128) * stride * 128 + p % 128; keys grow with the place, so
+                            // the real scores (key <= t) are the first n_valid places
+                            const int64_t tile_span = static_cast<int64_t>(ord.stride) * kTileKeys;
+                            const int64_t j_last = t / tile_span;
+                            int n_valid = ord.ns * kTileKeys;
+                            if (j_last < ord.ns) {
+                                const int64_t in_tile = t - j_last * tile_span + 1;
+                                n_valid = static_cast<int>(j_last) * kTileKeys + static_cast<int>(in_tile < kTileKeys ? in_tile : kTileKeys);
+                            }
+                            // rank (from the top) of the sample score wanted as threshold: where the k_top-th largest of the
+                            // t + 1 scores is expected in a sample of n_valid, plus 4.5 standard deviations of that count
+                            const float frac = static_cast<float>(n_valid) / static_cast<float>(t + 1);
+                            const float expect = static_cast<float>(p.st.k_top) * frac;
+                            const float rank_f = ceilf(expect + 4.5f * sqrtf(expect * fmaxf(1.f - frac, 0.f)) + 2.f);
+                            float tau = -INFINITY;
+                            if (rank_f < static_cast<float>(n_valid)) {
+                                const uint32_t rank = static_cast<uint32_t>(rank_f);
+                                // mean and spread of the sample, then 32 bins of 3/32 spreads around where a normal sample
+                                // has that rank; the threshold is the lower edge of the highest bin that, with the bins
+                                // above it, holds `rank` scores (a sample score of at least that rank: never too high)
+                                float s1 = 0.f, s2 = 0.f;
+                                for (int place = lane; place < n_valid; place += 32) {
+                                    const float x = smp[place];
+                                    s1 += x;
+                                    s2 = fmaf(x, x, s2);
+                                }
+#pragma unroll
+                                for (int o = 16; o > 0; o >>= 1) {
+                                    s1 += __shfl_xor_sync(0xFFFFFFFFu, s1, o);
+                                    s2 += __shfl_xor_sync(0xFFFFFFFFu, s2, o);
+                                }
+                                const float inv_n = 1.f / static_cast<float>(n_valid);
+                                const float mean = s1 * inv_n;
+                                const float sd = sqrtf(fmaxf(s2 * inv_n - mean * mean, 0.f));
+                                const float z = topk::upper_quantile_z(static_cast<float>(rank) * inv_n);
+                                const float lo_edge = mean + (z - 1.5f) * sd;
+                                const float scale = 32.f / (3.f * sd);
+                                if (sd > 0.f && fabsf(scale) < 3.0e38f && fabsf(lo_edge) < 3.0e38f) {      // finite, not constant
+                                    uint32_t* hist = warp_hist + (warp - kEpilogueWarp0) * 32;
+                                    hist[lane] = 0u;
+                                    __syncwarp();
+                                    for (int place = lane; place < n_valid; place += 32) {
+                                        const int bin = __float2int_rd((smp[place] - lo_edge) * scale);
+                                        if (bin >= 0) atomicAdd(&hist[bin < 31 ? bin : 31], 1u);
+                                    }
+                                    __syncwarp();
+                                    uint32_t from_top = hist[lane];                       // scores in bins lane .. 31
+#pragma unroll
+                                    for (int o = 1; o < 32; o <<= 1) {
+                                        const uint32_t y = __shfl_down_sync(0xFFFFFFFFu, from_top, o);
+                                        if (lane + o < 32) from_top += y;
+                                    }
+                                    const uint32_t reach = __ballot_sync(0xFFFFFFFFu, from_top >= rank);
+                                    if (reach != 0u) tau = lo_edge + static_cast<float>(31 - __clz(reach)) / scale;
+                                    __syncwarp();
+                                }
+                            }
+                            // the sample's own scores that are not below the threshold open the row's list
+                            uint32_t mine_mask = 0;                                   // bit e: place lane + 32 e passes
+                            for (int e = 0; e < Cfg::kSampleMax / 32; ++e) {
+                                const int place = lane + 32 * e;
+                                if (place < n_valid && !(smp[place] < tau)) mine_mask |= 1u << e;
+                            }
+                            uint32_t total;
+                            uint32_t pos = topk::warp_excl_scan(static_cast<uint32_t>(__popc(mine_mask)), lane, total);
+                            while (mine_mask != 0u) {
+                                const int e = __ffs(mine_mask) - 1;
+                                mine_mask &= mine_mask - 1u;
+                                const int place = lane + 32 * e;
+                                if (pos < static_cast<uint32_t>(kStreamSampleCap))
+                                    p.st.cand[row * kStreamRowSlots + pos] =
+                                        make_uint2(__float_as_uint(smp[place]), static_cast<uint32_t>((place >> 7) * tile_span + (place & 127)));
+                                ++pos;
+                            }
+                            if (lane == 0) p.st.sample_count[row] = total;       // (never above kStreamSampleCap: the sample is no larger)
+                            if (lane == 0) row_tau[r_item] = tau;
+                        }
+                        ok = group_sync();
+                        if (!ok) break;
+                    }
+                }
+            }
+            if constexpr (STREAM) {
+                // ---- end of the item: this warp's sub-list lengths go out (and the thresholds of the rows it owns)
+                if (!ok) break;
+#pragma unroll
+                for (int c = 0; c < 2 * QPW; ++c) {
+                    const int r_item = (c / QPW) * QPA + colhalf * QPW + c % QPW;
+                    const int64_t row = row_base + r_item;
+                    if (row < p.n_rows) {
+                        p.st.lane_count[row * kStreamLanes + quarter * 32 + lane] = static_cast<uint8_t>(my_count[c] < 255u ? my_count[c] : 255u);
+                        if (lane == 0 && (c & 3) == quarter) p.st.tau[row] = row_tau[r_item];
                     }
                 }
             }
@@ -362,18 +543,30 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
     }
 }
 
-template <int NKH, int H, bool FP8>
-cudaError_t launch_prefill_instance(const ScoreArgs& a, const CUtensorMap& q_map, const CUtensorMap& k_map,
-                                    unsigned int* status, int sm_count, cudaStream_t stream) {
-    using Cfg = PrefillCfg<NKH>;
-    auto kern = score_prefill_tc_kernel<NKH, H, FP8>;
+template <int NKH, int H, bool FP8, bool STREAM>
+cudaError_t launch_prefill_variant(const ScoreArgs& a, const CUtensorMap& q_map, const CUtensorMap& k_map,
+                                   unsigned int* status, int sm_count, cudaStream_t stream) {
+    using Cfg = PrefillCfg<NKH, H, STREAM>;
+    auto kern = score_prefill_tc_kernel<NKH, H, FP8, STREAM>;
     if (cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(kern), Cfg::kSmemBytes); e != cudaSuccess) return e;
     constexpr int QB = 2 * (kTileCols / H);
     const int64_t n_items = (a.n_rows + QB - 1) / QB;
     const int grid = static_cast<int>(n_items < sm_count ? n_items : sm_count);
-    PrefillParams p{a.w, a.q_scale, a.k_scale, a.scores, a.ld, a.q_begin, a.n_rows, a.k_rows, status};
+    PrefillParams p{a.w, a.q_scale, a.k_scale, a.scores, a.ld, a.q_begin, a.n_rows, a.k_rows, status, a.stream, a.item_mask};
     kern<<<grid, kPrefillThreads, Cfg::kSmemBytes, stream>>>(q_map, k_map, p);
     return cudaGetLastError();
+}
+
+template <int NKH, int H, bool FP8>
+cudaError_t launch_prefill_instance(const ScoreArgs& a, const CUtensorMap& q_map, const CUtensorMap& k_map,
+                                    unsigned int* status, int sm_count, cudaStream_t stream) {
+    if (a.stream.cand != nullptr) {
+        if constexpr (PrefillCfg<NKH, H, true>::kFits)
+            return launch_prefill_variant<NKH, H, FP8, true>(a, q_map, k_map, status, sm_count, stream);
+        else
+            return cudaErrorInvalidValue;
+    }
+    return launch_prefill_variant<NKH, H, FP8, false>(a, q_map, k_map, status, sm_count, stream);
 }
 
 }  // namespace
@@ -383,6 +576,18 @@ bool score_tc_supported(int H, int d, int fp8) {
     if (fp8) return d == 128;
     return d == 64 || d == 128;
 }
+
+bool score_prefill_stream_supported(int H, int d, int fp8) {
+    if (!score_tc_supported(H, d, fp8)) return false;
+    const int nkh = fp8 ? 1 : d / 64;
+    switch (H) {
+        case 16: return nkh == 2 ? PrefillCfg<2, 16, true>::kFits : PrefillCfg<1, 16, true>::kFits;
+        case 32: return nkh == 2 ? PrefillCfg<2, 32, true>::kFits : PrefillCfg<1, 32, true>::kFits;
+        default: return nkh == 2 ? PrefillCfg<2, 64, true>::kFits : PrefillCfg<1, 64, true>::kFits;
+    }
+}
+
+int score_prefill_rows_per_item(int H) { return 2 * (kTileCols / H); }
 
 cudaError_t launch_score_prefill_tc(const ScoreArgs& a, const CUtensorMap& q_map, const CUtensorMap& k_map,
                                     unsigned int* status, int sm_count, cudaStream_t stream) {

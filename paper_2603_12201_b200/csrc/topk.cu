@@ -47,7 +47,8 @@ struct alignas(16) TopkRowSmem : SampleSmem {
 template <int THREADS, int MIN_BLOCKS, int CAP>
 __global__ void __launch_bounds__(THREADS, MIN_BLOCKS)
 topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int64_t n_rows, int64_t first_len, int64_t len_step,
-                 const int32_t* __restrict__ lens, int k_top, int32_t* __restrict__ out, int map_scores) {
+                 const int32_t* __restrict__ lens, int k_top, int32_t* __restrict__ out, int map_scores,
+                 const uint8_t* __restrict__ row_mask) {
     constexpr int WARPS = THREADS / 32;
     constexpr int U = TK_UNROLL;
     __shared__ __align__(16) TopkSmem<WARPS, 2048> sm;           // 2048 bins: the keys-only path needs them
@@ -62,6 +63,7 @@ topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int64_t n_rows, i
     // longest rows first when lengths grow with the row number
     for (int64_t blk = blockIdx.x; blk < n_rows; blk += gridDim.x) {
         const int64_t row = n_rows - 1 - blk;
+        if (row_mask != nullptr && row_mask[row] == 0) continue;
         int64_t len = lens ? static_cast<int64_t>(lens[row]) : first_len + row * len_step;
         len = len < 0 ? 0 : (len > ld ? ld : len);
         const int n = static_cast<int>(len);
@@ -227,12 +229,13 @@ topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int64_t n_rows, i
 
 template <int THREADS, int MIN_BLOCKS, int CAP>
 cudaError_t launch_instance(const float* scores, int64_t ld, int64_t n_rows, int64_t first_len, int64_t len_step,
-                            const int32_t* lens, int k_top, int32_t* out, int map_bytes, cudaStream_t stream) {
+                            const int32_t* lens, int k_top, int32_t* out, int map_bytes, cudaStream_t stream,
+                            const uint8_t* row_mask) {
     auto kern = topk_rows_kernel<THREADS, MIN_BLOCKS, CAP>;
     if (cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(kern), TK_MAP_MAX_BYTES + 8 * CAP); e != cudaSuccess) return e;
     const int64_t max_grid = 1 << 20;
     const unsigned grid = static_cast<unsigned>(n_rows < max_grid ? n_rows : max_grid);
-    kern<<<grid, THREADS, map_bytes + 8 * CAP, stream>>>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, map_bytes * 4);
+    kern<<<grid, THREADS, map_bytes + 8 * CAP, stream>>>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, map_bytes * 4, row_mask);
     return cudaGetLastError();
 }
 
@@ -252,20 +255,20 @@ cudaError_t preload_topk_rows() {
 }
 
 cudaError_t launch_topk_rows(const float* scores, int64_t ld, int64_t n_rows, int64_t first_len, int64_t len_step,
-                             const int32_t* lens, int k_top, int32_t* out, cudaStream_t stream) {
+                             const int32_t* lens, int k_top, int32_t* out, cudaStream_t stream, const uint8_t* row_mask) {
     if (n_rows <= 0) return cudaSuccess;
     // the selection map covers the longest row of this launch, rounded up to a whole 128-score block
     int64_t longest = lens ? ld : first_len + (n_rows - 1) * len_step;
     if (longest > ld) longest = ld;
     if (longest < 0) longest = 0;
     if (topk_cluster_applicable(n_rows, longest))
-        return launch_topk_rows_cluster(scores, ld, n_rows, first_len, len_step, lens, k_top, out, longest, stream);
+        return launch_topk_rows_cluster(scores, ld, n_rows, first_len, len_step, lens, k_top, out, longest, stream, row_mask);
     int64_t map_bytes = (longest + 127) / 128 * 32;
     if (map_bytes > TK_MAP_MAX_BYTES) map_bytes = TK_MAP_MAX_BYTES;
     // many rows: small CTAs, many per SM; few rows: more threads per row
     if (n_rows >= 1024)
-        return launch_instance<128, 8, kCapMany>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, static_cast<int>(map_bytes), stream);
-    return launch_instance<1024, 1, kCapFew>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, static_cast<int>(map_bytes), stream);
+        return launch_instance<128, 8, kCapMany>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, static_cast<int>(map_bytes), stream, row_mask);
+    return launch_instance<1024, 1, kCapFew>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, static_cast<int>(map_bytes), stream, row_mask);
 }
 
 }  // namespace idxc

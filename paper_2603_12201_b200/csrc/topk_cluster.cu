@@ -54,7 +54,8 @@ struct ClusterRowSmem : SampleSmem {
 
 __global__ void __launch_bounds__(CL_THREADS, 2)
 topk_rows_cluster_kernel(const float* __restrict__ scores, int64_t ld, int64_t n_rows, int64_t first_len, int64_t len_step,
-                         const int32_t* __restrict__ lens, int k_top, int32_t* __restrict__ out, int map_bytes) {
+                         const int32_t* __restrict__ lens, int k_top, int32_t* __restrict__ out, int map_bytes,
+                         const uint8_t* __restrict__ row_mask) {
     cg::cluster_group cluster = cg::this_cluster();
     __shared__ __align__(16) TopkSmem<CL_WARPS, 2048> sm;      // [0, 1024): sample histogram, then the summed fine histogram;
                                                                // [1024, 2048): this CTA's fine histogram; all 2048: keys-only path
@@ -74,6 +75,7 @@ topk_rows_cluster_kernel(const float* __restrict__ scores, int64_t ld, int64_t n
 
     int par = 1;
     for (int64_t row = blockIdx.x / CL_SIZE; row < n_rows; row += n_clusters) {
+        if (row_mask != nullptr && row_mask[row] == 0) continue;      // the same for every CTA of the cluster
         par ^= 1;                                              // which copy of the exchanged counts this row uses
         int64_t len = lens ? static_cast<int64_t>(lens[row]) : first_len + row * len_step;
         len = len < 0 ? 0 : (len > ld ? ld : len);
@@ -287,7 +289,8 @@ bool topk_cluster_applicable(int64_t n_rows, int64_t longest) {
 }
 
 cudaError_t launch_topk_rows_cluster(const float* scores, int64_t ld, int64_t n_rows, int64_t first_len, int64_t len_step,
-                                     const int32_t* lens, int k_top, int32_t* out, int64_t longest, cudaStream_t stream) {
+                                     const int32_t* lens, int k_top, int32_t* out, int64_t longest, cudaStream_t stream,
+                                     const uint8_t* row_mask) {
     const int64_t part = (((longest + CL_SIZE - 1) / CL_SIZE) + 127) & ~int64_t(127);
     const int map_bytes = static_cast<int>(part / 4);
     const int dyn_bytes = map_bytes + 2 * CL_CAP * 4;
@@ -304,7 +307,7 @@ cudaError_t launch_topk_rows_cluster(const float* scores, int64_t ld, int64_t n_
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, topk_rows_cluster_kernel, scores, ld, n_rows, first_len, len_step, lens, k_top, out, map_bytes);
+    return cudaLaunchKernelEx(&cfg, topk_rows_cluster_kernel, scores, ld, n_rows, first_len, len_step, lens, k_top, out, map_bytes, row_mask);
 }
 
 }  // namespace idxc

@@ -81,6 +81,12 @@ def test_argument_validation_happens_before_any_device_work(idxc):
     # tensor-map row coordinates are 32-bit: (query, head) rows and (sequence, head) rows must stay below 2^31
     assert L.idxc_indexer_prefill(one, one, one, None, None, 0, 1 << 25, 1 << 25, 64, 128, 8, idxc.BF16, None, 0, one, one, 1 << 20, 0, None) == idxc.ERR_INVALID_ARG
     assert L.idxc_indexer_decode(one, one, 100, one, None, None, one, one, 1 << 25, 10, 64, 128, 8, idxc.BF16, None, 0, one, one, 1 << 20, 0, None) == idxc.ERR_INVALID_ARG
+    # streaming top-k: index output only, not with the CUDA-core scorer, rows no longer than its position bitmap
+    S = idxc.FLAG_STREAM_TOPK
+    assert L.idxc_indexer_prefill(one, one, one, None, None, 0, 8, 8, 64, 128, 8, idxc.BF16, one, 8, one, one, 1 << 20, S, None) == idxc.ERR_INVALID_ARG
+    assert L.idxc_indexer_prefill(one, one, one, None, None, 0, 8, 8, 64, 128, 8, idxc.BF16, None, 0, None, one, 1 << 20, S, None) == idxc.ERR_INVALID_ARG
+    assert L.idxc_indexer_prefill(one, one, one, None, None, 0, 8, 8, 64, 128, 8, idxc.BF16, None, 0, one, one, 1 << 20, S | idxc.FLAG_SIMT_SCORER, None) == idxc.ERR_INVALID_ARG
+    assert L.idxc_indexer_prefill(one, one, one, None, None, 0, 8, 1 << 19, 64, 128, 8, idxc.BF16, None, 0, one, one, 1 << 20, S, None) == idxc.ERR_UNSUPPORTED
 
 
 
@@ -115,6 +121,9 @@ def test_workspace_queries(idxc):
     big = idxc.prefill_workspace_bytes(131072, 131072, 64, 128, 2048)
     assert big <= 8 << 30 and big % (131072 * 4 * 32) == 0
     assert idxc.decode_workspace_bytes(32, 131072, 64, 128, 2048) == 32 * 131072 * 4
+    # streaming top-k: per row the full scores (rows that are computed again), 9216 candidate slots of 8 bytes, 128 list
+    # lengths, sample length, threshold, two flag bytes; plus alignment slack for seven regions
+    assert idxc.prefill_workspace_bytes(2048, 2048, 64, 128, 256, idxc.BF16, idxc.FLAG_STREAM_TOPK) == 2048 * (2048 * 4 + 9216 * 8 + 128 + 10) + 7 * 256
 
 
 def test_binding_refuses_cpu_tensors(idxc):
