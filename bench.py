@@ -604,6 +604,42 @@ def time_fp8_chunked(idxc, synth, dev, peaks, L, chunk, H, d, k_top, seed, decod
     return out
 
 
+def time_stream_topk(idxc, synth, dev, L, H, d, k_top, seed):
+    """Config 2 with the streaming top-k (IDXC_FLAG_STREAM_TOPK: the scorer's epilogue keeps per-row candidate lists instead
+    of writing the scores) next to the ordinary step, calls interleaved; the index tensors must be identical."""
+    inp = synth.prefill_inputs(L, H, d, seed=seed, device=dev, clustered=True)
+    F = idxc.FLAG_STREAM_TOPK
+    ws0 = idxc.alloc_workspace(idxc.prefill_workspace_bytes(L, L, H, d, k_top, idxc.BF16), dev)
+    ws1 = idxc.alloc_workspace(idxc.prefill_workspace_bytes(L, L, H, d, k_top, idxc.BF16, F), dev)
+    t0 = torch.empty((L, k_top), dtype=torch.int32, device=dev)
+    t1 = torch.empty((L, k_top), dtype=torch.int32, device=dev)
+    f0 = lambda: idxc.indexer_prefill(inp.q, inp.k, inp.w, k_top, topk_out=t0, workspace=ws0)
+    f1 = lambda: idxc.indexer_prefill(inp.q, inp.k, inp.w, k_top, topk_out=t1, workspace=ws1, flags=F)
+    for _ in range(2):
+        f0(); f1()
+    torch.cuda.synchronize()
+    idxc.poll_device_status()
+    ta, tb = [], []
+    for _ in range(5):
+        for f, acc in ((f0, ta), (f1, tb)):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(2):
+                f()
+            b.record()
+            torch.cuda.synchronize()
+            acc.append(a.elapsed_time(b) / 2)
+    idxc.poll_device_status()
+    pairs = L * (L + 1) / 2
+    ms0, ms1 = statistics.median(ta), statistics.median(tb)
+    return {"workload": f"cfg2 shape: L={L}, H_I={H}, d_I={d}, k_top={k_top}, bf16, clustered keys, seed {seed}",
+            "ms_ordinary": ms0, "ms_streaming": ms1, "gpairs_per_s_streaming": pairs / (ms1 * 1e-3) / 1e9,
+            "indices_identical": bool(torch.equal(t0, t1)),
+            "launches_per_call": {"ordinary": 2, "streaming": 4},
+            "note": "streaming = scorer with per-row candidate lists + list select + the two ordinary kernels restricted to flagged rows; "
+                    "the ordinary step is the default because the scorer's epilogue is the pace-setter and every per-score operation added to it costs more than the select saves"}
+
+
 def time_quantize(idxc, dev, peaks, n_tokens, H, d):
     """Per-token bf16 -> e4m3 quantiser on query-shaped rows [n_tokens, H*d] and key-shaped rows [16 * n_tokens, d]
     (both larger than L2). Algorithmic bytes: 2 read + 1 written per element + 4 per token."""
@@ -749,6 +785,7 @@ def main():
     ap.add_argument("--L", type=int, default=0, help="override the workload's sequence length (small profiling cases)")
     ap.add_argument("--only-decode", action="store_true", help="run only the decode section (profiling)")
     ap.add_argument("--only-decode-fp8", action="store_true", help="run only the batch-8 e4m3 decode step of config 5 (profiling)")
+    ap.add_argument("--only-stream-topk", action="store_true", help="run only the streaming top-k section (profiling; --L sets the length)")
     ap.add_argument("--only-sparse-attention", action="store_true", help="run only the sparse-attention section (profiling)")
     ap.add_argument("--only-layer-loop", action="store_true", help="run only the indexer + attention layer loop section")
     ap.add_argument("--only-fp8", action="store_true", help="run only the FP8 chunked-prefill section (profiling; --L sets the length)")
@@ -798,6 +835,10 @@ def main():
     if args.only_decode_fp8:
         print(json.dumps({"decode_fp8": section(time_decode_fp8, idxc, synth, dev, peaks, args.L or c5["L"], c5["H"], c5["d"], c5["k_top"],
                                                 c5["seed"], c5["decode_B"])}), flush=True)
+        return
+    if args.only_stream_topk:
+        c2 = synth.CONFIGS["cfg2"]
+        print(json.dumps({"stream_topk": section(time_stream_topk, idxc, synth, dev, args.L or c2["L"], c2["H"], c2["d"], c2["k_top"], c2["seed"])}), flush=True)
         return
     if args.only_layer_loop:
         print(json.dumps({"layer_loop": section(time_layer_loop, idxc, synth, dev, args.L or 32768, 2048, 4, 4, seed=8)}), flush=True)
@@ -999,6 +1040,8 @@ def main():
             line["topk_overlap"] = section(time_overlap, idxc, dev, peaks, 8192, c5["k_top"], 6)
             line["quantize_e4m3"] = section(time_quantize, idxc, dev, peaks, 32768, c5["H"], c5["d"])
             line["tmem_readout"] = section(time_tmem_readout, idxc, dev)
+            c2 = synth.CONFIGS["cfg2"]
+            line["stream_topk"] = section(time_stream_topk, idxc, synth, dev, c2["L"], c2["H"], c2["d"], c2["k_top"], c2["seed"])
             fp8_L, fp8_layers = (32768, 8) if args.quick else (c5["L"], c5["N"])
             line["fp8_chunked"] = section(time_fp8_chunked, idxc, synth, dev, peaks, fp8_L, c5["chunk"], c5["H"], c5["d"], c5["k_top"],
                                           c5["seed"], c5["decode_B"], fp8_layers, c5["every"], line["tmem_readout"])
@@ -1007,7 +1050,8 @@ def main():
             by_config = {
                 "cfg1": {"us_per_call": line["cfg1"]["us_per_call"], "us_back_to_back": line["cfg1"]["us_per_call_back_to_back"]},
                 "cfg2": {"gpairs_per_s": value, "ms_per_step": ms_per_step, "scorer_frac_of_bf16_peak": roofline["frac"],
-                         "topk_frac_of_hbm": roofline["topk_kernel"]["frac"]},
+                         "topk_frac_of_hbm": roofline["topk_kernel"]["frac"],
+                         "streaming_topk_ms": line["stream_topk"]["ms_streaming"], "streaming_topk_identical": line["stream_topk"]["indices_identical"]},
                 "cfg3": {"us_per_step": dc["us_per_step"], "scorer_frac_of_hbm": dc["roofline"]["frac"], "step_frac_of_hbm": dc["frac_step_vs_hbm"]},
                 "cfg4": {"workload": sc["workload"], "ms_scheduled": sc["ms_scheduled"], "ms_all_full": sc["ms_all_full"], "ratio": sc["ratio"],
                          "gpairs_per_s_full_layers": sc["gpairs_per_s_full_layers"], "checks": sc["checks"]},

@@ -11,9 +11,9 @@
 // One CTA per block of rows_per_item rows (the scorer's work item), so that the CTA can also say whether any row of
 // the block was flagged: the scorer's second run visits only flagged blocks.
 //
-// Selection: the list's keys (order-preserving 32-bit images of the scores) sit in registers; three histogram passes
-// (11 + 11 + 10 bits) find the key of the wanted rank; the chosen key indices are set in a bitmap over the row's
-// positions and read out in ascending order.
+// Selection: three histogram passes (11 + 11 + 10 bits) over the list's keys (order-preserving 32-bit images of the
+// scores) find the key of the wanted rank; the chosen key indices are set in a bitmap over the row's positions and read
+// out in ascending order.
 #include "kernels.h"
 #include "topk_common.cuh"
 
@@ -23,20 +23,8 @@ namespace {
 
 constexpr int FS_THREADS = 256;
 constexpr int FS_WARPS = FS_THREADS / 32;
-constexpr int FS_SAMPLE_PER = kStreamSampleCap / FS_THREADS;                 // sample slots per thread
-constexpr int FS_LIST_PER = kStreamLaneCap / (FS_THREADS / kStreamLanes);     // slots of a per-thread list that one thread covers
-constexpr int FS_PER = FS_SAMPLE_PER + FS_LIST_PER;                           // entries a thread may hold
 constexpr int FS_EQ_MAX = 256;                           // entries equal to the threshold key ranked by direct comparison
-static_assert(kStreamSampleCap % FS_THREADS == 0 && FS_THREADS % kStreamLanes == 0 && kStreamLaneCap % (FS_THREADS / kStreamLanes) == 0,
-              "list slots per thread");
-static_assert(FS_PER <= 64, "one bit per slot of a thread");
-// Entry e of thread tid: e < FS_SAMPLE_PER: slot tid + 256 e of the sample part; else position
-// tid / 128 + 2 (e - FS_SAMPLE_PER) of per-thread list tid % 128 (lists are filled from position 0, so a thread's
-// entries of a list end where the list does, and the whole block can stop at the longest list).
-__device__ __forceinline__ int fs_slot(int tid, int e) {
-    if (e < FS_SAMPLE_PER) return tid + FS_THREADS * e;
-    return kStreamSampleCap + (tid % kStreamLanes) * kStreamLaneCap + tid / kStreamLanes + (FS_THREADS / kStreamLanes) * (e - FS_SAMPLE_PER);
-}
+static_assert(FS_THREADS % kStreamLanes == 0, "whole threads per per-thread list");
 
 __global__ void __launch_bounds__(FS_THREADS)
 finish_topk_stream_kernel(const uint2* __restrict__ cand, const uint32_t* __restrict__ sample_count,
@@ -47,7 +35,7 @@ finish_topk_stream_kernel(const uint2* __restrict__ cand, const uint32_t* __rest
     extern __shared__ uint32_t bitmap[];                       // one bit per key position of the longest row of the launch
     __shared__ uint32_t eq_idx[FS_EQ_MAX];
     __shared__ uint32_t lane_len[kStreamLanes];
-    __shared__ uint32_t eq_count, ge_count, over_count, longest_list;
+    __shared__ uint32_t eq_count, ge_count, over_count, longest_list, key_lo, key_hi;
     const int tid = threadIdx.x;
     int slot = 0;
     for (int64_t item = blockIdx.x; item * rows_per_item < n_rows; item += gridDim.x) {
@@ -63,13 +51,11 @@ finish_topk_stream_kernel(const uint2* __restrict__ cand, const uint32_t* __rest
             const bool no_tau = t_row == -INFINITY;
             const uint32_t t_key = score_key(t_row);
             __syncthreads();                                   // the previous row's readers of the shared arrays are done
-            if (tid == 0) { eq_count = 0u; ge_count = 0u; over_count = 0u; longest_list = 0u; }
+            if (tid == 0) { eq_count = 0u; ge_count = 0u; over_count = 0u; longest_list = 0u; key_lo = 0xFFFFFFFFu; key_hi = 0u; }
             if (tid < kStreamLanes) lane_len[tid] = lane_count[row * kStreamLanes + tid];
-            zero_hist<FS_THREADS>(sm, 2048);
             __syncthreads();
-            // ---- the list's keys into registers; entries >= tau counted; first histogram
-            uint32_t key[FS_PER];
-            uint64_t have = 0;                                 // bit e: entry e of this thread exists
+            // ---- first pass over the list: entries >= tau counted; first histogram. The list is read again in every
+            // pass (it is in L2, most of it in L1): holding its keys in registers would leave two CTAs per SM
             uint32_t c_ge = 0;
             const uint2* lst = cand + row * static_cast<int64_t>(kStreamRowSlots);
             if (tid < kStreamLanes) {
@@ -77,70 +63,86 @@ finish_topk_stream_kernel(const uint2* __restrict__ cand, const uint32_t* __rest
                 atomicMax(&longest_list, lane_len[tid] < static_cast<uint32_t>(kStreamLaneCap) ? lane_len[tid] : static_cast<uint32_t>(kStreamLaneCap));
             }
             __syncthreads();
-            const uint32_t my_len = lane_len[tid % kStreamLanes];
-            const int n_list_iter = static_cast<int>((longest_list + (FS_THREADS / kStreamLanes) - 1) / (FS_THREADS / kStreamLanes));
-#pragma unroll
-            for (int e = 0; e < FS_PER; ++e) {
-                key[e] = 0u;
-                if (e >= FS_SAMPLE_PER && e - FS_SAMPLE_PER >= n_list_iter) continue;                  // (the same for every thread)
-                const bool there = e < FS_SAMPLE_PER ? static_cast<uint32_t>(tid + FS_THREADS * e) < n_sample
-                                                     : static_cast<uint32_t>(tid / kStreamLanes + (FS_THREADS / kStreamLanes) * (e - FS_SAMPLE_PER)) < my_len;
-                if (there) {
-                    have |= 1ull << e;
-                    key[e] = score_key(__uint_as_float(__ldg(&lst[fs_slot(tid, e)].x)));
-                    c_ge += no_tau || key[e] >= t_key;
-                    atomicAdd(&sm.hist[key[e] >> 21], 1u);
+            // f(slot, key) for every entry of the list: the sample part thread by thread; the 128 per-thread lists one
+            // list per warp at a time, a lane per position (a list is a contiguous run of slots: one 256-byte load covers
+            // 32 of them; a thread per list would touch 32 lines with every load)
+            constexpr int kListsPerWarp = kStreamLanes / FS_WARPS;
+            const int lane = tid & 31, wid = tid >> 5;
+            auto for_each_entry = [&](auto f) {
+                for (uint32_t i = tid; i < n_sample; i += FS_THREADS)
+                    f(static_cast<int>(i), score_key(__uint_as_float(__ldg(&lst[i].x))));
+#pragma unroll 4
+                for (int j = 0; j < kListsPerWarp; ++j) {
+                    const int list = wid * kListsPerWarp + j;
+                    const uint32_t len = lane_len[list] < static_cast<uint32_t>(kStreamLaneCap) ? lane_len[list] : static_cast<uint32_t>(kStreamLaneCap);
+                    const int base = kStreamSampleCap + list * kStreamLaneCap;
+                    for (uint32_t pos = lane; pos < len; pos += 32)
+                        f(base + static_cast<int>(pos), score_key(__uint_as_float(__ldg(&lst[base + pos].x))));
                 }
-            }
+            };
+            // smallest and largest key, entries >= tau
+            uint32_t k_lo = 0xFFFFFFFFu, k_hi = 0u;
+            if (n_sample <= static_cast<uint32_t>(kStreamSampleCap))
+                for_each_entry([&](int, uint32_t key) {
+                    c_ge += no_tau || key >= t_key;
+                    k_lo = key < k_lo ? key : k_lo;
+                    k_hi = key > k_hi ? key : k_hi;
+                });
             c_ge = __reduce_add_sync(0xFFFFFFFFu, c_ge);
-            if ((tid & 31) == 0 && c_ge != 0u) atomicAdd(&ge_count, c_ge);
+            k_lo = __reduce_min_sync(0xFFFFFFFFu, k_lo);
+            k_hi = __reduce_max_sync(0xFFFFFFFFu, k_hi);
+            if ((tid & 31) == 0) {
+                if (c_ge != 0u) atomicAdd(&ge_count, c_ge);
+                atomicMin(&key_lo, k_lo);
+                atomicMax(&key_hi, k_hi);
+            }
             __syncthreads();
-            // flagged: overflow, fewer than kk entries reach tau, or an index that cannot be a key of this row (the
-            // same for every thread)
+            // flagged: overflow, or fewer than kk entries reach tau (the same for every thread)
             if (over_count != 0u || n_sample > static_cast<uint32_t>(kStreamSampleCap) || ge_count < kk) {
                 if (tid == 0) row_fail[row] = 1;
                 any_fail = true;
                 continue;
             }
-            // ---- the key of rank kk: 11 + 11 + 10 bits
-            uint32_t need = kk, b1, b2, b3, above;
-            select_bucket<2048, FS_THREADS>(sm, need, slot, b1, above);
-            need -= above;
-            zero_hist<FS_THREADS>(sm, 2048);
-            __syncthreads();
-#pragma unroll
-            for (int e = 0; e < FS_PER; ++e)
-                if (((have >> e) & 1ull) && (key[e] >> 21) == b1) atomicAdd(&sm.hist[(key[e] >> 10) & 2047u], 1u);
-            __syncthreads();
-            select_bucket<2048, FS_THREADS>(sm, need, slot, b2, above);
-            need -= above;
-            zero_hist<FS_THREADS>(sm, 1024);
-            __syncthreads();
-            const uint32_t p2 = (b1 << 11) | b2;
-#pragma unroll
-            for (int e = 0; e < FS_PER; ++e)
-                if (((have >> e) & 1ull) && (key[e] >> 10) == p2) atomicAdd(&sm.hist[key[e] & 1023u], 1u);
-            __syncthreads();
-            select_bucket<1024, FS_THREADS>(sm, need, slot, b3, above);
-            need -= above;                                     // entries to take among those equal to the threshold key, >= 1
-            const uint32_t T = (p2 << 10) | b3;
+            // ---- the key of rank kk. The keys of a list are close together (scores at or above one threshold), so the
+            // top bits of the key would put them all into a few bins; the bins are laid over [smallest, largest] instead,
+            // 2048 at a time, and narrowed to the bin that holds the rank until a bin is one key wide
+            uint32_t need = kk;
+            uint32_t base = key_lo;                            // the window of keys still in play starts here ...
+            uint32_t window_bits = 32u - static_cast<uint32_t>(__clz(key_hi - key_lo));   // ... and is < 2^window_bits wide (0: one key)
+            for (;;) {
+                const uint32_t shift = window_bits > 11u ? window_bits - 11u : 0u;
+                const uint32_t window_last = window_bits >= 32u ? 0xFFFFFFFFu : (1u << window_bits) - 1u;   // largest key - base in the window
+                __syncthreads();
+                zero_hist<FS_THREADS>(sm, 2048);
+                __syncthreads();
+                for_each_entry([&](int, uint32_t key) {
+                    if (key >= base && key - base <= window_last) atomicAdd(&sm.hist[(key - base) >> shift], 1u);
+                });
+                __syncthreads();
+                uint32_t bin, above;
+                select_bucket<2048, FS_THREADS>(sm, need, slot, bin, above);
+                need -= above;
+                base += bin << shift;
+                if (shift == 0u) break;
+                window_bits = shift;
+            }
+            const uint32_t T = base;                           // need = entries to take among those equal to T, >= 1
             // ---- bitmap of the chosen positions
             const int n_words = (n + 31) >> 5;
             for (int w = tid; w < n_words; w += FS_THREADS) bitmap[w] = 0u;
             __syncthreads();
             bool bad_index = false;
-#pragma unroll
-            for (int e = 0; e < FS_PER; ++e) {
-                if (!((have >> e) & 1ull) || key[e] < T) continue;
-                const uint32_t idx = __ldg(&lst[fs_slot(tid, e)].y);
-                if (idx >= static_cast<uint32_t>(n)) { bad_index = true; continue; }      // cannot happen with a list the scorer wrote
-                if (key[e] > T) {
+            for_each_entry([&](int slot_i, uint32_t key) {
+                if (key < T) return;
+                const uint32_t idx = __ldg(&lst[slot_i].y);
+                if (idx >= static_cast<uint32_t>(n)) { bad_index = true; return; }      // cannot happen with a list the scorer wrote
+                if (key > T) {
                     atomicOr(&bitmap[idx >> 5], 1u << (idx & 31u));
                 } else {
                     const uint32_t pos = atomicAdd(&eq_count, 1u);
                     if (pos < static_cast<uint32_t>(FS_EQ_MAX)) eq_idx[pos] = idx;
                 }
-            }
+            });
             const bool any_bad = __syncthreads_or(bad_index);
             const uint32_t n_eq = eq_count;
             if (any_bad || n_eq > static_cast<uint32_t>(FS_EQ_MAX)) {          // many equal scores at the threshold: the ordinary path
