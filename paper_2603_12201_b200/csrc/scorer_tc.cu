@@ -398,16 +398,20 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
                             if (r == j) mine = v;                      // thread j of the group stores key g + 8j
                         }
                         const int r_item = half * QPA + colhalf * QPW + i;
-                        const int64_t row = row_base + r_item;
+                        const int64_t row = row_base + half * QPA + colhalf * QPW + i;
                         const int64_t t = p.q_begin + row;
-                        if constexpr (FP8) mine *= ksc;
                         if constexpr (!STREAM) {
-                            if (row < p.n_rows && s <= t) p.scores[row * p.ld + s] = mine;
+                            if (row < p.n_rows && s <= t) {
+                                if constexpr (FP8) mine *= ksc;
+                                p.scores[row * p.ld + s] = mine;
+                            }
                         } else if (jt < ord.ns) {
+                            if constexpr (FP8) mine *= ksc;
                             // a sample tile: every score goes to the row's sample (which of them are real is worked out
                             // from their place when the sample is read)
                             sample[r_item * Cfg::kSampleMax + jt * kTileKeys + key_written] = mine;
                         } else {
+                            if constexpr (FP8) mine *= ksc;
                             // past the sample: only scores that are not below the row's threshold (a NaN stays in)
                             if (row < p.n_rows && s <= t && !(mine < row_tau[r_item])) {
                                 const uint32_t pos = my_count[half * QPW + i]++;
