@@ -11,9 +11,10 @@
 // One CTA per block of rows_per_item rows (the scorer's work item), so that the CTA can also say whether any row of
 // the block was flagged: the scorer's second run visits only flagged blocks.
 //
-// Selection: three histogram passes (11 + 11 + 10 bits) over the list's keys (order-preserving 32-bit images of the
-// scores) find the key of the wanted rank; the chosen key indices are set in a bitmap over the row's positions and read
-// out in ascending order.
+// Selection: the list (a sample part and 128 short per-thread lists) is read from global memory once and its keys
+// (order-preserving 32-bit images of the scores) packed into shared memory; histogram passes over the packed keys, with
+// 2048 bins laid over [smallest, largest] and narrowed to the bin of the wanted rank, find that rank's key; the chosen
+// key indices are set in a bitmap over the row's positions and read out in ascending order.
 #include "kernels.h"
 #include "topk_common.cuh"
 
@@ -26,17 +27,23 @@ constexpr int FS_WARPS = FS_THREADS / 32;
 constexpr int FS_EQ_MAX = 256;                           // entries equal to the threshold key ranked by direct comparison
 static_assert(FS_THREADS % kStreamLanes == 0, "whole threads per per-thread list");
 
+constexpr int FS_DENSE_MAX = 6144;                        // list entries the shared-memory copy holds; longer lists are flagged
+
 __global__ void __launch_bounds__(FS_THREADS)
 finish_topk_stream_kernel(const uint2* __restrict__ cand, const uint32_t* __restrict__ sample_count,
                           const uint8_t* __restrict__ lane_count, const float* __restrict__ tau,
                           int64_t n_rows, int64_t q_begin, int rows_per_item, int k_top, int32_t* __restrict__ out,
                           uint8_t* __restrict__ row_fail, uint8_t* __restrict__ item_fail) {
     __shared__ __align__(16) TopkSmem<FS_WARPS, 2048> sm;
-    extern __shared__ uint32_t bitmap[];                       // one bit per key position of the longest row of the launch
+    __shared__ uint32_t dense_key[FS_DENSE_MAX];               // the list's keys, packed
+    __shared__ uint16_t dense_slot[FS_DENSE_MAX];              // ... and the slot of the row's list each came from
     __shared__ uint32_t eq_idx[FS_EQ_MAX];
-    __shared__ uint32_t lane_len[kStreamLanes];
-    __shared__ uint32_t eq_count, ge_count, over_count, longest_list, key_lo, key_hi;
+    __shared__ uint32_t list_off[kStreamLanes + 1];            // where per-thread list j starts in the packed copy
+    __shared__ uint32_t eq_count, ge_count, over_count, key_lo, key_hi;
+    extern __shared__ uint32_t bitmap[];                       // one bit per key position of the longest row of the launch
     const int tid = threadIdx.x;
+    const int lane = tid & 31, wid = tid >> 5;
+    constexpr int kListsPerWarp = kStreamLanes / FS_WARPS;
     int slot = 0;
     for (int64_t item = blockIdx.x; item * rows_per_item < n_rows; item += gridDim.x) {
         bool any_fail = false;
@@ -50,55 +57,57 @@ finish_topk_stream_kernel(const uint2* __restrict__ cand, const uint32_t* __rest
             const float t_row = tau[row];
             const bool no_tau = t_row == -INFINITY;
             const uint32_t t_key = score_key(t_row);
-            __syncthreads();                                   // the previous row's readers of the shared arrays are done
-            if (tid == 0) { eq_count = 0u; ge_count = 0u; over_count = 0u; longest_list = 0u; key_lo = 0xFFFFFFFFu; key_hi = 0u; }
-            if (tid < kStreamLanes) lane_len[tid] = lane_count[row * kStreamLanes + tid];
-            __syncthreads();
-            // ---- first pass over the list: entries >= tau counted; first histogram. The list is read again in every
-            // pass (it is in L2, most of it in L1): holding its keys in registers would leave two CTAs per SM
-            uint32_t c_ge = 0;
             const uint2* lst = cand + row * static_cast<int64_t>(kStreamRowSlots);
+            __syncthreads();                                   // the previous row's readers of the shared arrays are done
+            if (tid == 0) { eq_count = 0u; ge_count = 0u; over_count = 0u; key_lo = 0xFFFFFFFFu; key_hi = 0u; }
+            // ---- where every per-thread list goes in the packed copy: a prefix sum over the 128 list lengths
+            uint32_t my_len = 0;
             if (tid < kStreamLanes) {
-                if (lane_len[tid] > static_cast<uint32_t>(kStreamLaneCap)) atomicAdd(&over_count, 1u);
-                atomicMax(&longest_list, lane_len[tid] < static_cast<uint32_t>(kStreamLaneCap) ? lane_len[tid] : static_cast<uint32_t>(kStreamLaneCap));
+                my_len = lane_count[row * kStreamLanes + tid];
+                if (my_len > static_cast<uint32_t>(kStreamLaneCap)) { atomicAdd(&over_count, 1u); my_len = kStreamLaneCap; }
             }
+            uint32_t m;                                        // entries of the list
+            const uint32_t off = block_excl_scan<FS_WARPS>(my_len, sm, slot, m) + n_sample;
+            if (tid < kStreamLanes) list_off[tid] = off;
+            m += n_sample;
+            if (tid == 0) list_off[kStreamLanes] = m;
             __syncthreads();
-            // f(slot, key) for every entry of the list: the sample part thread by thread; the 128 per-thread lists one
-            // list per warp at a time, a lane per position (a list is a contiguous run of slots: one 256-byte load covers
-            // 32 of them; a thread per list would touch 32 lines with every load)
-            constexpr int kListsPerWarp = kStreamLanes / FS_WARPS;
-            const int lane = tid & 31, wid = tid >> 5;
-            auto for_each_entry = [&](auto f) {
-                for (uint32_t i = tid; i < n_sample; i += FS_THREADS)
-                    f(static_cast<int>(i), score_key(__uint_as_float(__ldg(&lst[i].x))));
-#pragma unroll 4
-                for (int j = 0; j < kListsPerWarp; ++j) {
-                    const int list = wid * kListsPerWarp + j;
-                    const uint32_t len = lane_len[list] < static_cast<uint32_t>(kStreamLaneCap) ? lane_len[list] : static_cast<uint32_t>(kStreamLaneCap);
-                    const int base = kStreamSampleCap + list * kStreamLaneCap;
-                    for (uint32_t pos = lane; pos < len; pos += 32)
-                        f(base + static_cast<int>(pos), score_key(__uint_as_float(__ldg(&lst[base + pos].x))));
-                }
+            // flagged: a list overflowed or is longer than the packed copy (the same for every thread)
+            if (over_count != 0u || n_sample > static_cast<uint32_t>(kStreamSampleCap) || m > static_cast<uint32_t>(FS_DENSE_MAX) || m < kk) {
+                if (tid == 0) row_fail[row] = 1;
+                any_fail = true;
+                continue;
+            }
+            // ---- one pass over global memory: keys into the packed copy (the sample part thread by thread; the per-thread
+            // lists a warp per list, a lane per position: a list is a contiguous run of slots), smallest and largest key,
+            // entries >= tau
+            uint32_t c_ge = 0, k_lo = 0xFFFFFFFFu, k_hi = 0u;
+            auto take = [&](uint32_t dst, int slot_i) {
+                const uint32_t key = score_key(__uint_as_float(__ldg(&lst[slot_i].x)));
+                dense_key[dst] = key;
+                dense_slot[dst] = static_cast<uint16_t>(slot_i);
+                c_ge += no_tau || key >= t_key;
+                k_lo = key < k_lo ? key : k_lo;
+                k_hi = key > k_hi ? key : k_hi;
             };
-            // smallest and largest key, entries >= tau
-            uint32_t k_lo = 0xFFFFFFFFu, k_hi = 0u;
-            if (n_sample <= static_cast<uint32_t>(kStreamSampleCap))
-                for_each_entry([&](int, uint32_t key) {
-                    c_ge += no_tau || key >= t_key;
-                    k_lo = key < k_lo ? key : k_lo;
-                    k_hi = key > k_hi ? key : k_hi;
-                });
+            for (uint32_t i = tid; i < n_sample; i += FS_THREADS) take(i, static_cast<int>(i));
+#pragma unroll 4
+            for (int j = 0; j < kListsPerWarp; ++j) {
+                const int list = wid * kListsPerWarp + j;
+                const uint32_t o = list_off[list], len = list_off[list + 1] - o;
+                for (uint32_t pos = lane; pos < len; pos += 32) take(o + pos, kStreamSampleCap + list * kStreamLaneCap + static_cast<int>(pos));
+            }
             c_ge = __reduce_add_sync(0xFFFFFFFFu, c_ge);
             k_lo = __reduce_min_sync(0xFFFFFFFFu, k_lo);
             k_hi = __reduce_max_sync(0xFFFFFFFFu, k_hi);
-            if ((tid & 31) == 0) {
+            if (lane == 0) {
                 if (c_ge != 0u) atomicAdd(&ge_count, c_ge);
                 atomicMin(&key_lo, k_lo);
                 atomicMax(&key_hi, k_hi);
             }
             __syncthreads();
-            // flagged: overflow, or fewer than kk entries reach tau (the same for every thread)
-            if (over_count != 0u || n_sample > static_cast<uint32_t>(kStreamSampleCap) || ge_count < kk) {
+            // flagged: fewer than kk entries reach tau (some score that was dropped could belong to the answer)
+            if (ge_count < kk) {
                 if (tid == 0) row_fail[row] = 1;
                 any_fail = true;
                 continue;
@@ -112,12 +121,12 @@ finish_topk_stream_kernel(const uint2* __restrict__ cand, const uint32_t* __rest
             for (;;) {
                 const uint32_t shift = window_bits > 11u ? window_bits - 11u : 0u;
                 const uint32_t window_last = window_bits >= 32u ? 0xFFFFFFFFu : (1u << window_bits) - 1u;   // largest key - base in the window
-                __syncthreads();
                 zero_hist<FS_THREADS>(sm, 2048);
                 __syncthreads();
-                for_each_entry([&](int, uint32_t key) {
+                for (uint32_t i = tid; i < m; i += FS_THREADS) {
+                    const uint32_t key = dense_key[i];
                     if (key >= base && key - base <= window_last) atomicAdd(&sm.hist[(key - base) >> shift], 1u);
-                });
+                }
                 __syncthreads();
                 uint32_t bin, above;
                 select_bucket<2048, FS_THREADS>(sm, need, slot, bin, above);
@@ -132,17 +141,18 @@ finish_topk_stream_kernel(const uint2* __restrict__ cand, const uint32_t* __rest
             for (int w = tid; w < n_words; w += FS_THREADS) bitmap[w] = 0u;
             __syncthreads();
             bool bad_index = false;
-            for_each_entry([&](int slot_i, uint32_t key) {
-                if (key < T) return;
-                const uint32_t idx = __ldg(&lst[slot_i].y);
-                if (idx >= static_cast<uint32_t>(n)) { bad_index = true; return; }      // cannot happen with a list the scorer wrote
+            for (uint32_t i = tid; i < m; i += FS_THREADS) {
+                const uint32_t key = dense_key[i];
+                if (key < T) continue;
+                const uint32_t idx = __ldg(&lst[dense_slot[i]].y);
+                if (idx >= static_cast<uint32_t>(n)) { bad_index = true; continue; }      // cannot happen with a list the scorer wrote
                 if (key > T) {
                     atomicOr(&bitmap[idx >> 5], 1u << (idx & 31u));
                 } else {
                     const uint32_t pos = atomicAdd(&eq_count, 1u);
                     if (pos < static_cast<uint32_t>(FS_EQ_MAX)) eq_idx[pos] = idx;
                 }
-            });
+            }
             const bool any_bad = __syncthreads_or(bad_index);
             const uint32_t n_eq = eq_count;
             if (any_bad || n_eq > static_cast<uint32_t>(FS_EQ_MAX)) {          // many equal scores at the threshold: the ordinary path
@@ -166,10 +176,10 @@ finish_topk_stream_kernel(const uint2* __restrict__ cand, const uint32_t* __rest
             uint32_t total;
             uint32_t pos = block_excl_scan<FS_WARPS>(c, sm, slot, total);
             for (int w = w0; w < w1; ++w) {
-                uint32_t b = bitmap[w];
-                while (b) {
-                    const int bit = __ffs(b) - 1;
-                    b &= b - 1;
+                uint32_t bw = bitmap[w];
+                while (bw) {
+                    const int bit = __ffs(bw) - 1;
+                    bw &= bw - 1;
                     if (pos < kk) out_row[pos] = 32 * w + bit;
                     ++pos;
                 }
@@ -192,6 +202,7 @@ cudaError_t launch_finish_topk_stream(const StreamTopk& st, int64_t n_rows, int6
     const int64_t longest = q_begin + n_rows;                  // keys of the last row
     if (longest > kStreamMaxKeys) return cudaErrorInvalidValue;
     const int map_bytes = static_cast<int>((longest + 31) / 32 * 4);
+    if (cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(finish_topk_stream_kernel), kStreamMaxKeys / 8); e != cudaSuccess) return e;
     finish_topk_stream_kernel<<<grid, FS_THREADS, map_bytes, stream>>>(st.cand, st.sample_count, st.lane_count, st.tau, n_rows, q_begin,
                                                                        rows_per_item, st.k_top, out, row_fail, item_fail);
     return cudaGetLastError();
