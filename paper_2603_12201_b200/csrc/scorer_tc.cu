@@ -388,14 +388,25 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
 #pragma unroll
                     for (int i = 0; i < QPW; ++i) {
                         float mine = 0.f;
+                        {
+                            // The four threads of a group each hold partial sums of the group's four keys; thread j wants
+                            // the whole sum of key j. A butterfly does it in three shuffles: with the neighbour (xor 1) a
+                            // thread keeps the two keys of its own parity and gives away the other two, with the thread
+                            // two further (xor 2) it keeps its own key. The sum is ((own + xor 1) + (xor 2 + xor 3)).
+                            float v[4];
 #pragma unroll
-                        for (int r = 0; r < 4; ++r) {
-                            float v, v_odd;
-                            unpack_f32x2(acc[r][i], v, v_odd);
-                            v += v_odd;
-                            v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
-                            v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
-                            if (r == j) mine = v;                      // thread j of the group stores key g + 8j
+                            for (int r = 0; r < 4; ++r) {
+                                float lo, hi;
+                                unpack_f32x2(acc[r][i], lo, hi);
+                                v[r] = lo + hi;
+                            }
+                            const bool odd = (j & 1) != 0, upper = (j & 2) != 0;
+                            float keep0 = odd ? v[1] : v[0], give0 = odd ? v[0] : v[1];
+                            float keep1 = odd ? v[3] : v[2], give1 = odd ? v[2] : v[3];
+                            keep0 += __shfl_xor_sync(0xFFFFFFFFu, give0, 1);
+                            keep1 += __shfl_xor_sync(0xFFFFFFFFu, give1, 1);
+                            const float keep = upper ? keep1 : keep0, give = upper ? keep0 : keep1;
+                            mine = keep + __shfl_xor_sync(0xFFFFFFFFu, give, 2);
                         }
                         const int r_item = half * QPA + colhalf * QPW + i;
                         const int64_t row = row_base + half * QPA + colhalf * QPW + i;
