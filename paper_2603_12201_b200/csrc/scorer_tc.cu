@@ -5,7 +5,7 @@
 // out with KEYS ON THE MMA's M axis (TMEM lanes) and (query, head) ON N (TMEM columns):
 // an epilogue thread then owns a few keys and a quarter of the (query, head) columns, so
 // the gate and the w-weighted head sum are register arithmetic with w held in registers,
-// finished by a two-step shuffle across the four threads that share a key.
+// finished by a butterfly of three shuffles across the four threads that share a group of four keys.
 //
 // Prefill kernel (persistent, one CTA per SM, warp-specialised):
 //   warp 0      TMA producer: a block of 2*256/H queries (two 256-column B tiles) is loaded
@@ -13,8 +13,8 @@
 //               through a ring of stages. Per-CTA loads only.
 //   warp 1      MMA issuer: per key tile, one 128 x 256 x d UMMA chain into each of the two
 //               256-column TMEM accumulators, so accumulator A is drained while B is filled.
-//   warps 2-9   epilogue: tcgen05.ld (16x256b), ReLU, FMA with w held in registers, two shuffles per
-//               score to join the four threads of a key, causal predicate, coalesced score store.
+//   warps 2-9   epilogue: tcgen05.ld (16x256b), ReLU, FMA with w held in registers, three shuffles per four
+//               scores to join the four threads of a key group, causal predicate, coalesced score store.
 // Causal structure: a work item only visits key tiles up to its last query's position;
 // items are handed out longest first in a boustrophedon order over the CTAs.
 //
@@ -282,7 +282,7 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
         // its warp's lane quarter, g = lane/4) and the columns 8i + 2j + {0,1} (j = lane%4) of every
         // 8-column group. Its share of w (64 values per work item) therefore lives in registers and
         // the gate/FMA loop issues no shared-memory loads; the four threads of a group add their
-        // partial head sums with two shuffles per score at the end.
+        // partial head sums with three shuffles per four scores at the end.
         constexpr int QPW = kColsPerEpiWarp / H;     // queries per warp per accumulator
         static_assert(QPW >= 1, "an epilogue warp must cover at least one query");
         const int ew = warp - kEpilogueWarp0;
