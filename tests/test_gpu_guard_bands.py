@@ -109,6 +109,28 @@ def test_prefill_outputs_and_workspace(L, H, d, k_top, fp8):
         assert torch.equal(part.t, ref_topk[q0:q1])
 
 
+@pytest.mark.parametrize("L,H,d,k_top,fp8,rows_ws", [(2049, 64, 128, 300, False, 0), (1300, 64, 128, 2048, True, 64), (777, 32, 64, 64, False, 0),
+                                                      (515, 16, 128, 40, True, 32)])
+def test_streaming_topk_outputs_and_workspace(L, H, d, k_top, fp8, rows_ws):
+    """The streaming top-k writes per-row candidate lists, list lengths, thresholds and flag bytes into regions of the
+    workspace: nothing of it may land outside the workspace or the index output, whole or in chunks of rows_ws rows."""
+    inp = _dev(synth.prefill_inputs(L, H, d, seed=2000 + L, fp8=fp8))
+    dt = idxc.FP8_E4M3 if fp8 else idxc.BF16
+    F = idxc.FLAG_STREAM_TOPK
+    topk = Guarded((L, k_top), torch.int32, fill=-7)
+    ws = Guarded((idxc.prefill_workspace_bytes(rows_ws or L, L, H, d, k_top, dt, F),), torch.uint8)
+
+    def run():
+        idxc.indexer_prefill(inp.q, inp.k, inp.w, k_top, inp.q_scale, inp.k_scale, topk_out=topk.t, workspace=ws.t, flags=F)
+    _twice(run, [topk], "streaming prefill")
+    ws.check("streaming prefill workspace")
+    # and it is the ordinary path's answer
+    ref = torch.empty((L, k_top), dtype=torch.int32, device=DEV)
+    idxc.indexer_prefill(inp.q, inp.k, inp.w, k_top, inp.q_scale, inp.k_scale, topk_out=ref,
+                         workspace=idxc.alloc_workspace(idxc.prefill_workspace_bytes(L, L, H, d, k_top, dt), DEV))
+    assert torch.equal(ref, topk.t)
+
+
 @pytest.mark.parametrize("H,d,k_top,fp8,lens", [(64, 128, 64, False, [1, 127, 129, 2049]), (16, 64, 16, False, [300, 5, 4097]),
                                                  (64, 128, 2048, True, [2047, 2049, 9000]), (32, 128, 100, True, [515])])
 def test_decode_outputs_workspace_and_builtin_scratch(H, d, k_top, fp8, lens):
