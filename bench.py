@@ -608,17 +608,24 @@ def time_fp8_chunked(idxc, synth, dev, peaks, L, chunk, H, d, k_top, seed, decod
     return out
 
 
-def time_stream_topk(idxc, synth, dev, L, H, d, k_top, seed):
+def time_stream_topk(idxc, synth, dev, L, H, d, k_top, seed, fp8=False, q_begin=0, q_len=0):
     """Config 2 with the streaming top-k (IDXC_FLAG_STREAM_TOPK: the scorer's epilogue keeps per-row candidate lists instead
-    of writing the scores) next to the ordinary step, calls interleaved; the index tensors must be identical."""
-    inp = synth.prefill_inputs(L, H, d, seed=seed, device=dev, clustered=True)
+    of writing the scores) next to the ordinary step, calls interleaved; the index tensors must be identical.
+    fp8 / q_begin / q_len: the same comparison on one query chunk [q_begin, q_begin + q_len) of an e4m3 prefill (config 5's
+    shape: long rows)."""
+    inp = synth.prefill_inputs(L, H, d, seed=seed, device=dev, clustered=not fp8, fp8=fp8)
     F = idxc.FLAG_STREAM_TOPK
-    ws0 = idxc.alloc_workspace(idxc.prefill_workspace_bytes(L, L, H, d, k_top, idxc.BF16), dev)
-    ws1 = idxc.alloc_workspace(idxc.prefill_workspace_bytes(L, L, H, d, k_top, idxc.BF16, F), dev)
-    t0 = torch.empty((L, k_top), dtype=torch.int32, device=dev)
-    t1 = torch.empty((L, k_top), dtype=torch.int32, device=dev)
-    f0 = lambda: idxc.indexer_prefill(inp.q, inp.k, inp.w, k_top, topk_out=t0, workspace=ws0)
-    f1 = lambda: idxc.indexer_prefill(inp.q, inp.k, inp.w, k_top, topk_out=t1, workspace=ws1, flags=F)
+    dt = idxc.FP8_E4M3 if fp8 else idxc.BF16
+    q_len = q_len or L - q_begin
+    sl = slice(q_begin, q_begin + q_len)
+    q, w = inp.q[sl], inp.w[sl]
+    qs = inp.q_scale[sl] if fp8 else None
+    ws0 = idxc.alloc_workspace(idxc.prefill_workspace_bytes(q_len, L, H, d, k_top, dt), dev)
+    ws1 = idxc.alloc_workspace(idxc.prefill_workspace_bytes(q_len, L, H, d, k_top, dt, F), dev)
+    t0 = torch.empty((q_len, k_top), dtype=torch.int32, device=dev)
+    t1 = torch.empty((q_len, k_top), dtype=torch.int32, device=dev)
+    f0 = lambda: idxc.indexer_prefill(q, inp.k, w, k_top, qs, inp.k_scale, q_begin=q_begin, topk_out=t0, workspace=ws0)
+    f1 = lambda: idxc.indexer_prefill(q, inp.k, w, k_top, qs, inp.k_scale, q_begin=q_begin, topk_out=t1, workspace=ws1, flags=F)
     for _ in range(2):
         f0(); f1()
     torch.cuda.synchronize()
@@ -634,9 +641,9 @@ def time_stream_topk(idxc, synth, dev, L, H, d, k_top, seed):
             torch.cuda.synchronize()
             acc.append(a.elapsed_time(b) / 2)
     idxc.poll_device_status()
-    pairs = L * (L + 1) / 2
+    pairs = sum(range(q_begin + 1, q_begin + q_len + 1))
     ms0, ms1 = statistics.median(ta), statistics.median(tb)
-    return {"workload": f"cfg2 shape: L={L}, H_I={H}, d_I={d}, k_top={k_top}, bf16, clustered keys, seed {seed}",
+    return {"workload": f"L={L}, rows {q_begin}..{q_begin + q_len - 1}, H_I={H}, d_I={d}, k_top={k_top}, {'e4m3' if fp8 else 'bf16, clustered keys'}, seed {seed}",
             "ms_ordinary": ms0, "ms_streaming": ms1, "gpairs_per_s_streaming": pairs / (ms1 * 1e-3) / 1e9,
             "indices_identical": bool(torch.equal(t0, t1)),
             "launches_per_call": {"ordinary": 2, "streaming": 4},
@@ -790,6 +797,7 @@ def main():
     ap.add_argument("--only-decode", action="store_true", help="run only the decode section (profiling)")
     ap.add_argument("--only-decode-fp8", action="store_true", help="run only the batch-8 e4m3 decode step of config 5 (profiling)")
     ap.add_argument("--only-stream-topk", action="store_true", help="run only the streaming top-k section (profiling; --L sets the length)")
+    ap.add_argument("--stream-fp8-chunk", type=int, default=-1, help="with --only-stream-topk: compare on the config-5 query chunk that starts at this row (e4m3, L = 131072 unless --L is given)")
     ap.add_argument("--only-sparse-attention", action="store_true", help="run only the sparse-attention section (profiling)")
     ap.add_argument("--only-layer-loop", action="store_true", help="run only the indexer + attention layer loop section")
     ap.add_argument("--only-fp8", action="store_true", help="run only the FP8 chunked-prefill section (profiling; --L sets the length)")
@@ -842,7 +850,11 @@ def main():
         return
     if args.only_stream_topk:
         c2 = synth.CONFIGS["cfg2"]
-        print(json.dumps({"stream_topk": section(time_stream_topk, idxc, synth, dev, args.L or c2["L"], c2["H"], c2["d"], c2["k_top"], c2["seed"])}), flush=True)
+        if args.stream_fp8_chunk >= 0:
+            print(json.dumps({"stream_topk": section(time_stream_topk, idxc, synth, dev, args.L or c5["L"], c5["H"], c5["d"], c5["k_top"], c5["seed"],
+                                                     fp8=True, q_begin=args.stream_fp8_chunk, q_len=c5["chunk"])}), flush=True)
+        else:
+            print(json.dumps({"stream_topk": section(time_stream_topk, idxc, synth, dev, args.L or c2["L"], c2["H"], c2["d"], c2["k_top"], c2["seed"])}), flush=True)
         return
     if args.only_layer_loop:
         print(json.dumps({"layer_loop": section(time_layer_loop, idxc, synth, dev, args.L or 32768, 2048, 4, 4, seed=8)}), flush=True)
