@@ -95,6 +95,10 @@ def test_stream_topk_rows_the_lists_cannot_answer_take_the_ordinary_path():
         kk = min(k_top, t + 1)
         assert np.array_equal(t_str[t, :kk], np.arange(kk)), f"row {t}"
         assert np.all(t_str[t, kk:] == -1)
+    # the same through a workspace of 96 rows: the flags of a chunk's rows and work items are the chunk's own
+    small = idxc.alloc_workspace(idxc.prefill_workspace_bytes(96, L, H, d, k_top, idxc.BF16, idxc.FLAG_STREAM_TOPK), DEV)
+    t_small, _ = _run(inp, k_top, stream=True, workspace=small)
+    assert np.array_equal(t_small, t_str)
     # scores that grow with the position: q = k = e_0 scaled by the position, one head with weight 1
     L = 6000
     inp = _to_dev(synth.prefill_inputs(L, H, d, seed=6))
