@@ -478,6 +478,10 @@ def time_decode_fp8(idxc, synth, dev, peaks, L, H, d, k_top, seed, decode_B, fir
     dld = (L + 31) // 32 * 32
     dscores = dws[: decode_B * dld * 4].view(torch.float32).view(decode_B, dld)
     ev_step, ev_score = [], []
+    # The calls are enqueued behind a 10 ms spin kernel, so that all of them are queued before the first one runs: a step
+    # of 50 us is otherwise as long as the host needs to issue it, and the events would time the host
+    torch.cuda.synchronize()
+    torch.cuda._sleep(20_000_000)
     for i in range(26):                                 # enqueued back to back: no host round trip inside a timed interval
         x = sets[i & 1]
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -485,6 +489,8 @@ def time_decode_fp8(idxc, synth, dev, peaks, L, H, d, k_top, seed, decode_B, fir
         idxc.indexer_decode(x.q_step, x.k_cache, x.w, x.k_offsets, x.lens, L, k_top, x.q_scale, x.k_scale, topk_out=dtop, workspace=dws)
         b.record()
         ev_step.append((a, b))
+    torch.cuda.synchronize()
+    torch.cuda._sleep(20_000_000)
     for i in range(26):
         x = sets[i & 1]
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

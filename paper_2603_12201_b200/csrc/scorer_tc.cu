@@ -992,16 +992,20 @@ cudaError_t launch_decode_instance(const ScoreArgs& a, const CUtensorMap& q_map,
     auto kern = score_decode_tc_kernel<NKH, H, FP8>;
     if (cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(kern), Cfg::kSmemBytes); e != cudaSuccess) return e;
     const int64_t tiles = (a.max_len + kTileKeys - 1) / kTileKeys;
-    // Tiles per work item: 512 KB of keys streams best (shorter items cost about 5 % at a large batch), but a small batch
-    // leaves the last round of the static schedule half empty. Estimated with every sequence at max_len (the lengths live
-    // on the device): the item size in 320..512 KB with the fewest rounds x size, the larger one on a tie (items of 192 to
-    // 256 KB make the CTAs walk HBM in lock-step at a stride that costs a fifth of the bandwidth).
-    const int cmax = Cfg::kMaxChunk, cmin = 10 * 2 / NKH;
+    // Tiles per work item, estimated with every sequence at max_len (the lengths live on the device): the size with the
+    // lowest rounds x (size + one tile's worth of hand-over per item). 512 KB of keys streams best at a large batch
+    // (shorter items cost about 5 %), but a small batch must be cut finer to give every SM an item (one sequence of
+    // 131072 e4m3 keys in items of 28 tiles is 37 items for 148 SMs). Items of 192 to 256 KB are left out: the CTAs then
+    // walk HBM in lock-step at a stride that costs a fifth of the bandwidth. The larger size wins a tie.
+    constexpr int kTileBytes = NKH * kKRegionBytes;
+    const int cmax = Cfg::kMaxChunk;
     int chunk = cmax;
     int64_t best = -1;
-    for (int c = cmax; c >= cmin; --c) {
+    for (int c = cmax; c >= 2; --c) {
+        const int item_bytes = c * kTileBytes;
+        if (item_bytes > 160 * 1024 && item_bytes < 320 * 1024) continue;
         const int64_t n_items = a.n_rows * ((tiles + c - 1) / c);
-        const int64_t cost = ((n_items + sm_count - 1) / sm_count) * c;
+        const int64_t cost = ((n_items + sm_count - 1) / sm_count) * (c + 1);
         if (best < 0 || cost < best) { best = cost; chunk = c; }
     }
     const int64_t items = a.n_rows * ((tiles + chunk - 1) / chunk);
