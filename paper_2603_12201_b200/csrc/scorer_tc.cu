@@ -995,17 +995,17 @@ cudaError_t launch_decode_instance(const ScoreArgs& a, const CUtensorMap& q_map,
     // Tiles per work item, estimated with every sequence at max_len (the lengths live on the device): the size with the
     // lowest rounds x (size + one tile's worth of hand-over per item). 512 KB of keys streams best at a large batch
     // (shorter items cost about 5 %), but a small batch must be cut finer to give every SM an item (one sequence of
-    // 131072 e4m3 keys in items of 28 tiles is 37 items for 148 SMs). Items of 192 to 256 KB are left out: the CTAs then
-    // walk HBM in lock-step at a stride that costs a fifth of the bandwidth. The larger size wins a tie.
+    // 131072 e4m3 keys in items of 28 tiles is 37 items for 148 SMs). Items of 192 to 256 KB count a quarter dearer: the CTAs
+    // then walk HBM in lock-step at a stride that costs a fifth of the bandwidth. The larger size wins a tie.
     constexpr int kTileBytes = NKH * kKRegionBytes;
     const int cmax = Cfg::kMaxChunk;
     int chunk = cmax;
     int64_t best = -1;
     for (int c = cmax; c >= 2; --c) {
         const int item_bytes = c * kTileBytes;
-        if (item_bytes > 160 * 1024 && item_bytes < 320 * 1024) continue;
+        const bool bad_stride = item_bytes > 160 * 1024 && item_bytes < 320 * 1024;
         const int64_t n_items = a.n_rows * ((tiles + c - 1) / c);
-        const int64_t cost = ((n_items + sm_count - 1) / sm_count) * (c + 1);
+        const int64_t cost = ((n_items + sm_count - 1) / sm_count) * (c + 1) * (bad_stride ? 5 : 4);   // (a quarter dearer)
         if (best < 0 || cost < best) { best = cost; chunk = c; }
     }
     const int64_t items = a.n_rows * ((tiles + chunk - 1) / chunk);
