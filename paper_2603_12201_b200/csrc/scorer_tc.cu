@@ -75,6 +75,8 @@ struct PrefillParams {
     unsigned int* status;
     StreamTopk st;
     const uint8_t* item_mask;
+    int sub_per_block;      // work items per block of QB query rows: 1, or (few blocks, long rows) the block's key tiles in
+    int key_split;          // ... sub_per_block runs of key_split tiles each, so that every SM gets work
 };
 
 // Order in which a work item of nkt key tiles is visited when the top-k streams: `ns` sample tiles 0, stride,
@@ -99,7 +101,7 @@ __device__ __forceinline__ void give_up(volatile uint32_t* abort_flag, unsigned 
 }
 
 // NKH: 128-byte chunks per operand row (d * element size / 128). H: indexer heads.
-template <int NKH, int H, bool FP8, bool STREAM>
+template <int NKH, int H, bool FP8, bool STREAM, bool SPLIT>
 __global__ void __launch_bounds__(kPrefillThreads, 1)
 score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                         const PrefillParams p) {
@@ -158,22 +160,35 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
     tcgen05_fence_after_sync();
     const uint32_t tmem_base = *tmem_base_slot;
 
-    const int64_t n_items = (p.n_rows + QB - 1) / QB;
+    const int n_sub = SPLIT ? p.sub_per_block : 1;       // (a compile-time 1 keeps the unsplit kernel's code as it was)
+    const int64_t n_items = (p.n_rows + QB - 1) / QB * n_sub;
     const int G = gridDim.x;
     const int cta = blockIdx.x;
-    // work item of this CTA in round `rho` (longest first, boustrophedon), or -1
-    // (-2: the item is masked out and every role passes over it)
+    // key tiles a block of QB query rows visits: positions 0 .. q_begin + (its last row)
+    auto key_tiles_of_block = [&](int64_t block) -> int {
+        int64_t last = block * QB + QB;
+        if (last > p.n_rows) last = p.n_rows;
+        return static_cast<int>((p.q_begin + last + kTileKeys - 1) / kTileKeys);
+    };
+    // A work item is a block of QB query rows with all its key tiles, or (n_sub > 1) run number item % n_sub of key_split
+    // of its key tiles. Work item of this CTA in round `rho` (longest first, boustrophedon), -1: none left,
+    // -2: the item is masked out or its run lies beyond the block's last tile, and every role passes over it
     auto item_of_round = [&](int64_t rho) -> int64_t {
         const int64_t seq = rho * G + ((rho & 1) ? (G - 1 - cta) : cta);
         if (seq >= n_items) return -1;
         const int64_t item = n_items - 1 - seq;
-        if (p.item_mask != nullptr && p.item_mask[item] == 0) return -2;
+        const int64_t block = n_sub == 1 ? item : item / n_sub;
+        if (p.item_mask != nullptr && p.item_mask[block] == 0) return -2;
+        if (n_sub > 1 && static_cast<int>(item % n_sub) * p.key_split >= key_tiles_of_block(block)) return -2;
         return item;
     };
+    // first key tile and number of key tiles of a work item
+    auto first_tile_of_item = [&](int64_t item) -> int { return n_sub == 1 ? 0 : static_cast<int>(item % n_sub) * p.key_split; };
     auto key_tiles_of_item = [&](int64_t item) -> int {
-        int64_t last = item * QB + QB;
-        if (last > p.n_rows) last = p.n_rows;
-        return static_cast<int>((p.q_begin + last + kTileKeys - 1) / kTileKeys);   // positions 0 .. q_begin+last-1
+        const int all = key_tiles_of_block(n_sub == 1 ? item : item / n_sub);
+        if (n_sub == 1) return all;
+        const int left = all - first_tile_of_item(item);
+        return left < p.key_split ? left : p.key_split;
     };
 
     if (warp == 0) {
@@ -185,13 +200,15 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
             uint32_t k_phase = 0, q_phase = 0;
             bool ok = true;
             for (int64_t rho = 0; ok; ++rho) {
-                const int64_t item = item_of_round(rho);
-                if (item == -2) continue;
-                if (item < 0) break;
-                const int nkt = key_tiles_of_item(item);
+                const int64_t item_id = item_of_round(rho);
+                if (item_id == -2) continue;
+                if (item_id < 0) break;
+                const int nkt = key_tiles_of_item(item_id);
+                const int kt0 = first_tile_of_item(item_id);
+                const int64_t item = n_sub == 1 ? item_id : item_id / n_sub;        // the block of query rows
                 const TileOrder ord(nkt, STREAM ? Cfg::kSampleTiles : nkt);
                 auto load_k = [&](int j) -> bool {
-                    const int kt = STREAM ? ord.tile(j) : j;
+                    const int kt = STREAM ? ord.tile(j) : kt0 + j;
                     if (!mbar_wait(bar_k_empty + 8 * stage, k_phase ^ 1u, abort_flag)) return false;
                     mbar_arrive_expect_tx(bar_k_full + 8 * stage, NKH * kKRegionBytes);
                     for (int kh = 0; kh < NKH; ++kh)
@@ -232,10 +249,10 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
             return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort_flag));
         };
         for (int64_t rho = 0; ok; ++rho) {
-            const int64_t item = item_of_round(rho);
-            if (item == -2) continue;
-            if (item < 0) break;
-            const int nkt = key_tiles_of_item(item);
+            const int64_t item_id = item_of_round(rho);
+            if (item_id == -2) continue;
+            if (item_id < 0) break;
+            const int nkt = key_tiles_of_item(item_id);
             for (int kt = 0; kt < nkt && ok; ++kt) {
                 ok = wait_bar(bar_k_full + 8 * stage, k_phase);
                 if (!ok) break;
@@ -303,10 +320,12 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
             return good;
         };
         for (int64_t rho = 0; ok; ++rho) {
-            const int64_t item = item_of_round(rho);
-            if (item == -2) continue;
-            if (item < 0) break;
-            const int nkt = key_tiles_of_item(item);
+            const int64_t item_id = item_of_round(rho);
+            if (item_id == -2) continue;
+            if (item_id < 0) break;
+            const int nkt = key_tiles_of_item(item_id);
+            const int kt0 = first_tile_of_item(item_id);
+            const int64_t item = n_sub == 1 ? item_id : item_id / n_sub;            // the block of query rows
             const TileOrder ord(nkt, STREAM ? Cfg::kSampleTiles : nkt);
             const int64_t row_base = item * QB;
             // STREAM: every thread has a list of its own per row (it sees one key of each tile), so it appends at a position
@@ -337,7 +356,7 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
                 }
             }
             for (int jt = 0; jt < nkt && ok; ++jt) {
-                const int kt = STREAM ? ord.tile(jt) : jt;
+                const int kt = STREAM ? ord.tile(jt) : kt0 + jt;
                 const int64_t s = static_cast<int64_t>(kt) * kTileKeys + key_written;
                 float ksc = 1.f;
                 if constexpr (FP8) ksc = s < p.k_rows ? __ldg(p.k_scale + s) : 0.f;
@@ -558,18 +577,50 @@ score_prefill_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_
     }
 }
 
+template <int NKH, int H, bool FP8, bool STREAM, bool SPLIT>
+cudaError_t launch_prefill_kernel(const PrefillParams& p, int grid, const CUtensorMap& q_map, const CUtensorMap& k_map, cudaStream_t stream) {
+    using Cfg = PrefillCfg<NKH, H, STREAM>;
+    auto kern = score_prefill_tc_kernel<NKH, H, FP8, STREAM, SPLIT>;
+    if (cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(kern), Cfg::kSmemBytes); e != cudaSuccess) return e;
+    kern<<<grid, kPrefillThreads, Cfg::kSmemBytes, stream>>>(q_map, k_map, p);
+    return cudaGetLastError();
+}
+
 template <int NKH, int H, bool FP8, bool STREAM>
 cudaError_t launch_prefill_variant(const ScoreArgs& a, const CUtensorMap& q_map, const CUtensorMap& k_map,
                                    unsigned int* status, int sm_count, cudaStream_t stream) {
-    using Cfg = PrefillCfg<NKH, H, STREAM>;
-    auto kern = score_prefill_tc_kernel<NKH, H, FP8, STREAM>;
-    if (cudaError_t e = ensure_max_dynamic_smem(reinterpret_cast<const void*>(kern), Cfg::kSmemBytes); e != cudaSuccess) return e;
     constexpr int QB = 2 * (kTileCols / H);
-    const int64_t n_items = (a.n_rows + QB - 1) / QB;
+    const int64_t n_blocks = (a.n_rows + QB - 1) / QB;
+    // Few blocks of query rows (a short prompt, or a short chunk of queries against a long context) leave SMs idle and
+    // the longest block sets the time: the blocks' key tiles are then cut into runs of key_split tiles (the scores of a
+    // row's keys are independent, so any cut is exact; the query tile is loaded once per run). The split with the
+    // shortest makespan rounds x run length among those that give the grid 1 to 4 items per SM; not with the streaming
+    // top-k, whose threshold needs a row's sample before the rest of its tiles.
+    int sub_per_block = 1, key_split = 0;
+    if (!STREAM && n_blocks < 2 * static_cast<int64_t>(sm_count)) {
+        const int64_t tiles_longest = (a.q_begin + a.n_rows + kTileKeys - 1) / kTileKeys;
+        const int64_t tiles_first = (a.q_begin + (a.n_rows < QB ? a.n_rows : QB) + kTileKeys - 1) / kTileKeys;
+        const int64_t total = (tiles_first + tiles_longest) * n_blocks / 2;          // the blocks' tile counts grow linearly
+        int64_t best = ((n_blocks + sm_count - 1) / sm_count) * (tiles_longest + 1);
+        for (int m = 1; m <= 4; ++m) {
+            int64_t split = (total + static_cast<int64_t>(m) * sm_count - 1) / (static_cast<int64_t>(m) * sm_count);
+            if (split < 4) split = 4;
+            if (split >= tiles_longest) continue;
+            const int64_t subs = (tiles_longest + split - 1) / split;
+            // runs that are not empty: block b has ceil(tiles_b / split) of them; estimated from the linear growth
+            const int64_t n_runs = n_blocks * ((tiles_first + tiles_longest) / 2 + split - 1) / split;
+            const int64_t cost = ((n_runs + sm_count - 1) / sm_count) * (split + 1);
+            if (cost < best) { best = cost; sub_per_block = static_cast<int>(subs); key_split = static_cast<int>(split); }
+        }
+    }
+    const int64_t n_items = n_blocks * sub_per_block;
     const int grid = static_cast<int>(n_items < sm_count ? n_items : sm_count);
-    PrefillParams p{a.w, a.q_scale, a.k_scale, a.scores, a.ld, a.q_begin, a.n_rows, a.k_rows, status, a.stream, a.item_mask};
-    kern<<<grid, kPrefillThreads, Cfg::kSmemBytes, stream>>>(q_map, k_map, p);
-    return cudaGetLastError();
+    PrefillParams p{a.w, a.q_scale, a.k_scale, a.scores, a.ld, a.q_begin, a.n_rows, a.k_rows, status, a.stream, a.item_mask,
+                    sub_per_block, key_split};
+    if constexpr (!STREAM) {
+        if (sub_per_block > 1) return launch_prefill_kernel<NKH, H, FP8, false, true>(p, grid, q_map, k_map, stream);
+    }
+    return launch_prefill_kernel<NKH, H, FP8, STREAM, false>(p, grid, q_map, k_map, stream);
 }
 
 template <int NKH, int H, bool FP8>

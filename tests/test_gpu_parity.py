@@ -250,6 +250,26 @@ def test_prefill_chunked_workspace_and_scoreless_paths_agree():
     assert e.value.status == idxc.ERR_WORKSPACE
 
 
+def test_prefill_short_chunk_against_long_context_equals_the_whole_prefill():
+    """A few hundred query rows against a long K are cut into runs of key tiles so that every SM gets work; a whole
+    prefill of the same length has enough blocks of rows and is not cut. Both must give the same bits."""
+    L, H, d, k_top = 20000, 64, 128, 512
+    inp = _to_dev(synth.prefill_inputs(L, H, d, seed=91))
+    s_full, t_full = _gpu_prefill(inp, k_top)
+    for q0, q1 in [(19400, 20000), (12345, 12601), (0, 300)]:
+        s_c, t_c = _gpu_prefill(inp, k_top, q_begin=q0, q_slice=slice(q0, q1))
+        assert np.array_equal(t_c, t_full[q0:q1])
+        for r in (0, 1, (q1 - q0) // 2, q1 - q0 - 1):
+            assert np.array_equal(s_c[r, : q0 + r + 1], s_full[q0 + r, : q0 + r + 1])
+            assert np.all(np.isnan(s_c[r, q0 + r + 1:]))
+    # and in e4m3
+    inp8 = _to_dev(synth.prefill_inputs(9000, H, d, seed=92, fp8=True))
+    s_full, t_full = _gpu_prefill(inp8, k_top)
+    s_c, t_c = _gpu_prefill(inp8, k_top, q_begin=8500, q_slice=slice(8500, 9000))
+    assert np.array_equal(t_c, t_full[8500:])
+    assert np.array_equal(s_c[499, :9000], s_full[8999, :9000])
+
+
 def test_prefill_duplicate_keys_pick_lowest_index_and_gate():
     L, H, d, k_top = 400, 16, 64, 8
     inp = synth.prefill_inputs(L, H, d, seed=3)
