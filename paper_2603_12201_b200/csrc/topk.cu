@@ -265,8 +265,12 @@ cudaError_t launch_topk_rows(const float* scores, int64_t ld, int64_t n_rows, in
         return launch_topk_rows_cluster(scores, ld, n_rows, first_len, len_step, lens, k_top, out, longest, stream, row_mask);
     int64_t map_bytes = (longest + 127) / 128 * 32;
     if (map_bytes > TK_MAP_MAX_BYTES) map_bytes = TK_MAP_MAX_BYTES;
-    // many rows: small CTAs, many per SM; few rows: more threads per row
-    if (n_rows >= 1024)
+    // Many rows of moderate length: small CTAs, eight per SM. Few rows, or long rows (a 128-thread CTA alone on a row of
+    // 100K scores has too few loads in flight: measured on 8192 rows, the small instance reads 2.5 / 2.1 / 1.8 / 1.4 TB/s
+    // at 16K / 32K / 64K / 128K scores per row, the large one 0.9 / 1.5 / 2.3 / 3.0 TB/s): 1024 threads per row.
+    int64_t mean_len = lens ? longest : first_len + (n_rows - 1) * len_step / 2;
+    if (mean_len > ld) mean_len = ld;
+    if (n_rows >= 1024 && mean_len < 49152)
         return launch_instance<128, 8, kCapMany>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, static_cast<int>(map_bytes), stream, row_mask);
     return launch_instance<1024, 1, kCapFew>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, static_cast<int>(map_bytes), stream, row_mask);
 }
