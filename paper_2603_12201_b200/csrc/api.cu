@@ -218,9 +218,10 @@ idxc_status idxc_indexer_prefill(const void* q, const void* k, const float* w, c
         idxc_status s2 = launch_scorer(a, false, flags, stream);
         if (s2 != IDXC_OK) return s2;
         if (topk_out) {
-            g_launches += 1;
-            if (launch_topk_rows(sc, ld, nr, q_begin + r0 + 1, 1, nullptr, k_top, topk_out + r0 * k_top, stream) != cudaSuccess)
-                return IDXC_ERR_CUDA;
+            int n_l = 0;
+            const cudaError_t e = launch_topk_rows(sc, ld, nr, q_begin + r0 + 1, 1, nullptr, k_top, topk_out + r0 * k_top, stream, nullptr, &n_l);
+            g_launches += n_l;
+            if (e != cudaSuccess) return IDXC_ERR_CUDA;
         }
         return IDXC_OK;
     };
@@ -272,9 +273,10 @@ idxc_status idxc_indexer_prefill(const void* q, const void* k, const float* w, c
             a.scores = sc; a.ld = ld; a.stream = StreamTopk{}; a.item_mask = item_fail;
             st = launch_scorer(a, false, flags, stream);
             if (st != IDXC_OK) return st;
-            g_launches += 1;
-            if (launch_topk_rows(sc, ld, nr, q_begin + r0 + 1, 1, nullptr, k_top, topk_out + r0 * k_top, stream, row_fail) != cudaSuccess)
-                return IDXC_ERR_CUDA;
+            int n_l = 0;
+            const cudaError_t e = launch_topk_rows(sc, ld, nr, q_begin + r0 + 1, 1, nullptr, k_top, topk_out + r0 * k_top, stream, row_fail, &n_l);
+            g_launches += n_l;
+            if (e != cudaSuccess) return IDXC_ERR_CUDA;
         }
         return IDXC_OK;
     }
@@ -347,9 +349,11 @@ idxc_status idxc_topk_rows(const float* scores, int64_t ld, int64_t n_rows, int6
     if (n_rows == 0) return IDXC_OK;
     if (!scores || !topk_out || !aligned(scores, 16) || !aligned(topk_out, 4)) return IDXC_ERR_INVALID_ARG;
     if (!lens && (first_len < 0 || len_step < 0)) return IDXC_ERR_INVALID_ARG;
-    g_launches += 1;
-    return launch_topk_rows(scores, ld, n_rows, first_len, len_step, lens, k_top, topk_out,
-                            static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? IDXC_OK : IDXC_ERR_CUDA;
+    int n_l = 0;
+    const cudaError_t e = launch_topk_rows(scores, ld, n_rows, first_len, len_step, lens, k_top, topk_out,
+                                           static_cast<cudaStream_t>(cuda_stream), nullptr, &n_l);
+    g_launches += n_l;
+    return e == cudaSuccess ? IDXC_OK : IDXC_ERR_CUDA;
 }
 
 // ------------------------------------------------------------------ schedule (Figure 2(b))

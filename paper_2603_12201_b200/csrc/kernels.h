@@ -13,10 +13,11 @@ cudaError_t ensure_max_dynamic_smem(const void* kernel, int bytes);
 
 // Row-wise top-k select (topk.cu). Row r has length lens[r] (device) if lens != nullptr,
 // else first_len + r * len_step, clamped to [0, ld]. row_mask: nullptr, or one byte per row: rows whose byte is 0 are
-// left alone (neither read nor written).
+// left alone (neither read nor written). launches: if given, receives the number of kernels launched (rows whose lengths
+// grow with the row number go out in up to three launches, one per range of lengths).
 cudaError_t launch_topk_rows(const float* scores, int64_t ld, int64_t n_rows, int64_t first_len,
                              int64_t len_step, const int32_t* lens, int k_top, int32_t* out,
-                             cudaStream_t stream, const uint8_t* row_mask = nullptr);
+                             cudaStream_t stream, const uint8_t* row_mask = nullptr, int* launches = nullptr);
 
 // Cluster variant for a few long rows (topk_cluster.cu): 8 CTAs per row exchanging through
 // distributed shared memory. `longest` = longest row of the launch.

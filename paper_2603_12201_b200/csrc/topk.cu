@@ -248,31 +248,91 @@ cudaError_t preload_topk_rows() {
     cudaFuncAttributes fa;
     const void* many = reinterpret_cast<const void*>(topk_rows_kernel<128, 8, kCapMany>);
     const void* few = reinterpret_cast<const void*>(topk_rows_kernel<1024, 1, kCapFew>);
+    const void* mid = reinterpret_cast<const void*>(topk_rows_kernel<256, 4, 3072>);
+    const void* half = reinterpret_cast<const void*>(topk_rows_kernel<512, 2, 4096>);
+    if (cudaError_t e = cudaFuncGetAttributes(&fa, mid); e != cudaSuccess) return e;
+    if (cudaError_t e = cudaFuncGetAttributes(&fa, half); e != cudaSuccess) return e;
+    if (cudaError_t e = ensure_max_dynamic_smem(mid, TK_MAP_MAX_BYTES + 8 * 3072); e != cudaSuccess) return e;
+    if (cudaError_t e = ensure_max_dynamic_smem(half, TK_MAP_MAX_BYTES + 8 * 4096); e != cudaSuccess) return e;
     if (cudaError_t e = cudaFuncGetAttributes(&fa, many); e != cudaSuccess) return e;
     if (cudaError_t e = cudaFuncGetAttributes(&fa, few); e != cudaSuccess) return e;
     if (cudaError_t e = ensure_max_dynamic_smem(many, TK_MAP_MAX_BYTES + 8 * kCapMany); e != cudaSuccess) return e;
     return ensure_max_dynamic_smem(few, TK_MAP_MAX_BYTES + 8 * kCapFew);
 }
 
+namespace {
+
+constexpr int kCapMid = 3072, kCapHalf = 4096;
+// Row lengths at which the next larger instance reads faster (8192 rows of one length, B200): 128 threads x 8 CTAs per SM
+// reads 2.3-2.6 TB/s up to 16K scores per row and falls off beyond (too few loads in flight per row: 1.8 TB/s at 64K,
+// 1.4 TB/s at 128K); 256 threads x 4 reads 2.6-3.9 TB/s from 20K to 56K; 512 threads x 2 reads 3.3-3.5 TB/s from 64K on;
+// 1024 threads x 1 is for launches of so few rows that the SMs would not fill otherwise.
+constexpr int64_t kLenMid = 18432, kLenHalf = 61440;
+
+cudaError_t launch_by_length(const float* scores, int64_t ld, int64_t n_rows, int64_t first_len, int64_t len_step,
+                             const int32_t* lens, int k_top, int32_t* out, int64_t longest, int64_t typical_len, cudaStream_t stream,
+                             const uint8_t* row_mask) {
+    int64_t map_bytes = (longest + 127) / 128 * 32;
+    if (map_bytes > TK_MAP_MAX_BYTES) map_bytes = TK_MAP_MAX_BYTES;
+    const int mb = static_cast<int>(map_bytes);
+    if (n_rows < 296)
+        return launch_instance<1024, 1, kCapFew>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, mb, stream, row_mask);
+    if (typical_len < kLenMid)
+        return launch_instance<128, 8, kCapMany>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, mb, stream, row_mask);
+    if (typical_len < kLenHalf)
+        return launch_instance<256, 4, kCapMid>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, mb, stream, row_mask);
+    return launch_instance<512, 2, kCapHalf>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, mb, stream, row_mask);
+}
+
+}  // namespace
+
 cudaError_t launch_topk_rows(const float* scores, int64_t ld, int64_t n_rows, int64_t first_len, int64_t len_step,
-                             const int32_t* lens, int k_top, int32_t* out, cudaStream_t stream, const uint8_t* row_mask) {
+                             const int32_t* lens, int k_top, int32_t* out, cudaStream_t stream, const uint8_t* row_mask,
+                             int* launches) {
+    if (launches) *launches = 0;
     if (n_rows <= 0) return cudaSuccess;
     // the selection map covers the longest row of this launch, rounded up to a whole 128-score block
     int64_t longest = lens ? ld : first_len + (n_rows - 1) * len_step;
     if (longest > ld) longest = ld;
     if (longest < 0) longest = 0;
-    if (topk_cluster_applicable(n_rows, longest))
+    if (topk_cluster_applicable(n_rows, longest)) {
+        if (launches) *launches = 1;
         return launch_topk_rows_cluster(scores, ld, n_rows, first_len, len_step, lens, k_top, out, longest, stream, row_mask);
-    int64_t map_bytes = (longest + 127) / 128 * 32;
-    if (map_bytes > TK_MAP_MAX_BYTES) map_bytes = TK_MAP_MAX_BYTES;
-    // Many rows of moderate length: small CTAs, eight per SM. Few rows, or long rows (a 128-thread CTA alone on a row of
-    // 100K scores has too few loads in flight: measured on 8192 rows, the small instance reads 2.5 / 2.1 / 1.8 / 1.4 TB/s
-    // at 16K / 32K / 64K / 128K scores per row, the large one 0.9 / 1.5 / 2.3 / 3.0 TB/s): 1024 threads per row.
-    int64_t mean_len = lens ? longest : first_len + (n_rows - 1) * len_step / 2;
-    if (mean_len > ld) mean_len = ld;
-    if (n_rows >= 1024 && mean_len < 49152)
-        return launch_instance<128, 8, kCapMany>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, static_cast<int>(map_bytes), stream, row_mask);
-    return launch_instance<1024, 1, kCapFew>(scores, ld, n_rows, first_len, len_step, lens, k_top, out, static_cast<int>(map_bytes), stream, row_mask);
+    }
+    if (lens != nullptr || len_step <= 0 || n_rows < 2048) {
+        // lengths on the device, one length for all rows, or few rows: one launch, sized for the longest (mean) row
+        if (launches) *launches = 1;
+        int64_t typical = lens ? longest : first_len + (n_rows - 1) * len_step / 2;
+        if (typical > ld) typical = ld;
+        return launch_by_length(scores, ld, n_rows, first_len, len_step, lens, k_top, out, longest, typical, stream, row_mask);
+    }
+    // Lengths that grow with the row number (a prefill): the rows are cut where the length crosses kLenMid and kLenHalf,
+    // and every stretch (of at least 1024 rows) goes to the instance that suits its lengths, as a launch of its own
+    // (the rows are independent).
+    int64_t cuts[4] = {0, (kLenMid - first_len + len_step - 1) / len_step, (kLenHalf - first_len + len_step - 1) / len_step, n_rows};
+    for (int i = 1; i <= 2; ++i) {
+        if (cuts[i] < cuts[i - 1]) cuts[i] = cuts[i - 1];
+        if (cuts[i] > n_rows) cuts[i] = n_rows;
+    }
+    // stretches shorter than 1024 rows join their neighbour
+    if (cuts[1] - cuts[0] < 1024) cuts[1] = cuts[0];
+    if (cuts[3] - cuts[2] < 1024) cuts[2] = cuts[3];
+    if (cuts[2] - cuts[1] < 1024) { if (cuts[1] > cuts[0]) cuts[1] = cuts[2]; else cuts[2] = cuts[1]; }
+    for (int i = 0; i < 3; ++i) {
+        const int64_t r0 = cuts[i], nr = cuts[i + 1] - cuts[i];
+        if (nr <= 0) continue;
+        const int64_t fl = first_len + r0 * len_step;
+        int64_t hi = fl + (nr - 1) * len_step;
+        if (hi > ld) hi = ld;
+        int64_t typical = fl + (nr - 1) * len_step / 2;
+        if (typical > ld) typical = ld;
+        if (cudaError_t e = launch_by_length(scores + r0 * ld, ld, nr, fl, len_step, nullptr, k_top, out + r0 * static_cast<int64_t>(k_top), hi,
+                                             typical, stream, row_mask ? row_mask + r0 : nullptr);
+            e != cudaSuccess)
+            return e;
+        if (launches) *launches += 1;
+    }
+    return cudaSuccess;
 }
 
 }  // namespace idxc
