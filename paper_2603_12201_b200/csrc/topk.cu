@@ -267,7 +267,7 @@ constexpr int kCapMid = 3072, kCapHalf = 4096;
 // reads 2.3-2.6 TB/s up to 16K scores per row and falls off beyond (too few loads in flight per row: 1.8 TB/s at 64K,
 // 1.4 TB/s at 128K); 256 threads x 4 reads 2.6-3.9 TB/s from 20K to 56K; 512 threads x 2 reads 3.3-3.5 TB/s from 64K on;
 // 1024 threads x 1 is for launches of so few rows that the SMs would not fill otherwise.
-constexpr int64_t kLenMid = 18432, kLenHalf = 61440;
+constexpr int64_t kLenMid = 20480, kLenHalf = 61440;
 
 cudaError_t launch_by_length(const float* scores, int64_t ld, int64_t n_rows, int64_t first_len, int64_t len_step,
                              const int32_t* lens, int k_top, int32_t* out, int64_t longest, int64_t typical_len, cudaStream_t stream,
