@@ -167,6 +167,19 @@ def test_config5_fp8_chunked_prefill_and_decode():
     o_sc, _ = oracle.indexer_prefill(codes(inp.q[t:t + 1]), codes_cached(inp), f32(inp.w[t:t + 1]), k_top, dt,
                                      f32(inp.q_scale[t:t + 1]), f32(inp.k_scale), q_begin=t)
     assert_scores_close(score_rows[t][: t + 1], o_sc[0, : t + 1], RTOL_BF16, what="fp8 row, tight bound")
+    # the streaming top-k on the first, a middle and the last chunk: the same indices entry for entry. The last chunk's rows
+    # are so long that the sample leaves the threshold loose, most of its work items overflow a list and are scored again by
+    # the ordinary kernels: the path that repairs is exercised at scale
+    F = idxc.FLAG_STREAM_TOPK
+    ws_s = idxc.alloc_workspace(idxc.prefill_workspace_bytes(chunk, L, H, d, k_top, idxc.FP8_E4M3, F), DEV)
+    for q0 in (0, 7 * chunk, L - chunk):
+        sl = slice(q0, q0 + chunk)
+        t_s = torch.full((chunk, k_top), -7, dtype=torch.int32, device=DEV)
+        idxc.indexer_prefill(inp.q[sl], inp.k, inp.w[sl], k_top, inp.q_scale[sl], inp.k_scale, q_begin=q0, topk_out=t_s,
+                             workspace=ws_s, flags=F)
+        idxc.poll_device_status()
+        assert torch.equal(t_s, topk[sl]), f"streaming top-k, chunk at {q0}"
+    del ws_s
     # one decode step at the workload's batch: the resulting cache (sequence 0) and fresh caches of the same length
     B = c["decode_B"]
     fresh = synth.decode_inputs(B, H, d, L, L, seed=c["seed"], device=DEV, layer=1, fp8=True, lens=[L] * B)
