@@ -256,10 +256,10 @@ def test_prefill_short_chunk_against_long_context_equals_the_whole_prefill():
     L, H, d, k_top = 20000, 64, 128, 512
     inp = _to_dev(synth.prefill_inputs(L, H, d, seed=91))
     s_full, t_full = _gpu_prefill(inp, k_top)
-    for q0, q1 in [(19400, 20000), (12345, 12601), (0, 300)]:
+    for q0, q1 in [(19400, 20000), (12345, 12601), (0, 300), (19995, 20000), (7, 8)]:      # (down to a handful of rows)
         s_c, t_c = _gpu_prefill(inp, k_top, q_begin=q0, q_slice=slice(q0, q1))
         assert np.array_equal(t_c, t_full[q0:q1])
-        for r in (0, 1, (q1 - q0) // 2, q1 - q0 - 1):
+        for r in sorted({0, min(1, q1 - q0 - 1), (q1 - q0) // 2, q1 - q0 - 1}):
             assert np.array_equal(s_c[r, : q0 + r + 1], s_full[q0 + r, : q0 + r + 1])
             assert np.all(np.isnan(s_c[r, q0 + r + 1:]))
     # and in e4m3
