@@ -1,0 +1,147 @@
+"""Seeded random shapes through the prefill and decode entry points: every accepted (H_I, d_I, dtype), ragged lengths,
+query chunks against a longer K, workspaces that force chunking, the streaming top-k, empty sequences, unaligned cache
+offsets. Each case is checked against the FP64 oracle on sampled rows and against the GPU's own scores (exact top-k with
+the lowest-index tie rule); the score-less and streaming paths must give the ordinary path's indices."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2603_12201_b200 import binding as idxc
+from paper_2603_12201_b200 import synth
+from tests.util import RTOL_BF16, RTOL_FP8, assert_scores_close, assert_topk_valid, codes, f32
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+SHAPES = [(16, 64, False), (32, 64, False), (64, 64, False), (16, 128, False), (32, 128, False), (64, 128, False),
+          (16, 128, True), (32, 128, True), (64, 128, True)]
+
+
+def to_dev(inp):
+    for name in ("q", "k", "w", "q_scale", "k_scale", "q_step", "k_cache", "k_offsets", "lens"):
+        if hasattr(inp, name) and getattr(inp, name) is not None:
+            setattr(inp, name, getattr(inp, name).to(DEV))
+    return inp
+
+
+def own_exact(g_scores, g_topk, rows, k_top, q_begin):
+    for r in rows:
+        n = q_begin + r + 1
+        kk = min(k_top, n)
+        order = np.argsort(-g_scores[r, :n].astype(np.float64), kind="stable")
+        assert np.array_equal(np.sort(order[:kk]), g_topk[r, :kk]), f"own top-k row {r}"
+        assert np.all(g_topk[r, kk:] == -1), f"tail row {r}"
+
+
+def prefill_case(rng, i, note):
+    H, d, fp8 = SHAPES[rng.integers(len(SHAPES))]
+    L = int(rng.choice([rng.integers(1, 300), rng.integers(300, 3000), rng.integers(3000, 9000)]))
+    k_top = int(rng.choice([rng.integers(1, 64), rng.integers(64, 1024), 2048, rng.integers(1024, 2049)]))
+    q0 = 0 if rng.random() < 0.4 else int(rng.integers(0, L))
+    q1 = L if rng.random() < 0.5 else int(rng.integers(q0 + 1, L + 1))
+    desc = f"prefill L={L} H={H} d={d} fp8={fp8} k={k_top} q=[{q0},{q1})"
+    note["case"] = desc
+    inp = to_dev(synth.prefill_inputs(L, H, d, seed=1000 + i, fp8=fp8))
+    q, w = inp.q[q0:q1].contiguous(), inp.w[q0:q1].contiguous()
+    qs = None if inp.q_scale is None else inp.q_scale[q0:q1].contiguous()
+    n = q1 - q0
+    ld = (L + 3) // 4 * 4
+    scores = torch.full((n, ld), float("nan"), device=DEV)
+    topk = torch.full((n, k_top), -7, dtype=torch.int32, device=DEV)
+    idxc.indexer_prefill(q, inp.k, w, k_top, qs, inp.k_scale, q_begin=q0, scores_out=scores, topk_out=topk)
+    idxc.poll_device_status()
+    dt = idxc.FP8_E4M3 if fp8 else idxc.BF16
+    # scoreless path, with a workspace that forces chunks sometimes
+    full = idxc.prefill_workspace_bytes(n, L, H, d, k_top, dt, 0)
+    ws_bytes = full if rng.random() < 0.5 else max(full // int(rng.integers(2, 6)), 1)
+    topk2 = torch.full((n, k_top), -7, dtype=torch.int32, device=DEV)
+    try:
+        idxc.indexer_prefill(q, inp.k, w, k_top, qs, inp.k_scale, q_begin=q0, topk_out=topk2, workspace=idxc.alloc_workspace(ws_bytes, DEV))
+        idxc.poll_device_status()
+        assert torch.equal(topk, topk2), "scoreless path differs"
+    except idxc.IdxcError as e:
+        if e.status != idxc.ERR_WORKSPACE:
+            raise
+    # streaming path
+    fl = idxc.FLAG_STREAM_TOPK
+    fulls = idxc.prefill_workspace_bytes(n, L, H, d, k_top, dt, fl)
+    ws_bytes = fulls if rng.random() < 0.5 else max(fulls // int(rng.integers(2, 6)), 1)
+    topk3 = torch.full((n, k_top), -7, dtype=torch.int32, device=DEV)
+    try:
+        idxc.indexer_prefill(q, inp.k, w, k_top, qs, inp.k_scale, q_begin=q0, topk_out=topk3, workspace=idxc.alloc_workspace(ws_bytes, DEV), flags=fl)
+        idxc.poll_device_status()
+        assert torch.equal(topk, topk3), "streaming path differs"
+    except idxc.IdxcError as e:
+        if e.status not in (idxc.ERR_WORKSPACE, idxc.ERR_INVALID_ARG):
+            raise
+    g_s, g_t = scores.cpu().numpy(), topk.cpu().numpy()
+    rows = sorted(set(int(x) for x in rng.integers(0, n, size=min(n, 24))) | {0, n - 1})
+    own_exact(g_s, g_t, rows, k_top, q0)
+    # nothing right of the diagonal
+    for r in rows:
+        assert np.all(np.isnan(g_s[r, q0 + r + 1:])), f"row {r} wrote past the diagonal"
+    orows = rows[:: max(1, len(rows) // 6)]
+    o_scores, _ = oracle.indexer_prefill(codes(q), codes(inp.k), f32(w), k_top, oracle.FP8_E4M3 if fp8 else oracle.BF16,
+                                         f32(qs), f32(inp.k_scale), q_begin=q0, rows=orows)
+    rtol = RTOL_FP8 if fp8 else RTOL_BF16
+    for j, r in enumerate(orows):
+        t = q0 + r
+        assert_scores_close(g_s[r, : t + 1], o_scores[j, : t + 1], rtol, what=f"row {r}")
+        assert_topk_valid(g_t[r], o_scores[j, : t + 1], k_top, rtol, what=f"row {r}")
+    return desc
+
+
+def decode_case(rng, i, note):
+    H, d, fp8 = SHAPES[rng.integers(len(SHAPES))]
+    B = int(rng.choice([1, 2, rng.integers(1, 9), rng.integers(9, 48)]))
+    hi = int(rng.choice([300, 5000, 40000, 140000])) if B <= 8 else int(rng.choice([300, 5000, 20000]))
+    lens = [int(x) for x in rng.integers(0, hi + 1, size=B)]
+    if rng.random() < 0.3:
+        lens[int(rng.integers(B))] = 0
+    k_top = int(rng.choice([rng.integers(1, 64), rng.integers(64, 1024), 2048]))
+    align = int(rng.choice([1, 8, 128]))
+    desc = f"decode B={B} H={H} d={d} fp8={fp8} k={k_top} align={align} lens={lens[:6]}..."
+    note["case"] = desc
+    inp = to_dev(synth.decode_inputs(B, H, d, 0, 0, seed=5000 + i, fp8=fp8, lens=lens, row_align=align))
+    if inp.max_len == 0:
+        return desc + " (skipped: all empty)"
+    ld = (inp.max_len + 3) // 4 * 4
+    scores = torch.full((B, ld), float("nan"), device=DEV)
+    topk = torch.full((B, k_top), -7, dtype=torch.int32, device=DEV)
+    idxc.indexer_decode(inp.q_step, inp.k_cache, inp.w, inp.k_offsets, inp.lens, inp.max_len, k_top, inp.q_scale,
+                        inp.k_scale, scores_out=scores, topk_out=topk)
+    idxc.poll_device_status()
+    topk2 = torch.full((B, k_top), -7, dtype=torch.int32, device=DEV)
+    dt = idxc.FP8_E4M3 if fp8 else idxc.BF16
+    ws = idxc.alloc_workspace(idxc.decode_workspace_bytes(B, inp.max_len, H, d, k_top, dt), DEV)
+    idxc.indexer_decode(inp.q_step, inp.k_cache, inp.w, inp.k_offsets, inp.lens, inp.max_len, k_top, inp.q_scale,
+                        inp.k_scale, topk_out=topk2, workspace=ws)
+    idxc.poll_device_status()
+    assert torch.equal(topk, topk2), "workspace path differs"
+    g_s, g_t = scores.cpu().numpy(), topk.cpu().numpy()
+    o_scores, _ = oracle.indexer_decode(codes(inp.q_step), codes(inp.k_cache), f32(inp.w), inp.k_offsets.cpu().numpy(),
+                                        inp.lens.cpu().numpy(), k_top, oracle.FP8_E4M3 if fp8 else oracle.BF16,
+                                        f32(inp.q_scale), f32(inp.k_scale))
+    rtol = RTOL_FP8 if fp8 else RTOL_BF16
+    for b in range(B):
+        n = lens[b]
+        assert_scores_close(g_s[b, :n], o_scores[b, :n], rtol, what=f"seq {b}")
+        assert np.all(np.isnan(g_s[b, n:])), f"seq {b} wrote past its length"
+        assert_topk_valid(g_t[b], o_scores[b, :n], k_top, rtol, what=f"seq {b}")
+        order = np.argsort(-g_s[b, :n].astype(np.float64), kind="stable")
+        kk = min(k_top, n)
+        assert np.array_equal(np.sort(order[:kk]), g_t[b, :kk]), f"own top-k seq {b}"
+        assert np.all(g_t[b, kk:] == -1)
+    return desc
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3, 4])
+def test_random_shapes(seed):
+    rng = np.random.default_rng(seed)
+    note = {}
+    for i in range(60):
+        fn = prefill_case if i % 2 else decode_case
+        try:
+            fn(rng, 100 * seed + i, note)
+        except (AssertionError, idxc.IdxcError) as e:
+            raise AssertionError(f"seed {seed} case {i} ({note.get('case')}): {e}") from e
