@@ -145,3 +145,98 @@ def test_random_shapes(seed):
             fn(rng, 100 * seed + i, note)
         except (AssertionError, idxc.IdxcError) as e:
             raise AssertionError(f"seed {seed} case {i} ({note.get('case')}): {e}") from e
+
+
+def make_scores(rng, g, n_rows, ld, kind):
+    if kind == "normal":
+        x = torch.randn((n_rows, ld), device=DEV, generator=g)
+    elif kind == "uniform":
+        x = torch.rand((n_rows, ld), device=DEV, generator=g)
+    elif kind == "relu":       # half of the scores exactly zero
+        x = torch.relu(torch.randn((n_rows, ld), device=DEV, generator=g))
+    elif kind == "cauchy":
+        x = torch.tan(3.14159 * (torch.rand((n_rows, ld), device=DEV, generator=g) - 0.5)).clamp(-1e30, 1e30)
+    elif kind == "quant":      # few distinct values
+        x = torch.randint(0, int(rng.integers(2, 40)), (n_rows, ld), device=DEV, generator=g).float()
+    elif kind == "asc":
+        x = torch.arange(ld, device=DEV).float().repeat(n_rows, 1) * 0.25 + torch.randn((n_rows, 1), device=DEV, generator=g)
+    elif kind == "desc":
+        x = -torch.arange(ld, device=DEV).float().repeat(n_rows, 1) * 0.25
+    elif kind == "spike":      # constant with a few outliers
+        x = torch.full((n_rows, ld), 1.5, device=DEV)
+        m = torch.rand((n_rows, ld), device=DEV, generator=g) < 0.001
+        x[m] = torch.randn((int(m.sum()),), device=DEV, generator=g) * 100
+    elif kind == "tiny":       # denormals and signed zeros
+        x = torch.randn((n_rows, ld), device=DEV, generator=g) * 1e-41
+        x[torch.rand((n_rows, ld), device=DEV, generator=g) < 0.2] = -0.0
+    elif kind == "huge":
+        x = torch.randn((n_rows, ld), device=DEV, generator=g) * 1e37
+    elif kind == "bimodal":
+        x = torch.randn((n_rows, ld), device=DEV, generator=g) + 50.0 * (torch.rand((n_rows, ld), device=DEV, generator=g) < float(rng.random())).float()
+    elif kind == "lognormal":
+        x = torch.exp(3 * torch.randn((n_rows, ld), device=DEV, generator=g))
+    elif kind == "bf16":       # scores rounded to 8 bits of mantissa: many ties
+        x = torch.randn((n_rows, ld), device=DEV, generator=g).bfloat16().float()
+    return x.contiguous()
+
+
+SCORE_KINDS = ["normal", "uniform", "relu", "cauchy", "quant", "asc", "desc", "spike", "tiny", "huge", "bimodal", "lognormal", "bf16"]
+
+
+def rows_not_exact(x, topk, lens, k_top):
+    """Rows whose indices are not the exact top-k (larger score first, lower index first among equal scores, -0 == +0;
+    ascending indices, -1 beyond the row's length), by a stable library sort on the GPU."""
+    n_rows, ld = x.shape
+    col = torch.arange(ld, device=DEV)
+    xm = torch.where(col[None, :] < lens[:, None], x, torch.full_like(x, float("-inf")))
+    xm = torch.where(xm == 0, torch.zeros_like(xm), xm)          # -0 == +0
+    order = torch.sort(xm, dim=1, descending=True, stable=True).indices[:, :k_top]
+    if order.shape[1] < k_top:
+        order = torch.nn.functional.pad(order, (0, k_top - order.shape[1]), value=0)
+    kk = torch.clamp(lens, max=k_top)
+    j = torch.arange(k_top, device=DEV)
+    valid = j[None, :] < kk[:, None]
+    want = torch.where(valid, order, torch.full_like(order, ld + 1))
+    want = torch.sort(want, dim=1).values
+    want = torch.where(valid, want, torch.full_like(want, -1)).int()
+    bad = (want != topk).any(dim=1)
+    return bad
+
+
+def test_topk_rows_adversarial_distributions():
+    """The select alone on score distributions chosen against its sampling step: heavy tails, a few distinct values,
+    sorted rows, constants with outliers, denormals and signed zeros, values near the float range's end; as a prefill
+    chunk (lengths growing by 0, 1 or 2 per row), as a decode step (few rows up to 600K scores) and as many ragged rows."""
+    rng = np.random.default_rng(7)
+    g = torch.Generator(device=DEV); g.manual_seed(11)
+    for i in range(400):
+        kind = SCORE_KINDS[rng.integers(len(SCORE_KINDS))]
+        mode = int(rng.integers(3))
+        k_top = int(rng.choice([1, rng.integers(1, 100), rng.integers(100, 2048), 2048]))
+        if mode == 0:
+            n_rows = int(rng.integers(1, 3000)); first = int(rng.integers(1, 70000)); step = int(rng.integers(0, 3))
+            n_rows = max(1, min(n_rows, int(2e8 // (first + step * n_rows))))
+            ld = (first + step * (n_rows - 1) + 3) // 4 * 4
+            lens_t = (first + step * torch.arange(n_rows, device=DEV)).int(); args = dict(first_len=first, len_step=step)
+        else:
+            if mode == 1:
+                n_rows = int(rng.integers(1, 140)); hi = int(rng.choice([3000, 40000, 200000, 600000]))
+            else:
+                n_rows = int(rng.integers(1, 5000)); hi = int(rng.choice([500, 5000, 30000]))
+            n_rows = max(1, min(n_rows, int(2e8 // hi)))
+            lens_np = rng.integers(0, hi + 1, size=n_rows); ld = max((int(lens_np.max()) + 3) // 4 * 4, 4)
+            lens_t = torch.tensor(lens_np, dtype=torch.int32, device=DEV); args = dict(lens=lens_t)
+        x = make_scores(rng, g, n_rows, ld, kind)
+        topk = torch.full((n_rows, k_top), -7, dtype=torch.int32, device=DEV)
+        idxc.topk_rows(x, k_top, topk, **args)
+        idxc.poll_device_status()
+        bad = rows_not_exact(x, topk, lens_t.long(), k_top)
+        assert not bool(bad.any()), f"case {i} {kind} mode {mode} rows {n_rows} ld {ld} k {k_top}: rows {torch.nonzero(bad).flatten()[:5].tolist()}"
+        if i % 50 == 0 and int(lens_t.max()) > 0:
+            # the checker itself: one spoiled entry must be reported, for its row only
+            r = int(torch.argmax(lens_t))
+            spoiled = topk.clone()
+            spoiled[r, 0] = -1
+            bad = rows_not_exact(x, spoiled, lens_t.long(), k_top)
+            assert bool(bad[r]) and int(bad.sum()) == 1
+        del x, topk
