@@ -1,4 +1,4 @@
-"""Seeded random shapes through the prefill and decode entry points: every accepted (H_I, d_I, dtype), ragged lengths,
+"""Seeded random shapes through every device entry point. Prefill and decode: every accepted (H_I, d_I, dtype), ragged lengths,
 query chunks against a longer K, workspaces that force chunking, the streaming top-k, empty sequences, unaligned cache
 offsets. Each case is checked against the FP64 oracle on sampled rows and against the GPU's own scores (exact top-k with
 the lowest-index tie rule); the score-less and streaming paths must give the ordinary path's indices."""
@@ -7,6 +7,8 @@ import pytest
 import torch
 
 import oracle
+from oracle import distill as odist
+from oracle import pattern as opat
 from paper_2603_12201_b200 import binding as idxc
 from paper_2603_12201_b200 import synth
 from tests.util import RTOL_BF16, RTOL_FP8, assert_scores_close, assert_topk_valid, codes, f32
@@ -240,3 +242,87 @@ def test_topk_rows_adversarial_distributions():
             bad = rows_not_exact(x, spoiled, lens_t.long(), k_top)
             assert bool(bad[r]) and int(bad.sum()) == 1
         del x, topk
+
+
+def quant_case(rng, i):
+    n = int(rng.choice([1, rng.integers(1, 50), rng.integers(50, 3000)]))
+    shape = [(128,), (64,), (256,), (64, 128), (16, 64), (8, 40), (8,), (32, 128), (576,), (24,)][rng.integers(10)]
+    desc = f"quant n={n} shape={shape}"
+    g = torch.Generator().manual_seed(i)
+    mag = torch.exp(torch.randn(n, generator=g) * float(rng.choice([0.1, 3.0, 8.0])))
+    x = (torch.randn((n,) + shape, generator=g) * mag[(...,) + (None,) * len(shape)]).to(torch.bfloat16)
+    if rng.random() < 0.3:
+        x[rng.integers(n)] = 0
+    if rng.random() < 0.3:
+        x[torch.rand(x.shape, generator=g) < 0.5] = 0
+    xd = x.to(DEV)
+    codes_out = torch.full((n,) + shape, 0x55, dtype=torch.uint8, device=DEV)
+    scale_out = torch.full((n,), -1.0, device=DEV)
+    idxc.quantize_e4m3(xd, codes_out, scale_out)
+    o_codes, o_scale = oracle.quantize_e4m3(codes(x))
+    g_codes = codes_out.cpu().numpy()
+    assert np.array_equal(scale_out.cpu().numpy(), o_scale), desc + " scales"
+    nz = (o_codes & 0x7F) != 0
+    assert np.array_equal(g_codes & 0x7F, o_codes & 0x7F) and np.array_equal(g_codes[nz], o_codes[nz]), desc + " codes"
+    return desc
+
+
+def overlap_case(rng, i):
+    n_layers = int(rng.integers(2, 7)); n_rows = int(rng.choice([1, rng.integers(1, 100), rng.integers(100, 3000)]))
+    k_top = int(rng.choice([1, rng.integers(1, 64), rng.integers(64, 2049)])); n_keys = int(rng.integers(k_top, 4 * k_top + 50))
+    desc = f"overlap layers={n_layers} rows={n_rows} k={k_top} keys={n_keys}"
+    tops = []
+    for l in range(n_layers):
+        key = torch.rand((n_rows, n_keys), device=DEV)
+        idx = torch.topk(key, k_top, dim=1).indices.sort(dim=1).values.int()
+        # ragged valid counts: -1 tails
+        valid = torch.randint(0, k_top + 1, (n_rows,), device=DEV)
+        if rng.random() < 0.5:
+            idx = torch.where(torch.arange(k_top, device=DEV)[None, :] < valid[:, None], idx, torch.full_like(idx, -1))
+        tops.append(idx.contiguous())
+    host = [t.cpu().numpy() for t in tops]
+    mean = idxc.topk_overlap(tops).cpu().numpy()
+    pairs = [(a, b) for a in range(n_layers) for b in range(a + 1, n_layers)]
+    for p, (a, b) in enumerate(pairs):
+        want = opat.overlap(host[a], host[b])
+        assert abs(mean[p] - want) <= 1e-9 or (np.isnan(want) and np.isnan(mean[p])), f"{desc} pair {a},{b}: {mean[p]} vs {want}"
+    a, b = int(rng.integers(n_layers)), int(rng.integers(n_layers))
+    m1, rows = idxc.topk_overlap(tops, pairs=[(a, b)], want_rows=True)
+    want_rows = opat.overlap_rows(host[a], host[b])
+    assert np.allclose(rows.cpu().numpy(), want_rows, atol=1e-6, equal_nan=True), desc + " rows"
+    return desc
+
+
+def distill_case(rng, i):
+    L = int(rng.choice([1, rng.integers(1, 100), rng.integers(100, 1500)])); n_t = int(rng.integers(1, 8))
+    first = int(rng.integers(1, 50)); step = int(rng.integers(0, 2))
+    ld = (first + step * (L - 1) + 3) // 4 * 4
+    desc = f"distill L={L} targets={n_t} first={first} step={step} ld={ld}"
+    gen = torch.Generator().manual_seed(i)
+    scores = (torch.randn((L, ld), generator=gen) * float(rng.choice([0.1, 1.0, 10.0]))).to(DEV).contiguous()
+    lens = first + step * torch.arange(L)
+    mask = (torch.arange(ld)[None, :] < lens[:, None]).float()
+    targets = []
+    for j in range(n_t):
+        p = torch.rand((L, ld), generator=gen) * mask
+        if rng.random() < 0.5:
+            p = p * (torch.rand((L, ld), generator=gen) < 0.5).float()
+            p[:, 0] += 1e-3 * mask[:, 0]
+        p = p / p.sum(dim=1, keepdim=True).clamp_min(1e-30)
+        targets.append(p.to(DEV).contiguous())
+    loss, rows = idxc.distill_kl(scores, targets, first_len=first, len_step=step, want_rows=True)
+    want, want_rows = odist.multi_layer_loss(scores.cpu().numpy(), [t.cpu().numpy() for t in targets], first_len=first, len_step=step)
+    assert abs(loss.item() - want) <= 2e-5 * abs(want) + 1e-7, f"{desc}: {loss.item()} vs {want}"
+    assert np.allclose(rows.cpu().numpy(), want_rows, rtol=1e-4, atol=1e-5), desc + " rows"
+    return desc
+
+
+@pytest.mark.parametrize("seed", [5])
+def test_random_shapes_of_the_quantiser_the_overlap_and_the_distillation_loss(seed):
+    """Seeded random cases of the three side entry points against their oracles: the quantiser bit for bit (token
+    magnitudes over many octaves, zero tokens, half-zero rows, every row width the tests use), the overlap ratios
+    (2..6 layers, ragged -1 tails), the distillation loss (1..7 targets, sparse targets, fixed or growing lengths)."""
+    rng = np.random.default_rng(seed)
+    fns = [quant_case, overlap_case, distill_case]
+    for i in range(1, 121):
+        fns[i % 3](rng, 1000 * seed + i)

@@ -228,3 +228,47 @@ def test_few_tiles_per_cta_after_unrelated_calls():
         out, lse = binding.sparse_attention(inp.q, inp.kv, topk, D_V, 0.06, kv_base=base)
         assert torch.equal(out, ref) and torch.equal(lse, ref_lse)
     binding.poll_device_status()
+
+
+@pytest.mark.parametrize("seed", [3, 4])
+def test_random_shapes(seed):
+    """Seeded random shapes: 1..700 queries (whole and split over CTAs), 1..128 heads, 1..5000 selected slots, caches of
+    1..20000 rows, per-query base offsets, holes anywhere, ragged tails, out-of-range entries, flat to peaked softmax;
+    sampled queries against the oracle, and a second call must reproduce the first bit for bit."""
+    rng = np.random.default_rng(seed)
+    for i in range(1, 101):
+        n_q = int(rng.choice([rng.integers(1, 8), rng.integers(8, 64), rng.integers(64, 160), rng.integers(160, 700)]))
+        n_kv = int(rng.choice([rng.integers(1, 100), rng.integers(100, 3000), rng.integers(3000, 20000)]))
+        h = int(rng.choice([1, 16, 64, 128, rng.integers(1, 129)]))
+        k_top = int(rng.choice([rng.integers(1, 64), 64, rng.integers(64, 600), 2048, rng.integers(600, 5000)]))
+        scale = float(rng.choice([1.0 / 24, 0.02, 0.1, 0.3]))
+        desc = f"n_q={n_q} n_kv={n_kv} h={h} k={k_top} scale={scale:.3f}"
+        inp = synth.attention_inputs(n_q, n_kv, h, D_QK, seed=100 * seed + i, device="cuda")
+        g = torch.Generator().manual_seed(1000 * seed + i)
+        use_base = rng.random() < 0.3
+        if use_base:
+            base_np = rng.integers(0, max(1, n_kv // 2), size=n_q)
+            span = n_kv - int(base_np.max())
+            topk = torch.randint(0, max(span, 1), (n_q, k_top), generator=g, dtype=torch.int32)
+            base = torch.as_tensor(base_np, dtype=torch.int64, device="cuda")
+        else:
+            topk = torch.randint(0, n_kv, (n_q, k_top), generator=g, dtype=torch.int32)
+            base = None
+        mode = rng.integers(4)
+        if mode == 1:
+            topk[torch.rand((n_q, k_top), generator=g) < float(rng.random())] = -1
+        elif mode == 2:      # ragged tails like an indexer's output
+            for r in range(n_q):
+                topk[r, int(rng.integers(0, k_top + 1)):] = -1
+        elif mode == 3:      # some out of range entries (skipped)
+            topk[torch.rand((n_q, k_top), generator=g) < 0.1] = n_kv + 5
+        topk = topk.cuda()
+        out, lse = binding.sparse_attention(inp.q, inp.kv, topk, D_V, scale, kv_base=base)
+        binding.poll_device_status()
+        n_rows = min(n_q, max(1, int(3e8 // (h * k_top * D_QK))))
+        rows = np.unique(np.concatenate([[0, n_q - 1], rng.integers(0, n_q, size=n_rows)]))
+        o_out, o_lse = osa.sparse_attention(codes(inp.q), codes(inp.kv), topk.cpu().numpy(), D_V, scale,
+                                            kv_base=None if base is None else base.cpu().numpy(), rows=rows)
+        _check(out, lse, o_out, o_lse, rows, f"seed {seed} case {i}: {desc} mode={mode} base={use_base}")
+        out2, lse2 = binding.sparse_attention(inp.q, inp.kv, topk, D_V, scale, kv_base=base)
+        assert torch.equal(out, out2) and torch.equal(lse, lse2), f"seed {seed} case {i}: {desc}: second call differs"
