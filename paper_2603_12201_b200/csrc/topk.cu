@@ -34,6 +34,7 @@ namespace {
 constexpr int TK_BINS = 1024;
 constexpr int TK_MAP_MAX_BYTES = 128 * 1024;      // rows up to 524288 scores use the map
 constexpr int TK_SMALL = 128;                     // scores ranked by direct comparison at most
+constexpr int TK_PREFETCH = 16384;                // bytes per L2 prefetch request of a row segment
 
 struct alignas(16) TopkRowSmem : SampleSmem {
     uint32_t part_a[32], part_c[32];
@@ -57,6 +58,8 @@ topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int64_t n_rows, i
     uint8_t* sel_bytes = reinterpret_cast<uint8_t*>(sel_map);
     uint32_t* cand_fb = sel_map + map_scores / 16;               // a candidate's fine bin ...
     uint32_t* cand_idx = cand_fb + CAP;                          // ... and position
+    int32_t* stage = reinterpret_cast<int32_t*>(cand_fb);        // the selected indices of a row before they are stored (the candidates are done with by then)
+    static_assert(2 * CAP >= 2048, "the staging area holds k_top indices");
     int slot = 0;
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const uint32_t k = static_cast<uint32_t>(k_top);
@@ -81,6 +84,17 @@ topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int64_t n_rows, i
         const int seg = (((n + WARPS - 1) / WARPS) + 127) & ~127;
         const int seg_begin = wid * seg < n ? wid * seg : n;
         const int seg_end = seg_begin + seg < n ? seg_begin + seg : n;
+        // ask the L2 for this warp's segment now: the sweep comes after the sample, its histogram and two scans, and
+        // then finds its scores on the chip (5 % of the kernel's time on 32K-score rows)
+        {
+            const int seg_bytes = ((seg_end - seg_begin) * 4) & ~15;
+            const char* seg_ptr = reinterpret_cast<const char*>(src + seg_begin);
+            for (int off = lane * TK_PREFETCH; off < seg_bytes; off += 32 * TK_PREFETCH) {
+                const int left = seg_bytes - off;
+                const uint32_t bytes = static_cast<uint32_t>(left < TK_PREFETCH ? left : TK_PREFETCH);
+                asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(seg_ptr + off), "r"(bytes) : "memory");
+            }
+        }
         // ---- the sample and the two pivot scores around the k-th largest (the same code serves the cluster kernel)
         __syncthreads();   // earlier readers of sm, rs and the map are done
         if (threadIdx.x == 0) { rs.cand_count = 0u; rs.small_count = 0u; }
@@ -219,9 +233,19 @@ topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int64_t n_rows, i
                 while (m) {
                     const int b = __ffs(m) - 1;
                     m &= m - 1;
-                    if (pos < k) out_row[pos] = idx0 + b;
+                    if (pos < k) stage[pos] = idx0 + b;
                     ++pos;
                 }
+            }
+            // the lanes' runs interleave in shared memory; the row leaves in whole 16-byte pieces (a lane's own stores
+            // would touch one 32-byte sector per index)
+            __syncthreads();
+            if ((k_top & 3) == 0 && (reinterpret_cast<uintptr_t>(out_row) & 15) == 0) {
+                const int4* s4 = reinterpret_cast<const int4*>(stage);
+                int4* o4 = reinterpret_cast<int4*>(out_row);
+                for (int j = threadIdx.x; j < (k_top >> 2); j += THREADS) o4[j] = s4[j];
+            } else {
+                for (int j = threadIdx.x; j < k_top; j += THREADS) out_row[j] = stage[j];
             }
         }
     }
