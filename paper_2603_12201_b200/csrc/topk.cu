@@ -34,7 +34,7 @@ namespace {
 constexpr int TK_BINS = 1024;
 constexpr int TK_MAP_MAX_BYTES = 128 * 1024;      // rows up to 524288 scores use the map
 constexpr int TK_SMALL = 128;                     // scores ranked by direct comparison at most
-constexpr int TK_PREFETCH = 16384;                // bytes per L2 prefetch request of a row segment
+constexpr int TK_PREFETCH = 16384;                // bytes of a warp's segment asked for ahead of the sweep
 
 struct alignas(16) TopkRowSmem : SampleSmem {
     uint32_t part_a[32], part_c[32];
@@ -84,16 +84,14 @@ topk_rows_kernel(const float* __restrict__ scores, int64_t ld, int64_t n_rows, i
         const int seg = (((n + WARPS - 1) / WARPS) + 127) & ~127;
         const int seg_begin = wid * seg < n ? wid * seg : n;
         const int seg_end = seg_begin + seg < n ? seg_begin + seg : n;
-        // ask the L2 for this warp's segment now: the sweep comes after the sample, its histogram and two scans, and
-        // then finds its scores on the chip (5 % of the kernel's time on 32K-score rows)
+        // ask the L2 for the head of this warp's segment now: the sweep comes after the sample, its histogram and two
+        // scans, and then finds its first scores on the chip (5 % of the kernel's time on rows of 12K..40K scores, which
+        // this covers whole; asking for all of a longer row, at once or as the sweep advances, measured slower: the rows
+        // of the resident blocks then no longer fit the L2 together)
         {
             const int seg_bytes = ((seg_end - seg_begin) * 4) & ~15;
-            const char* seg_ptr = reinterpret_cast<const char*>(src + seg_begin);
-            for (int off = lane * TK_PREFETCH; off < seg_bytes; off += 32 * TK_PREFETCH) {
-                const int left = seg_bytes - off;
-                const uint32_t bytes = static_cast<uint32_t>(left < TK_PREFETCH ? left : TK_PREFETCH);
-                asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(seg_ptr + off), "r"(bytes) : "memory");
-            }
+            if (lane == 0 && seg_bytes > 0)
+                asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src + seg_begin), "r"(static_cast<uint32_t>(seg_bytes < TK_PREFETCH ? seg_bytes : TK_PREFETCH)) : "memory");
         }
         // ---- the sample and the two pivot scores around the k-th largest (the same code serves the cluster kernel)
         __syncthreads();   // earlier readers of sm, rs and the map are done

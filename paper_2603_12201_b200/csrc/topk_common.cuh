@@ -381,35 +381,52 @@ __device__ __forceinline__ Pivots sample_pivots(SM& sm, RS& rs, const float* __r
     S = S < U ? U : S;
     S = S > seg_blocks ? seg_blocks : S;
     const int stride = (seg_blocks / S) << 7;
-    // calls f(float4, index of its first score) for the lane's part of every sample block
-    auto for_sample = [&](auto f) {
-        for (int j0 = 0; j0 < S; j0 += U) {
+    // The lane's part of sample block j: four scores from index base on (base >= seg_end: none)
+    auto sample_base = [&](int j) -> int { return j < S ? seg_begin + j * stride + 4 * lane : seg_end; };
+    auto sample_load = [&](int base) -> float4 {
+        return base < seg_end ? __ldg(reinterpret_cast<const float4*>(src + base)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    };
+    // calls f(float4, index of its first score) for the lane's part of every sample block after the first U
+    auto for_rest = [&](auto f) {
+        for (int j0 = U; j0 < S; j0 += U) {
             float4 x[U];
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int base = seg_begin + (j0 + u) * stride + 4 * lane;
-                x[u] = (j0 + u < S && base < seg_end) ? __ldg(reinterpret_cast<const float4*>(src + base))
-                                                     : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
+            for (int u = 0; u < U; ++u) x[u] = sample_load(sample_base(j0 + u));
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                const int base = seg_begin + (j0 + u) * stride + 4 * lane;
-                if (j0 + u < S && base < seg_end) f(x[u], base);
+                const int base = sample_base(j0 + u);
+                if (base < seg_end) f(x[u], base);
             }
         }
     };
+    // the first U blocks (all of the sample unless the row is longer than 32768 scores per 16 blocks of the block's
+    // warps) stay in registers for both passes
+    float4 x0[U];
+    int base0[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) { base0[u] = sample_base(u); x0[u] = sample_load(base0[u]); }
     Pivots pv;
     // ---- mean and spread
     zero_hist<THREADS>(sm, BINS);
     {
         float s1 = 0.f, s2 = 0.f;
         uint32_t m = 0;
-        for_sample([&](const float4& x, int base) {
-            const float xs[4] = {x.x, x.y, x.z, x.w};
+        auto add = [&](const float4& x, int base) {
+            if (base + 3 < n) {                                   // all but the last load of a row
+                s1 += (x.x + x.y) + (x.z + x.w);
+                s2 = fmaf(x.x, x.x, fmaf(x.y, x.y, fmaf(x.z, x.z, fmaf(x.w, x.w, s2))));
+                m += 4u;
+            } else {
+                const float xs[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
-            for (int e = 0; e < 4; ++e)
-                if (base + e < n) { s1 += xs[e]; s2 = fmaf(xs[e], xs[e], s2); ++m; }
-        });
+                for (int e = 0; e < 4; ++e)
+                    if (base + e < n) { s1 += xs[e]; s2 = fmaf(xs[e], xs[e], s2); ++m; }
+            }
+        };
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (base0[u] < seg_end) add(x0[u], base0[u]);
+        for_rest(add);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             s1 += __shfl_xor_sync(0xFFFFFFFFu, s1, o);
@@ -439,16 +456,22 @@ __device__ __forceinline__ Pivots sample_pivots(SM& sm, RS& rs, const float* __r
     }
     if (!pv.usable) return pv;                                // the same for every thread
     // ---- histogram of the sample
-    for_sample([&](const float4& x, int base) {
-        const float xs[4] = {x.x, x.y, x.z, x.w};
+    {
+        auto count = [&](const float4& x, int base) {
+            const float xs[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            if (base + e < n) {
-                const int b = __float2int_rd(__fmaf_rn(xs[e], pv.scale, pv.offset));     // NaN -> 0; saturates
-                atomicAdd(&sm.hist[min(max(b, 0), BINS - 1)], 1u);
+            for (int e = 0; e < 4; ++e) {
+                if (base + e < n) {
+                    const int b = __float2int_rd(__fmaf_rn(xs[e], pv.scale, pv.offset));     // NaN -> 0; saturates
+                    atomicAdd(&sm.hist[min(max(b, 0), BINS - 1)], 1u);
+                }
             }
-        }
-    });
+        };
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (base0[u] < seg_end) count(x0[u], base0[u]);
+        for_rest(count);
+    }
     __syncthreads();
     // ---- rank of the k-th largest of the row inside the sample, and its standard deviation under sampling without replacement
     const float mf = static_cast<float>(m_sample), nf = static_cast<float>(n);
