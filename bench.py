@@ -943,7 +943,10 @@ def main():
                    "on the fractions of the peaks MEASURED on this box (cuBLAS bf16 GEMM, copy bandwidth); frac_of_nominal gives the "
                    "same against the data-sheet figures (2250 TFLOP/s, 7.7 TB/s)",
         "algorithmic_flops_per_launch": flops,
-        "topk_kernel": {"ms_per_launch": topk_ms, "bound": "hbm", "achieved": topk_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+        "topk_kernel": {"ms_per_launch": topk_ms, "launches": max(1, launches // K - 1),
+                        "note": "one idxc_topk_rows call; a long prefill's rows are cut by length into up to three launches of "
+                                "topk_rows_kernel instances, timed and counted together (traffic: their sum)",
+                        "bound": "hbm", "achieved": topk_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                         "frac": topk_gbs / peaks["hbm_gbs"], "frac_of_nominal": topk_gbs / NOMINAL["hbm_gbs"],
                         "algorithmic_bytes": topk_bytes, "traffic": dram_traffic("topk_rows_kernel", case)},
     }
