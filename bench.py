@@ -236,6 +236,35 @@ def time_cfg1(idxc, synth, dev, reps=200):
             "note": "latency-bound: 4.3 GFLOP and 10 MB of output per call are about 3 us of roofline work"}
 
 
+def graph_replay_us(step, n_steps, reps=7):
+    """n_steps calls step(0), step(1), ... captured ONCE into a CUDA graph on a side stream and replayed: microseconds per
+    step of the median replay. The library's calls allocate nothing, never synchronise and only enqueue kernels on the
+    caller's stream, so a serving loop can capture its decode step this way; the replay removes the host's launch cost and
+    most of the launch-to-launch gap between the step's kernels."""
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        step(0)
+        with torch.cuda.graph(g, stream=side):
+            for i in range(n_steps):
+                step(i)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    g.replay()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b) * 1e3 / n_steps)
+    del g
+    return statistics.median(ts)
+
+
 def time_decode(idxc, synth, dev, peaks, steps, warmup):
     c = synth.CONFIGS["cfg3"]
     x = synth.decode_inputs(c["B"], c["H"], c["d"], c["len_lo"], c["len_hi"], seed=c["seed"], device=dev)
@@ -269,6 +298,9 @@ def time_decode(idxc, synth, dev, peaks, steps, warmup):
     keys = int(x.lens.sum().item())
     bytes_k = keys * c["d"] * 2
     us_score, us_total = statistics.median(t_score), statistics.median(t_total)
+    us_graph = graph_replay_us(lambda i: idxc.indexer_decode(x.q_step, x.k_cache, x.w, x.k_offsets, x.lens, x.max_len, k_top,
+                                                             topk_out=topk, workspace=ws), 16)
+    idxc.poll_device_status()
     gbs = bytes_k / (us_score * 1e-6) / 1e9
     # the consumer of the step's indices: sparse attention of the B new tokens over their selected cache rows
     # (128 heads, 576/512-column latent rows in a cache with the same row offsets; few queries: rows split over CTAs)
@@ -292,7 +324,9 @@ def time_decode(idxc, synth, dev, peaks, steps, warmup):
                                    "note": "B queries x k_top selected rows; with 32 queries four CTAs share a query and a second kernel merges their results"},
         "workload": f"cfg3: decode B={B} H_I={c['H']} d_I={c['d']} k_top={k_top}, sum(lens)={keys}",
         "us_per_step": us_total, "us_scorer": us_score, "us_topk": us_total - us_score,
-        "timing": "us_per_step: one idxc_indexer_decode call; us_scorer: the scorer kernel alone (scores only); us_topk: the difference",
+        "us_per_step_graph": us_graph,
+        "timing": "us_per_step: one idxc_indexer_decode call; us_scorer: the scorer kernel alone (scores only); us_topk: the difference; "
+                  "us_per_step_graph: 16 such calls captured once into a CUDA graph, per step of the median replay",
         "k_cache_bytes": bytes_k,
         "l2": "766 MB of keys per step exceed the 126 MB L2: every step streams them from HBM",
         "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -300,6 +334,7 @@ def time_decode(idxc, synth, dev, peaks, steps, warmup):
                      "algorithmic_bytes": bytes_k, "kernel": "score_decode_tc_kernel",
                      "of": peaks["source"], "frac_of_nominal": gbs / NOMINAL["hbm_gbs"]},
         "frac_step_vs_hbm": bytes_k / (us_total * 1e-6) / 1e9 / peaks["hbm_gbs"],
+        "frac_step_vs_hbm_graph": bytes_k / (us_graph * 1e-6) / 1e9 / peaks["hbm_gbs"],
     }
 
 
@@ -503,7 +538,15 @@ def time_decode_fp8(idxc, synth, dev, peaks, L, H, d, k_top, seed, decode_B, fir
     us = median_event_ms(ev_step[6:]) * 1e3
     us_sc = median_event_ms(ev_score[6:]) * 1e3
     nbytes = decode_B * L * (d + 4)
+
+    def graph_step(i):
+        x = sets[i & 1]
+        idxc.indexer_decode(x.q_step, x.k_cache, x.w, x.k_offsets, x.lens, L, k_top, x.q_scale, x.k_scale, topk_out=dtop, workspace=dws)
+    us_graph = graph_replay_us(graph_step, 24)          # the same alternation of the two cache sets, captured once
+    idxc.poll_device_status()
     return {"B": decode_B, "us_per_step": us, "us_scorer": us_sc, "us_topk": us - us_sc, "bytes": nbytes,
+            "us_per_step_graph": us_graph, "frac_of_hbm_graph": nbytes / (us_graph * 1e-6) / 1e9 / peaks["hbm_gbs"],
+            "graph": "24 calls captured once into a CUDA graph, per step of the median replay",
             "frac_of_hbm": nbytes / (us * 1e-6) / 1e9 / peaks["hbm_gbs"],
             "scorer_frac_of_hbm": nbytes / (us_sc * 1e-6) / 1e9 / peaks["hbm_gbs"],
             "l2": f"two cache sets of {nbytes >> 20} MiB alternate between steps ({2 * nbytes >> 20} MiB > 126 MB L2): every step streams its keys from HBM"}
@@ -1086,7 +1129,8 @@ def main():
                 "cfg2": {"gpairs_per_s": value, "ms_per_step": ms_per_step, "scorer_frac_of_bf16_peak": roofline["frac"],
                          "topk_frac_of_hbm": roofline["topk_kernel"]["frac"],
                          "streaming_topk_ms": line["stream_topk"]["ms_streaming"], "streaming_topk_identical": line["stream_topk"]["indices_identical"]},
-                "cfg3": {"us_per_step": dc["us_per_step"], "scorer_frac_of_hbm": dc["roofline"]["frac"], "step_frac_of_hbm": dc["frac_step_vs_hbm"]},
+                "cfg3": {"us_per_step": dc["us_per_step"], "scorer_frac_of_hbm": dc["roofline"]["frac"], "step_frac_of_hbm": dc["frac_step_vs_hbm"],
+                         "us_per_step_graph": dc["us_per_step_graph"], "step_frac_of_hbm_graph": dc["frac_step_vs_hbm_graph"]},
                 "cfg4": {"workload": sc["workload"], "ms_scheduled": sc["ms_scheduled"], "ms_all_full": sc["ms_all_full"], "ratio": sc["ratio"],
                          "gpairs_per_s_full_layers": sc["gpairs_per_s_full_layers"], "checks": sc["checks"]},
                 "cfg5": {"workload": f8["workload"], "ms_per_full_layer": f8["ms_per_layer"], "gpairs_per_s": f8["gpairs_per_s"],
@@ -1094,7 +1138,8 @@ def main():
                          "scorer_frac_of_2x_bf16_sustained": f8["roofline_tensor"]["frac_of_sustained"],
                          "scorer_frac_of_tmem_readout": f8.get("roofline_readout", {}).get("frac"),
                          "schedule_ratio": f8["schedule"]["ratio"], "decode_B8_us": f8["decode"]["us_per_step"],
-                         "decode_frac_of_hbm": f8["decode"]["frac_of_hbm"]},
+                         "decode_frac_of_hbm": f8["decode"]["frac_of_hbm"], "decode_B8_us_graph": f8["decode"]["us_per_step_graph"],
+                         "decode_frac_of_hbm_graph": f8["decode"]["frac_of_hbm_graph"]},
             }
             line["roofline"]["by_config"] = by_config
             line["summary"] = by_config
