@@ -513,6 +513,34 @@ def test_quantize_e4m3_bit_exact(n, shape):
     assert np.array_equal(g_codes & 0x7F, o_codes & 0x7F) and np.array_equal(g_codes[nz], o_codes[nz])
 
 
+def test_quantize_e4m3_every_value_under_many_row_maxima():
+    """The kernel divides by the row's scale through a reciprocal and one residual step instead of a division per
+    element. Here rows whose largest entry is a chosen bf16 value hold EVERY bf16 value not above it, both signs: the
+    codes must be the oracle's for all of them (edge maxima: subnormal, smallest normal, around the 1e-12 floor, powers
+    of two, the largest finite value; plus 200 seeded ones)."""
+    g = torch.Generator().manual_seed(5)
+    edge = [1, 2, 0x7F, 0x80, 0x81, 0x2B8C, 0x2B8D, 0x2B8E, 0x3F80, 0x3F81, 0x3FFF, 0x4000, 0x43E0, 0x7F00, 0x7F7F]
+    maxima = edge + torch.randint(1, 0x7F80, (200,), generator=g).tolist()
+    rows = []
+    for a in maxima:
+        mag = torch.arange(0, a + 1, dtype=torch.int32)
+        bits = torch.cat([mag, mag | 0x8000])
+        pad = (-bits.numel()) % 127
+        bits = torch.cat([bits, torch.zeros(pad, dtype=torch.int32)]).reshape(-1, 127)
+        rows.append(torch.cat([torch.full((bits.shape[0], 1), a, dtype=torch.int32), bits], dim=1))
+    bits = torch.cat(rows).to(torch.uint16)
+    x = bits.view(torch.bfloat16)
+    n = x.shape[0]
+    codes_out = torch.full((n, 128), 0x55, dtype=torch.uint8, device=DEV)
+    scale_out = torch.full((n,), -1.0, device=DEV)
+    idxc.quantize_e4m3(x.to(DEV), codes_out, scale_out)
+    o_codes, o_scale = oracle.quantize_e4m3(codes(x))
+    g_codes = codes_out.cpu().numpy()
+    assert np.array_equal(scale_out.cpu().numpy(), o_scale)
+    nz = (o_codes & 0x7F) != 0
+    assert np.array_equal(g_codes & 0x7F, o_codes & 0x7F) and np.array_equal(g_codes[nz], o_codes[nz])
+
+
 def test_quantize_e4m3_appends_to_a_k_cache_that_the_indexer_reads():
     # new keys of three sequences are appended at the end of their cache rows, then one decode step reads the cache
     B, H, d, k_top = 3, 64, 128, 32
