@@ -594,6 +594,42 @@ def test_topk_overlap_matches_oracle():
     assert idxc.topk_overlap([tops[0], tops[0]]).item() == 1.0          # identical tensors overlap fully
 
 
+@pytest.mark.parametrize("k_top,max_index", [(2048, 16384), (2048, 131072), (2048, 400000), (37, 5000), (37, 300000), (512, 131073)])
+def test_topk_overlap_near_and_far_rows_mixed(k_top, max_index):
+    """Rows whose largest index is below 131072 are intersected through a bitmap, the others by merging; here both kinds
+    alternate inside one launch (so a merged row must leave the bitmap clean), with padded, empty and identical rows."""
+    from oracle import pattern as opat
+    rows = 97
+    g = torch.Generator().manual_seed(k_top + max_index)
+
+    def tensor(shift):
+        t = torch.full((rows, k_top), -1, dtype=torch.int32)
+        for r in range(rows):
+            hi = max_index if r % 3 else min(max_index, 9000)             # every third row stays near
+            n = k_top if r % 5 else int(torch.randint(0, k_top + 1, (1,), generator=g))
+            n = min(n, hi)
+            if r == 11:
+                n = 0                                                     # an empty row
+            pick = torch.randperm(hi, generator=g)[:n]
+            if shift and r % 2:
+                pick = torch.cat([pick[: n // 2], torch.randperm(hi, generator=g)[: n - n // 2]]).unique()
+            vals = torch.sort(pick.unique()).values
+            t[r, : vals.numel()] = vals.to(torch.int32)
+        return t
+    a, b = tensor(False), tensor(True)
+    b[20] = a[20]                                                         # an identical row
+    tops = [a.to(DEV), b.to(DEV)]
+    for pair, (x, y) in (((0, 1), (a, b)), ((1, 0), (b, a))):
+        mean, per_row = idxc.topk_overlap(tops, pairs=[pair], want_rows=True)
+        want = opat.overlap_rows(x.numpy(), y.numpy())
+        assert np.allclose(per_row.cpu().numpy(), want, atol=1e-6)
+        assert mean.item() == pytest.approx(float(np.mean(want)), abs=1e-9)
+    both = idxc.topk_overlap(tops, pairs=[(0, 1), (1, 0), (0, 0)]).cpu().numpy()
+    assert both[0] == pytest.approx(opat.overlap(a.numpy(), b.numpy()), abs=1e-9)
+    assert both[1] == pytest.approx(opat.overlap(b.numpy(), a.numpy()), abs=1e-9)
+    assert both[2] == pytest.approx(opat.overlap(a.numpy(), a.numpy()), abs=1e-9)
+
+
 # ------------------------------------------------------------------------------ multi-layer distillation loss (Eq. 1)
 def test_distill_kl_matches_oracle():
     from oracle import distill as odist
