@@ -231,7 +231,10 @@ def time_cfg1(idxc, synth, dev, reps=200):
     torch.cuda.synchronize()
     us_stream = a.elapsed_time(b) * 1e3 / reps
     pairs = causal_pairs(L)
+    us_graph = graph_replay_us(lambda i: call(), 50)
+    idxc.poll_device_status()
     return {"workload": workload_name("cfg1", c) + ", scores + indices", "us_per_call": us, "us_per_call_back_to_back": us_stream,
+            "us_per_call_graph": us_graph,
             "gpairs_per_s": pairs / (us_stream * 1e-6) / 1e9, "kernels_per_call": 2,
             "note": "latency-bound: 4.3 GFLOP and 10 MB of output per call are about 3 us of roofline work"}
 
@@ -853,6 +856,7 @@ def main():
     ap.add_argument("--only-sparse-attention", action="store_true", help="run only the sparse-attention section (profiling)")
     ap.add_argument("--only-layer-loop", action="store_true", help="run only the indexer + attention layer loop section")
     ap.add_argument("--only-fp8", action="store_true", help="run only the FP8 chunked-prefill section (profiling; --L sets the length)")
+    ap.add_argument("--only-tools", action="store_true", help="run only the distillation-loss, overlap and quantiser sections (profiling)")
     ap.add_argument("--sa-queries", type=int, default=8192, help="queries of the sparse-attention section")
     args = ap.parse_args()
     if args.warmup < 3:
@@ -917,6 +921,11 @@ def main():
         print(json.dumps({"tmem_readout": ro,
                           "fp8_chunked": section(time_fp8_chunked, idxc, synth, dev, peaks, L5, min(c5["chunk"], L5), c5["H"], c5["d"],
                                                  c5["k_top"], c5["seed"], c5["decode_B"], 8 if args.quick else c5["N"], c5["every"], ro)}), flush=True)
+        return
+    if args.only_tools:
+        print(json.dumps({"distill_kl": section(time_distill, idxc, dev, peaks, 16384, 2),
+                          "topk_overlap": section(time_overlap, idxc, dev, peaks, 8192, c5["k_top"], 6),
+                          "quantize_e4m3": section(time_quantize, idxc, dev, peaks, 32768, c5["H"], c5["d"])}), flush=True)
         return
     if args.only_sparse_attention:
         print(json.dumps({"sparse_attention": section(time_sparse_attention, idxc, synth, dev, peaks, args.L or 32768, args.sa_queries, 2048,
@@ -1125,7 +1134,8 @@ def main():
             # the five workloads in one place, inside the roofline block and again at the very end of the line
             f8, dc, sc = line["fp8_chunked"], line["decode"], line["schedule"]
             by_config = {
-                "cfg1": {"us_per_call": line["cfg1"]["us_per_call"], "us_back_to_back": line["cfg1"]["us_per_call_back_to_back"]},
+                "cfg1": {"us_per_call": line["cfg1"]["us_per_call"], "us_back_to_back": line["cfg1"]["us_per_call_back_to_back"],
+                         "us_graph": line["cfg1"]["us_per_call_graph"]},
                 "cfg2": {"gpairs_per_s": value, "ms_per_step": ms_per_step, "scorer_frac_of_bf16_peak": roofline["frac"],
                          "topk_frac_of_hbm": roofline["topk_kernel"]["frac"],
                          "streaming_topk_ms": line["stream_topk"]["ms_streaming"], "streaming_topk_identical": line["stream_topk"]["indices_identical"]},
