@@ -320,9 +320,12 @@ def time_decode(idxc, synth, dev, peaks, steps, warmup):
     torch.cuda.synchronize()
     idxc.poll_device_status()
     us_attn = ea.elapsed_time(eb) * 1e3 / 10
+    us_attn_graph = graph_replay_us(lambda i: idxc.sparse_attention(att.q, att.kv, topk, 512, 1.0 / 24.0, kv_base=x.k_offsets, out=a_out,
+                                                                    workspace=a_ws, want_lse=False), 10)
+    idxc.poll_device_status()
     attn_tf = 2.0 * 128 * (576 + 512) * B * k_top / (us_attn * 1e-6) / 1e12
     return {
-        "sparse_attention_after": {"us": us_attn, "tflops_useful": attn_tf, "frac_of_bf16_peak": attn_tf / peaks["bf16_tflops"],
+        "sparse_attention_after": {"us": us_attn, "us_graph": us_attn_graph, "tflops_useful": attn_tf, "frac_of_bf16_peak": attn_tf / peaks["bf16_tflops"],
                                    "gathered_bytes": B * k_top * (576 + 256) * 2,
                                    "note": "B queries x k_top selected rows; with 32 queries four CTAs share a query and a second kernel merges their results"},
         "workload": f"cfg3: decode B={B} H_I={c['H']} d_I={c['d']} k_top={k_top}, sum(lens)={keys}",
