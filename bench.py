@@ -39,7 +39,7 @@ METRIC = "indexer+top-k Gpairs/s (prefill)"
 UNIT = "Gpairs/s"
 
 # Nominal chip figures (dense, no sparsity), for the second fraction of every roofline block.
-NOMINAL = {"bf16_tflops": 2250.0, "fp8_tflops": 4500.0, "hbm_gbs": 7700.0}
+NOMINAL = {"bf16_tflops": 2250.0, "fp8_tflops": 4500.0, "hbm_gbs": 7700.0, "sm_max_mhz": 1965.0}
 
 
 def dram_traffic(kernel: str, case: str):
@@ -499,8 +499,29 @@ def time_tmem_readout(idxc, dev, accumulators_per_warp=4096):
     torch.cuda.synchronize()
     idxc.poll_device_status()
     ms = min(a.elapsed_time(b) for a, b in evs)
-    return {"bytes_per_launch": nbytes, "ms": ms, "tbytes_per_s": nbytes / (ms * 1e-3) / 1e12,
-            "what": "fp32 accumulator bytes read out of tensor memory per second over all SMs, the scorer's load pattern alone"}
+    out = {"bytes_per_launch": nbytes, "ms": ms, "tbytes_per_s": nbytes / (ms * 1e-3) / 1e12,
+           "what": "fp32 accumulator bytes read out of tensor memory per second over all SMs, the scorer's load pattern alone"}
+    # the same loads while a ninth warp keeps the tensor pipe filling the two accumulators with the scorer's MMAs
+    counters = torch.zeros(2, dtype=torch.int64, device=dev)
+    for name, fp8 in (("under_fp8_mma", True), ("under_bf16_mma", False)):
+        best = None
+        for _ in range(4):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            nb = idxc.selftest_tmem_readout_under_mma(accumulators_per_warp, fp8, counters)
+            b.record()
+            torch.cuda.synchronize()
+            t = a.elapsed_time(b)
+            if best is None or t < best[0]:
+                best = (t, int(counters[0].item()), int(counters[1].item()))
+        idxc.poll_device_status()
+        t, fills, cycles = best
+        out[name] = {"ms": t, "tbytes_per_s": nb / (t * 1e-3) / 1e12, "accumulator_fills": fills,
+                     "mma_tflops": fills * 2.0 * 128 * 256 * 128 / (t * 1e-3) / 1e12,
+                     "reader_cycles_per_accumulator": cycles / accumulators_per_warp}
+    out["under_mma_note"] = ("readers and MMAs run unordered beside each other on every SM; mma_tflops counts the fills completed while the "
+                             "readers ran (2 x 128 x 256 x 128 flops each) over the launch time")
+    return out
 
 
 def time_decode_fp8(idxc, synth, dev, peaks, L, H, d, k_top, seed, decode_B, first_k=None, first_k_scale=None):
@@ -626,6 +647,19 @@ def time_fp8_chunked(idxc, synth, dev, peaks, L, chunk, H, d, k_top, seed, decod
                                    "frac": ach / readout["tbytes_per_s"],
                                    "derivation": f"4 B x H_I = {4 * H} accumulator bytes per causal pair, {acc_bytes:.3e} B per layer, / scorer time; "
                                                  "peak = the same loads alone, measured in this run (tmem_readout section)"}
+        if "under_fp8_mma" in readout:
+            out["roofline_readout"]["peak_under_fp8_mma"] = readout["under_fp8_mma"]["tbytes_per_s"]
+            out["roofline_readout"]["frac_under_fp8_mma"] = ach / readout["under_fp8_mma"]["tbytes_per_s"]
+    # the gate: one min/max instruction per accumulator element on a pipe that issues 16 lanes per clock and scheduler
+    # (measured: a warp's FMNMX every 2.0 cycles per scheduler), 4 schedulers per SM, at the SM clock's maximum
+    props = torch.cuda.get_device_properties(dev)
+    gate_peak = props.multi_processor_count * 4 * 16 * (NOMINAL["sm_max_mhz"] * 1e6) / 1e12          # T elements / s
+    gate_ach = acc_bytes / 4 / (t_sc * 1e-3) / 1e12
+    out["roofline_gate"] = {"bound": "alu", "achieved": gate_ach, "peak": gate_peak, "unit": "T accumulator elements gated per second",
+                            "frac": gate_ach / gate_peak,
+                            "derivation": "ReLU = one min/max per accumulator element; that pipe takes a warp instruction every 2 cycles per scheduler: "
+                                          f"{props.multi_processor_count} SMs x 4 schedulers x 16 lanes x {NOMINAL['sm_max_mhz']} MHz; with e4m3 inputs this equals the tensor time "
+                                          "of the accumulator (512 cycles per 128 x 256), and the epilogue's selects, compares and address arithmetic share the pipe"}
     fp8_peak = measure_fp8_gemm_peak(dev)
     if fp8_peak:
         out["fp8_gemm_peak_measured_here_tflops"] = fp8_peak
@@ -1150,6 +1184,7 @@ def main():
                          "scorer_frac_of_2x_bf16_peak": f8["roofline_tensor"]["frac"],
                          "scorer_frac_of_2x_bf16_sustained": f8["roofline_tensor"]["frac_of_sustained"],
                          "scorer_frac_of_tmem_readout": f8.get("roofline_readout", {}).get("frac"),
+                         "scorer_frac_of_gate_rate": f8["roofline_gate"]["frac"],
                          "schedule_ratio": f8["schedule"]["ratio"], "decode_B8_us": f8["decode"]["us_per_step"],
                          "decode_frac_of_hbm": f8["decode"]["frac_of_hbm"], "decode_B8_us_graph": f8["decode"]["us_per_step_graph"],
                          "decode_frac_of_hbm_graph": f8["decode"]["frac_of_hbm_graph"]},

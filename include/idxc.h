@@ -333,6 +333,15 @@ idxc_status idxc_selftest_bounded_wait(uint32_t wait_cycles, void* cuda_stream);
  * over all SMs; time the launch with events around the call to get bytes per second. 1 <= accumulators_per_warp <= 2^24. */
 idxc_status idxc_selftest_tmem_readout(uint32_t accumulators_per_warp, int64_t* bytes_read_out, void* cuda_stream);
 
+/* Measurement aid (no counterpart in the paper): the same read-out while one more warp per SM keeps the tensor pipe busy
+ * filling the two 128 x 256 accumulators with MMAs of the scorer's shape (fp8 != 0: e4m3, four K = 32 steps per fill;
+ * else bf16, eight K = 16 steps; operands are zero tiles in shared memory) until the reading warps are done. It tells
+ * whether tensor-memory reads and MMAs slow each other down. counters (DEVICE, uint64 [2], zeroed by the call):
+ * [0] = accumulator fills completed over all SMs while the readers ran (each 2 * 128 * 256 * 128 flops),
+ * [1] = cycles of the slowest reading warp. *bytes_read_out (HOST, may be NULL) as above; time the launch with events. */
+idxc_status idxc_selftest_tmem_readout_under_mma(uint32_t accumulators_per_warp, int fp8, int64_t* bytes_read_out,
+                                                 uint64_t* counters, void* cuda_stream);
+
 /* Number of kernel launches this library has made in this process (all streams). */
 int64_t idxc_launch_count(void);
 

@@ -27,7 +27,7 @@ EXPORTED_SYMBOLS = [
     "idxc_indexer_decode", "idxc_topk_rows", "idxc_schedule_create", "idxc_schedule_destroy",
     "idxc_schedule_begin_pass", "idxc_schedule_source", "idxc_schedule_stats", "idxc_schedule_prefill_layer",
     "idxc_schedule_decode_layer", "idxc_poll_device_status", "idxc_launch_count", "idxc_indexer_decode_noalloc",
-    "idxc_selftest_bounded_wait", "idxc_selftest_tmem_readout", "idxc_quantize_e4m3", "idxc_topk_overlap", "idxc_pattern_search_dp",
+    "idxc_selftest_bounded_wait", "idxc_selftest_tmem_readout", "idxc_selftest_tmem_readout_under_mma", "idxc_quantize_e4m3", "idxc_topk_overlap", "idxc_pattern_search_dp",
     "idxc_pattern_search_greedy", "idxc_distill_kl", "idxc_sparse_attention_workspace_bytes", "idxc_sparse_attention",
 ]
 NOALLOC_SCRATCH_BYTES = 16 << 20
@@ -104,6 +104,8 @@ def lib() -> ctypes.CDLL:
         L.idxc_selftest_bounded_wait.argtypes = [u32, vp]
         L.idxc_selftest_tmem_readout.restype = i32
         L.idxc_selftest_tmem_readout.argtypes = [u32, ctypes.POINTER(i64), vp]
+        L.idxc_selftest_tmem_readout_under_mma.restype = i32
+        L.idxc_selftest_tmem_readout_under_mma.argtypes = [u32, ctypes.c_int, ctypes.POINTER(i64), vp, vp]
         L.idxc_poll_device_status.restype = i32
         L.idxc_poll_device_status.argtypes = [vp]
         _lib = L
@@ -364,6 +366,16 @@ def selftest_tmem_readout(accumulators_per_warp: int, stream=None) -> int:
     nbytes = ctypes.c_int64()
     _check(lib().idxc_selftest_tmem_readout(int(accumulators_per_warp), ctypes.byref(nbytes), _stream(stream)),
            "idxc_selftest_tmem_readout")
+    return int(nbytes.value)
+
+
+def selftest_tmem_readout_under_mma(accumulators_per_warp: int, fp8: bool, counters, stream=None) -> int:
+    """idxc_selftest_tmem_readout_under_mma: the read-out measurement with MMAs running beside it; counters is a device
+    int64 tensor of two entries (accumulator fills completed, cycles of the slowest reader). Returns the bytes read."""
+    _dev(counters, "counters", torch.int64)
+    nbytes = ctypes.c_int64()
+    _check(lib().idxc_selftest_tmem_readout_under_mma(int(accumulators_per_warp), int(bool(fp8)), ctypes.byref(nbytes),
+                                                      _ptr(counters), _stream(stream)), "idxc_selftest_tmem_readout_under_mma")
     return int(nbytes.value)
 
 

@@ -540,6 +540,19 @@ idxc_status idxc_selftest_tmem_readout(uint32_t accumulators_per_warp, int64_t* 
                ? IDXC_OK : IDXC_ERR_CUDA;
 }
 
+idxc_status idxc_selftest_tmem_readout_under_mma(uint32_t accumulators_per_warp, int fp8, int64_t* bytes_read_out,
+                                                 uint64_t* counters, void* cuda_stream) {
+    DeviceInfo& di = device_info();
+    if (!di.ok) return IDXC_ERR_CUDA;
+    if (accumulators_per_warp == 0 || accumulators_per_warp > (1u << 24) || !counters) return IDXC_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (bytes_read_out) *bytes_read_out = static_cast<int64_t>(di.sm_count) * 8 * accumulators_per_warp * (32 * 128 * 4);
+    if (cudaMemsetAsync(counters, 0, 2 * sizeof(uint64_t), stream) != cudaSuccess) return IDXC_ERR_CUDA;
+    g_launches += 1;
+    return launch_selftest_tmem_readout_mma(accumulators_per_warp, fp8 != 0, di.status_ptr, reinterpret_cast<unsigned long long*>(counters),
+                                            di.status_ptr, di.sm_count, stream) == cudaSuccess ? IDXC_OK : IDXC_ERR_CUDA;
+}
+
 idxc_status idxc_poll_device_status(void* cuda_stream) {
     if (!device_info().ok) return IDXC_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
