@@ -1,7 +1,8 @@
 // Pattern tooling on index tensors (the paper's Appendix A, Appendix C and Algorithm 1).
 //   * overlap kernel: per query row |T_a n T_b| / (valid entries of T_a), for one pair of index tensors or
-//     for every pair of N layers in one launch. Both rows are ascending: runs of one row are merged against the
-//     other in shared memory. 2 * 4 * k bytes per row pair (the pairs of a row run together: repeats hit the L2).
+//     for every pair of N layers in one launch. One row's entries set bits of a shared-memory bitmap, the other row's
+//     entries test them (indices below 131072); rows that reach further are ascending runs merged in shared memory.
+//     2 * 4 * k bytes per row pair (the pairs of a row run together: repeats hit the L2).
 //   * similarity DP (host): the exact pattern with M Full layers that maximises the summed similarity of
 //     the Shared layers to their source layers.
 //   * greedy layer selection (host): Algorithm 1 with the caller's loss function.
