@@ -1055,6 +1055,26 @@ def main():
     torch.cuda.synchronize()
     combined_ms = c0.elapsed_time(c1) / K
 
+    # ---- the select by itself, after a pause in which the board leaves the power limit the scorer holds it at: the
+    # select's time follows the SM clock (it is bound by instruction issue, not by bytes), so both figures are given
+    # with the clock they were taken at
+    time.sleep(0.5)
+    with ClockSampler(local) as clk_alone:
+        for _ in range(3):
+            idxc.topk_rows(scores, k_top, topk, first_len=1, len_step=1)
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record()
+        for _ in range(20):
+            idxc.topk_rows(scores, k_top, topk, first_len=1, len_step=1)
+        a1.record()
+        torch.cuda.synchronize()
+    topk_alone_ms = a0.elapsed_time(a1) / 20
+    alone_gbs = topk_bytes / (topk_alone_ms * 1e-3) / 1e9
+    roofline["topk_kernel"]["alone"] = {"ms_per_launch": topk_alone_ms, "achieved": alone_gbs, "frac": alone_gbs / peaks["hbm_gbs"],
+                                        "sm_mhz": clk_alone.summary()["sm_mhz"],
+                                        "note": "20 calls back to back without the scorer between them; the figure above is taken inside the "
+                                                "timed loop, at the clock the top-level `clocks` entry records"}
+
     # ---- e2e: host buffers; every step copies its inputs H2D (pinned) and its result D2H inside the timed
     # region. Steps are software-pipelined over three streams with double-buffered device inputs and outputs
     # (copy-in of step i+1 and copy-out of step i-1 overlap the kernels of step i), as a serving loop would.
