@@ -929,10 +929,16 @@ def main():
     peaks = load_peaks()
 
     def section(fn, *a, **kw):
-        """Runs one section with the clock sampler around it; the section's dict gets a `clocks` entry."""
+        """Runs one section with the clock sampler around it; the section's dict gets a `clocks` entry. A section that
+        raises is reported as {"error": ...} (and on stderr) instead of taking the headline line with it."""
         with ClockSampler(local) as clk:
-            res = fn(*a, **kw)
-            torch.cuda.synchronize()
+            try:
+                res = fn(*a, **kw)
+                torch.cuda.synchronize()
+            except Exception as e:
+                import traceback
+                traceback.print_exc()
+                res = {"error": f"{type(e).__name__}: {e}"[:400]}
         res["clocks"] = clk.summary()
         torch.cuda.empty_cache()
         return res
@@ -1195,25 +1201,30 @@ def main():
             line["stream_topk"] = section(time_stream_topk, idxc, synth, dev, c2["L"], c2["H"], c2["d"], c2["k_top"], c2["seed"])
             # the five workloads in one place, inside the roofline block and again at the very end of the line
             f8, dc, sc = line["fp8_chunked"], line["decode"], line["schedule"]
-            by_config = {
-                "cfg1": {"us_per_call": line["cfg1"]["us_per_call"], "us_back_to_back": line["cfg1"]["us_per_call_back_to_back"],
-                         "us_graph": line["cfg1"]["us_per_call_graph"]},
-                "cfg2": {"gpairs_per_s": value, "ms_per_step": ms_per_step, "scorer_frac_of_bf16_peak": roofline["frac"],
-                         "topk_frac_of_hbm": roofline["topk_kernel"]["frac"],
-                         "streaming_topk_ms": line["stream_topk"]["ms_streaming"], "streaming_topk_identical": line["stream_topk"]["indices_identical"]},
-                "cfg3": {"us_per_step": dc["us_per_step"], "scorer_frac_of_hbm": dc["roofline"]["frac"], "step_frac_of_hbm": dc["frac_step_vs_hbm"],
-                         "us_per_step_graph": dc["us_per_step_graph"], "step_frac_of_hbm_graph": dc["frac_step_vs_hbm_graph"]},
-                "cfg4": {"workload": sc["workload"], "ms_scheduled": sc["ms_scheduled"], "ms_all_full": sc["ms_all_full"], "ratio": sc["ratio"],
-                         "gpairs_per_s_full_layers": sc["gpairs_per_s_full_layers"], "checks": sc["checks"]},
-                "cfg5": {"workload": f8["workload"], "ms_per_full_layer": f8["ms_per_layer"], "gpairs_per_s": f8["gpairs_per_s"],
-                         "scorer_frac_of_2x_bf16_peak": f8["roofline_tensor"]["frac"],
-                         "scorer_frac_of_2x_bf16_sustained": f8["roofline_tensor"]["frac_of_sustained"],
-                         "scorer_frac_of_tmem_readout": f8.get("roofline_readout", {}).get("frac"),
-                         "scorer_frac_of_gate_rate": f8["roofline_gate"]["frac"],
-                         "schedule_ratio": f8["schedule"]["ratio"], "decode_B8_us": f8["decode"]["us_per_step"],
-                         "decode_frac_of_hbm": f8["decode"]["frac_of_hbm"], "decode_B8_us_graph": f8["decode"]["us_per_step_graph"],
-                         "decode_frac_of_hbm_graph": f8["decode"]["frac_of_hbm_graph"]},
-            }
+            def summarise():
+                return {
+                    "cfg1": {"us_per_call": line["cfg1"]["us_per_call"], "us_back_to_back": line["cfg1"]["us_per_call_back_to_back"],
+                             "us_graph": line["cfg1"]["us_per_call_graph"]},
+                    "cfg2": {"gpairs_per_s": value, "ms_per_step": ms_per_step, "scorer_frac_of_bf16_peak": roofline["frac"],
+                             "topk_frac_of_hbm": roofline["topk_kernel"]["frac"],
+                             "streaming_topk_ms": line["stream_topk"]["ms_streaming"], "streaming_topk_identical": line["stream_topk"]["indices_identical"]},
+                    "cfg3": {"us_per_step": dc["us_per_step"], "scorer_frac_of_hbm": dc["roofline"]["frac"], "step_frac_of_hbm": dc["frac_step_vs_hbm"],
+                             "us_per_step_graph": dc["us_per_step_graph"], "step_frac_of_hbm_graph": dc["frac_step_vs_hbm_graph"]},
+                    "cfg4": {"workload": sc["workload"], "ms_scheduled": sc["ms_scheduled"], "ms_all_full": sc["ms_all_full"], "ratio": sc["ratio"],
+                             "gpairs_per_s_full_layers": sc["gpairs_per_s_full_layers"], "checks": sc["checks"]},
+                    "cfg5": {"workload": f8["workload"], "ms_per_full_layer": f8["ms_per_layer"], "gpairs_per_s": f8["gpairs_per_s"],
+                             "scorer_frac_of_2x_bf16_peak": f8["roofline_tensor"]["frac"],
+                             "scorer_frac_of_2x_bf16_sustained": f8["roofline_tensor"]["frac_of_sustained"],
+                             "scorer_frac_of_tmem_readout": f8.get("roofline_readout", {}).get("frac"),
+                             "scorer_frac_of_gate_rate": f8["roofline_gate"]["frac"],
+                             "schedule_ratio": f8["schedule"]["ratio"], "decode_B8_us": f8["decode"]["us_per_step"],
+                             "decode_frac_of_hbm": f8["decode"]["frac_of_hbm"], "decode_B8_us_graph": f8["decode"]["us_per_step_graph"],
+                             "decode_frac_of_hbm_graph": f8["decode"]["frac_of_hbm_graph"]},
+                }
+            try:
+                by_config = summarise()
+            except (KeyError, TypeError) as e:      # a section reported an error instead of its figures
+                by_config = {"error": f"summary incomplete: {type(e).__name__}: {e}"}
             line["roofline"]["by_config"] = by_config
             line["summary"] = by_config
     if rank == 0:
