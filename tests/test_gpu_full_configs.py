@@ -59,11 +59,12 @@ _codes_cache = {}
 
 
 def codes_cached(inp):
-    key = id(inp.k)
-    if key not in _codes_cache:
-        _codes_cache.clear()
-        _codes_cache[key] = codes(inp.k)
-    return _codes_cache[key]
+    """Host copy of the current inputs' key codes, made once per input set. The cache keeps the tensor itself and compares
+    by identity: an `id()` alone can come back for a new tensor once the old one has been freed."""
+    if _codes_cache.get("k") is not inp.k:
+        _codes_cache["k"] = inp.k
+        _codes_cache["codes"] = codes(inp.k)
+    return _codes_cache["codes"]
 
 
 def _gpu_row_scores(inp, t, k_top):
