@@ -524,6 +524,8 @@ def time_tmem_readout(idxc, dev, accumulators_per_warp=4096):
         out[name] = {"ms": t, "tbytes_per_s": nb / (t * 1e-3) / 1e12, "accumulator_fills": fills,
                      "mma_tflops": fills * 2.0 * 128 * 256 * 128 / (t * 1e-3) / 1e12,
                      "reader_cycles_per_accumulator": cycles / accumulators_per_warp}
+    # what one scheduler takes per warp instruction of the kinds the epilogue and the select are made of
+    out["issue_cycles_per_warp_instruction"] = idxc.selftest_issue_rates(4096)
     out["under_mma_note"] = ("readers and MMAs run unordered beside each other on every SM; mma_tflops counts the fills completed while the "
                              "readers ran (2 x 128 x 256 x 128 flops each) over the launch time")
     return out
@@ -658,12 +660,14 @@ def time_fp8_chunked(idxc, synth, dev, peaks, L, chunk, H, d, k_top, seed, decod
     # the gate: one min/max instruction per accumulator element on a pipe that issues 16 lanes per clock and scheduler
     # (measured: a warp's FMNMX every 2.0 cycles per scheduler), 4 schedulers per SM, at the SM clock's maximum
     props = torch.cuda.get_device_properties(dev)
-    gate_peak = props.multi_processor_count * 4 * 16 * (NOMINAL["sm_max_mhz"] * 1e6) / 1e12          # T elements / s
+    fmnmx_cycles = (readout or {}).get("issue_cycles_per_warp_instruction", {}).get("fmnmx", 2.0)     # measured in this run
+    gate_peak = props.multi_processor_count * 4 * (32.0 / fmnmx_cycles) * (NOMINAL["sm_max_mhz"] * 1e6) / 1e12   # T elements / s
     gate_ach = acc_bytes / 4 / (t_sc * 1e-3) / 1e12
     out["roofline_gate"] = {"bound": "alu", "achieved": gate_ach, "peak": gate_peak, "unit": "T accumulator elements gated per second",
                             "frac": gate_ach / gate_peak,
-                            "derivation": "ReLU = one min/max per accumulator element; that pipe takes a warp instruction every 2 cycles per scheduler: "
-                                          f"{props.multi_processor_count} SMs x 4 schedulers x 16 lanes x {NOMINAL['sm_max_mhz']} MHz; with e4m3 inputs this equals the tensor time "
+                            "derivation": f"ReLU = one min/max per accumulator element; a scheduler takes one such warp instruction every {fmnmx_cycles:.2f} cycles "
+                                          "(measured in this run, tmem_readout.issue_cycles_per_warp_instruction): "
+                                          f"{props.multi_processor_count} SMs x 4 schedulers x 32 lanes / {fmnmx_cycles:.2f} x {NOMINAL['sm_max_mhz']} MHz; with e4m3 inputs this equals the tensor time "
                                           "of the accumulator (512 cycles per 128 x 256), and the epilogue's selects, compares and address arithmetic share the pipe"}
     fp8_peak = measure_fp8_gemm_peak(dev)
     if fp8_peak:

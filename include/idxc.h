@@ -342,6 +342,17 @@ idxc_status idxc_selftest_tmem_readout(uint32_t accumulators_per_warp, int64_t* 
 idxc_status idxc_selftest_tmem_readout_under_mma(uint32_t accumulators_per_warp, int fp8, int64_t* bytes_read_out,
                                                  uint64_t* counters, void* cuda_stream);
 
+/* Measurement aid (no counterpart in the paper): how fast one scheduler of an SM takes instructions of seven kinds,
+ * which is what bounds the scorer's epilogue and the select (both are limited by instruction issue, not by bytes).
+ * Enqueues seven kernels (one CTA of 256 threads per SM: two warps per scheduler); in each, every thread runs `rounds`
+ * rounds of 16 independent instructions of one kind (8 for the packed kind). cycles (DEVICE, uint64
+ * [IDXC_ISSUE_RATE_KINDS], zeroed by the call) receives the slowest warp's cycles per kind, in this order: 0 float min/max,
+ * 1 add with |x|, 2 fma, 3 packed fma.rn.f32x2 (8 per round), 4 compare + select (a pair per slot), 5 three-input logic,
+ * 6 warp shuffle. cycles[i] / (rounds * 16 * 2) (8 for kind 3) = scheduler cycles per
+ * warp instruction. 1 <= rounds <= 2^20. */
+#define IDXC_ISSUE_RATE_KINDS 7
+idxc_status idxc_selftest_issue_rates(uint32_t rounds, uint64_t* cycles, void* cuda_stream);
+
 /* Number of kernel launches this library has made in this process (all streams). */
 int64_t idxc_launch_count(void);
 

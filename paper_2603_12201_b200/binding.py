@@ -27,7 +27,7 @@ EXPORTED_SYMBOLS = [
     "idxc_indexer_decode", "idxc_topk_rows", "idxc_schedule_create", "idxc_schedule_destroy",
     "idxc_schedule_begin_pass", "idxc_schedule_source", "idxc_schedule_stats", "idxc_schedule_prefill_layer",
     "idxc_schedule_decode_layer", "idxc_poll_device_status", "idxc_launch_count", "idxc_indexer_decode_noalloc",
-    "idxc_selftest_bounded_wait", "idxc_selftest_tmem_readout", "idxc_selftest_tmem_readout_under_mma", "idxc_quantize_e4m3", "idxc_topk_overlap", "idxc_pattern_search_dp",
+    "idxc_selftest_bounded_wait", "idxc_selftest_tmem_readout", "idxc_selftest_tmem_readout_under_mma", "idxc_selftest_issue_rates", "idxc_quantize_e4m3", "idxc_topk_overlap", "idxc_pattern_search_dp",
     "idxc_pattern_search_greedy", "idxc_distill_kl", "idxc_sparse_attention_workspace_bytes", "idxc_sparse_attention",
 ]
 NOALLOC_SCRATCH_BYTES = 16 << 20
@@ -106,6 +106,8 @@ def lib() -> ctypes.CDLL:
         L.idxc_selftest_tmem_readout.argtypes = [u32, ctypes.POINTER(i64), vp]
         L.idxc_selftest_tmem_readout_under_mma.restype = i32
         L.idxc_selftest_tmem_readout_under_mma.argtypes = [u32, ctypes.c_int, ctypes.POINTER(i64), vp, vp]
+        L.idxc_selftest_issue_rates.restype = i32
+        L.idxc_selftest_issue_rates.argtypes = [u32, vp, vp]
         L.idxc_poll_device_status.restype = i32
         L.idxc_poll_device_status.argtypes = [vp]
         _lib = L
@@ -377,6 +379,20 @@ def selftest_tmem_readout_under_mma(accumulators_per_warp: int, fp8: bool, count
     _check(lib().idxc_selftest_tmem_readout_under_mma(int(accumulators_per_warp), int(bool(fp8)), ctypes.byref(nbytes),
                                                       _ptr(counters), _stream(stream)), "idxc_selftest_tmem_readout_under_mma")
     return int(nbytes.value)
+
+
+ISSUE_RATE_KINDS = ("fmnmx", "fadd_abs", "ffma", "ffma2_packed", "fsetp_sel_pair", "lop3", "shfl")
+
+
+def selftest_issue_rates(rounds: int = 4096, stream=None) -> dict:
+    """idxc_selftest_issue_rates: scheduler cycles per warp instruction for seven instruction kinds (two warps per
+    scheduler). Synchronises the stream to read the counters back."""
+    s = torch.cuda.current_stream() if stream is None else stream
+    cycles = torch.zeros(len(ISSUE_RATE_KINDS), dtype=torch.int64, device=f"cuda:{torch.cuda.current_device()}")
+    _check(lib().idxc_selftest_issue_rates(int(rounds), _ptr(cycles), _stream(s)), "idxc_selftest_issue_rates")
+    s.synchronize()
+    c = cycles.tolist()
+    return {name: c[i] / (rounds * (8 if name == "ffma2_packed" else 16) * 2.0) for i, name in enumerate(ISSUE_RATE_KINDS)}
 
 
 def poll_device_status(stream=None):

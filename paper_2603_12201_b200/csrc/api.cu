@@ -553,6 +553,18 @@ idxc_status idxc_selftest_tmem_readout_under_mma(uint32_t accumulators_per_warp,
                                             di.status_ptr, di.sm_count, stream) == cudaSuccess ? IDXC_OK : IDXC_ERR_CUDA;
 }
 
+idxc_status idxc_selftest_issue_rates(uint32_t rounds, uint64_t* cycles, void* cuda_stream) {
+    DeviceInfo& di = device_info();
+    if (!di.ok) return IDXC_ERR_CUDA;
+    if (rounds == 0 || rounds > (1u << 20) || !cycles) return IDXC_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemsetAsync(cycles, 0, IDXC_ISSUE_RATE_KINDS * sizeof(uint64_t), stream) != cudaSuccess) return IDXC_ERR_CUDA;
+    g_launches += IDXC_ISSUE_RATE_KINDS;
+    // the status word doubles as the sink: the kernels never write it in practice (see selftest.cu)
+    return launch_selftest_issue_rates(rounds, reinterpret_cast<unsigned long long*>(cycles), reinterpret_cast<float*>(di.status_ptr),
+                                       di.sm_count, stream) == cudaSuccess ? IDXC_OK : IDXC_ERR_CUDA;
+}
+
 idxc_status idxc_poll_device_status(void* cuda_stream) {
     if (!device_info().ok) return IDXC_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);

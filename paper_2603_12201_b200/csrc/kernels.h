@@ -122,6 +122,8 @@ cudaError_t launch_selftest_bounded_wait(unsigned int* status, long long budget_
 // selftest.cu: every SM reads `iters` 128 x 256 fp32 accumulators per reading warp out of tensor memory with the
 // prefill epilogue's load pattern (8 warps per SM); `sink` is a device word that is never written in practice.
 cudaError_t launch_selftest_tmem_readout(uint32_t iters, uint32_t* sink, int sm_count, cudaStream_t stream);
+// Issue rates of seven instruction kinds (selftest.cu); cycles: DEVICE [7], zeroed by the caller.
+cudaError_t launch_selftest_issue_rates(uint32_t iters, unsigned long long* cycles, float* sink, int sm_count, cudaStream_t stream);
 // The same read-out with a warp filling the accumulators by MMAs beside it; counters: DEVICE [2], see selftest.cu.
 cudaError_t launch_selftest_tmem_readout_mma(uint32_t iters, bool fp8, uint32_t* sink, unsigned long long* counters,
                                              unsigned int* status, int sm_count, cudaStream_t stream);

@@ -183,7 +183,60 @@ selftest_tmem_readout_mma_kernel(uint32_t iters, uint32_t* sink, unsigned long l
     }
 }
 
+// Issue rate of single instructions: every thread runs `iters` rounds of 16 independent operations of one kind (8 for the
+// packed two-wide ones) on registers, 256 threads per CTA and one CTA per SM, i.e. two warps per scheduler. cycles[OP] = the
+// slowest warp's cycles over all CTAs; divided by iters x 16 (or 8) x 2 it is the scheduler's cycles per warp instruction.
+// The operands rotate through the registers so that no round can be folded into the one before.
+template <int OP>
+__global__ void __launch_bounds__(256, 1)
+selftest_issue_rate_kernel(uint32_t iters, float seed, unsigned long long* cycles, float* sink) {
+    float x[16];
+    uint64_t pk[8];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) x[i] = seed * static_cast<float>(threadIdx.x + i) - 3.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) pk[i] = pack_f32x2(x[2 * i], x[2 * i + 1]);
+    const uint64_t w = pack_f32x2(seed, 1.0001f);
+    const long long t0 = clock64();
+    for (uint32_t it = 0; it < iters; ++it) {
+        if constexpr (OP == 3) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) pk[i] = fma_f32x2(pk[i], w, pk[i]);                                   // fma.rn.f32x2
+        } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float a = x[(i + 1) & 15], b = x[(i + 5) & 15];
+                if constexpr (OP == 0) x[i] = fmaxf(a, b);                                                    // min/max
+                if constexpr (OP == 1) x[i] = x[i] + fabsf(x[i]);                                             // add with |x|
+                if constexpr (OP == 2) x[i] = fmaf(x[i], seed, 0.5f);                                         // fma
+                if constexpr (OP == 4) x[i] = (x[i] > seed) ? x[i] : a;                                       // compare + select
+                if constexpr (OP == 5) x[i] = __uint_as_float(__float_as_uint(a) ^ __float_as_uint(b));       // three-input logic
+                if constexpr (OP == 6) x[i] = __shfl_xor_sync(0xFFFFFFFFu, x[i], 1);                          // shuffle
+            }
+        }
+    }
+    const long long t1 = clock64();
+    float sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) sum += x[i];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { float lo, hi; unpack_f32x2(pk[i], lo, hi); sum += lo + hi; }
+    if (sum == 1234.5678f && iters == 0xFFFFFFFFu) *sink = sum;      // keeps the chains alive; never true in practice
+    if ((threadIdx.x & 31) == 0) atomicMax(&cycles[OP], static_cast<unsigned long long>(t1 - t0));
+}
+
 }  // namespace
+
+cudaError_t launch_selftest_issue_rates(uint32_t iters, unsigned long long* cycles, float* sink, int sm_count, cudaStream_t stream) {
+    selftest_issue_rate_kernel<0><<<sm_count, 256, 0, stream>>>(iters, 0.37f, cycles, sink);
+    selftest_issue_rate_kernel<1><<<sm_count, 256, 0, stream>>>(iters, 0.37f, cycles, sink);
+    selftest_issue_rate_kernel<2><<<sm_count, 256, 0, stream>>>(iters, 0.37f, cycles, sink);
+    selftest_issue_rate_kernel<3><<<sm_count, 256, 0, stream>>>(iters, 0.37f, cycles, sink);
+    selftest_issue_rate_kernel<4><<<sm_count, 256, 0, stream>>>(iters, 0.37f, cycles, sink);
+    selftest_issue_rate_kernel<5><<<sm_count, 256, 0, stream>>>(iters, 0.37f, cycles, sink);
+    selftest_issue_rate_kernel<6><<<sm_count, 256, 0, stream>>>(iters, 0.37f, cycles, sink);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_selftest_tmem_readout_mma(uint32_t iters, bool fp8, uint32_t* sink, unsigned long long* counters,
                                              unsigned int* status, int sm_count, cudaStream_t stream) {
